@@ -1,0 +1,163 @@
+/*
+ * osdp.h -- C ABI of the operator-split linear layer for NVIDIA B200 (sm_100a).
+ *
+ * The operation is the paper's "Operator Splitting" (Section 3.3): a large MatMul operator
+ * is cut into `slice granularity` slices that are processed one after another, and the
+ * partial results are combined.  Here the operator is a linear layer
+ *
+ *      Y = act(X W^T + b)        X [M,K] tokens x in_features,  W [N,K] row-major,
+ *      dX = G W,  dW = G^T X,  db = column sums of G,   G = dY (.) act'(X W^T + b)
+ *
+ * and k = k_split slices are taken along
+ *      OSDP_SPLIT_OUT : the N rows of W (outputs Y, dW, db concatenate; dX is summed), or
+ *      OSDP_SPLIT_RED : the K columns of W and X -- the paper's own wording ("the last
+ *                       dimension of the input data and the first dimension of the operator
+ *                       ... all computation results are summed") -- Y is summed; dX, dW concatenate.
+ * Slices are visited in ascending order (slice-major).  A summed output is carried between
+ * slices as an fp32 running sum in the caller's workspace.
+ *
+ * Slice rule (the paper gives none for non-divisible extents): slice length
+ * L = ceil(D/k) rounded up to a multiple of 8 elements; slice s = [s*L, min(D,(s+1)*L)); a
+ * k for which the last slice would be empty is rejected.  k_split 0 means 1 (the paper plots
+ * "granularity 0" as no splitting).
+ *
+ * Conventions for every call
+ *  - All tensor pointers are DEVICE pointers unless stated; they stay owned by the caller and
+ *    must stay valid until the stream has passed the call.  Nothing is allocated or freed.
+ *  - bf16 tensors are row-major, 16-byte aligned; N and K must be multiples of 8.
+ *  - W lives inside a flat bf16 parameter buffer `w_flat` at ELEMENT offset `w_offset`
+ *    (multiple of 8); it is read in place through TMA descriptors, never copied or unflattened.
+ *    dW is written at `dw_offset` of a flat gradient buffer `dw_flat` (bf16 or fp32 elements).
+ *  - Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = default
+ *    stream) and never synchronise, except osdp_read_device_status.
+ *  - `ws` is scratch of at least osdp_split_linear_workspace_bytes(...) bytes, 256-byte
+ *    aligned.  Its first word is a device status word (see osdp_read_device_status); the
+ *    caller zeroes the first 256 bytes once after allocating it.
+ *  - Return value: OSDP_OK or an error code; nothing is launched when an argument check
+ *    fails.  Never aborts, never prints.
+ */
+#ifndef OSDP_H_
+#define OSDP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define OSDP_VERSION 100
+
+/* status codes */
+#define OSDP_OK 0
+#define OSDP_ERR_NULL_POINTER 1
+#define OSDP_ERR_BAD_SHAPE 2          /* M, N or K <= 0, or too large for 32-bit tile coordinates */
+#define OSDP_ERR_BAD_SPLIT 3          /* k < 0, empty slice, bad split_dim, slice_idx out of range */
+#define OSDP_ERR_ALIGNMENT 4          /* pointer / offset not 16-byte aligned, N or K not a multiple of 8 */
+#define OSDP_ERR_WORKSPACE_TOO_SMALL 5
+#define OSDP_ERR_UNSUPPORTED 6        /* unknown activation, dtype or op */
+#define OSDP_ERR_CUDA 7               /* a CUDA call failed; see osdp_last_cuda_error */
+#define OSDP_ERR_DEVICE_TIMEOUT 8     /* a bounded device-side wait ran out (status word) */
+
+#define OSDP_SPLIT_OUT 0
+#define OSDP_SPLIT_RED 1
+
+#define OSDP_ACT_NONE 0
+#define OSDP_ACT_GELU_TANH 1
+#define OSDP_ACT_GELU_ERF 2
+
+#define OSDP_DTYPE_BF16 0
+#define OSDP_DTYPE_FP32 1
+
+#define OSDP_OP_LINEAR_FWD 0
+#define OSDP_OP_LINEAR_BWD 1
+#define OSDP_OP_MLP_FWD 2
+#define OSDP_OP_MLP_BWD 3
+
+#define OSDP_MAX_SPLIT 1024
+
+int osdp_version(void);
+const char *osdp_status_string(int status);
+/* The cudaError_t (as int) of the most recent failed CUDA call made by this library on the
+ * calling thread, 0 if none. */
+int osdp_last_cuda_error(void);
+
+/* Section 3.3 step 1 (partition): [begin,end) of slice s of an extent D cut into k slices by
+ * the slice rule above.  Host-only integer arithmetic.  OSDP_ERR_BAD_SPLIT if a slice is empty
+ * or s is out of range. */
+int osdp_slice_range(int64_t D, int k_split, int slice_idx, int64_t *begin, int64_t *end);
+
+/* Exact scratch bytes a call with these arguments uses (the "staging" figure).  For the linear
+ * ops (M,N,K) are the layer's; for the MLP ops pass M = tokens, N = ffn, K = hidden.
+ * The query assumes every optional output (dx, dbias, ...) is requested. */
+int osdp_split_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int k_split, int split_dim,
+                                      int act, int op, size_t *bytes);
+
+/* Forward of all k slices in slice-major order (Section 3.3 steps 1-3).
+ *   x [M,K] bf16; bias [N] fp32 or NULL; out [M,N] bf16 = act(X W^T + bias);
+ *   z_save [M,N] bf16 or NULL: receives the pre-activation (what the backward needs when act != NONE).
+ * OUT: slice s writes columns R_s of out.  RED: partial products are summed (fp32 carry in ws);
+ * bias and activation are applied once, after the last slice. */
+int osdp_split_linear_fwd(const void *x, const void *w_flat, int64_t w_offset, const float *bias,
+                          int64_t M, int64_t N, int64_t K, int k_split, int split_dim, int act,
+                          void *out, void *z_save, void *ws, size_t ws_bytes, void *stream);
+
+/* One slice of the forward (Section 3.3 step 2, "the computation of each slice is executed
+ * sequentially"): lets a caller put other work between slices.  Slices must be issued in
+ * ascending order on one stream with the same arguments and workspace: under RED slice 0
+ * starts the carry and slice k-1 writes `out`. */
+int osdp_split_linear_fwd_slice(const void *x, const void *w_flat, int64_t w_offset, const float *bias,
+                                int64_t M, int64_t N, int64_t K, int k_split, int split_dim, int act,
+                                int slice_idx, void *out, void *z_save, void *ws, size_t ws_bytes,
+                                void *stream);
+
+/* Backward of all k slices in slice-major order.
+ *   dy [M,N] bf16; x [M,K] bf16; z_saved [M,N] bf16 (pre-activation; required iff act != NONE);
+ *   dx [M,K] bf16 or NULL; dw_flat + dw_offset: dW [N,K] in dw_dtype (bf16 or fp32), NULL to skip;
+ *   accumulate: 0 dW = ..., 1 dW += ...; dbias [N] fp32 or NULL (always overwritten).
+ * OUT: dW[R_s,:], db[R_s] per slice, dX = sum over slices (fp32 carry in ws).
+ * RED: dX[:,C_s], dW[:,C_s] per slice. */
+int osdp_split_linear_bwd(const void *dy, const void *x, const void *w_flat, int64_t w_offset,
+                          const void *z_saved, int64_t M, int64_t N, int64_t K, int k_split,
+                          int split_dim, int act, void *dx, void *dw_flat, int64_t dw_offset,
+                          int dw_dtype, int accumulate, float *dbias, void *ws, size_t ws_bytes,
+                          void *stream);
+
+/* One slice of the backward; same ordering rule as osdp_split_linear_fwd_slice.  Under RED
+ * dbias is produced by slice 0. */
+int osdp_split_linear_bwd_slice(const void *dy, const void *x, const void *w_flat, int64_t w_offset,
+                                const void *z_saved, int64_t M, int64_t N, int64_t K, int k_split,
+                                int split_dim, int act, int slice_idx, void *dx, void *dw_flat,
+                                int64_t dw_offset, int dw_dtype, int accumulate, float *dbias,
+                                void *ws, size_t ws_bytes, void *stream);
+
+/* Transformer MLP block split along the ffn dimension (first layer OUT-split + activation,
+ * second layer RED-split, Section 3.3 applied to both MatMuls of the block):
+ *   out [M,hidden] = sum_s act(X W1[F_s,:]^T + b1[F_s]) W2[:,F_s]^T + b2, slice by slice.
+ * W1 [ffn,hidden] at off_w1 and W2 [hidden,ffn] at off_w2 of the same flat buffer; b1 [ffn],
+ * b2 [hidden] fp32 or NULL.  Only a slice-sized intermediate A_s [M, ffn/k] lives in ws.
+ * z1_save [M,ffn] bf16 or NULL receives the first layer's pre-activation for the backward. */
+int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const float *b1,
+                       int64_t off_w2, const float *b2, int64_t M, int64_t hidden, int64_t ffn,
+                       int k_split, int act, void *out, void *z1_save, void *ws, size_t ws_bytes,
+                       void *stream);
+
+/* Backward of the split MLP block, slice by slice, from the saved pre-activation z1_saved
+ * [M,ffn] bf16:  dA_s = dY W2[:,F_s]; dZ_s = dA_s (.) act'(Z1_s); dW2[:,F_s] = dY^T act(Z1_s);
+ * dW1[F_s,:] = dZ_s^T X; db1[F_s] = colsum dZ_s; dX = sum_s dZ_s W1[F_s,:]; db2 = colsum dY.
+ * dW1/dW2 land at dw_off_w1/dw_off_w2 of dw_flat (dw_dtype).  Slice-sized dZ_s and A_s live in ws. */
+int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_t off_w1,
+                       int64_t off_w2, const void *z1_saved, int64_t M, int64_t hidden, int64_t ffn,
+                       int k_split, int act, void *dx, void *dw_flat, int64_t dw_off_w1,
+                       int64_t dw_off_w2, int dw_dtype, int accumulate, float *db1, float *db2,
+                       void *ws, size_t ws_bytes, void *stream);
+
+/* Synchronises `stream`, copies the device status word at the start of `ws` to *status
+ * (OSDP_OK, or OSDP_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel ran out) and
+ * clears it.  Every device-side wait in this library is bounded; none can hang the GPU. */
+int osdp_read_device_status(void *ws, int *status, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OSDP_H_ */

@@ -1,0 +1,203 @@
+"""ctypes binding with the same names as the C ABI in include/osdp.h (argument marshalling only).
+
+Tensor arguments may be torch CUDA tensors (their data pointer is passed) or integers
+(raw device addresses) or None.  ``stream`` may be a torch.cuda.Stream, an integer handle or
+None (torch's current stream).  Functions return the library's status code; ``check=True``
+raises OsdpError on a non-zero status instead.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+SPLIT_OUT, SPLIT_RED = 0, 1
+ACT_NONE, ACT_GELU_TANH, ACT_GELU_ERF = 0, 1, 2
+DTYPE_BF16, DTYPE_FP32 = 0, 1
+OP_LINEAR_FWD, OP_LINEAR_BWD, OP_MLP_FWD, OP_MLP_BWD = 0, 1, 2, 3
+
+EXPORTS = [
+    "osdp_version", "osdp_status_string", "osdp_last_cuda_error", "osdp_slice_range",
+    "osdp_split_linear_workspace_bytes", "osdp_split_linear_fwd", "osdp_split_linear_fwd_slice",
+    "osdp_split_linear_bwd", "osdp_split_linear_bwd_slice", "osdp_split_mlp_fwd", "osdp_split_mlp_bwd",
+    "osdp_read_device_status",
+]
+
+_lib = None
+
+
+class OsdpError(RuntimeError):
+    def __init__(self, status, where=""):
+        self.status = status
+        msg = osdp_status_string(status)
+        if status == 7:
+            msg += " (cuda error %d)" % osdp_last_cuda_error()
+        super().__init__("%s: %s" % (where, msg) if where else msg)
+
+
+def lib_path() -> str:
+    return os.path.join(HERE, "libosdp.so")
+
+
+def lib():
+    """Loads libosdp.so (built in-tree by paper_2209_13258_b200/build.py).  No fallback."""
+    global _lib
+    if _lib is None:
+        path = lib_path()
+        if not os.path.exists(path):
+            raise OSError("%s is missing: run `python -m paper_2209_13258_b200.build` (needs nvcc); "
+                          "there is no CPU fallback" % path)
+        L = ctypes.CDLL(path)
+        vp, i64, ci, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
+        L.osdp_version.restype = ci
+        L.osdp_status_string.restype = ctypes.c_char_p
+        L.osdp_status_string.argtypes = [ci]
+        L.osdp_last_cuda_error.restype = ci
+        L.osdp_slice_range.argtypes = [i64, ci, ci, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+        L.osdp_split_linear_workspace_bytes.argtypes = [i64, i64, i64, ci, ci, ci, ci, ctypes.POINTER(sz)]
+        fwd = [vp, vp, i64, vp, i64, i64, i64, ci, ci, ci]
+        L.osdp_split_linear_fwd.argtypes = fwd + [vp, vp, vp, sz, vp]
+        L.osdp_split_linear_fwd_slice.argtypes = fwd + [ci, vp, vp, vp, sz, vp]
+        bwd = [vp, vp, vp, i64, vp, i64, i64, i64, ci, ci, ci]
+        L.osdp_split_linear_bwd.argtypes = bwd + [vp, vp, i64, ci, ci, vp, vp, sz, vp]
+        L.osdp_split_linear_bwd_slice.argtypes = bwd + [ci, vp, vp, i64, ci, ci, vp, vp, sz, vp]
+        L.osdp_split_mlp_fwd.argtypes = [vp, vp, i64, vp, i64, vp, i64, i64, i64, ci, ci, vp, vp, vp, sz, vp]
+        L.osdp_split_mlp_bwd.argtypes = [vp, vp, vp, i64, i64, vp, i64, i64, i64, ci, ci, vp, vp, i64, i64, ci, ci,
+                                         vp, vp, vp, sz, vp]
+        L.osdp_read_device_status.argtypes = [vp, ctypes.POINTER(ci), vp]
+        for name in EXPORTS:
+            getattr(L, name)
+            if name not in ("osdp_status_string",):
+                getattr(L, name).restype = ci
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return ctypes.c_void_p(t)
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(s):
+    if s is None:
+        import torch
+        return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    if isinstance(s, int):
+        return ctypes.c_void_p(s)
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _ws(ws):
+    if ws is None:
+        return None, 0
+    if isinstance(ws, tuple):
+        return ctypes.c_void_p(ws[0]), int(ws[1])
+    return ctypes.c_void_p(ws.data_ptr()), ws.numel() * ws.element_size()
+
+
+def _ret(rc, check, where):
+    if check and rc != 0:
+        raise OsdpError(rc, where)
+    return rc
+
+
+def osdp_version() -> int:
+    return lib().osdp_version()
+
+
+def osdp_status_string(status: int) -> str:
+    return lib().osdp_status_string(int(status)).decode()
+
+
+def osdp_last_cuda_error() -> int:
+    return lib().osdp_last_cuda_error()
+
+
+def osdp_slice_range(D, k_split, slice_idx):
+    """Returns (status, begin, end)."""
+    b, e = ctypes.c_int64(), ctypes.c_int64()
+    rc = lib().osdp_slice_range(int(D), int(k_split), int(slice_idx), ctypes.byref(b), ctypes.byref(e))
+    return rc, b.value, e.value
+
+
+def osdp_split_linear_workspace_bytes(M, N, K, k_split, split_dim, act, op):
+    """Returns (status, bytes)."""
+    n = ctypes.c_size_t()
+    rc = lib().osdp_split_linear_workspace_bytes(int(M), int(N), int(K), int(k_split), int(split_dim), int(act),
+                                                 int(op), ctypes.byref(n))
+    return rc, n.value
+
+
+def new_workspace(nbytes: int, device="cuda"):
+    """A zeroed torch byte tensor usable as `ws` (torch allocations are 512-byte aligned)."""
+    import torch
+    return torch.zeros(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def osdp_split_linear_fwd(x, w_flat, w_offset, bias, M, N, K, k_split, split_dim, act, out, z_save, ws,
+                          stream=None, check=False):
+    wp, wn = _ws(ws)
+    rc = lib().osdp_split_linear_fwd(_ptr(x), _ptr(w_flat), int(w_offset), _ptr(bias), int(M), int(N), int(K),
+                                     int(k_split), int(split_dim), int(act), _ptr(out), _ptr(z_save), wp, wn,
+                                     _stream(stream))
+    return _ret(rc, check, "osdp_split_linear_fwd")
+
+
+def osdp_split_linear_fwd_slice(x, w_flat, w_offset, bias, M, N, K, k_split, split_dim, act, slice_idx, out,
+                                z_save, ws, stream=None, check=False):
+    wp, wn = _ws(ws)
+    rc = lib().osdp_split_linear_fwd_slice(_ptr(x), _ptr(w_flat), int(w_offset), _ptr(bias), int(M), int(N), int(K),
+                                           int(k_split), int(split_dim), int(act), int(slice_idx), _ptr(out),
+                                           _ptr(z_save), wp, wn, _stream(stream))
+    return _ret(rc, check, "osdp_split_linear_fwd_slice")
+
+
+def osdp_split_linear_bwd(dy, x, w_flat, w_offset, z_saved, M, N, K, k_split, split_dim, act, dx, dw_flat,
+                          dw_offset, dw_dtype, accumulate, dbias, ws, stream=None, check=False):
+    wp, wn = _ws(ws)
+    rc = lib().osdp_split_linear_bwd(_ptr(dy), _ptr(x), _ptr(w_flat), int(w_offset), _ptr(z_saved), int(M), int(N),
+                                     int(K), int(k_split), int(split_dim), int(act), _ptr(dx), _ptr(dw_flat),
+                                     int(dw_offset), int(dw_dtype), int(accumulate), _ptr(dbias), wp, wn,
+                                     _stream(stream))
+    return _ret(rc, check, "osdp_split_linear_bwd")
+
+
+def osdp_split_linear_bwd_slice(dy, x, w_flat, w_offset, z_saved, M, N, K, k_split, split_dim, act, slice_idx, dx,
+                                dw_flat, dw_offset, dw_dtype, accumulate, dbias, ws, stream=None, check=False):
+    wp, wn = _ws(ws)
+    rc = lib().osdp_split_linear_bwd_slice(_ptr(dy), _ptr(x), _ptr(w_flat), int(w_offset), _ptr(z_saved), int(M),
+                                           int(N), int(K), int(k_split), int(split_dim), int(act), int(slice_idx),
+                                           _ptr(dx), _ptr(dw_flat), int(dw_offset), int(dw_dtype), int(accumulate),
+                                           _ptr(dbias), wp, wn, _stream(stream))
+    return _ret(rc, check, "osdp_split_linear_bwd_slice")
+
+
+def osdp_split_mlp_fwd(x, w_flat, off_w1, b1, off_w2, b2, M, hidden, ffn, k_split, act, out, z1_save, ws,
+                       stream=None, check=False):
+    wp, wn = _ws(ws)
+    rc = lib().osdp_split_mlp_fwd(_ptr(x), _ptr(w_flat), int(off_w1), _ptr(b1), int(off_w2), _ptr(b2), int(M),
+                                  int(hidden), int(ffn), int(k_split), int(act), _ptr(out), _ptr(z1_save), wp, wn,
+                                  _stream(stream))
+    return _ret(rc, check, "osdp_split_mlp_fwd")
+
+
+def osdp_split_mlp_bwd(dy, x, w_flat, off_w1, off_w2, z1_saved, M, hidden, ffn, k_split, act, dx, dw_flat,
+                       dw_off_w1, dw_off_w2, dw_dtype, accumulate, db1, db2, ws, stream=None, check=False):
+    wp, wn = _ws(ws)
+    rc = lib().osdp_split_mlp_bwd(_ptr(dy), _ptr(x), _ptr(w_flat), int(off_w1), int(off_w2), _ptr(z1_saved), int(M),
+                                  int(hidden), int(ffn), int(k_split), int(act), _ptr(dx), _ptr(dw_flat),
+                                  int(dw_off_w1), int(dw_off_w2), int(dw_dtype), int(accumulate), _ptr(db1),
+                                  _ptr(db2), wp, wn, _stream(stream))
+    return _ret(rc, check, "osdp_split_mlp_bwd")
+
+
+def osdp_read_device_status(ws, stream=None):
+    """Returns (status of the call, device status)."""
+    wp, _ = _ws(ws)
+    st = ctypes.c_int(0)
+    rc = lib().osdp_read_device_status(wp, ctypes.byref(st), _stream(stream))
+    return rc, st.value

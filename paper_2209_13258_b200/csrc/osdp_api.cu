@@ -1,0 +1,776 @@
+// Host side of the C ABI declared in include/osdp.h: argument checks, the slice table, the
+// workspace plan, TMA descriptor encoding and kernel launches.  No allocation, no stream
+// synchronisation (except osdp_read_device_status), no CPU fallback: if the CUDA path cannot
+// run, the call returns an error.
+#include "../../include/osdp.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <string.h>
+
+#include "osdp_aux.cuh"
+#include "osdp_gemm.cuh"
+
+using namespace osdp;
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+int cuda_fail(cudaError_t e) {
+  g_last_cuda_error = (int)e;
+  return OSDP_ERR_CUDA;
+}
+int cu_fail(CUresult r) {
+  g_last_cuda_error = 100000 + (int)r;   // driver-API codes are reported offset by 100000
+  return OSDP_ERR_CUDA;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+int get_encode_fn(EncodeTiledFn *out) {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (q != cudaDriverEntryPointSuccess || !p) return cuda_fail(cudaErrorNotSupported);
+    fn = (EncodeTiledFn)p;
+  }
+  *out = fn;
+  return OSDP_OK;
+}
+
+struct DeviceInfo {
+  int sms;
+  bool attrs_set;
+};
+DeviceInfo g_dev[64];
+
+int device_sms(int *sms) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= 64) return cuda_fail(cudaErrorInvalidDevice);
+  if (g_dev[dev].sms == 0) {
+    int n = 0;
+    e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    g_dev[dev].sms = n;
+  }
+  *sms = g_dev[dev].sms;
+  return OSDP_OK;
+}
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ------------------------------------------------------------------------------------------------
+// Slice table (Section 3.3, step 1)
+
+int slice_len(int64_t D, int k, int64_t *L) {
+  if (k < 0 || k > OSDP_MAX_SPLIT) return OSDP_ERR_BAD_SPLIT;
+  if (k == 0) k = 1;
+  if (D <= 0) return OSDP_ERR_BAD_SHAPE;
+  int64_t l = (D + k - 1) / k;
+  l = (l + 7) / 8 * 8;
+  if ((int64_t)(k - 1) * l >= D) return OSDP_ERR_BAD_SPLIT;
+  *L = l;
+  return OSDP_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Workspace plan.  Region 0 is always the 256-byte status block.
+
+struct WsPlan {
+  size_t carry_off, carry_bytes;      // fp32 running sum of the summed output
+  size_t stage0_off, stage0_bytes;    // bf16 slice staging (G_s, A_s)
+  size_t stage1_off, stage1_bytes;    // second bf16 slice staging (dZ_s)
+  size_t part_off, part_bytes;        // column-sum partials
+  size_t total;
+};
+
+int plan_workspace(int64_t M, int64_t N, int64_t K, int k, int split_dim, int act, int op, WsPlan *w) {
+  memset(w, 0, sizeof(*w));
+  if (M <= 0 || N <= 0 || K <= 0) return OSDP_ERR_BAD_SHAPE;
+  if (k == 0) k = 1;
+  size_t off = 256;
+  auto take = [&](size_t bytes, size_t *o, size_t *b) {
+    *o = off;
+    *b = bytes;
+    off = align_up(off + bytes, 256);
+  };
+  const size_t chunks = (size_t)((M + COLSUM_ROWS_PER_CHUNK - 1) / COLSUM_ROWS_PER_CHUNK);
+  int64_t L = 0;
+  int rc;
+  switch (op) {
+    case OSDP_OP_LINEAR_FWD:
+      if (split_dim != OSDP_SPLIT_OUT && split_dim != OSDP_SPLIT_RED) return OSDP_ERR_BAD_SPLIT;
+      rc = slice_len(split_dim == OSDP_SPLIT_OUT ? N : K, k, &L);
+      if (rc) return rc;
+      if (split_dim == OSDP_SPLIT_RED && k > 1) take((size_t)M * N * 4, &w->carry_off, &w->carry_bytes);
+      break;
+    case OSDP_OP_LINEAR_BWD:
+      if (split_dim != OSDP_SPLIT_OUT && split_dim != OSDP_SPLIT_RED) return OSDP_ERR_BAD_SPLIT;
+      rc = slice_len(split_dim == OSDP_SPLIT_OUT ? N : K, k, &L);
+      if (rc) return rc;
+      if (split_dim == OSDP_SPLIT_OUT && k > 1) take((size_t)M * K * 4, &w->carry_off, &w->carry_bytes);
+      if (act != OSDP_ACT_NONE)
+        take((size_t)M * (split_dim == OSDP_SPLIT_OUT ? L : N) * 2, &w->stage0_off, &w->stage0_bytes);
+      take(chunks * (size_t)N * 4, &w->part_off, &w->part_bytes);
+      break;
+    case OSDP_OP_MLP_FWD:   // N = ffn, K = hidden
+      rc = slice_len(N, k, &L);
+      if (rc) return rc;
+      if (k > 1) take((size_t)M * K * 4, &w->carry_off, &w->carry_bytes);
+      take((size_t)M * L * 2, &w->stage0_off, &w->stage0_bytes);
+      break;
+    case OSDP_OP_MLP_BWD:
+      rc = slice_len(N, k, &L);
+      if (rc) return rc;
+      if (k > 1) take((size_t)M * K * 4, &w->carry_off, &w->carry_bytes);
+      take((size_t)M * L * 2, &w->stage0_off, &w->stage0_bytes);
+      take((size_t)M * L * 2, &w->stage1_off, &w->stage1_bytes);
+      take(chunks * (size_t)(L > K ? L : K) * 4, &w->part_off, &w->part_bytes);
+      break;
+    default:
+      return OSDP_ERR_UNSUPPORTED;
+  }
+  w->total = off;
+  return OSDP_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// GEMM launch
+
+// A row-major bf16 matrix view used as a GEMM operand.  `inner` is the contiguous extent.
+// K-major: inner is the reduction dimension; MN-major: inner is the output dimension.
+struct Operand {
+  const void *base;
+  int64_t inner, outer, ld;
+  bool mn_major;
+  bool whole;   // true: the view is the whole operator and the launch's slices cut it;
+                // false: the view is already one slice (or is not cut at all)
+};
+
+struct GemmCall {
+  Operand a, b;
+  int64_t P, Q, R;
+  int mode;
+  int64_t L;
+  int k_total, s_begin, s_end;
+  int64_t bn_P, bn_Q;   // extents that choose the tile width (the unsplit operator's, so k never changes it)
+  Epilogue epi;
+  int *status;
+};
+
+int encode3d(CUtensorMap *m, const void *base, const cuuint64_t dims[3], const cuuint64_t strides_bytes[2],
+             const cuuint32_t box[3]) {
+  EncodeTiledFn fn;
+  int rc = get_encode_fn(&fn);
+  if (rc) return rc;
+  const cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides_bytes, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return cu_fail(r);
+  return OSDP_OK;
+}
+
+// Builds the two 3-D maps of one operand.  The slice index is a tensor coordinate: for slices
+// 0..k-2 the map has a dimension of extent k-1 and stride L (in the cut dimension's units); the
+// last slice, which may be shorter, gets a map of its own so that out-of-range elements are
+// zero-filled instead of running into the neighbouring slice.
+int make_operand_maps(const Operand &op, bool is_a, int mode, int64_t L, int k, int tile_rows, CUtensorMap *main_map,
+                      CUtensorMap *tail_map, int *sc_mul) {
+  const bool mid = op.mn_major ? (mode == (is_a ? MODE_ROWS : MODE_COLS)) : (mode == MODE_RED);
+  const bool role_sliced = is_a ? (mode == MODE_ROWS || mode == MODE_RED) : (mode == MODE_COLS || mode == MODE_RED);
+  const bool cut = role_sliced && op.whole && k > 1;
+  *sc_mul = cut ? 1 : 0;
+  const cuuint32_t box_outer = op.mn_major ? (cuuint32_t)BK : (cuuint32_t)tile_rows;
+  const char *base = static_cast<const char *>(op.base);
+  const cuuint64_t ldb = (cuuint64_t)op.ld * 2;
+  int rc;
+  if (!cut) {
+    if (mid) {
+      const cuuint64_t dims[3] = {(cuuint64_t)op.inner, 1, (cuuint64_t)op.outer};
+      const cuuint64_t str[2] = {(cuuint64_t)op.inner * 2, ldb};
+      const cuuint32_t box[3] = {64, 1, box_outer};
+      rc = encode3d(tail_map, base, dims, str, box);
+    } else {
+      const cuuint64_t dims[3] = {(cuuint64_t)op.inner, (cuuint64_t)op.outer, 1};
+      const cuuint64_t str[2] = {ldb, ldb * (cuuint64_t)op.outer};
+      const cuuint32_t box[3] = {64, box_outer, 1};
+      rc = encode3d(tail_map, base, dims, str, box);
+    }
+    if (rc) return rc;
+    *main_map = *tail_map;
+    return OSDP_OK;
+  }
+  if (mid) {   // the slices cut the contiguous dimension
+    const cuuint64_t str[2] = {(cuuint64_t)L * 2, ldb};
+    const cuuint32_t box[3] = {64, 1, box_outer};
+    const cuuint64_t dims_main[3] = {(cuuint64_t)L, (cuuint64_t)(k - 1), (cuuint64_t)op.outer};
+    rc = encode3d(main_map, base, dims_main, str, box);
+    if (rc) return rc;
+    const cuuint64_t dims_tail[3] = {(cuuint64_t)(op.inner - (int64_t)(k - 1) * L), 1, (cuuint64_t)op.outer};
+    return encode3d(tail_map, base + (int64_t)(k - 1) * L * 2, dims_tail, str, box);
+  }
+  // the slices cut the strided dimension
+  const cuuint64_t str[2] = {ldb, ldb * (cuuint64_t)L};
+  const cuuint32_t box[3] = {64, box_outer, 1};
+  const cuuint64_t dims_main[3] = {(cuuint64_t)op.inner, (cuuint64_t)L, (cuuint64_t)(k - 1)};
+  rc = encode3d(main_map, base, dims_main, str, box);
+  if (rc) return rc;
+  const cuuint64_t dims_tail[3] = {(cuuint64_t)op.inner, (cuuint64_t)(op.outer - (int64_t)(k - 1) * L), 1};
+  return encode3d(tail_map, base + (int64_t)(k - 1) * L * (int64_t)ldb, dims_tail, str, box);
+}
+
+template <int BN, bool A_MN, bool B_MN>
+int launch_variant(const GemmParams &p, int grid, cudaStream_t stream) {
+  static bool attr_done[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (!attr_done[dev & 63]) {
+    e = cudaFuncSetAttribute(gemm_kernel<BN, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             SmemLayout<BN>::TOTAL);
+    if (e != cudaSuccess) return cuda_fail(e);
+    attr_done[dev & 63] = true;
+  }
+  gemm_kernel<BN, A_MN, B_MN><<<grid, NUM_THREADS, SmemLayout<BN>::TOTAL, stream>>>(p);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  return OSDP_OK;
+}
+
+template <int BN>
+int launch_bn(const GemmParams &p, bool a_mn, bool b_mn, int grid, cudaStream_t stream) {
+  if (!a_mn && !b_mn) return launch_variant<BN, false, false>(p, grid, stream);
+  if (!a_mn && b_mn) return launch_variant<BN, false, true>(p, grid, stream);
+  if (a_mn && b_mn) return launch_variant<BN, true, true>(p, grid, stream);
+  return OSDP_ERR_UNSUPPORTED;
+}
+
+inline int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+int launch_gemm(const GemmCall &c, cudaStream_t stream) {
+  int sms = 0;
+  int rc = device_sms(&sms);
+  if (rc) return rc;
+  // Tile width from the unsplit operator's shape: the same for every k, so that concatenated
+  // outputs are computed by exactly the same instruction sequence whatever the split.
+  int bn = 64;
+  const int64_t want = (int64_t)sms * 4 / 5;
+  if (cdiv(c.bn_P, BM) * cdiv(c.bn_Q, 256) >= want) bn = 256;
+  else if (cdiv(c.bn_P, BM) * cdiv(c.bn_Q, 128) >= want) bn = 128;
+
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  rc = make_operand_maps(c.a, true, c.mode, c.L, c.k_total, BM, &p.a_main, &p.a_tail, &p.a_sc_mul);
+  if (rc) return rc;
+  rc = make_operand_maps(c.b, false, c.mode, c.L, c.k_total, bn, &p.b_main, &p.b_tail, &p.b_sc_mul);
+  if (rc) return rc;
+  p.P = (int)c.P; p.Q = (int)c.Q; p.R = (int)c.R;
+  p.mode = c.mode; p.L = (int)c.L; p.k_total = c.k_total; p.s_begin = c.s_begin; p.s_end = c.s_end;
+  p.epi = c.epi;
+  p.status = c.status;
+
+  // Work items of this launch -> grid size (one CTA per SM at most).
+  int64_t items;
+  if (c.mode == MODE_RED) {
+    items = cdiv(c.P, BM) * cdiv(c.Q, bn);
+  } else {
+    const int64_t rows_full = (c.mode == MODE_ROWS) ? c.L : c.P;
+    const int64_t cols_full = (c.mode == MODE_COLS) ? c.L : c.Q;
+    const int nsl = c.s_end - c.s_begin;
+    const int last = c.s_end - 1;
+    const int64_t rows_last = (c.mode == MODE_ROWS) ? ((c.P - last * c.L) < c.L ? (c.P - last * c.L) : c.L) : c.P;
+    const int64_t cols_last = (c.mode == MODE_COLS) ? ((c.Q - last * c.L) < c.L ? (c.Q - last * c.L) : c.L) : c.Q;
+    items = (int64_t)(nsl - 1) * cdiv(rows_full, BM) * cdiv(cols_full, bn) + cdiv(rows_last, BM) * cdiv(cols_last, bn);
+  }
+  const int grid = (int)(items < sms ? items : sms);
+  if (grid <= 0) return OSDP_OK;
+  switch (bn) {
+    case 256: return launch_bn<256>(p, c.a.mn_major, c.b.mn_major, grid, stream);
+    case 128: return launch_bn<128>(p, c.a.mn_major, c.b.mn_major, grid, stream);
+    default: return launch_bn<64>(p, c.a.mn_major, c.b.mn_major, grid, stream);
+  }
+}
+
+Epilogue plain_epilogue(void *out, int64_t ld, int fp32) {
+  Epilogue e;
+  memset(&e, 0, sizeof(e));
+  e.out = out;
+  e.ld_out = ld;
+  e.out_fp32 = fp32;
+  return e;
+}
+
+int launch_colsum(const void *g, int64_t ld, int64_t M, int c0, int ncols, float *partial, float *out,
+                  cudaStream_t stream) {
+  const int chunks = (int)cdiv(M, COLSUM_ROWS_PER_CHUNK);
+  dim3 grid((unsigned)cdiv(ncols, 64), (unsigned)chunks);
+  colsum_partial_kernel<<<grid, 256, 0, stream>>>((const __nv_bfloat16 *)g, ld, M, c0, ncols, partial, ncols);
+  colsum_final_kernel<<<(unsigned)cdiv(ncols, 256), 256, 0, stream>>>(partial, ncols, chunks, ncols, out + c0);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  return OSDP_OK;
+}
+
+int launch_act_backward(const void *dy, int64_t ld_dy, const void *z, int64_t ld_z, void *g, int64_t ld_g, int64_t M,
+                        int c0, int ncols, int act, cudaStream_t stream) {
+  int sms = 0;
+  int rc = device_sms(&sms);
+  if (rc) return rc;
+  const int64_t total = M * (ncols / 8);
+  int64_t blocks = cdiv(total, 256);
+  if (blocks > (int64_t)sms * 16) blocks = (int64_t)sms * 16;
+  act_backward_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const __nv_bfloat16 *)dy, ld_dy, (const __nv_bfloat16 *)z,
+                                                           ld_z, (__nv_bfloat16 *)g, ld_g, M, c0, ncols, act);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  return OSDP_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Argument checks shared by the linear entry points
+
+int check_common(int64_t M, int64_t N, int64_t K, int k, int split_dim, int act, int64_t *L) {
+  if (M <= 0 || N <= 0 || K <= 0) return OSDP_ERR_BAD_SHAPE;
+  const int64_t lim = (int64_t)1 << 30;
+  if (M > lim || N > lim || K > lim) return OSDP_ERR_BAD_SHAPE;
+  if ((N & 7) || (K & 7)) return OSDP_ERR_ALIGNMENT;
+  if (split_dim != OSDP_SPLIT_OUT && split_dim != OSDP_SPLIT_RED) return OSDP_ERR_BAD_SPLIT;
+  if (act != OSDP_ACT_NONE && act != OSDP_ACT_GELU_TANH && act != OSDP_ACT_GELU_ERF) return OSDP_ERR_UNSUPPORTED;
+  return slice_len(split_dim == OSDP_SPLIT_OUT ? N : K, k, L);
+}
+
+int check_ws(const void *ws, size_t ws_bytes, const WsPlan &plan) {
+  if (!ws) return OSDP_ERR_NULL_POINTER;
+  if (reinterpret_cast<uintptr_t>(ws) & 255u) return OSDP_ERR_ALIGNMENT;
+  if (ws_bytes < plan.total) return OSDP_ERR_WORKSPACE_TOO_SMALL;
+  return OSDP_OK;
+}
+
+int fwd_impl(const void *x, const void *w_flat, int64_t w_offset, const float *bias, int64_t M, int64_t N, int64_t K,
+             int k, int split_dim, int act, int s_begin, int s_end, bool single, void *out, void *z_save, void *ws,
+             size_t ws_bytes, void *stream) {
+  if (!x || !w_flat || !out) return OSDP_ERR_NULL_POINTER;
+  int64_t L = 0;
+  int rc = check_common(M, N, K, k, split_dim, act, &L);
+  if (rc) return rc;
+  if (k == 0) k = 1;
+  if (single) {
+    if (s_begin < 0 || s_begin >= k) return OSDP_ERR_BAD_SPLIT;
+    s_end = s_begin + 1;
+  } else {
+    s_begin = 0;
+    s_end = k;
+  }
+  if (w_offset < 0 || (w_offset & 7)) return OSDP_ERR_ALIGNMENT;
+  if (!aligned16(x) || !aligned16(w_flat) || !aligned16(out) || !aligned16(z_save) || !aligned16(bias))
+    return OSDP_ERR_ALIGNMENT;
+  WsPlan plan;
+  rc = plan_workspace(M, N, K, k, split_dim, act, OSDP_OP_LINEAR_FWD, &plan);
+  if (rc) return rc;
+  rc = check_ws(ws, ws_bytes, plan);
+  if (rc) return rc;
+
+  const __nv_bfloat16 *w = static_cast<const __nv_bfloat16 *>(w_flat) + w_offset;
+  GemmCall c;
+  memset(&c, 0, sizeof(c));
+  c.a = Operand{x, K, M, K, false, true};
+  c.b = Operand{w, K, N, K, false, true};
+  c.P = M; c.Q = N; c.R = K;
+  c.bn_P = M; c.bn_Q = N;
+  c.mode = (k == 1) ? MODE_NONE : (split_dim == OSDP_SPLIT_OUT ? MODE_COLS : MODE_RED);
+  c.L = L; c.k_total = k; c.s_begin = s_begin; c.s_end = s_end;
+  c.epi = plain_epilogue(out, N, 0);
+  c.epi.bias = bias;
+  c.epi.z_save = static_cast<__nv_bfloat16 *>(z_save);
+  c.epi.ld_z = N;
+  c.epi.act = act;
+  c.epi.carry = reinterpret_cast<float *>(static_cast<char *>(ws) + plan.carry_off);
+  c.epi.ld_carry = N;
+  c.status = static_cast<int *>(ws);
+  return launch_gemm(c, static_cast<cudaStream_t>(stream));
+}
+
+int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset, const void *z_saved, int64_t M,
+             int64_t N, int64_t K, int k, int split_dim, int act, int s_begin, int s_end, bool single, void *dx,
+             void *dw_flat, int64_t dw_offset, int dw_dtype, int accumulate, float *dbias, void *ws, size_t ws_bytes,
+             void *stream_) {
+  if (!dy || !x || !w_flat) return OSDP_ERR_NULL_POINTER;
+  int64_t L = 0;
+  int rc = check_common(M, N, K, k, split_dim, act, &L);
+  if (rc) return rc;
+  if (k == 0) k = 1;
+  if (single) {
+    if (s_begin < 0 || s_begin >= k) return OSDP_ERR_BAD_SPLIT;
+    s_end = s_begin + 1;
+  } else {
+    s_begin = 0;
+    s_end = k;
+  }
+  if (act != OSDP_ACT_NONE && !z_saved) return OSDP_ERR_NULL_POINTER;
+  if (dw_dtype != OSDP_DTYPE_BF16 && dw_dtype != OSDP_DTYPE_FP32) return OSDP_ERR_UNSUPPORTED;
+  if (w_offset < 0 || (w_offset & 7) || dw_offset < 0 || (dw_offset & 7)) return OSDP_ERR_ALIGNMENT;
+  if (!aligned16(dy) || !aligned16(x) || !aligned16(w_flat) || !aligned16(z_saved) || !aligned16(dx) ||
+      !aligned16(dw_flat) || !aligned16(dbias))
+    return OSDP_ERR_ALIGNMENT;
+  WsPlan plan;
+  rc = plan_workspace(M, N, K, k, split_dim, act, OSDP_OP_LINEAR_BWD, &plan);
+  if (rc) return rc;
+  rc = check_ws(ws, ws_bytes, plan);
+  if (rc) return rc;
+
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  char *wsb = static_cast<char *>(ws);
+  const __nv_bfloat16 *w = static_cast<const __nv_bfloat16 *>(w_flat) + w_offset;
+  float *partial = reinterpret_cast<float *>(wsb + plan.part_off);
+  float *carry = reinterpret_cast<float *>(wsb + plan.carry_off);
+  __nv_bfloat16 *stage = reinterpret_cast<__nv_bfloat16 *>(wsb + plan.stage0_off);
+  int *status = static_cast<int *>(ws);
+  void *dw = nullptr;
+  if (dw_flat)
+    dw = (dw_dtype == OSDP_DTYPE_FP32) ? (void *)(static_cast<float *>(dw_flat) + dw_offset)
+                                       : (void *)(static_cast<__nv_bfloat16 *>(dw_flat) + dw_offset);
+  const bool out_split = (split_dim == OSDP_SPLIT_OUT);
+  const int mode_sum = (k == 1) ? MODE_NONE : MODE_RED;
+
+  auto dx_call = [&](const Operand &g, int sb, int se) {
+    GemmCall c;
+    memset(&c, 0, sizeof(c));
+    c.a = g;                                        // G [M,N], reduction N contiguous
+    c.b = Operand{w, K, N, K, true, true};          // W [N,K]: output dim K contiguous
+    c.P = M; c.Q = K; c.R = N; c.bn_P = M; c.bn_Q = K;
+    c.mode = (k == 1) ? MODE_NONE : (out_split ? MODE_RED : MODE_COLS);
+    c.L = L; c.k_total = k; c.s_begin = sb; c.s_end = se;
+    c.epi = plain_epilogue(dx, K, 0);
+    c.epi.carry = carry;
+    c.epi.ld_carry = K;
+    c.status = status;
+    return launch_gemm(c, stream);
+  };
+  auto dw_call = [&](const Operand &gt, int sb, int se) {
+    GemmCall c;
+    memset(&c, 0, sizeof(c));
+    c.a = gt;                                       // G^T: output dim N contiguous in G
+    c.b = Operand{x, K, M, K, true, true};          // X [M,K]: output dim K contiguous
+    c.P = N; c.Q = K; c.R = M; c.bn_P = N; c.bn_Q = K;
+    c.mode = (k == 1) ? MODE_NONE : (out_split ? MODE_ROWS : MODE_COLS);
+    c.L = L; c.k_total = k; c.s_begin = sb; c.s_end = se;
+    c.epi = plain_epilogue(dw, K, dw_dtype == OSDP_DTYPE_FP32);
+    c.epi.accumulate = accumulate;
+    c.status = status;
+    return launch_gemm(c, stream);
+  };
+  (void)mode_sum;
+
+  if (act == OSDP_ACT_NONE) {
+    if (dx) { rc = dx_call(Operand{dy, N, M, N, false, true}, s_begin, s_end); if (rc) return rc; }
+    if (dw) { rc = dw_call(Operand{dy, N, M, N, true, true}, s_begin, s_end); if (rc) return rc; }
+    if (dbias) {
+      if (out_split) {
+        const int64_t c0 = (int64_t)s_begin * L;
+        const int64_t c1 = ((int64_t)s_end * L < N) ? (int64_t)s_end * L : N;
+        rc = launch_colsum(dy, N, M, (int)c0, (int)(c1 - c0), partial, dbias, stream);
+      } else if (s_begin == 0) {
+        rc = launch_colsum(dy, N, M, 0, (int)N, partial, dbias, stream);
+      }
+      if (rc) return rc;
+    }
+    return OSDP_OK;
+  }
+
+  if (out_split) {
+    // Slice by slice: G_s = dY[:,R_s] (.) act'(Z[:,R_s]) into slice-sized staging, then the slice's GEMMs.
+    for (int s = s_begin; s < s_end; ++s) {
+      const int64_t c0 = (int64_t)s * L;
+      const int64_t ls = (c0 + L < N ? c0 + L : N) - c0;
+      rc = launch_act_backward(dy, N, z_saved, N, stage, L, M, (int)c0, (int)ls, act, stream);
+      if (rc) return rc;
+      if (dx) { rc = dx_call(Operand{stage, ls, M, L, false, false}, s, s + 1); if (rc) return rc; }
+      if (dw) { rc = dw_call(Operand{stage, ls, M, L, true, false}, s, s + 1); if (rc) return rc; }
+      if (dbias) { rc = launch_colsum(stage, L, M, 0, (int)ls, partial, dbias + c0, stream); if (rc) return rc; }
+    }
+    return OSDP_OK;
+  }
+  // RED split: G is needed whole by every slice.
+  if (s_begin == 0) {
+    rc = launch_act_backward(dy, N, z_saved, N, stage, N, M, 0, (int)N, act, stream);
+    if (rc) return rc;
+    if (dbias) { rc = launch_colsum(stage, N, M, 0, (int)N, partial, dbias, stream); if (rc) return rc; }
+  }
+  if (dx) { rc = dx_call(Operand{stage, N, M, N, false, true}, s_begin, s_end); if (rc) return rc; }
+  if (dw) { rc = dw_call(Operand{stage, N, M, N, true, true}, s_begin, s_end); if (rc) return rc; }
+  return OSDP_OK;
+}
+
+}  // namespace
+
+// ================================================================================================
+// C ABI
+
+extern "C" {
+
+int osdp_version(void) { return OSDP_VERSION; }
+
+const char *osdp_status_string(int status) {
+  switch (status) {
+    case OSDP_OK: return "ok";
+    case OSDP_ERR_NULL_POINTER: return "null pointer";
+    case OSDP_ERR_BAD_SHAPE: return "bad shape";
+    case OSDP_ERR_BAD_SPLIT: return "bad split";
+    case OSDP_ERR_ALIGNMENT: return "alignment";
+    case OSDP_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case OSDP_ERR_UNSUPPORTED: return "unsupported";
+    case OSDP_ERR_CUDA: return "CUDA error";
+    case OSDP_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+int osdp_last_cuda_error(void) { return g_last_cuda_error; }
+
+int osdp_slice_range(int64_t D, int k_split, int slice_idx, int64_t *begin, int64_t *end) {
+  if (!begin || !end) return OSDP_ERR_NULL_POINTER;
+  int64_t L = 0;
+  int rc = slice_len(D, k_split, &L);
+  if (rc) return rc;
+  const int k = k_split == 0 ? 1 : k_split;
+  if (slice_idx < 0 || slice_idx >= k) return OSDP_ERR_BAD_SPLIT;
+  *begin = (int64_t)slice_idx * L;
+  *end = (*begin + L < D) ? *begin + L : D;
+  return OSDP_OK;
+}
+
+int osdp_split_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int k_split, int split_dim, int act, int op,
+                                      size_t *bytes) {
+  if (!bytes) return OSDP_ERR_NULL_POINTER;
+  if (act != OSDP_ACT_NONE && act != OSDP_ACT_GELU_TANH && act != OSDP_ACT_GELU_ERF) return OSDP_ERR_UNSUPPORTED;
+  WsPlan plan;
+  int rc = plan_workspace(M, N, K, k_split, split_dim, act, op, &plan);
+  if (rc) return rc;
+  *bytes = plan.total;
+  return OSDP_OK;
+}
+
+int osdp_split_linear_fwd(const void *x, const void *w_flat, int64_t w_offset, const float *bias, int64_t M,
+                          int64_t N, int64_t K, int k_split, int split_dim, int act, void *out, void *z_save,
+                          void *ws, size_t ws_bytes, void *stream) {
+  return fwd_impl(x, w_flat, w_offset, bias, M, N, K, k_split, split_dim, act, 0, 0, false, out, z_save, ws, ws_bytes,
+                  stream);
+}
+
+int osdp_split_linear_fwd_slice(const void *x, const void *w_flat, int64_t w_offset, const float *bias, int64_t M,
+                                int64_t N, int64_t K, int k_split, int split_dim, int act, int slice_idx, void *out,
+                                void *z_save, void *ws, size_t ws_bytes, void *stream) {
+  return fwd_impl(x, w_flat, w_offset, bias, M, N, K, k_split, split_dim, act, slice_idx, 0, true, out, z_save, ws,
+                  ws_bytes, stream);
+}
+
+int osdp_split_linear_bwd(const void *dy, const void *x, const void *w_flat, int64_t w_offset, const void *z_saved,
+                          int64_t M, int64_t N, int64_t K, int k_split, int split_dim, int act, void *dx,
+                          void *dw_flat, int64_t dw_offset, int dw_dtype, int accumulate, float *dbias, void *ws,
+                          size_t ws_bytes, void *stream) {
+  return bwd_impl(dy, x, w_flat, w_offset, z_saved, M, N, K, k_split, split_dim, act, 0, 0, false, dx, dw_flat,
+                  dw_offset, dw_dtype, accumulate, dbias, ws, ws_bytes, stream);
+}
+
+int osdp_split_linear_bwd_slice(const void *dy, const void *x, const void *w_flat, int64_t w_offset,
+                                const void *z_saved, int64_t M, int64_t N, int64_t K, int k_split, int split_dim,
+                                int act, int slice_idx, void *dx, void *dw_flat, int64_t dw_offset, int dw_dtype,
+                                int accumulate, float *dbias, void *ws, size_t ws_bytes, void *stream) {
+  return bwd_impl(dy, x, w_flat, w_offset, z_saved, M, N, K, k_split, split_dim, act, slice_idx, 0, true, dx, dw_flat,
+                  dw_offset, dw_dtype, accumulate, dbias, ws, ws_bytes, stream);
+}
+
+int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const float *b1, int64_t off_w2,
+                       const float *b2, int64_t M, int64_t hidden, int64_t ffn, int k_split, int act, void *out,
+                       void *z1_save, void *ws, size_t ws_bytes, void *stream_) {
+  if (!x || !w_flat || !out) return OSDP_ERR_NULL_POINTER;
+  int64_t L = 0;
+  int rc = check_common(M, ffn, hidden, k_split, OSDP_SPLIT_OUT, act, &L);
+  if (rc) return rc;
+  const int k = k_split == 0 ? 1 : k_split;
+  if (off_w1 < 0 || off_w2 < 0 || (off_w1 & 7) || (off_w2 & 7)) return OSDP_ERR_ALIGNMENT;
+  if (!aligned16(x) || !aligned16(w_flat) || !aligned16(out) || !aligned16(z1_save) || !aligned16(b1) ||
+      !aligned16(b2))
+    return OSDP_ERR_ALIGNMENT;
+  WsPlan plan;
+  rc = plan_workspace(M, ffn, hidden, k, OSDP_SPLIT_OUT, act, OSDP_OP_MLP_FWD, &plan);
+  if (rc) return rc;
+  rc = check_ws(ws, ws_bytes, plan);
+  if (rc) return rc;
+
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  char *wsb = static_cast<char *>(ws);
+  const __nv_bfloat16 *w1 = static_cast<const __nv_bfloat16 *>(w_flat) + off_w1;   // [ffn, hidden]
+  const __nv_bfloat16 *w2 = static_cast<const __nv_bfloat16 *>(w_flat) + off_w2;   // [hidden, ffn]
+  __nv_bfloat16 *a_s = reinterpret_cast<__nv_bfloat16 *>(wsb + plan.stage0_off);   // A_s [M, ls], ld L
+  float *carry = reinterpret_cast<float *>(wsb + plan.carry_off);
+  int *status = static_cast<int *>(ws);
+
+  for (int s = 0; s < k; ++s) {
+    const int64_t lo = (int64_t)s * L;
+    const int64_t ls = (lo + L < ffn ? lo + L : ffn) - lo;
+    // A_s = act(X W1[F_s,:]^T + b1[F_s])
+    GemmCall c;
+    memset(&c, 0, sizeof(c));
+    c.a = Operand{x, hidden, M, hidden, false, false};
+    c.b = Operand{w1 + lo * hidden, hidden, ls, hidden, false, false};
+    c.P = M; c.Q = ls; c.R = hidden; c.bn_P = M; c.bn_Q = L;
+    c.mode = MODE_NONE; c.L = ls; c.k_total = 1; c.s_begin = 0; c.s_end = 1;
+    c.epi = plain_epilogue(a_s, L, 0);
+    c.epi.bias = b1 ? b1 + lo : nullptr;
+    c.epi.z_save = z1_save ? static_cast<__nv_bfloat16 *>(z1_save) + lo : nullptr;
+    c.epi.ld_z = ffn;
+    c.epi.act = act;
+    c.status = status;
+    rc = launch_gemm(c, stream);
+    if (rc) return rc;
+    // Y (+)= A_s W2[:,F_s]^T ; + b2 after the last slice
+    memset(&c, 0, sizeof(c));
+    c.a = Operand{a_s, ls, M, L, false, false};
+    c.b = Operand{w2, ffn, hidden, ffn, false, true};
+    c.P = M; c.Q = hidden; c.R = ffn; c.bn_P = M; c.bn_Q = hidden;
+    c.mode = (k == 1) ? MODE_NONE : MODE_RED;
+    c.L = L; c.k_total = k; c.s_begin = s; c.s_end = s + 1;
+    c.epi = plain_epilogue(out, hidden, 0);
+    c.epi.bias = b2;
+    c.epi.carry = carry;
+    c.epi.ld_carry = hidden;
+    c.status = status;
+    rc = launch_gemm(c, stream);
+    if (rc) return rc;
+  }
+  return OSDP_OK;
+}
+
+int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_t off_w1, int64_t off_w2,
+                       const void *z1_saved, int64_t M, int64_t hidden, int64_t ffn, int k_split, int act, void *dx,
+                       void *dw_flat, int64_t dw_off_w1, int64_t dw_off_w2, int dw_dtype, int accumulate, float *db1,
+                       float *db2, void *ws, size_t ws_bytes, void *stream_) {
+  if (!dy || !x || !w_flat || !z1_saved) return OSDP_ERR_NULL_POINTER;
+  int64_t L = 0;
+  int rc = check_common(M, ffn, hidden, k_split, OSDP_SPLIT_OUT, act, &L);
+  if (rc) return rc;
+  const int k = k_split == 0 ? 1 : k_split;
+  if (dw_dtype != OSDP_DTYPE_BF16 && dw_dtype != OSDP_DTYPE_FP32) return OSDP_ERR_UNSUPPORTED;
+  if (off_w1 < 0 || off_w2 < 0 || (off_w1 & 7) || (off_w2 & 7) || dw_off_w1 < 0 || dw_off_w2 < 0 ||
+      (dw_off_w1 & 7) || (dw_off_w2 & 7))
+    return OSDP_ERR_ALIGNMENT;
+  if (!aligned16(dy) || !aligned16(x) || !aligned16(w_flat) || !aligned16(z1_saved) || !aligned16(dx) ||
+      !aligned16(dw_flat) || !aligned16(db1) || !aligned16(db2))
+    return OSDP_ERR_ALIGNMENT;
+  WsPlan plan;
+  rc = plan_workspace(M, ffn, hidden, k, OSDP_SPLIT_OUT, act, OSDP_OP_MLP_BWD, &plan);
+  if (rc) return rc;
+  rc = check_ws(ws, ws_bytes, plan);
+  if (rc) return rc;
+
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  char *wsb = static_cast<char *>(ws);
+  const __nv_bfloat16 *w1 = static_cast<const __nv_bfloat16 *>(w_flat) + off_w1;
+  const __nv_bfloat16 *w2 = static_cast<const __nv_bfloat16 *>(w_flat) + off_w2;
+  const __nv_bfloat16 *z1 = static_cast<const __nv_bfloat16 *>(z1_saved);
+  __nv_bfloat16 *a_s = reinterpret_cast<__nv_bfloat16 *>(wsb + plan.stage0_off);
+  __nv_bfloat16 *dz_s = reinterpret_cast<__nv_bfloat16 *>(wsb + plan.stage1_off);
+  float *carry = reinterpret_cast<float *>(wsb + plan.carry_off);
+  float *partial = reinterpret_cast<float *>(wsb + plan.part_off);
+  int *status = static_cast<int *>(ws);
+  const int fp32 = dw_dtype == OSDP_DTYPE_FP32;
+  auto dw_ptr = [&](int64_t off) -> void * {
+    if (!dw_flat) return nullptr;
+    return fp32 ? (void *)(static_cast<float *>(dw_flat) + off) : (void *)(static_cast<__nv_bfloat16 *>(dw_flat) + off);
+  };
+
+  if (db2) { rc = launch_colsum(dy, hidden, M, 0, (int)hidden, partial, db2, stream); if (rc) return rc; }
+  for (int s = 0; s < k; ++s) {
+    const int64_t lo = (int64_t)s * L;
+    const int64_t ls = (lo + L < ffn ? lo + L : ffn) - lo;
+    GemmCall c;
+    // dZ_s = (dY W2[:,F_s]) (.) act'(Z1_s);  A_s = act(Z1_s)
+    memset(&c, 0, sizeof(c));
+    c.a = Operand{dy, hidden, M, hidden, false, false};
+    c.b = Operand{w2 + lo, ls, hidden, ffn, true, false};
+    c.P = M; c.Q = ls; c.R = hidden; c.bn_P = M; c.bn_Q = L;
+    c.mode = MODE_NONE; c.L = ls; c.k_total = 1; c.s_begin = 0; c.s_end = 1;
+    c.epi = plain_epilogue(dz_s, L, 0);
+    c.epi.gz = z1 + lo;
+    c.epi.ld_gz = ffn;
+    c.epi.gz_act = act;
+    c.epi.act_out = a_s;
+    c.epi.ld_act_out = L;
+    c.status = status;
+    rc = launch_gemm(c, stream);
+    if (rc) return rc;
+    if (dw_flat) {
+      // dW2[:,F_s] = dY^T A_s
+      memset(&c, 0, sizeof(c));
+      c.a = Operand{dy, hidden, M, hidden, true, false};
+      c.b = Operand{a_s, ls, M, L, true, false};
+      c.P = hidden; c.Q = ls; c.R = M; c.bn_P = hidden; c.bn_Q = L;
+      c.mode = MODE_NONE; c.L = ls; c.k_total = 1; c.s_begin = 0; c.s_end = 1;
+      c.epi = plain_epilogue(dw_ptr(dw_off_w2 + lo), ffn, fp32);
+      c.epi.accumulate = accumulate;
+      c.status = status;
+      rc = launch_gemm(c, stream);
+      if (rc) return rc;
+      // dW1[F_s,:] = dZ_s^T X
+      memset(&c, 0, sizeof(c));
+      c.a = Operand{dz_s, ls, M, L, true, false};
+      c.b = Operand{x, hidden, M, hidden, true, false};
+      c.P = ls; c.Q = hidden; c.R = M; c.bn_P = L; c.bn_Q = hidden;
+      c.mode = MODE_NONE; c.L = ls; c.k_total = 1; c.s_begin = 0; c.s_end = 1;
+      c.epi = plain_epilogue(dw_ptr(dw_off_w1 + lo * hidden), hidden, fp32);
+      c.epi.accumulate = accumulate;
+      c.status = status;
+      rc = launch_gemm(c, stream);
+      if (rc) return rc;
+    }
+    if (db1) { rc = launch_colsum(dz_s, L, M, 0, (int)ls, partial, db1 + lo, stream); if (rc) return rc; }
+    if (dx) {
+      // dX (+)= dZ_s W1[F_s,:]
+      memset(&c, 0, sizeof(c));
+      c.a = Operand{dz_s, ls, M, L, false, false};
+      c.b = Operand{w1, hidden, ffn, hidden, true, true};
+      c.P = M; c.Q = hidden; c.R = ffn; c.bn_P = M; c.bn_Q = hidden;
+      c.mode = (k == 1) ? MODE_NONE : MODE_RED;
+      c.L = L; c.k_total = k; c.s_begin = s; c.s_end = s + 1;
+      c.epi = plain_epilogue(dx, hidden, 0);
+      c.epi.carry = carry;
+      c.epi.ld_carry = hidden;
+      c.status = status;
+      rc = launch_gemm(c, stream);
+      if (rc) return rc;
+    }
+  }
+  return OSDP_OK;
+}
+
+int osdp_read_device_status(void *ws, int *status, void *stream_) {
+  if (!ws || !status) return OSDP_ERR_NULL_POINTER;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  int word = 0;
+  cudaError_t e = cudaMemcpyAsync(&word, ws, sizeof(int), cudaMemcpyDeviceToHost, stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (word != 0) {
+    e = cudaMemsetAsync(ws, 0, sizeof(int), stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  *status = (word == 0) ? OSDP_OK : OSDP_ERR_DEVICE_TIMEOUT;
+  return OSDP_OK;
+}
+
+}  // extern "C"

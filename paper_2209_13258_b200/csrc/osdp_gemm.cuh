@@ -1,0 +1,589 @@
+// Persistent, warp-specialised bf16 GEMM for sm_100a: TMA -> shared-memory ring -> tcgen05.mma
+// with fp32 accumulators in tensor memory -> fused epilogue.  One CTA per SM.
+//
+// It computes, for a range of slices of the operator (Section 3.3 of the paper: partition,
+// process the slices one after another, combine), tiles of  OUT[P,Q] = A[P,R] * B[Q,R]^T  where
+// the slice cuts either the output columns, the output rows, or the reduction dimension R:
+//   MODE_COLS / MODE_ROWS : slices write disjoint parts of OUT (concatenation); the tile list is
+//                           walked in slice-major order, no dependence between slices.
+//   MODE_RED              : every slice contributes to every tile (sum over slices); each CTA owns
+//                           a fixed set of tiles and walks slices in the outer loop, carrying the
+//                           fp32 partial sum of a tile through global memory between slices.  The
+//                           same thread writes and later re-reads a carry element, so no
+//                           cross-CTA synchronisation exists anywhere in this kernel.
+// Both operands may be K-major (reduction contiguous) or MN-major (output dim contiguous); the three
+// GEMMs of a linear layer need (K,K) forward, (K,MN) dX and (MN,MN) dW.
+//
+// Warp roles (256 threads): warp 0 TMA producer, warp 1 MMA issuer, warp 2 TMEM allocator,
+// warps 4-7 epilogue (warp w reads TMEM lanes 32*(w%4) ...).  Two TMEM accumulators so that the
+// epilogue of tile i overlaps the main loop of tile i+1.
+// Every mbarrier wait is bounded in time; on expiry the CTA records a status code and unwinds.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace osdp {
+
+constexpr int BM = 128;       // tile rows  (UMMA M, cta_group::1)
+constexpr int BK = 64;        // reduction elements per pipeline stage (one 128-byte swizzle span)
+constexpr int UMMA_K = 16;    // reduction elements per tcgen05.mma (bf16)
+constexpr int NUM_THREADS = 256;
+constexpr int GROUP_M = 16;   // tile rasterisation: tiles of 16 tile-rows share operand tiles in L2
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s per wait
+
+enum : int { MODE_NONE = 0, MODE_COLS = 1, MODE_ROWS = 2, MODE_RED = 3 };
+enum : int { ACT_NONE = 0, ACT_GELU_TANH = 1, ACT_GELU_ERF = 2 };
+enum : int { STATUS_TIMEOUT_PRODUCER = 101, STATUS_TIMEOUT_MMA = 102, STATUS_TIMEOUT_EPILOGUE = 103 };
+
+struct Epilogue {
+  void *out;                 // [P,Q] final output (bf16 or fp32)
+  long long ld_out;
+  int out_fp32;
+  int accumulate;            // out += instead of out =
+  float *carry;              // [P,Q] fp32 running sum for MODE_RED (unused otherwise)
+  long long ld_carry;
+  const float *bias;         // [Q] or null; added when the tile is finalised
+  __nv_bfloat16 *z_save;     // [P,Q] or null; pre-activation written when finalised
+  long long ld_z;
+  int act;                   // activation applied when finalised
+  const __nv_bfloat16 *gz;   // [P,Q] or null: multiply the result by act'(gz) (activation backward)
+  long long ld_gz;
+  int gz_act;
+  __nv_bfloat16 *act_out;    // [P,Q] or null: also write act(gz) here
+  long long ld_act_out;
+};
+
+struct GemmParams {
+  CUtensorMap a_main, a_tail, b_main, b_tail;   // 3-D maps: slices 0..k-2 / the last slice
+  int P, Q, R;               // output rows, output cols, reduction extent (whole operator)
+  int mode;                  // which dimension the slices cut
+  int L;                     // slice length in that dimension
+  int k_total;               // number of slices of the operator
+  int s_begin, s_end;        // slices processed by this launch
+  int a_sc_mul, b_sc_mul;    // 1: the operand map has a slice coordinate; 0: the operand is one slice already
+  Epilogue epi;
+  int *status;               // device status word or null
+};
+
+// ------------------------------------------------------------------------------------------------
+// PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the CTA is unwinding (this wait or another one ran out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          int *status, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  uint32_t polls = 0;
+  unsigned long long t0 = 0;
+  for (;;) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++polls & 255u) == 0u) {
+      if (*abort_flag) return false;
+      unsigned long long now = globaltimer_ns();
+      if (t0 == 0) {
+        t0 = now;
+      } else if (now - t0 > WAIT_LIMIT_NS) {
+        *abort_flag = 1;
+        if (status) atomicCAS(status, 0, code);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap *m) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(m) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0,
+                                            int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// mbarrier arrives once every tcgen05.mma issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld_x32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// ------------------------------------------------------------------------------------------------
+// Descriptors
+
+// Shared-memory matrix descriptor, 128-byte swizzle, version 1 (sm_100).
+//  K-major tile  [rows][64 bf16]: rows are 128 B apart, groups of 8 rows 1024 B apart (SBO).
+//  MN-major tile [chunks of 64 MN][64 k-rows of 128 B]: 8 k-rows = 1024 B (SBO), MN chunks
+//  8192 B apart (LBO).
+template <bool MN_MAJOR>
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
+  constexpr uint64_t lbo = MN_MAJOR ? (uint64_t)((BK * 128) >> 4) : 1ull;
+  constexpr uint64_t sbo = 1024 >> 4;
+  uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= lbo << 16;
+  d |= sbo << 32;
+  d |= 1ull << 46;   // descriptor version
+  d |= 2ull << 61;   // SWIZZLE_128B
+  return d;
+}
+// Bytes the start address moves per UMMA_K step inside a stage.
+template <bool MN_MAJOR>
+__device__ __forceinline__ constexpr uint32_t desc_k_advance() {
+  return MN_MAJOR ? (UMMA_K * 128) : (UMMA_K * 2);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = BN.
+template <int BN, bool A_MN, bool B_MN>
+__device__ __forceinline__ constexpr uint32_t make_idesc() {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16) |
+         ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+template <int BN>
+struct SmemLayout {
+  static constexpr int A_BYTES = BM * BK * 2;
+  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
+  static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+  static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;   // barriers + alignment slack
+  static constexpr int TMEM_COLS = 2 * BN;
+};
+
+// ------------------------------------------------------------------------------------------------
+// Tile schedule (identical in every warp role)
+
+struct Work {
+  int s;                     // slice
+  int row0, row_end;         // output rows of the tile, clipped extent of the slice
+  int col0, col_end;
+  int kblocks;               // reduction blocks of this slice
+  int a_row, b_col;          // TMA coordinates (slice-relative where that dimension is sliced)
+  int carry_in, carry_out;
+};
+
+__device__ __forceinline__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+template <int BN>
+__device__ __forceinline__ bool get_work(const GemmParams &p, int i, Work &w) {
+  const int nsl = p.s_end - p.s_begin;
+  int s, t, rows, cols;
+  if (p.mode == MODE_RED) {
+    const int tiles = ceil_div(p.P, BM) * ceil_div(p.Q, BN);
+    const int bid = blockIdx.x, G = gridDim.x;
+    if (bid >= tiles) return false;
+    const int n_my = (tiles - bid + G - 1) / G;
+    const int srel = i / n_my;
+    if (srel >= nsl) return false;
+    s = p.s_begin + srel;
+    t = bid + (i - srel * n_my) * G;
+    rows = p.P;
+    cols = p.Q;
+  } else {
+    const int rows_full = (p.mode == MODE_ROWS) ? p.L : p.P;
+    const int cols_full = (p.mode == MODE_COLS) ? p.L : p.Q;
+    const int t_full = ceil_div(rows_full, BM) * ceil_div(cols_full, BN);
+    const long long widx = (long long)blockIdx.x + (long long)i * gridDim.x;
+    long long srel = widx / t_full;
+    if (srel > nsl - 1) srel = nsl - 1;
+    s = p.s_begin + (int)srel;
+    const long long tl = widx - srel * t_full;
+    rows = (p.mode == MODE_ROWS) ? min(p.L, p.P - s * p.L) : p.P;
+    cols = (p.mode == MODE_COLS) ? min(p.L, p.Q - s * p.L) : p.Q;
+    if (tl >= (long long)ceil_div(rows, BM) * ceil_div(cols, BN)) return false;
+    t = (int)tl;
+  }
+  const int tiles_m = ceil_div(rows, BM), tiles_n = ceil_div(cols, BN);
+  const int group = GROUP_M * tiles_n;
+  const int g = t / group;
+  const int first_m = g * GROUP_M;
+  const int gm = min(GROUP_M, tiles_m - first_m);
+  const int tm = first_m + (t - g * group) % gm;
+  const int tn = (t - g * group) / gm;
+  const int row_base = (p.mode == MODE_ROWS) ? s * p.L : 0;
+  const int col_base = (p.mode == MODE_COLS) ? s * p.L : 0;
+  w.s = s;
+  w.a_row = tm * BM;
+  w.b_col = tn * BN;
+  w.row0 = row_base + w.a_row;
+  w.col0 = col_base + w.b_col;
+  w.row_end = row_base + rows;
+  w.col_end = col_base + cols;
+  const int red = (p.mode == MODE_RED) ? min(p.L, p.R - s * p.L) : p.R;
+  w.kblocks = ceil_div(red, BK);
+  w.carry_in = (p.mode == MODE_RED) && (s > 0);
+  w.carry_out = (p.mode == MODE_RED) && (s < p.k_total - 1);
+  return true;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Epilogue arithmetic on 8 consecutive columns of one row
+
+__device__ __forceinline__ float gelu_f(float x, int act) {
+  if (act == ACT_GELU_TANH) {
+    const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
+    return 0.5f * x * (1.0f + tanhf(u));
+  }
+  if (act == ACT_GELU_ERF) return 0.5f * x * (1.0f + erff(x * 0.7071067811865476f));
+  return x;
+}
+__device__ __forceinline__ float gelu_grad_f(float x, int act) {
+  if (act == ACT_GELU_TANH) {
+    const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
+    const float t = tanhf(u);
+    const float du = 0.7978845608028654f * (1.0f + 0.134145f * x * x);
+    return 0.5f * (1.0f + t) + 0.5f * x * (1.0f - t * t) * du;
+  }
+  if (act == ACT_GELU_ERF) {
+    const float Phi = 0.5f * (1.0f + erff(x * 0.7071067811865476f));
+    const float phi = 0.3989422804014327f * __expf(-0.5f * x * x);
+    return Phi + x * phi;
+  }
+  return 1.0f;
+}
+__device__ __forceinline__ void unpack_bf16x8(const uint4 &u, float (&f)[8]) {
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    f[2 * j] = __uint_as_float(w[j] << 16);
+    f[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+  }
+}
+__device__ __forceinline__ uint4 pack_bf16x8(const float (&f)[8]) {
+  uint32_t w[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * j], f[2 * j + 1]);
+    w[j] = *reinterpret_cast<uint32_t *>(&h);
+  }
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+__device__ __forceinline__ void epilogue8(const Epilogue &e, long long row, int col, float (&f)[8],
+                                          int carry_in, int carry_out) {
+  if (carry_in) {
+    const float4 *c = reinterpret_cast<const float4 *>(e.carry + row * e.ld_carry + col);
+    const float4 c0 = c[0], c1 = c[1];
+    f[0] += c0.x; f[1] += c0.y; f[2] += c0.z; f[3] += c0.w;
+    f[4] += c1.x; f[5] += c1.y; f[6] += c1.z; f[7] += c1.w;
+  }
+  if (carry_out) {
+    float4 *c = reinterpret_cast<float4 *>(e.carry + row * e.ld_carry + col);
+    c[0] = make_float4(f[0], f[1], f[2], f[3]);
+    c[1] = make_float4(f[4], f[5], f[6], f[7]);
+    return;
+  }
+  if (e.bias) {
+    const float4 b0 = *reinterpret_cast<const float4 *>(e.bias + col);
+    const float4 b1 = *reinterpret_cast<const float4 *>(e.bias + col + 4);
+    f[0] += b0.x; f[1] += b0.y; f[2] += b0.z; f[3] += b0.w;
+    f[4] += b1.x; f[5] += b1.y; f[6] += b1.z; f[7] += b1.w;
+  }
+  if (e.z_save) *reinterpret_cast<uint4 *>(e.z_save + row * e.ld_z + col) = pack_bf16x8(f);
+  if (e.act != ACT_NONE) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) f[j] = gelu_f(f[j], e.act);
+  }
+  if (e.gz) {
+    float z[8];
+    unpack_bf16x8(*reinterpret_cast<const uint4 *>(e.gz + row * e.ld_gz + col), z);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) f[j] *= gelu_grad_f(z[j], e.gz_act);
+    if (e.act_out) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) z[j] = gelu_f(z[j], e.gz_act);
+      *reinterpret_cast<uint4 *>(e.act_out + row * e.ld_act_out + col) = pack_bf16x8(z);
+    }
+  }
+  if (e.out_fp32) {
+    float4 *o = reinterpret_cast<float4 *>(reinterpret_cast<float *>(e.out) + row * e.ld_out + col);
+    if (e.accumulate) {
+      const float4 o0 = o[0], o1 = o[1];
+      f[0] += o0.x; f[1] += o0.y; f[2] += o0.z; f[3] += o0.w;
+      f[4] += o1.x; f[5] += o1.y; f[6] += o1.z; f[7] += o1.w;
+    }
+    o[0] = make_float4(f[0], f[1], f[2], f[3]);
+    o[1] = make_float4(f[4], f[5], f[6], f[7]);
+  } else {
+    uint4 *o = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(e.out) + row * e.ld_out + col);
+    if (e.accumulate) {
+      float old[8];
+      unpack_bf16x8(*o, old);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) f[j] += old[j];
+    }
+    *o = pack_bf16x8(f);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// The kernel
+
+template <int BN, bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
+  using SL = SmemLayout<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+
+  const uint32_t bar_base = smem_base + SL::BAR_OFFSET;
+  auto full_bar = [&](int st) { return bar_base + 8u * st; };
+  auto empty_bar = [&](int st) { return bar_base + 8u * (SL::STAGES + st); };
+  auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * SL::STAGES + b); };
+  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * SL::STAGES + 2 + b); };
+  uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(smem_gen + SL::BAR_OFFSET + 8 * (2 * SL::STAGES + 4));
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int st = 0; st < SL::STAGES; ++st) {
+      mbar_init(full_bar(st), 1);
+      mbar_init(empty_bar(st), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(tfull_bar(b), 1);
+      mbar_init(tempty_bar(b), 4);
+    }
+    *abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tmap(&p.a_main);
+    prefetch_tmap(&p.a_tail);
+    prefetch_tmap(&p.b_main);
+    prefetch_tmap(&p.b_tail);
+  }
+  if (warp == 2) {
+    tmem_alloc(smem_u32(tmem_holder), SL::TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+
+  // Which operand dimension the slice coordinate belongs to (fixed by mode and operand major).
+  const bool a_sliced = (p.mode == MODE_ROWS) || (p.mode == MODE_RED);
+  const bool b_sliced = (p.mode == MODE_COLS) || (p.mode == MODE_RED);
+  const bool a_mid = A_MN ? (p.mode == MODE_ROWS) : (p.mode == MODE_RED);   // slice cuts A's contiguous dim
+  const bool b_mid = B_MN ? (p.mode == MODE_COLS) : (p.mode == MODE_RED);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    int stage = 0;
+    uint32_t phase = 0;
+    uint32_t armed = 0, armed_phase = 0;   // per-stage bookkeeping for the unwind path
+    bool ok = true;
+    Work w;
+    for (int i = 0; ok && get_work<BN>(p, i, w); ++i) {
+      const bool tail = (w.s == p.k_total - 1);
+      const CUtensorMap *amap = (a_sliced && !tail) ? &p.a_main : &p.a_tail;
+      const CUtensorMap *bmap = (b_sliced && !tail) ? &p.b_main : &p.b_tail;
+      const int a_sc = (a_sliced && !tail) ? w.s * p.a_sc_mul : 0;
+      const int b_sc = (b_sliced && !tail) ? w.s * p.b_sc_mul : 0;
+      for (int kb = 0; kb < w.kblocks; ++kb) {
+        ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER);
+        if (!ok) break;
+        if (lane == 0) {
+          const uint32_t sa = smem_base + stage * SL::STAGE_BYTES;
+          const uint32_t sb = sa + SL::A_BYTES;
+          const uint32_t fb = full_bar(stage);
+          mbar_expect_tx(fb, SL::STAGE_BYTES);
+          const int kc = kb * BK;
+          if (A_MN) {
+#pragma unroll
+            for (int j = 0; j < BM / 64; ++j) {
+              const int in = w.a_row + j * 64;
+              if (a_mid) tma_load_3d(sa + j * (BK * 128), amap, fb, in, a_sc, kc);
+              else tma_load_3d(sa + j * (BK * 128), amap, fb, in, kc, a_sc);
+            }
+          } else {
+            if (a_mid) tma_load_3d(sa, amap, fb, kc, a_sc, w.a_row);
+            else tma_load_3d(sa, amap, fb, kc, w.a_row, a_sc);
+          }
+          if (B_MN) {
+#pragma unroll
+            for (int j = 0; j < BN / 64; ++j) {
+              const int in = w.b_col + j * 64;
+              if (b_mid) tma_load_3d(sb + j * (BK * 128), bmap, fb, in, b_sc, kc);
+              else tma_load_3d(sb + j * (BK * 128), bmap, fb, in, kc, b_sc);
+            }
+          } else {
+            if (b_mid) tma_load_3d(sb, bmap, fb, kc, b_sc, w.b_col);
+            else tma_load_3d(sb, bmap, fb, kc, w.b_col, b_sc);
+          }
+        }
+        armed |= 1u << stage;
+        armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
+        __syncwarp();
+        if (++stage == SL::STAGES) { stage = 0; phase ^= 1u; }
+      }
+    }
+    if (!ok) {
+      // Unwinding: let the copies already issued land before the CTA's shared memory goes away.
+      for (int st = 0; st < SL::STAGES; ++st) {
+        if (!((armed >> st) & 1u)) continue;
+        const unsigned long long t0 = globaltimer_ns();
+        while (!mbar_try_wait(full_bar(st), (armed_phase >> st) & 1u)) {
+          if (globaltimer_ns() - t0 > 2000000ull) break;   // 2 ms
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    constexpr uint32_t idesc = make_idesc<BN, A_MN, B_MN>();
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    Work w;
+    for (int i = 0; ok && get_work<BN>(p, i, w); ++i) {
+      const int buf = i & 1;
+      const uint32_t bphase = (uint32_t)(i >> 1) & 1u;
+      ok = mbar_wait(tempty_bar(buf), bphase ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+      for (int kb = 0; kb < w.kblocks; ++kb) {
+        ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status, STATUS_TIMEOUT_MMA);
+        if (!ok) break;
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t sa = smem_base + stage * SL::STAGE_BYTES;
+          const uint32_t sb = sa + SL::A_BYTES;
+          const uint64_t adesc = make_smem_desc<A_MN>(sa);
+          const uint64_t bdesc = make_smem_desc<B_MN>(sb);
+#pragma unroll
+          for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+            umma_bf16(d_tmem, adesc + (uint64_t)((kk * desc_k_advance<A_MN>()) >> 4),
+                      bdesc + (uint64_t)((kk * desc_k_advance<B_MN>()) >> 4), idesc,
+                      (kb > 0 || kk > 0) ? 1u : 0u);
+          }
+          umma_commit(empty_bar(stage));                      // frees the stage when the MMAs retire
+          if (kb == w.kblocks - 1) umma_commit(tfull_bar(buf));   // accumulator complete
+        }
+        __syncwarp();
+        if (++stage == SL::STAGES) { stage = 0; phase ^= 1u; }
+      }
+    }
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------------ epilogue
+    const int quarter = warp & 3;
+    bool ok = true;
+    Work w;
+    for (int i = 0; ok && get_work<BN>(p, i, w); ++i) {
+      const int buf = i & 1;
+      const uint32_t bphase = (uint32_t)(i >> 1) & 1u;
+      ok = mbar_wait(tfull_bar(buf), bphase, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE);
+      if (!ok) break;
+      tc_fence_after();
+      const long long row = (long long)w.row0 + quarter * 32 + lane;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        const int cbase = w.col0 + c * 32;
+        if (cbase >= w.col_end) break;
+        uint32_t v[32];
+        tmem_ld_x32(taddr + (uint32_t)(c * 32), v);
+        tmem_ld_wait();
+        if (row < w.row_end) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            const int col = cbase + g * 8;
+            if (col < w.col_end) {
+              float f[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[g * 8 + j]);
+              epilogue8(p.epi, row, col, f, w.carry_in, w.carry_out);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(buf));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, SL::TMEM_COLS);
+  }
+}
+
+}  // namespace osdp
