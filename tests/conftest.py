@@ -15,3 +15,12 @@ def pytest_configure(config):
 def pytest_collection_modifyitems(config, items):
     # keep the file that must run last at the end whatever the collection order
     items.sort(key=lambda it: 1 if "test_zz_" in it.nodeid else 0)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_libraries():
+    """Both shared libraries are built in-tree if missing or stale (nvcc / gcc, seconds)."""
+    from oracle.build import build as build_oracle
+    from paper_2209_13258_b200.build import build as build_osdp
+    build_oracle()
+    build_osdp()

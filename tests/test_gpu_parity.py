@@ -1,0 +1,332 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded bf16 inputs.  Tolerances: relative Frobenius <= 5e-3 and max abs <= 3e-2 (see util.py);
+concatenated outputs of a split must be bit-identical to the GPU's own k = 1 result."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2209_13258_b200 import inputs
+from util import Guarded, assert_close, to_dev, to_f64
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def P():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2209_13258_b200 as pkg
+    pkg.lib()   # fails loudly if the extension is missing: there is no fallback
+    return pkg
+
+
+def run_linear(P, c, k, split, act=0, dw_fp32=True, use_bias=True, accumulate=0, dw_init=None, per_slice=False):
+    """fwd + bwd through the C ABI; returns dict of cuda tensors."""
+    M, N, K, off = c["M"], c["N"], c["K"], c["w_offset"]
+    x, dy, wf = to_dev(c["x"]), to_dev(c["dy"]), to_dev(c["w_flat"])
+    b = to_dev(c["bias"]) if use_bias else None
+    out, z, dx = Guarded((M, N), torch.bfloat16), Guarded((M, N), torch.bfloat16), Guarded((M, K), torch.bfloat16)
+    dwf = Guarded((wf.numel(),), torch.float32 if dw_fp32 else torch.bfloat16)
+    if dw_init is not None:
+        dwf.t.copy_(dw_init)
+    db = Guarded((N,), torch.float32)
+    rc, n1 = P.osdp_split_linear_workspace_bytes(M, N, K, k, split, act, P.OP_LINEAR_FWD)
+    rc2, n2 = P.osdp_split_linear_workspace_bytes(M, N, K, k, split, act, P.OP_LINEAR_BWD)
+    assert rc == 0 and rc2 == 0
+    ws = P.new_workspace(max(n1, n2))
+    zs = z.t if act else None
+    dt = P.DTYPE_FP32 if dw_fp32 else P.DTYPE_BF16
+    if per_slice:
+        for s in range(max(k, 1)):
+            P.osdp_split_linear_fwd_slice(x, wf, off, b, M, N, K, k, split, act, s, out.t, zs, ws, check=True)
+        for s in range(max(k, 1)):
+            P.osdp_split_linear_bwd_slice(dy, x, wf, off, zs, M, N, K, k, split, act, s, dx.t, dwf.t, off, dt,
+                                          accumulate, db.t, ws, check=True)
+    else:
+        P.osdp_split_linear_fwd(x, wf, off, b, M, N, K, k, split, act, out.t, zs, ws, check=True)
+        P.osdp_split_linear_bwd(dy, x, wf, off, zs, M, N, K, k, split, act, dx.t, dwf.t, off, dt, accumulate, db.t,
+                                ws, check=True)
+    rc, st = P.osdp_read_device_status(ws)
+    assert rc == 0 and st == 0
+    for g in (out, dx, dwf, db) + ((z,) if act else ()):
+        g.check()
+    dw = dwf.t[off:off + N * K].view(N, K)
+    # nothing outside W's window of the flat gradient buffer may be written
+    if dw_init is None:
+        assert bool(torch.isnan(dwf.t[:off]).all()) and bool(torch.isnan(dwf.t[off + N * K:]).all())
+    return {"y": out.t, "z": z.t if act else None, "dx": dx.t, "dw": dw, "db": db.t}
+
+
+def oracle_linear(c, act, k=1, split=None, use_bias=True):
+    b = c["bias"] if use_bias else None
+    z, y = oracle.linear_fwd(c["x"], c["w"], b, act, k, split)
+    dX, dW, db = oracle.linear_bwd(c["dy"], c["x"], c["w"], z, act, k, split)
+    return {"y": y, "z": z, "dx": dX, "dw": dW, "db": db}
+
+
+def compare(g, o, act, dw_fp32=True):
+    assert_close(to_f64(g["y"]), o["y"], "Y")
+    if act:
+        assert_close(to_f64(g["z"]), o["z"], "Z")
+    assert_close(to_f64(g["dx"]), o["dx"], "dX")
+    assert_close(to_f64(g["dw"]), o["dw"], "dW")
+    assert_close(to_f64(g["db"]), o["db"], "db")
+
+
+# ---------------------------------------------------------------------------------------------
+# config 1: X [256,512], W [2048,512] ~N(0,0.02), bias zeros, k=4 along the output dim
+
+def test_config1_exact_shapes(P):
+    c = inputs.linear_case(256, 2048, 512)
+    g = run_linear(P, c, 4, P.SPLIT_OUT)
+    o = oracle_linear(c, 0, 4, oracle.SPLIT_OUT)
+    compare(g, o, 0)
+    # fp32 dW, fp32 db: the literal bounds hold with a wide margin
+    relf, maxabs = assert_close(to_f64(g["dw"]), o["dw"], "dW fp32", relf_tol=1e-5)
+    assert maxabs <= 3e-2
+    # bit identity of the concatenated outputs with the GPU's own k = 1 result
+    g1 = run_linear(P, c, 1, P.SPLIT_OUT)
+    for name in ("y", "dw", "db"):
+        assert torch.equal(g[name].view(torch.int32 if g[name].dtype == torch.float32 else torch.int16),
+                           g1[name].view(torch.int32 if g1[name].dtype == torch.float32 else torch.int16)), name
+
+
+def test_config1_with_bias_and_offset(P):
+    c = inputs.linear_case(256, 2048, 512, bias_std=0.02, w_offset=4096 + 8, flat_pad=24)
+    for split in (P.SPLIT_OUT, P.SPLIT_RED):
+        g = run_linear(P, c, 4, split)
+        compare(g, oracle_linear(c, 0, 4, split), 0)
+
+
+# ---------------------------------------------------------------------------------------------
+# ragged shapes spanning several tiles, every split / activation / dtype combination
+
+RAGGED = [(200, 264, 136), (300, 520, 328), (77, 1032, 72), (513, 8, 520), (130, 392, 264)]
+
+
+@pytest.mark.parametrize("shape", RAGGED)
+@pytest.mark.parametrize("split", [0, 1])
+def test_ragged_shapes_all_k(P, shape, split):
+    M, N, K = shape
+    c = inputs.linear_case(M, N, K, w_std=0.1, bias_std=0.3, w_offset=72, flat_pad=8, layer=2)
+    D = N if split == 0 else K
+    for k in (1, 2, 3, 5, 8, D // 8):
+        if k < 1 or P.osdp_slice_range(D, k, 0)[0] != 0:
+            continue
+        g = run_linear(P, c, k, split)
+        compare(g, oracle_linear(c, 0, k, split), 0)
+
+
+@pytest.mark.parametrize("act", [1, 2])
+@pytest.mark.parametrize("split,k", [(0, 1), (0, 3), (1, 4), (0, 6)])
+def test_activation_forward_backward(P, act, split, k):
+    c = inputs.linear_case(260, 528, 200, w_std=0.08, bias_std=0.3, layer=4)
+    g = run_linear(P, c, k, split, act=act)
+    o = oracle_linear(c, act, k, split)
+    compare(g, o, act)
+
+
+def test_bf16_dw_and_accumulate(P):
+    c = inputs.linear_case(384, 512, 256, w_std=0.1, layer=5)
+    o = oracle_linear(c, 0)
+    g = run_linear(P, c, 2, P.SPLIT_OUT, dw_fp32=False)
+    assert g["dw"].dtype == torch.bfloat16
+    assert_close(to_f64(g["dw"]), o["dw"], "dW bf16")
+    # accumulate: dW += ..., starting from a known fp32 buffer
+    init = torch.arange(c["w_flat"].size, dtype=torch.float32, device="cuda") * 1e-3
+    for split in (0, 1):
+        g = run_linear(P, c, 2, split, accumulate=1, dw_init=init)
+        want = o["dw"] + to_f64(init)[c["w_offset"]:c["w_offset"] + 512 * 256].reshape(512, 256)
+        assert_close(to_f64(g["dw"]), want, "dW accumulate", relf_tol=1e-5)
+
+
+# ---------------------------------------------------------------------------------------------
+# bit identity, per-slice calls, determinism
+
+def _bits(t):
+    return t.contiguous().view(torch.int32 if t.dtype == torch.float32 else torch.int16)
+
+
+@pytest.mark.parametrize("shape", [(512, 2048, 1024), (300, 520, 328)])
+def test_bit_identity_of_concatenated_outputs(P, shape):
+    M, N, K = shape
+    c = inputs.linear_case(M, N, K, bias_std=0.1, layer=6)
+    g1 = run_linear(P, c, 1, 0, act=1)
+    for k in (2, 4, 8):
+        g = run_linear(P, c, k, P.SPLIT_OUT, act=1)
+        for name in ("y", "z"):
+            assert torch.equal(_bits(g[name]), _bits(g1[name])), (name, k)
+    # without activation the backward's concatenated outputs are bit-identical too
+    g1 = run_linear(P, c, 1, 0)
+    for k in (2, 4, 8):
+        g = run_linear(P, c, k, P.SPLIT_OUT)
+        for name in ("y", "dw", "db"):
+            assert torch.equal(_bits(g[name]), _bits(g1[name])), (name, k)
+        if P.osdp_slice_range(K, k, 0)[0] != 0:
+            continue
+        g = run_linear(P, c, k, P.SPLIT_RED)
+        for name in ("dx", "dw", "db"):
+            assert torch.equal(_bits(g[name]), _bits(g1[name])), (name, k)
+
+
+@pytest.mark.parametrize("split", [0, 1])
+@pytest.mark.parametrize("act", [0, 1])
+def test_per_slice_calls_equal_whole_call(P, split, act):
+    c = inputs.linear_case(300, 520, 328, w_std=0.1, bias_std=0.2, layer=7)
+    a = run_linear(P, c, 3, split, act=act)
+    b = run_linear(P, c, 3, split, act=act, per_slice=True)
+    for name in ("y", "dx", "dw", "db"):
+        assert torch.equal(_bits(a[name]), _bits(b[name])), name
+
+
+def test_repeated_runs_are_bitwise_equal(P):
+    c = inputs.linear_case(1024, 1024, 512, layer=8)
+    ref = run_linear(P, c, 4, P.SPLIT_RED)
+    for _ in range(5):
+        g = run_linear(P, c, 4, P.SPLIT_RED)
+        for name in ("y", "dx", "dw", "db"):
+            assert torch.equal(_bits(g[name]), _bits(ref[name])), name
+
+
+def test_maximum_split_and_tiny_shapes(P):
+    # slices of length 8 (the minimum), and a 1-token batch
+    c = inputs.linear_case(1, 64, 64, w_std=0.2, layer=9)
+    for split in (0, 1):
+        g = run_linear(P, c, 8, split)
+        compare(g, oracle_linear(c, 0, 8, split), 0)
+    c = inputs.linear_case(8, 8, 8, w_std=0.5, layer=10)
+    compare(run_linear(P, c, 1, 0), oracle_linear(c, 0), 0)
+
+
+# ---------------------------------------------------------------------------------------------
+# config 2: transformer MLP block, hidden 1024, ffn 4096, tokens 8 x 512, split along ffn
+
+def run_mlp(P, c, k, act=1, dw_fp32=True):
+    M, H, F = c["M"], c["hidden"], c["ffn"]
+    x, dy, wf = to_dev(c["x"]), to_dev(c["dy"]), to_dev(c["w_flat"])
+    b1, b2 = to_dev(c["b1"]), to_dev(c["b2"])
+    out, z1, dx = Guarded((M, H), torch.bfloat16), Guarded((M, F), torch.bfloat16), Guarded((M, H), torch.bfloat16)
+    dwf = Guarded((wf.numel(),), torch.float32 if dw_fp32 else torch.bfloat16)
+    db1, db2 = Guarded((F,), torch.float32), Guarded((H,), torch.float32)
+    _, n1 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, act, P.OP_MLP_FWD)
+    _, n2 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, act, P.OP_MLP_BWD)
+    ws = P.new_workspace(max(n1, n2))
+    P.osdp_split_mlp_fwd(x, wf, c["off_w1"], b1, c["off_w2"], b2, M, H, F, k, act, out.t, z1.t, ws, check=True)
+    P.osdp_split_mlp_bwd(dy, x, wf, c["off_w1"], c["off_w2"], z1.t, M, H, F, k, act, dx.t, dwf.t, c["off_w1"],
+                         c["off_w2"], P.DTYPE_FP32 if dw_fp32 else P.DTYPE_BF16, 0, db1.t, db2.t, ws, check=True)
+    rc, st = P.osdp_read_device_status(ws)
+    assert rc == 0 and st == 0
+    for g in (out, z1, dx, dwf, db1, db2):
+        g.check()
+    return {"y": out.t, "dx": dx.t, "dw1": dwf.t[c["off_w1"]:c["off_w1"] + F * H].view(F, H),
+            "dw2": dwf.t[c["off_w2"]:c["off_w2"] + H * F].view(H, F), "db1": db1.t, "db2": db2.t,
+            "staging": (n1, n2)}
+
+
+def compare_mlp(g, o):
+    names = ("y", "dx", "dw1", "db1", "dw2", "db2")
+    for name, ref in zip(names, o):
+        assert_close(to_f64(g[name]), ref, name)
+
+
+@pytest.mark.parametrize("k", [1, 2, 3, 5])
+def test_mlp_small_ragged(P, k):
+    c = inputs.mlp_case(200, 264, 520, w_std=0.08, layer=11)
+    g = run_mlp(P, c, k)
+    _, y = oracle.mlp_fwd(c["x"], c["w1"], c["b1"], c["w2"], c["b2"], oracle.ACT_GELU_TANH, k)
+    grads = oracle.mlp_bwd(c["dy"], c["x"], c["w1"], c["b1"], c["w2"], oracle.ACT_GELU_TANH, k)
+    compare_mlp(g, (y,) + tuple(grads))
+
+
+def test_config2_mlp_block_all_k(P):
+    c = inputs.mlp_case(8 * 512, 1024, 4096)
+    _, y = oracle.mlp_fwd(c["x"], c["w1"], c["b1"], c["w2"], c["b2"], oracle.ACT_GELU_TANH, None)
+    grads = oracle.mlp_bwd(c["dy"], c["x"], c["w1"], c["b1"], c["w2"], oracle.ACT_GELU_TANH, None)
+    staging = {}
+    for k in (1, 2, 4, 8):
+        g = run_mlp(P, c, k)
+        compare_mlp(g, (y,) + tuple(grads))
+        staging[k] = g["staging"]
+    # the slice-sized intermediates shrink as 1/k (the fp32 carry of the summed output does not)
+    M, H = 4096, 1024
+    carry = M * H * 4
+    for k in (2, 4, 8):
+        slice_part_1 = staging[1][0] - 256
+        slice_part_k = staging[k][0] - 256 - carry
+        assert abs(slice_part_k - slice_part_1 / k) <= 1024, (k, staging)
+
+
+# ---------------------------------------------------------------------------------------------
+# full-size shapes: sampled rows/columns against the oracle + matrix-vector identities over
+# every output element (launch configuration = the one bench.py times)
+
+def _sample_idx(n, boundaries, rng, extra=6):
+    idx = {0, n - 1}
+    for b in boundaries:
+        for d in (-1, 0):
+            if 0 <= b + d < n:
+                idx.add(b + d)
+    idx.update(int(v) for v in rng.integers(0, n, extra))
+    return np.array(sorted(idx))
+
+
+def check_large_linear(P, M, N, K, k, split, w_std, layer):
+    c = inputs.linear_case(M, N, K, w_std=w_std, layer=layer)
+    g = run_linear(P, c, k, split, dw_fp32=False, use_bias=False)
+    rng = np.random.default_rng(layer)
+    D = N if split == 0 else K
+    L = P.osdp_slice_range(D, k, 0)[2]
+    bounds = list(range(L, D, L))
+    rows = _sample_idx(M, [128, 256, M // 2], rng)
+    # sampled rows of Y and dX: the oracle on the row subset (same slicing along N or K)
+    sub = dict(c, x=c["x"][rows], dy=c["dy"][rows], M=len(rows))
+    z, y = oracle.linear_fwd(sub["x"], c["w"], None, 0, k, split)
+    dX, _, _ = oracle.linear_bwd(sub["dy"], sub["x"], c["w"], None, 0, k, split)
+    idx = torch.from_numpy(rows).cuda()
+    assert_close(to_f64(g["y"][idx]), y, "Y rows")
+    assert_close(to_f64(g["dx"][idx]), dX, "dX rows")
+    # sampled rows of dW (= columns of dY) and db: dW[n,:] = sum_m dY[m,n] X[m,:]
+    ncols = _sample_idx(N, bounds if split == 0 else [256, 512], rng)
+    dy_sub = np.ascontiguousarray(c["dy"][:, ncols])
+    _, dW, db = oracle.linear_bwd(dy_sub, c["x"], np.ascontiguousarray(c["w"][ncols]), None, 0)
+    nidx = torch.from_numpy(ncols).cuda()
+    assert_close(to_f64(g["dw"][nidx]), dW, "dW rows")
+    assert_close(to_f64(g["db"][nidx]), db, "db")
+    # identities over every element: Y r = X (W^T r),  dX r = dY (W r),  r^T dW = (dY r)^T X
+    Xf = inputs.bf16_bits_to_f32(c["x"]).astype(np.float64)
+    Wf = inputs.bf16_bits_to_f32(c["w"]).astype(np.float64)
+    Gf = inputs.bf16_bits_to_f32(c["dy"]).astype(np.float64)
+    rN, rK = rng.standard_normal(N), rng.standard_normal(K)
+    def close(a, b, scale, name):
+        # every element of the GPU output carries one bf16 rounding (2^-9 relative): a random
+        # combination of n of them has error ~ 2^-9 * rms * sqrt(n); allow 8x that
+        err = np.abs(a - b).max()
+        assert err <= 8 * scale, "%s identity: %.3e > %.3e" % (name, err, 8 * scale)
+    Y = to_f64(g["y"]); dXg = to_f64(g["dx"]); dWg = to_f64(g["dw"])
+    close(Y @ rN, Xf @ (Wf.T @ rN), 2.0 ** -9 * np.sqrt(np.mean(Y * Y)) * np.sqrt(N), "Y")
+    close(dXg @ rK, Gf @ (Wf @ rK), 2.0 ** -9 * np.sqrt(np.mean(dXg * dXg)) * np.sqrt(K), "dX")
+    close(rN @ dWg, (Gf @ rN) @ Xf, 2.0 ** -9 * np.sqrt(np.mean(dWg * dWg)) * np.sqrt(N), "dW")
+    return g
+
+
+def test_config5_split_sweep_shape_k8_out(P):
+    check_large_linear(P, 16384, 8192, 8192, 8, 0, 0.02, 20)
+
+
+def test_config5_split_sweep_shape_k8_red(P):
+    check_large_linear(P, 16384, 8192, 8192, 8, 1, 0.02, 21)
+
+
+@pytest.mark.parametrize("NK", [(6144, 2048), (2048, 2048), (8192, 2048), (2048, 8192)])
+def test_config3_decoder_linears_k4(P, NK):
+    N, K = NK
+    check_large_linear(P, 8192, N, K, 4, 0, 0.02, 30 + N // 2048 + K // 8192)
+
+
+def test_config4_wide_layer_k8(P):
+    # hidden 8192, ffn 32768, tokens 4 x 2048: the first MLP linear, split along the output dim,
+    # and the second, split along the reduction dim
+    check_large_linear(P, 8192, 32768, 8192, 8, 0, 0.01, 40)
+    check_large_linear(P, 8192, 8192, 32768, 8, 1, 0.01, 41)

@@ -1,0 +1,136 @@
+"""Host-side behaviour of the C ABI that needs no GPU: the library loads and exports every symbol
+the header declares, the slice table matches the hand-computed one, argument checks reject bad
+calls before anything is launched, and the workspace plan has the stated shape."""
+import os
+import re
+
+import pytest
+
+import paper_2209_13258_b200 as P
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    hdr = open(os.path.join(ROOT, "include", "osdp.h")).read()
+    declared = set(re.findall(r"\b(osdp_[a-z0-9_]+)\s*\(", hdr))
+    assert len(declared) >= 12
+    L = P.lib()
+    for name in declared:
+        assert hasattr(L, name), name
+    assert P.osdp_version() == 100
+    assert P.osdp_status_string(0) == "ok" and "split" in P.osdp_status_string(3)
+
+
+def test_slice_range_matches_golden_table():
+    path = os.path.join(ROOT, "tests", "golden", "slice_table.txt")
+    for line in open(path):
+        if line.startswith("#") or not line.strip():
+            continue
+        head, tail = line.split(":")
+        D, k = (int(v) for v in head.split())
+        want = [tuple(int(v) for v in pair.split(",")) for pair in tail.split()]
+        got = [P.osdp_slice_range(D, k, s) for s in range(k)]
+        assert [g[0] for g in got] == [0] * k
+        assert [(g[1], g[2]) for g in got] == want
+    assert P.osdp_slice_range(40, 6, 0)[0] == 3          # empty last slice
+    assert P.osdp_slice_range(40, 5, 5)[0] == 3          # slice index out of range
+    assert P.osdp_slice_range(40, 0, 0) == (0, 0, 40)    # granularity 0 = unsplit
+    assert P.osdp_slice_range(0, 1, 0)[0] == 2
+
+
+def test_workspace_plan():
+    M, N, K = 16384, 8192, 8192
+    q = lambda k, split, act, op: P.osdp_split_linear_workspace_bytes(M, N, K, k, split, act, op)
+    # forward: nothing but the status block unless the reduction dim is split (fp32 carry of Y)
+    assert q(1, 0, 0, P.OP_LINEAR_FWD) == (0, 256)
+    assert q(8, 0, 0, P.OP_LINEAR_FWD) == (0, 256)
+    assert q(8, 1, 0, P.OP_LINEAR_FWD) == (0, 256 + M * N * 4)
+    # backward: column-sum partials always; fp32 carry of dX when the output dim is split
+    part = 16 * N * 4
+    assert q(1, 0, 0, P.OP_LINEAR_BWD) == (0, 256 + part)
+    assert q(8, 0, 0, P.OP_LINEAR_BWD) == (0, 256 + M * K * 4 + part)
+    assert q(8, 1, 0, P.OP_LINEAR_BWD) == (0, 256 + part)
+    # activation backward stages G for one slice (output split) or whole (reduction split)
+    assert q(8, 0, 1, P.OP_LINEAR_BWD)[1] - q(8, 0, 0, P.OP_LINEAR_BWD)[1] == M * (N // 8) * 2
+    assert q(8, 1, 1, P.OP_LINEAR_BWD)[1] - q(8, 1, 0, P.OP_LINEAR_BWD)[1] == M * N * 2
+    # MLP chain: slice-sized intermediates shrink as 1/k
+    f = lambda k: P.osdp_split_linear_workspace_bytes(8192, 32768, 8192, k, 0, 1, P.OP_MLP_FWD)[1]
+    carry = 8192 * 8192 * 4
+    assert f(1) == 256 + 8192 * 32768 * 2
+    for k in (2, 4, 8, 16):
+        assert f(k) == 256 + carry + 8192 * (32768 // k) * 2
+    assert P.osdp_split_linear_workspace_bytes(8, 8, 8, 1, 0, 0, 9)[0] == 6
+    assert P.osdp_split_linear_workspace_bytes(8, 8, 8, 1, 0, 7, 0)[0] == 6
+    assert P.osdp_split_linear_workspace_bytes(8, 16, 8, 3, 0, 0, 0)[0] == 3
+
+
+A = 1 << 20   # a fake, 16-byte aligned "device address": argument checks never dereference it
+
+
+def _fwd(**kw):
+    a = dict(x=A, w_flat=A, w_offset=0, bias=None, M=64, N=64, K=64, k_split=2, split_dim=0, act=0, out=A,
+             z_save=None, ws=(A, 1 << 30), stream=0)
+    a.update(kw)
+    return P.osdp_split_linear_fwd(**a)
+
+
+def _bwd(**kw):
+    a = dict(dy=A, x=A, w_flat=A, w_offset=0, z_saved=None, M=64, N=64, K=64, k_split=2, split_dim=0, act=0,
+             dx=A, dw_flat=A, dw_offset=0, dw_dtype=1, accumulate=0, dbias=A, ws=(A, 1 << 30), stream=0)
+    a.update(kw)
+    return P.osdp_split_linear_bwd(**a)
+
+
+def test_forward_argument_checks():
+    assert _fwd(x=None) == 1 and _fwd(w_flat=None) == 1 and _fwd(out=None) == 1 and _fwd(ws=None) == 1
+    assert _fwd(M=0) == 2 and _fwd(N=-8) == 2 and _fwd(K=1 << 40) == 2
+    assert _fwd(N=60) == 4 and _fwd(K=12) == 4
+    assert _fwd(w_offset=4) == 4 and _fwd(w_offset=-8) == 4
+    assert _fwd(x=A + 2) == 4 and _fwd(out=A + 8) == 4 and _fwd(ws=(A + 16, 1 << 30)) == 4
+    assert _fwd(k_split=-1) == 3 and _fwd(k_split=9) == 3 and _fwd(split_dim=2) == 3
+    assert _fwd(act=3) == 6
+    assert _fwd(split_dim=1, ws=(A, 256)) == 5          # the carry does not fit
+    assert P.osdp_split_linear_fwd_slice(A, A, 0, None, 64, 64, 64, 2, 0, 0, 2, A, None, (A, 1 << 20), stream=0) == 3
+    # a well-formed call gets past the checks and fails only because there is no device / fake pointers
+    if not _cuda():
+        assert _fwd() == 7 and P.osdp_last_cuda_error() != 0
+
+
+def test_backward_argument_checks():
+    assert _bwd(dy=None) == 1 and _bwd(x=None) == 1 and _bwd(w_flat=None) == 1
+    assert _bwd(act=1, z_saved=None) == 1
+    assert _bwd(dw_dtype=2) == 6
+    assert _bwd(dw_offset=12) == 4 and _bwd(dx=A + 4) == 4 and _bwd(dbias=A + 4) == 4
+    assert _bwd(k_split=9) == 3
+    assert _bwd(ws=(A, 1024)) == 5
+    assert P.osdp_split_linear_bwd_slice(A, A, A, 0, None, 64, 64, 64, 2, 0, 0, -1, A, A, 0, 1, 0, A, (A, 1 << 20),
+                                         stream=0) == 3
+
+
+def test_mlp_argument_checks():
+    f = lambda **kw: P.osdp_split_mlp_fwd(**dict(dict(x=A, w_flat=A, off_w1=0, b1=None, off_w2=64 * 256, b2=None,
+                                                      M=32, hidden=64, ffn=256, k_split=4, act=1, out=A,
+                                                      z1_save=None, ws=(A, 1 << 30), stream=0), **kw))
+    assert f(x=None) == 1 and f(off_w2=3) == 4 and f(k_split=64) == 3 and f(ws=(A, 256)) == 5 and f(ffn=100) == 4
+    b = lambda **kw: P.osdp_split_mlp_bwd(**dict(dict(dy=A, x=A, w_flat=A, off_w1=0, off_w2=64 * 256, z1_saved=A,
+                                                      M=32, hidden=64, ffn=256, k_split=4, act=1, dx=A, dw_flat=A,
+                                                      dw_off_w1=0, dw_off_w2=64 * 256, dw_dtype=1, accumulate=0,
+                                                      db1=A, db2=A, ws=(A, 1 << 30), stream=0), **kw))
+    assert b(z1_saved=None) == 1 and b(dw_dtype=5) == 6 and b(dw_off_w1=4) == 4 and b(ws=(A, 4096)) == 5
+
+
+def _cuda():
+    try:
+        import torch
+        return torch.cuda.is_available()
+    except Exception:
+        return False
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    from paper_2209_13258_b200 import binding
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "HERE", str(tmp_path))
+    with pytest.raises(OSError, match="no CPU fallback"):
+        binding.lib()
