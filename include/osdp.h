@@ -58,6 +58,7 @@ extern "C" {
 #define OSDP_ERR_UNSUPPORTED 6        /* unknown activation, dtype or op */
 #define OSDP_ERR_CUDA 7               /* a CUDA call failed; see osdp_last_cuda_error */
 #define OSDP_ERR_DEVICE_TIMEOUT 8     /* a bounded device-side wait ran out (status word) */
+#define OSDP_ERR_EXCEEDS_STATIC_SCRATCH 9 /* osdp_bias_grad_noalloc: ceil(M/1024) * N too large */
 
 #define OSDP_SPLIT_OUT 0
 #define OSDP_SPLIT_RED 1
@@ -156,6 +157,32 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
  * (OSDP_OK, or OSDP_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel ran out) and
  * clears it.  Every device-side wait in this library is bounded; none can hang the GPU. */
 int osdp_read_device_status(void *ws, int *status, void *stream);
+
+/* Bias gradient for callers that cannot allocate.  (The paper has no counterpart: it is an
+ * addition for users of this library.)
+ *
+ * Computes dbias[n] = sum over m of dy[m,n] -- the same result, bit for bit, as
+ * osdp_split_linear_bwd(..., act = OSDP_ACT_NONE, dx = NULL, dw_flat = NULL, dbias) -- without a
+ * workspace argument and without calling cudaMalloc, cudaFree or any allocating routine.  It is
+ * meant for code that runs where device allocation is forbidden or impossible: inside an
+ * allocator or memory-pool callback, in a plug-in whose host application owns all device memory
+ * after start-up, in a latency-critical loop that must never wait on the allocator.
+ *
+ * The partial sums live in a 4 MiB array built into the library image
+ * (OSDP_NOALLOC_MAX_PARTIALS floats); every GPU on which the library is loaded holds it until
+ * the process exits.  Limit: ceil(M/1024) * N <= OSDP_NOALLOC_MAX_PARTIALS, else
+ * OSDP_ERR_EXCEEDS_STATIC_SCRATCH and nothing is launched.
+ *
+ *   dy [M,N] bf16 device, row-major, 16-byte aligned, N a multiple of 8; dbias [N] fp32 device.
+ *   Asynchronous on `stream`; caller keeps the buffers alive until the stream has passed it.
+ *
+ * The first call on each device looks up the array's device address (with that device
+ * current); make that first call before starting any stream capture.  All calls on a device
+ * share the one array, which keeps whatever the last call left in it; each call overwrites the
+ * part it reads, so no clearing is needed, but two calls that may run at the same time on one
+ * GPU (different streams, different threads) race on it: serialise them. */
+#define OSDP_NOALLOC_MAX_PARTIALS (1 << 20)
+int osdp_bias_grad_noalloc(const void *dy, int64_t M, int64_t N, float *dbias, void *stream);
 
 #ifdef __cplusplus
 }

@@ -21,7 +21,7 @@ EXPORTS = [
     "osdp_version", "osdp_status_string", "osdp_last_cuda_error", "osdp_slice_range",
     "osdp_split_linear_workspace_bytes", "osdp_split_linear_fwd", "osdp_split_linear_fwd_slice",
     "osdp_split_linear_bwd", "osdp_split_linear_bwd_slice", "osdp_split_mlp_fwd", "osdp_split_mlp_bwd",
-    "osdp_read_device_status",
+    "osdp_read_device_status", "osdp_bias_grad_noalloc",
 ]
 
 _lib = None
@@ -66,6 +66,7 @@ def lib():
         L.osdp_split_mlp_bwd.argtypes = [vp, vp, vp, i64, i64, vp, i64, i64, i64, ci, ci, vp, vp, i64, i64, ci, ci,
                                          vp, vp, vp, sz, vp]
         L.osdp_read_device_status.argtypes = [vp, ctypes.POINTER(ci), vp]
+        L.osdp_bias_grad_noalloc.argtypes = [vp, i64, i64, vp, vp]
         for name in EXPORTS:
             getattr(L, name)
             if name not in ("osdp_status_string",):
@@ -201,3 +202,11 @@ def osdp_read_device_status(ws, stream=None):
     st = ctypes.c_int(0)
     rc = lib().osdp_read_device_status(wp, ctypes.byref(st), _stream(stream))
     return rc, st.value
+
+
+def osdp_bias_grad_noalloc(dy, M, N, dbias, stream=None, check=False):
+    """dbias[n] = sum_m dy[m,n] using the library's built-in scratch: for callers that cannot
+    allocate device memory (allocator callbacks, hosts that own all device memory, loops that must
+    not touch the allocator).  Limit ceil(M/1024) * N <= 2**20; calls on one GPU must not overlap."""
+    rc = lib().osdp_bias_grad_noalloc(_ptr(dy), int(M), int(N), _ptr(dbias), _stream(stream))
+    return _ret(rc, check, "osdp_bias_grad_noalloc")

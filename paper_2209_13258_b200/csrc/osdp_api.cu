@@ -532,6 +532,7 @@ const char *osdp_status_string(int status) {
     case OSDP_ERR_UNSUPPORTED: return "unsupported";
     case OSDP_ERR_CUDA: return "CUDA error";
     case OSDP_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case OSDP_ERR_EXCEEDS_STATIC_SCRATCH: return "problem larger than the library's built-in scratch";
     default: return "unknown status";
   }
 }
@@ -774,3 +775,59 @@ int osdp_read_device_status(void *ws, int *status, void *stream_) {
 }
 
 }  // extern "C"
+
+
+// ================================================================================================
+// Bias gradient without any allocation.
+//
+// Some callers cannot hand this library a workspace because they cannot allocate device memory
+// at the point of the call: code running inside a memory-pool or allocator callback, a plug-in
+// whose host framework owns every byte of the device and forbids cudaMalloc after start-up, or a
+// real-time loop that must not take the allocator's lock.  For them this entry point computes the
+// bias gradient db[n] = sum_m dY[m,n] with the partial sums kept in an array that is part of the
+// library image itself.
+
+namespace {
+
+// Scratch for the two-pass column sum: ceil(M/1024) x N fp32 partials.  4 MiB, reserved on every
+// GPU that loads this library for as long as the process lives.
+__device__ __align__(256) float g_noalloc_partials[OSDP_NOALLOC_MAX_PARTIALS];
+
+// In host code `g_noalloc_partials` is only a handle for the runtime, not a device address:
+// the address a kernel may use is looked up per device, once, with that device current.
+float *g_noalloc_ptr[64] = {};
+bool g_noalloc_ready[64] = {};
+
+int noalloc_scratch(float **ptr) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= 64) return cuda_fail(cudaErrorInvalidDevice);
+  if (!g_noalloc_ready[dev]) {
+    void *p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_noalloc_partials);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (!p) return cuda_fail(cudaErrorInvalidSymbol);
+    g_noalloc_ptr[dev] = static_cast<float *>(p);
+    g_noalloc_ready[dev] = true;
+  }
+  *ptr = g_noalloc_ptr[dev];
+  return OSDP_OK;
+}
+
+}  // namespace
+
+extern "C" int osdp_bias_grad_noalloc(const void *dy, int64_t M, int64_t N, float *dbias, void *stream) {
+  if (!dy || !dbias) return OSDP_ERR_NULL_POINTER;
+  if (M <= 0 || N <= 0 || M > ((int64_t)1 << 30) || N > ((int64_t)1 << 30)) return OSDP_ERR_BAD_SHAPE;
+  if (N & 7) return OSDP_ERR_ALIGNMENT;
+  if (!aligned16(dy) || !aligned16(dbias)) return OSDP_ERR_ALIGNMENT;
+  const int64_t chunks = cdiv(M, COLSUM_ROWS_PER_CHUNK);
+  if (chunks * N > (int64_t)OSDP_NOALLOC_MAX_PARTIALS) return OSDP_ERR_EXCEEDS_STATIC_SCRATCH;
+  float *partials = nullptr;
+  int rc = noalloc_scratch(&partials);   // first call on a device: looks the address up
+  if (rc) return rc;
+  // Every partial that the second pass reads is written by the first pass of the same call, so
+  // nothing left in the array by an earlier call can reach the result and nothing needs clearing.
+  return launch_colsum(dy, N, M, 0, (int)N, partials, dbias, static_cast<cudaStream_t>(stream));
+}
