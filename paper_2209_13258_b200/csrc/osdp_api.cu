@@ -168,66 +168,108 @@ struct GemmCall {
   int *status;
 };
 
-int encode3d(CUtensorMap *m, const void *base, const cuuint64_t dims[3], const cuuint64_t strides_bytes[2],
-             const cuuint32_t box[3]) {
+int encode3d(CUtensorMap *m, CUtensorMapDataType dt, const void *base, const cuuint64_t dims[3],
+             const cuuint64_t strides_bytes[2], const cuuint32_t box[3], bool swizzle = true) {
   EncodeTiledFn fn;
   int rc = get_encode_fn(&fn);
   if (rc) return rc;
   const cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides_bytes, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = fn(m, dt, 3, const_cast<void *>(base), dims, strides_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return cu_fail(r);
   return OSDP_OK;
 }
 
-// Builds the two 3-D maps of one operand.  The slice index is a tensor coordinate: for slices
-// 0..k-2 the map has a dimension of extent k-1 and stride L (in the cut dimension's units); the
-// last slice, which may be shorter, gets a map of its own so that out-of-range elements are
-// zero-filled instead of running into the neighbouring slice.
-int make_operand_maps(const Operand &op, bool is_a, int mode, int64_t L, int k, int tile_rows, CUtensorMap *main_map,
-                      CUtensorMap *tail_map, int *sc_mul) {
-  const bool mid = op.mn_major ? (mode == (is_a ? MODE_ROWS : MODE_COLS)) : (mode == MODE_RED);
-  const bool role_sliced = is_a ? (mode == MODE_ROWS || mode == MODE_RED) : (mode == MODE_COLS || mode == MODE_RED);
-  const bool cut = role_sliced && op.whole && k > 1;
-  *sc_mul = cut ? 1 : 0;
-  const cuuint32_t box_outer = op.mn_major ? (cuuint32_t)BK : (cuuint32_t)tile_rows;
-  const char *base = static_cast<const char *>(op.base);
-  const cuuint64_t ldb = (cuuint64_t)op.ld * 2;
+// A row-major matrix view [outer][inner] (leading dimension ld, elements of elem_bytes) as the
+// two 3-D maps the kernel uses.  The slice index is a tensor coordinate: for slices 0..k-2 the map
+// has a dimension of extent k-1 and stride L (in the cut dimension's units); the last slice, which
+// may be shorter, gets a map of its own so that out-of-range elements are zero-filled on loads and
+// dropped on stores instead of running into the neighbouring slice.
+//   mid : the slice coordinate is dimension 1 (the slices cut the contiguous dimension), else 2
+//   cut : the view is the whole matrix and is cut into k slices of length L; otherwise both maps
+//         describe the view as it is (slice extent 1)
+struct ViewSpec {
+  const void *base;
+  int elem_bytes;
+  CUtensorMapDataType dt;
+  int64_t inner, outer, ld;
+  bool mid, cut;
+  int64_t L;
+  int k;
+  cuuint32_t box_inner, box_outer;
+};
+
+int make_sliced_maps(const ViewSpec &v, CUtensorMap *main_map, CUtensorMap *tail_map) {
+  const char *base = static_cast<const char *>(v.base);
+  const cuuint64_t es = (cuuint64_t)v.elem_bytes;
+  const cuuint64_t ldb = (cuuint64_t)v.ld * es;
   int rc;
-  if (!cut) {
-    if (mid) {
-      const cuuint64_t dims[3] = {(cuuint64_t)op.inner, 1, (cuuint64_t)op.outer};
-      const cuuint64_t str[2] = {(cuuint64_t)op.inner * 2, ldb};
-      const cuuint32_t box[3] = {64, 1, box_outer};
-      rc = encode3d(tail_map, base, dims, str, box);
+  if (!v.cut) {
+    if (v.mid) {
+      const cuuint64_t dims[3] = {(cuuint64_t)v.inner, 1, (cuuint64_t)v.outer};
+      const cuuint64_t str[2] = {(cuuint64_t)v.inner * es, ldb};
+      const cuuint32_t box[3] = {v.box_inner, 1, v.box_outer};
+      rc = encode3d(tail_map, v.dt, base, dims, str, box);
     } else {
-      const cuuint64_t dims[3] = {(cuuint64_t)op.inner, (cuuint64_t)op.outer, 1};
-      const cuuint64_t str[2] = {ldb, ldb * (cuuint64_t)op.outer};
-      const cuuint32_t box[3] = {64, box_outer, 1};
-      rc = encode3d(tail_map, base, dims, str, box);
+      const cuuint64_t dims[3] = {(cuuint64_t)v.inner, (cuuint64_t)v.outer, 1};
+      const cuuint64_t str[2] = {ldb, ldb * (cuuint64_t)v.outer};
+      const cuuint32_t box[3] = {v.box_inner, v.box_outer, 1};
+      rc = encode3d(tail_map, v.dt, base, dims, str, box);
     }
     if (rc) return rc;
     *main_map = *tail_map;
     return OSDP_OK;
   }
-  if (mid) {   // the slices cut the contiguous dimension
-    const cuuint64_t str[2] = {(cuuint64_t)L * 2, ldb};
-    const cuuint32_t box[3] = {64, 1, box_outer};
-    const cuuint64_t dims_main[3] = {(cuuint64_t)L, (cuuint64_t)(k - 1), (cuuint64_t)op.outer};
-    rc = encode3d(main_map, base, dims_main, str, box);
+  const int64_t k1 = v.k - 1;
+  if (v.mid) {   // the slices cut the contiguous dimension
+    const cuuint64_t str[2] = {(cuuint64_t)v.L * es, ldb};
+    const cuuint32_t box[3] = {v.box_inner, 1, v.box_outer};
+    const cuuint64_t dims_main[3] = {(cuuint64_t)v.L, (cuuint64_t)k1, (cuuint64_t)v.outer};
+    rc = encode3d(main_map, v.dt, base, dims_main, str, box);
     if (rc) return rc;
-    const cuuint64_t dims_tail[3] = {(cuuint64_t)(op.inner - (int64_t)(k - 1) * L), 1, (cuuint64_t)op.outer};
-    return encode3d(tail_map, base + (int64_t)(k - 1) * L * 2, dims_tail, str, box);
+    const cuuint64_t dims_tail[3] = {(cuuint64_t)(v.inner - k1 * v.L), 1, (cuuint64_t)v.outer};
+    return encode3d(tail_map, v.dt, base + k1 * v.L * (int64_t)es, dims_tail, str, box);
   }
   // the slices cut the strided dimension
-  const cuuint64_t str[2] = {ldb, ldb * (cuuint64_t)L};
-  const cuuint32_t box[3] = {64, box_outer, 1};
-  const cuuint64_t dims_main[3] = {(cuuint64_t)op.inner, (cuuint64_t)L, (cuuint64_t)(k - 1)};
-  rc = encode3d(main_map, base, dims_main, str, box);
+  const cuuint64_t str[2] = {ldb, ldb * (cuuint64_t)v.L};
+  const cuuint32_t box[3] = {v.box_inner, v.box_outer, 1};
+  const cuuint64_t dims_main[3] = {(cuuint64_t)v.inner, (cuuint64_t)v.L, (cuuint64_t)k1};
+  rc = encode3d(main_map, v.dt, base, dims_main, str, box);
   if (rc) return rc;
-  const cuuint64_t dims_tail[3] = {(cuuint64_t)op.inner, (cuuint64_t)(op.outer - (int64_t)(k - 1) * L), 1};
-  return encode3d(tail_map, base + (int64_t)(k - 1) * L * (int64_t)ldb, dims_tail, str, box);
+  const cuuint64_t dims_tail[3] = {(cuuint64_t)v.inner, (cuuint64_t)(v.outer - k1 * v.L), 1};
+  return encode3d(tail_map, v.dt, base + k1 * v.L * (int64_t)ldb, dims_tail, str, box);
+}
+
+int make_operand_maps(const Operand &op, bool is_a, int mode, int64_t L, int k, int tile_rows, CUtensorMap *main_map,
+                      CUtensorMap *tail_map, int *sc_mul) {
+  ViewSpec v;
+  v.base = op.base; v.elem_bytes = 2; v.dt = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+  v.inner = op.inner; v.outer = op.outer; v.ld = op.ld;
+  v.mid = op.mn_major ? (mode == (is_a ? MODE_ROWS : MODE_COLS)) : (mode == MODE_RED);
+  const bool role_sliced = is_a ? (mode == MODE_ROWS || mode == MODE_RED) : (mode == MODE_COLS || mode == MODE_RED);
+  v.cut = role_sliced && op.whole && k > 1;
+  v.L = L; v.k = k;
+  v.box_inner = 64;
+  v.box_outer = op.mn_major ? (cuuint32_t)BK : (cuuint32_t)tile_rows;
+  *sc_mul = v.cut ? 1 : 0;
+  return make_sliced_maps(v, main_map, tail_map);
+}
+
+// Output-side maps: boxes of 32 rows x 128 bytes written by one epilogue warp.
+int make_output_maps(void *base, bool fp32, int64_t P, int64_t Q, int64_t ld, int mode, int64_t L, int k,
+                     CUtensorMap *main_map, CUtensorMap *tail_map, int *sc_mul) {
+  ViewSpec v;
+  v.base = base; v.elem_bytes = fp32 ? 4 : 2;
+  v.dt = fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+  v.inner = Q; v.outer = P; v.ld = ld;
+  v.mid = (mode == MODE_COLS);
+  v.cut = (mode == MODE_COLS || mode == MODE_ROWS) && k > 1;
+  v.L = L; v.k = k;
+  v.box_inner = fp32 ? 32 : 64;
+  v.box_outer = 32;
+  if (sc_mul) *sc_mul = v.cut ? 1 : 0;
+  return make_sliced_maps(v, main_map, tail_map);
 }
 
 template <int BN, bool A_MN, bool B_MN>
@@ -279,6 +321,29 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   p.mode = c.mode; p.L = (int)c.L; p.k_total = c.k_total; p.s_begin = c.s_begin; p.s_end = c.s_end;
   p.epi = c.epi;
   p.status = c.status;
+  // Outputs leave through TMA unless the epilogue has to read a second tensor element-wise.
+  p.tma_epilogue = (c.epi.gz == nullptr) ? 1 : 0;
+  if (p.tma_epilogue) {
+    rc = make_output_maps(c.epi.out, c.epi.out_fp32 != 0, c.P, c.Q, c.epi.ld_out, c.mode, c.L, c.k_total, &p.out_main,
+                          &p.out_tail, &p.out_sc_mul);
+    if (rc) return rc;
+    if (c.epi.z_save) {
+      rc = make_output_maps(c.epi.z_save, false, c.P, c.Q, c.epi.ld_z, c.mode, c.L, c.k_total, &p.z_main, &p.z_tail,
+                            nullptr);
+      if (rc) return rc;
+    }
+    if (c.mode == MODE_RED && c.k_total > 1) {
+      CUtensorMap unused;
+      rc = make_output_maps(c.epi.carry, true, c.P, c.Q, c.epi.ld_carry, MODE_NONE, c.L, 1, &unused, &p.carry_map,
+                            nullptr);
+      if (rc) return rc;
+      const cuuint64_t dims[3] = {(cuuint64_t)c.Q, (cuuint64_t)c.P, 1};
+      const cuuint64_t str[2] = {(cuuint64_t)c.epi.ld_carry * 4, (cuuint64_t)c.epi.ld_carry * 4 * (cuuint64_t)c.P};
+      const cuuint32_t box[3] = {(cuuint32_t)bn, 32, 1};
+      rc = encode3d(&p.carry_pf_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, c.epi.carry, dims, str, box, false);
+      if (rc) return rc;
+    }
+  }
 
   // Work items of this launch -> grid size (one CTA per SM at most).
   int64_t items;

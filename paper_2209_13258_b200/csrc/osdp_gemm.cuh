@@ -64,6 +64,11 @@ struct GemmParams {
   int k_total;               // number of slices of the operator
   int s_begin, s_end;        // slices processed by this launch
   int a_sc_mul, b_sc_mul;    // 1: the operand map has a slice coordinate; 0: the operand is one slice already
+  // Output-side maps (3-D, same slice-coordinate scheme): final output, saved pre-activation, fp32 carry.
+  CUtensorMap out_main, out_tail, z_main, z_tail, carry_map;
+  CUtensorMap carry_pf_map;  // same tensor as carry_map, unswizzled box of 32 rows x BN columns, for L2 prefetch
+  int out_sc_mul;
+  int tma_epilogue;          // 1: outputs leave through shared-memory staging + TMA; 0: direct stores
   Epilogue epi;
   int *status;               // device status word or null
 };
@@ -136,6 +141,34 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
       "[%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
+}
+// Shared -> global tensor store / reduce-add; completion is tracked in bulk async-groups of the issuing thread.
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap *map, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+}
+// Asks the memory system to bring a box of a tensor into L2 (no shared-memory destination, no completion).
+__device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap *map, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ float4 ld_shared_f4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
 }
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols)
@@ -219,7 +252,9 @@ struct SmemLayout {
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
-  static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+  static constexpr int STG_OFFSET = STAGES * STAGE_BYTES;   // epilogue staging: 4 warps x 2 x 4 KB
+  static constexpr int STG_BYTES = 4 * 2 * 4096;
+  static constexpr int BAR_OFFSET = STG_OFFSET + STG_BYTES;
   static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;   // barriers + alignment slack
   static constexpr int TMEM_COLS = 2 * BN;
 };
@@ -234,6 +269,7 @@ struct Work {
   int kblocks;               // reduction blocks of this slice
   int a_row, b_col;          // TMA coordinates (slice-relative where that dimension is sliced)
   int carry_in, carry_out;
+  int first_of_slice;        // MODE_RED: this CTA's first tile of slice s
 };
 
 __device__ __forceinline__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
@@ -253,7 +289,9 @@ __device__ __forceinline__ bool get_work(const GemmParams &p, int i, Work &w) {
     t = bid + (i - srel * n_my) * G;
     rows = p.P;
     cols = p.Q;
+    w.first_of_slice = (i == srel * n_my);
   } else {
+    w.first_of_slice = 0;
     const int rows_full = (p.mode == MODE_ROWS) ? p.L : p.P;
     const int cols_full = (p.mode == MODE_COLS) ? p.L : p.Q;
     const int t_full = ceil_div(rows_full, BM) * ceil_div(cols_full, BN);
@@ -420,12 +458,18 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
       mbar_init(tfull_bar(b), 1);
       mbar_init(tempty_bar(b), 4);
     }
+    for (int b = 0; b < 8; ++b) mbar_init(bar_base + 8u * (2 * SL::STAGES + 5 + b), 1);   // carry prefetch, 2 per epilogue warp
     *abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&p.a_main);
     prefetch_tmap(&p.a_tail);
     prefetch_tmap(&p.b_main);
     prefetch_tmap(&p.b_tail);
+    if (p.tma_epilogue) {
+      prefetch_tmap(&p.out_main);
+      prefetch_tmap(&p.out_tail);
+      prefetch_tmap(&p.carry_map);
+    }
   }
   if (warp == 2) {
     tmem_alloc(smem_u32(tmem_holder), SL::TMEM_COLS);
@@ -541,7 +585,20 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ epilogue
+    // Each warp owns 32 rows of the tile and two 4 KB staging buffers (32 rows x 128 bytes, 128-byte
+    // swizzle).  Outputs leave as TMA stores (or reduce-adds) of 32 x 128-byte boxes, which the
+    // tensor maps clip at the end of the matrix or of the slice.  The carry of a summed output:
+    // slice 0 stores the fp32 partial, later slices reduce-add theirs into it (the addition is
+    // done by the memory system, nothing is read back), the last slice prefetches the carry
+    // with TMA loads, adds its own partial and writes the final result.
     const int quarter = warp & 3;
+    const uint32_t stg = smem_base + SL::STG_OFFSET + (uint32_t)quarter * 8192u;
+    const uint32_t row_off = (uint32_t)lane * 128u;
+    const uint32_t swz = (uint32_t)(lane & 7);
+    const bool out_sliced = (p.mode == MODE_COLS) || (p.mode == MODE_ROWS);
+    const bool out_mid = (p.mode == MODE_COLS);
+    uint32_t n_store = 0;   // staged boxes issued by this warp (selects the staging buffer)
+    uint32_t n_cload = 0;   // carry boxes loaded by this warp
     bool ok = true;
     Work w;
     for (int i = 0; ok && get_work<BN>(p, i, w); ++i) {
@@ -550,25 +607,230 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
       ok = mbar_wait(tfull_bar(buf), bphase, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE);
       if (!ok) break;
       tc_fence_after();
-      const long long row = (long long)w.row0 + quarter * 32 + lane;
+      const int wrow0 = w.row0 + quarter * 32;
+      const long long row = (long long)wrow0 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
+      if (p.tma_epilogue && p.mode == MODE_RED && lane == 0) {
+        // The carry of this CTA's next tile is touched one main loop from now: have it in L2 by then.
+        Work nx;
+        if (get_work<BN>(p, i + 1, nx) && nx.carry_in)
+          tma_prefetch_l2_3d(&p.carry_pf_map, nx.col0, nx.row0 + quarter * 32, 0);
+      }
+      if (!p.tma_epilogue) {
+        // direct stores from registers (used when the epilogue also reads a second tensor)
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        const int cbase = w.col0 + c * 32;
-        if (cbase >= w.col_end) break;
-        uint32_t v[32];
-        tmem_ld_x32(taddr + (uint32_t)(c * 32), v);
-        tmem_ld_wait();
-        if (row < w.row_end) {
+        for (int c = 0; c < BN / 32; ++c) {
+          const int cbase = w.col0 + c * 32;
+          if (cbase >= w.col_end) break;
+          uint32_t v[32];
+          tmem_ld_x32(taddr + (uint32_t)(c * 32), v);
+          tmem_ld_wait();
+          if (row < w.row_end) {
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            const int col = cbase + g * 8;
-            if (col < w.col_end) {
+            for (int g = 0; g < 4; ++g) {
+              const int col = cbase + g * 8;
+              if (col < w.col_end) {
+                float f[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[g * 8 + j]);
+                epilogue8(p.epi, row, col, f, w.carry_in, w.carry_out);
+              }
+            }
+          }
+        }
+      } else if (wrow0 < w.row_end) {
+        const bool tail = (w.s == p.k_total - 1);
+        const int sc = (out_sliced && !tail) ? w.s * p.out_sc_mul : 0;
+        const CUtensorMap *omap = (out_sliced && !tail) ? &p.out_main : &p.out_tail;
+        const CUtensorMap *zmap = (out_sliced && !tail) ? &p.z_main : &p.z_tail;
+        const int r_in = w.a_row + quarter * 32;
+        // One staged box: wait until the buffer's previous box has been read, fill it, hand it to TMA.
+        auto stage_begin = [&]() -> uint32_t {
+          if (lane == 0) bulk_wait_read_1();
+          __syncwarp();
+          return stg + (n_store & 1u) * 4096u;
+        };
+        auto stage_issue = [&](const CUtensorMap *map, uint32_t src, int col_in, bool reduce) {
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            if (out_mid && map != &p.carry_map) {
+              if (reduce) tma_reduce_add_3d(map, src, col_in, sc, r_in);
+              else tma_store_3d(map, src, col_in, sc, r_in);
+            } else {
+              const int c2 = (map == &p.carry_map) ? 0 : sc;
+              if (reduce) tma_reduce_add_3d(map, src, col_in, r_in, c2);
+              else tma_store_3d(map, src, col_in, r_in, c2);
+            }
+            bulk_commit();
+          }
+          ++n_store;
+        };
+        if (w.carry_out || (w.carry_in && w.first_of_slice)) {
+          // Slice boundary: everything this warp sent for the previous slice must have landed
+          // before the same addresses are added to (or read) again.
+          if (w.first_of_slice && w.carry_in) {
+            if (lane == 0) bulk_wait_all();
+            __syncwarp();
+          }
+        }
+        if (w.carry_out) {
+          // fp32 partial -> carry, 32 columns (128 bytes per row) per box
+#pragma unroll 1
+          for (int c = 0; c < BN / 32; ++c) {
+            const int cbase = w.col0 + c * 32;
+            if (cbase >= w.col_end) break;
+            uint32_t v[32];
+            tmem_ld_x32(taddr + (uint32_t)(c * 32), v);
+            tmem_ld_wait();
+            const uint32_t dst = stage_begin();
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              st_shared_v4(dst + row_off + (((uint32_t)j ^ swz) << 4), v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            stage_issue(&p.carry_map, dst, cbase, w.carry_in != 0);
+          }
+        } else if (w.carry_in) {
+          // last slice: carry (prefetched by TMA, one box ahead) + accumulator -> bias/act -> out
+          const uint32_t cbar = bar_base + 8u * (2 * SL::STAGES + 5 + quarter * 2);
+          int nchunks = (w.col_end - w.col0 + 31) / 32;
+          if (nchunks > BN / 32) nchunks = BN / 32;
+          auto issue_load = [&](int c) {
+            if (lane == 0) {
+              const uint32_t b = n_cload & 1u;
+              mbar_expect_tx(cbar + 8u * b, 4096u);
+              tma_load_3d(stg + b * 4096u, &p.carry_map, cbar + 8u * b, w.col0 + c * 32, wrow0, 0);
+            }
+            ++n_cload;
+          };
+          const uint32_t first = n_cload;
+          issue_load(0);
+#pragma unroll 1
+          for (int c = 0; c < nchunks; ++c) {
+            if (c + 1 < nchunks) issue_load(c + 1);
+            uint32_t v[32];
+            tmem_ld_x32(taddr + (uint32_t)(c * 32), v);
+            tmem_ld_wait();
+            const uint32_t n = first + (uint32_t)c;
+            ok = mbar_wait(cbar + 8u * (n & 1u), (n >> 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE);
+            if (!ok) break;
+            const uint32_t src = stg + (n & 1u) * 4096u + row_off;
+            const int cbase = w.col0 + c * 32;
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              const float4 c0 = ld_shared_f4(src + (((uint32_t)(2 * g) ^ swz) << 4));
+              const float4 c1 = ld_shared_f4(src + (((uint32_t)(2 * g + 1) ^ swz) << 4));
+              const int col = cbase + g * 8;
+              if (row < w.row_end && col < w.col_end) {
+                float f[8];
+                f[0] = __uint_as_float(v[g * 8 + 0]) + c0.x; f[1] = __uint_as_float(v[g * 8 + 1]) + c0.y;
+                f[2] = __uint_as_float(v[g * 8 + 2]) + c0.z; f[3] = __uint_as_float(v[g * 8 + 3]) + c0.w;
+                f[4] = __uint_as_float(v[g * 8 + 4]) + c1.x; f[5] = __uint_as_float(v[g * 8 + 5]) + c1.y;
+                f[6] = __uint_as_float(v[g * 8 + 6]) + c1.z; f[7] = __uint_as_float(v[g * 8 + 7]) + c1.w;
+                epilogue8(p.epi, row, col, f, 0, 0);
+              }
+            }
+            __syncwarp();   // the buffer may be refilled once every lane has read it
+          }
+          if (!ok) break;
+        } else if (p.epi.out_fp32) {
+          // fp32 output, 32 columns per box; += is a reduce-add
+#pragma unroll 1
+          for (int c = 0; c < BN / 32; ++c) {
+            const int cbase = w.col0 + c * 32;
+            if (cbase >= w.col_end) break;
+            uint32_t v[32];
+            tmem_ld_x32(taddr + (uint32_t)(c * 32), v);
+            tmem_ld_wait();
+            if (p.epi.bias) {
+#pragma unroll
+              for (int g = 0; g < 4; ++g) {
+                if (cbase + g * 8 < w.col_end) {
+                  const float4 b0 = *reinterpret_cast<const float4 *>(p.epi.bias + cbase + g * 8);
+                  const float4 b1 = *reinterpret_cast<const float4 *>(p.epi.bias + cbase + g * 8 + 4);
+                  v[g * 8 + 0] = __float_as_uint(__uint_as_float(v[g * 8 + 0]) + b0.x);
+                  v[g * 8 + 1] = __float_as_uint(__uint_as_float(v[g * 8 + 1]) + b0.y);
+                  v[g * 8 + 2] = __float_as_uint(__uint_as_float(v[g * 8 + 2]) + b0.z);
+                  v[g * 8 + 3] = __float_as_uint(__uint_as_float(v[g * 8 + 3]) + b0.w);
+                  v[g * 8 + 4] = __float_as_uint(__uint_as_float(v[g * 8 + 4]) + b1.x);
+                  v[g * 8 + 5] = __float_as_uint(__uint_as_float(v[g * 8 + 5]) + b1.y);
+                  v[g * 8 + 6] = __float_as_uint(__uint_as_float(v[g * 8 + 6]) + b1.z);
+                  v[g * 8 + 7] = __float_as_uint(__uint_as_float(v[g * 8 + 7]) + b1.w);
+                }
+              }
+            }
+            if (p.epi.act != ACT_NONE) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(gelu_f(__uint_as_float(v[j]), p.epi.act));
+            }
+            const uint32_t dst = stage_begin();
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              st_shared_v4(dst + row_off + (((uint32_t)j ^ swz) << 4), v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            stage_issue(omap, dst, w.b_col + c * 32, p.epi.accumulate != 0);
+          }
+        } else {
+          // bf16 output, 64 columns (128 bytes per row) per box
+#pragma unroll 1
+          for (int c = 0; c < (BN + 63) / 64; ++c) {
+            const int cbase = w.col0 + c * 64;
+            if (cbase >= w.col_end) break;
+            uint32_t v[64];
+            {
+              uint32_t lo[32], hi[32];
+              tmem_ld_x32(taddr + (uint32_t)(c * 64), lo);
+              if (BN >= 64) tmem_ld_x32(taddr + (uint32_t)(c * 64 + 32), hi);
+              tmem_ld_wait();
+#pragma unroll
+              for (int j = 0; j < 32; ++j) { v[j] = lo[j]; v[32 + j] = hi[j]; }
+            }
+            uint4 packed[8];
+            if (p.epi.bias) {
+#pragma unroll
+              for (int g = 0; g < 8; ++g) {
+                if (cbase + g * 8 < w.col_end) {
+                  const float4 b0 = *reinterpret_cast<const float4 *>(p.epi.bias + cbase + g * 8);
+                  const float4 b1 = *reinterpret_cast<const float4 *>(p.epi.bias + cbase + g * 8 + 4);
+                  v[g * 8 + 0] = __float_as_uint(__uint_as_float(v[g * 8 + 0]) + b0.x);
+                  v[g * 8 + 1] = __float_as_uint(__uint_as_float(v[g * 8 + 1]) + b0.y);
+                  v[g * 8 + 2] = __float_as_uint(__uint_as_float(v[g * 8 + 2]) + b0.z);
+                  v[g * 8 + 3] = __float_as_uint(__uint_as_float(v[g * 8 + 3]) + b0.w);
+                  v[g * 8 + 4] = __float_as_uint(__uint_as_float(v[g * 8 + 4]) + b1.x);
+                  v[g * 8 + 5] = __float_as_uint(__uint_as_float(v[g * 8 + 5]) + b1.y);
+                  v[g * 8 + 6] = __float_as_uint(__uint_as_float(v[g * 8 + 6]) + b1.z);
+                  v[g * 8 + 7] = __float_as_uint(__uint_as_float(v[g * 8 + 7]) + b1.w);
+                }
+              }
+            }
+            if (p.epi.z_save) {
+#pragma unroll
+              for (int g = 0; g < 8; ++g) {
+                float f[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[g * 8 + j]);
+                packed[g] = pack_bf16x8(f);
+              }
+              const uint32_t dstz = stage_begin();
+#pragma unroll
+              for (int g = 0; g < 8; ++g)
+                st_shared_v4(dstz + row_off + (((uint32_t)g ^ swz) << 4), packed[g].x, packed[g].y, packed[g].z, packed[g].w);
+              stage_issue(zmap, dstz, w.b_col + c * 64, false);
+            }
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
               float f[8];
 #pragma unroll
               for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[g * 8 + j]);
-              epilogue8(p.epi, row, col, f, w.carry_in, w.carry_out);
+              if (p.epi.act != ACT_NONE) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) f[j] = gelu_f(f[j], p.epi.act);
+              }
+              packed[g] = pack_bf16x8(f);
             }
+            const uint32_t dst = stage_begin();
+#pragma unroll
+            for (int g = 0; g < 8; ++g)
+              st_shared_v4(dst + row_off + (((uint32_t)g ^ swz) << 4), packed[g].x, packed[g].y, packed[g].z, packed[g].w);
+            stage_issue(omap, dst, w.b_col + c * 64, p.epi.accumulate != 0);
           }
         }
       }
@@ -576,6 +838,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(buf));
     }
+    // Nothing this warp handed to TMA may still be reading shared memory (or be in flight) at exit.
+    if (lane == 0) bulk_wait_all();
+    __syncwarp();
   }
 
   tc_fence_before();
