@@ -272,29 +272,60 @@ int make_output_maps(void *base, bool fp32, int64_t P, int64_t Q, int64_t ld, in
   return make_sliced_maps(v, main_map, tail_map);
 }
 
-template <int BN, bool A_MN, bool B_MN>
-int launch_variant(const GemmParams &p, int grid, cudaStream_t stream) {
+// One kernel variant: sets its attributes once per device, sizes the grid and launches.
+// `units` = work items of the launch (tiles, summed over slices for concatenated outputs).
+template <int BN, bool A_MN, bool B_MN, bool CTA2>
+int launch_variant(const GemmParams &p, int64_t units, int sms, cudaStream_t stream) {
   static bool attr_done[64] = {};
+  static int max_clusters[64] = {};
+  using SL = SmemLayout<BN, CTA2>;
+  auto kernel = gemm_kernel<BN, A_MN, B_MN, CTA2>;
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return cuda_fail(e);
-  if (!attr_done[dev & 63]) {
-    e = cudaFuncSetAttribute(gemm_kernel<BN, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             SmemLayout<BN>::TOTAL);
+  dev &= 63;
+  if (!attr_done[dev]) {
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::TOTAL);
     if (e != cudaSuccess) return cuda_fail(e);
-    attr_done[dev & 63] = true;
+    if (CTA2) {
+      cudaLaunchConfig_t q = {};
+      q.gridDim = dim3(2 * sms, 1, 1);
+      q.blockDim = dim3(NUM_THREADS, 1, 1);
+      q.dynamicSmemBytes = SL::TOTAL;
+      cudaLaunchAttribute qa[1];
+      qa[0].id = cudaLaunchAttributeClusterDimension;
+      qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+      q.attrs = qa; q.numAttrs = 1;
+      int n = 0;
+      e = cudaOccupancyMaxActiveClusters(&n, kernel, &q);
+      if (e != cudaSuccess) return cuda_fail(e);
+      if (n < 1) return cuda_fail(cudaErrorLaunchOutOfResources);
+      max_clusters[dev] = n;
+    }
+    attr_done[dev] = true;
   }
-  gemm_kernel<BN, A_MN, B_MN><<<grid, NUM_THREADS, SmemLayout<BN>::TOTAL, stream>>>(p);
-  e = cudaGetLastError();
+  const int64_t cap = CTA2 ? max_clusters[dev] : sms;
+  const int n_units = (int)(units < cap ? units : cap);
+  if (n_units <= 0) return OSDP_OK;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(CTA2 ? 2 * n_units : n_units, 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = SL::TOTAL;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CTA2 ? 2 : 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  e = cudaLaunchKernelEx(&cfg, kernel, p);
   if (e != cudaSuccess) return cuda_fail(e);
   return OSDP_OK;
 }
 
-template <int BN>
-int launch_bn(const GemmParams &p, bool a_mn, bool b_mn, int grid, cudaStream_t stream) {
-  if (!a_mn && !b_mn) return launch_variant<BN, false, false>(p, grid, stream);
-  if (!a_mn && b_mn) return launch_variant<BN, false, true>(p, grid, stream);
-  if (a_mn && b_mn) return launch_variant<BN, true, true>(p, grid, stream);
+template <int BN, bool CTA2>
+int launch_bn(const GemmParams &p, bool a_mn, bool b_mn, int64_t units, int sms, cudaStream_t stream) {
+  if (!a_mn && !b_mn) return launch_variant<BN, false, false, CTA2>(p, units, sms, stream);
+  if (!a_mn && b_mn) return launch_variant<BN, false, true, CTA2>(p, units, sms, stream);
+  if (a_mn && b_mn) return launch_variant<BN, true, true, CTA2>(p, units, sms, stream);
   return OSDP_ERR_UNSUPPORTED;
 }
 
@@ -304,18 +335,22 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   int sms = 0;
   int rc = device_sms(&sms);
   if (rc) return rc;
-  // Tile width from the unsplit operator's shape: the same for every k, so that concatenated
+  // Tile shape from the unsplit operator's extents only: the same for every k, so that concatenated
   // outputs are computed by exactly the same instruction sequence whatever the split.
+  // Large operators: CTA pairs on 256 x 256 tiles.  Smaller ones: single CTAs, narrower tiles, so
+  // that there are enough tiles to occupy the SMs.
+  const bool pair = cdiv(c.bn_P, 2 * BM) * cdiv(c.bn_Q, 256) >= (int64_t)sms / 2;
   int bn = 64;
   const int64_t want = (int64_t)sms * 4 / 5;
-  if (cdiv(c.bn_P, BM) * cdiv(c.bn_Q, 256) >= want) bn = 256;
+  if (pair || cdiv(c.bn_P, BM) * cdiv(c.bn_Q, 256) >= want) bn = 256;
   else if (cdiv(c.bn_P, BM) * cdiv(c.bn_Q, 128) >= want) bn = 128;
+  const int tm = pair ? 2 * BM : BM;
 
   GemmParams p;
   memset(&p, 0, sizeof(p));
   rc = make_operand_maps(c.a, true, c.mode, c.L, c.k_total, BM, &p.a_main, &p.a_tail, &p.a_sc_mul);
   if (rc) return rc;
-  rc = make_operand_maps(c.b, false, c.mode, c.L, c.k_total, bn, &p.b_main, &p.b_tail, &p.b_sc_mul);
+  rc = make_operand_maps(c.b, false, c.mode, c.L, c.k_total, pair ? bn / 2 : bn, &p.b_main, &p.b_tail, &p.b_sc_mul);
   if (rc) return rc;
   p.P = (int)c.P; p.Q = (int)c.Q; p.R = (int)c.R;
   p.mode = c.mode; p.L = (int)c.L; p.k_total = c.k_total; p.s_begin = c.s_begin; p.s_end = c.s_end;
@@ -345,10 +380,10 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
     }
   }
 
-  // Work items of this launch -> grid size (one CTA per SM at most).
+  // Work items of this launch (one per scheduling unit and tile).
   int64_t items;
   if (c.mode == MODE_RED) {
-    items = cdiv(c.P, BM) * cdiv(c.Q, bn);
+    items = cdiv(c.P, tm) * cdiv(c.Q, bn);
   } else {
     const int64_t rows_full = (c.mode == MODE_ROWS) ? c.L : c.P;
     const int64_t cols_full = (c.mode == MODE_COLS) ? c.L : c.Q;
@@ -356,14 +391,13 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
     const int last = c.s_end - 1;
     const int64_t rows_last = (c.mode == MODE_ROWS) ? ((c.P - last * c.L) < c.L ? (c.P - last * c.L) : c.L) : c.P;
     const int64_t cols_last = (c.mode == MODE_COLS) ? ((c.Q - last * c.L) < c.L ? (c.Q - last * c.L) : c.L) : c.Q;
-    items = (int64_t)(nsl - 1) * cdiv(rows_full, BM) * cdiv(cols_full, bn) + cdiv(rows_last, BM) * cdiv(cols_last, bn);
+    items = (int64_t)(nsl - 1) * cdiv(rows_full, tm) * cdiv(cols_full, bn) + cdiv(rows_last, tm) * cdiv(cols_last, bn);
   }
-  const int grid = (int)(items < sms ? items : sms);
-  if (grid <= 0) return OSDP_OK;
+  if (pair) return launch_bn<256, true>(p, c.a.mn_major, c.b.mn_major, items, sms, stream);
   switch (bn) {
-    case 256: return launch_bn<256>(p, c.a.mn_major, c.b.mn_major, grid, stream);
-    case 128: return launch_bn<128>(p, c.a.mn_major, c.b.mn_major, grid, stream);
-    default: return launch_bn<64>(p, c.a.mn_major, c.b.mn_major, grid, stream);
+    case 256: return launch_bn<256, false>(p, c.a.mn_major, c.b.mn_major, items, sms, stream);
+    case 128: return launch_bn<128, false>(p, c.a.mn_major, c.b.mn_major, items, sms, stream);
+    default: return launch_bn<64, false>(p, c.a.mn_major, c.b.mn_major, items, sms, stream);
   }
 }
 

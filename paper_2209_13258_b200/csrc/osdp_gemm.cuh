@@ -160,7 +160,8 @@ __device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap *map, int c
                : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
@@ -170,15 +171,52 @@ __device__ __forceinline__ float4 ld_shared_f4(uint32_t addr) {
   asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
   return v;
 }
+// ---- CTA-pair (cluster of 2) forms.  The pair shares one MMA: the even CTA (rank 0) issues it.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+// Both CTAs of the pair load into their own shared memory; the bytes are counted on the
+// barrier of the even CTA (the barrier address with the pair bit cleared).
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0,
+                                                 int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar & 0xFEFFFFFFu), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t bar, uint32_t cta_rank) {
+  asm volatile(
+      "{\n\t.reg .b32 ra;\n\t"
+      "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
+      "mbarrier.arrive.shared::cluster.b64 _, [ra];\n\t}"
+      ::"r"(bar), "r"(cta_rank)
+      : "memory");
+}
+template <bool CTA2>
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols)
-               : "memory");
+  if (CTA2)
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols)
+                 : "memory");
+  else
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols)
+                 : "memory");
 }
+template <bool CTA2>
 __device__ __forceinline__ void tmem_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  if (CTA2) asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  else asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
 }
+template <bool CTA2>
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+  if (CTA2) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+  else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -186,19 +224,38 @@ __device__ __forceinline__ void tc_fence_before() {
 __device__ __forceinline__ void tc_fence_after() {
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
+template <bool CTA2>
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                           uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
+  if (CTA2)
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  else
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
 }
-// mbarrier arrives once every tcgen05.mma issued so far by this thread has completed.
+// mbarrier arrives once every tcgen05.mma issued so far by this thread has completed; in the
+// pair form the arrival is delivered to the same barrier in both CTAs.
+template <bool CTA2>
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
-               : "memory");
+  if (CTA2) {
+    const uint16_t mask = 3;
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"(mask)
+        : "memory");
+  } else {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+  }
 }
 __device__ __forceinline__ void tmem_ld_x32(uint32_t taddr, uint32_t (&v)[32]) {
   asm volatile(
@@ -240,20 +297,24 @@ __device__ __forceinline__ constexpr uint32_t desc_k_advance() {
   return MN_MAJOR ? (UMMA_K * 128) : (UMMA_K * 2);
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = BN.
-template <int BN, bool A_MN, bool B_MN>
+template <int UM, int BN, bool A_MN, bool B_MN>
 __device__ __forceinline__ constexpr uint32_t make_idesc() {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16) |
-         ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+         ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(UM >> 4) << 24);
 }
 
-template <int BN>
+template <int BN, bool CTA2>
 struct SmemLayout {
+  static constexpr int BNL = CTA2 ? BN / 2 : BN;   // B rows held by one CTA (a pair splits B between its CTAs)
   static constexpr int A_BYTES = BM * BK * 2;
-  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int B_BYTES = BNL * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
-  static constexpr int STG_OFFSET = STAGES * STAGE_BYTES;   // epilogue staging: 4 warps x 2 x 4 KB
-  static constexpr int STG_BYTES = 4 * 2 * 4096;
+  // Epilogue staging: STG_BUFS boxes of 4 KB per epilogue warp (boxes in flight to/from global memory).
+  static constexpr int STG_BUFS = 2;
+  static constexpr int STG_BYTES = 4 * STG_BUFS * 4096;
+  static constexpr int RING_BYTES = 229376 - STG_BYTES;
+  static constexpr int STAGES = (RING_BYTES / STAGE_BYTES) > 8 ? 8 : (RING_BYTES / STAGE_BYTES);
+  static constexpr int STG_OFFSET = STAGES * STAGE_BYTES;
   static constexpr int BAR_OFFSET = STG_OFFSET + STG_BYTES;
   static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;   // barriers + alignment slack
   static constexpr int TMEM_COLS = 2 * BN;
@@ -274,13 +335,14 @@ struct Work {
 
 __device__ __forceinline__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
-template <int BN>
-__device__ __forceinline__ bool get_work(const GemmParams &p, int i, Work &w) {
+// TM x BN is the tile of one scheduling unit (a CTA, or a CTA pair); bid / G are the unit's index
+// and the number of units in the grid.
+template <int TM, int BN>
+__device__ __forceinline__ bool get_work(const GemmParams &p, int i, int bid, int G, Work &w) {
   const int nsl = p.s_end - p.s_begin;
   int s, t, rows, cols;
   if (p.mode == MODE_RED) {
-    const int tiles = ceil_div(p.P, BM) * ceil_div(p.Q, BN);
-    const int bid = blockIdx.x, G = gridDim.x;
+    const int tiles = ceil_div(p.P, TM) * ceil_div(p.Q, BN);
     if (bid >= tiles) return false;
     const int n_my = (tiles - bid + G - 1) / G;
     const int srel = i / n_my;
@@ -294,28 +356,29 @@ __device__ __forceinline__ bool get_work(const GemmParams &p, int i, Work &w) {
     w.first_of_slice = 0;
     const int rows_full = (p.mode == MODE_ROWS) ? p.L : p.P;
     const int cols_full = (p.mode == MODE_COLS) ? p.L : p.Q;
-    const int t_full = ceil_div(rows_full, BM) * ceil_div(cols_full, BN);
-    const long long widx = (long long)blockIdx.x + (long long)i * gridDim.x;
+    const int t_full = ceil_div(rows_full, TM) * ceil_div(cols_full, BN);
+    const long long widx = (long long)bid + (long long)i * G;
     long long srel = widx / t_full;
     if (srel > nsl - 1) srel = nsl - 1;
     s = p.s_begin + (int)srel;
     const long long tl = widx - srel * t_full;
     rows = (p.mode == MODE_ROWS) ? min(p.L, p.P - s * p.L) : p.P;
     cols = (p.mode == MODE_COLS) ? min(p.L, p.Q - s * p.L) : p.Q;
-    if (tl >= (long long)ceil_div(rows, BM) * ceil_div(cols, BN)) return false;
+    if (tl >= (long long)ceil_div(rows, TM) * ceil_div(cols, BN)) return false;
     t = (int)tl;
   }
-  const int tiles_m = ceil_div(rows, BM), tiles_n = ceil_div(cols, BN);
-  const int group = GROUP_M * tiles_n;
+  const int tiles_m = ceil_div(rows, TM), tiles_n = ceil_div(cols, BN);
+  constexpr int GM = GROUP_M * BM / TM;   // same number of rows per group whatever the unit
+  const int group = GM * tiles_n;
   const int g = t / group;
-  const int first_m = g * GROUP_M;
-  const int gm = min(GROUP_M, tiles_m - first_m);
+  const int first_m = g * GM;
+  const int gm = min(GM, tiles_m - first_m);
   const int tm = first_m + (t - g * group) % gm;
   const int tn = (t - g * group) / gm;
   const int row_base = (p.mode == MODE_ROWS) ? s * p.L : 0;
   const int col_base = (p.mode == MODE_COLS) ? s * p.L : 0;
   w.s = s;
-  w.a_row = tm * BM;
+  w.a_row = tm * TM;
   w.b_col = tn * BN;
   w.row0 = row_base + w.a_row;
   w.col0 = col_base + w.b_col;
@@ -431,9 +494,19 @@ __device__ __forceinline__ void epilogue8(const Epilogue &e, long long row, int 
 // ------------------------------------------------------------------------------------------------
 // The kernel
 
-template <int BN, bool A_MN, bool B_MN>
+// CTA2 = true: the scheduling unit is a cluster of two CTAs working on a 256 x BN tile with one
+// tcgen05.mma.cta_group::2 issued by the even CTA.  Each CTA loads its own 128 rows of A and half
+// of the B tile (BN/2 rows), holds the accumulator of its 128 rows in its own tensor memory and
+// runs its own epilogue.  Per CTA a stage is 32 KB instead of 48 KB (6 stages instead of 4) and
+// half as many B bytes cross from L2 to shared memory per flop.
+template <int BN, bool A_MN, bool B_MN, bool CTA2>
 __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
-  using SL = SmemLayout<BN>;
+  using SL = SmemLayout<BN, CTA2>;
+  constexpr int TM = CTA2 ? 2 * BM : BM;
+  constexpr int BNL = SL::BNL;
+  const uint32_t rank = CTA2 ? cluster_ctarank() : 0u;
+  const int bid = CTA2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int G = CTA2 ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -456,9 +529,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull_bar(b), 1);
-      mbar_init(tempty_bar(b), 4);
+      mbar_init(tempty_bar(b), CTA2 ? 8 : 4);
     }
-    for (int b = 0; b < 8; ++b) mbar_init(bar_base + 8u * (2 * SL::STAGES + 5 + b), 1);   // carry prefetch, 2 per epilogue warp
+    for (int b = 0; b < 4 * SL::STG_BUFS; ++b) mbar_init(bar_base + 8u * (2 * SL::STAGES + 5 + b), 1);   // carry prefetch
     *abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&p.a_main);
@@ -472,11 +545,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
     }
   }
   if (warp == 2) {
-    tmem_alloc(smem_u32(tmem_holder), SL::TMEM_COLS);
-    tmem_relinquish();
+    tmem_alloc<CTA2>(smem_u32(tmem_holder), SL::TMEM_COLS);
+    tmem_relinquish<CTA2>();
   }
   tc_fence_before();
   __syncthreads();
+  if (CTA2) cluster_sync_all();   // the peer's barriers exist before anything is signalled across the pair
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
 
@@ -493,7 +567,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
     uint32_t armed = 0, armed_phase = 0;   // per-stage bookkeeping for the unwind path
     bool ok = true;
     Work w;
-    for (int i = 0; ok && get_work<BN>(p, i, w); ++i) {
+    for (int i = 0; ok && get_work<TM, BN>(p, i, bid, G, w); ++i) {
+      w.a_row += (int)rank * BM;            // this CTA's rows of the pair's tile
+      w.b_col += (int)rank * BNL;           // ... and its half of the B tile
       const bool tail = (w.s == p.k_total - 1);
       const CUtensorMap *amap = (a_sliced && !tail) ? &p.a_main : &p.a_tail;
       const CUtensorMap *bmap = (b_sliced && !tail) ? &p.b_main : &p.b_tail;
@@ -506,29 +582,33 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
           const uint32_t sa = smem_base + stage * SL::STAGE_BYTES;
           const uint32_t sb = sa + SL::A_BYTES;
           const uint32_t fb = full_bar(stage);
-          mbar_expect_tx(fb, SL::STAGE_BYTES);
+          if (!CTA2 || rank == 0) mbar_expect_tx(fb, SL::STAGE_BYTES * (CTA2 ? 2 : 1));
           const int kc = kb * BK;
+          auto tma_load = [&](uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2) {
+            if (CTA2) tma_load_3d_pair(dst, map, fb, c0, c1, c2);
+            else tma_load_3d(dst, map, fb, c0, c1, c2);
+          };
           if (A_MN) {
 #pragma unroll
             for (int j = 0; j < BM / 64; ++j) {
               const int in = w.a_row + j * 64;
-              if (a_mid) tma_load_3d(sa + j * (BK * 128), amap, fb, in, a_sc, kc);
-              else tma_load_3d(sa + j * (BK * 128), amap, fb, in, kc, a_sc);
+              if (a_mid) tma_load(sa + j * (BK * 128), amap, in, a_sc, kc);
+              else tma_load(sa + j * (BK * 128), amap, in, kc, a_sc);
             }
           } else {
-            if (a_mid) tma_load_3d(sa, amap, fb, kc, a_sc, w.a_row);
-            else tma_load_3d(sa, amap, fb, kc, w.a_row, a_sc);
+            if (a_mid) tma_load(sa, amap, kc, a_sc, w.a_row);
+            else tma_load(sa, amap, kc, w.a_row, a_sc);
           }
           if (B_MN) {
 #pragma unroll
-            for (int j = 0; j < BN / 64; ++j) {
+            for (int j = 0; j < BNL / 64; ++j) {
               const int in = w.b_col + j * 64;
-              if (b_mid) tma_load_3d(sb + j * (BK * 128), bmap, fb, in, b_sc, kc);
-              else tma_load_3d(sb + j * (BK * 128), bmap, fb, in, kc, b_sc);
+              if (b_mid) tma_load(sb + j * (BK * 128), bmap, in, b_sc, kc);
+              else tma_load(sb + j * (BK * 128), bmap, in, kc, b_sc);
             }
           } else {
-            if (b_mid) tma_load_3d(sb, bmap, fb, kc, b_sc, w.b_col);
-            else tma_load_3d(sb, bmap, fb, kc, w.b_col, b_sc);
+            if (b_mid) tma_load(sb, bmap, kc, b_sc, w.b_col);
+            else tma_load(sb, bmap, kc, w.b_col, b_sc);
           }
         }
         armed |= 1u << stage;
@@ -537,7 +617,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
         if (++stage == SL::STAGES) { stage = 0; phase ^= 1u; }
       }
     }
-    if (!ok) {
+    if (!ok && rank == 0) {
       // Unwinding: let the copies already issued land before the CTA's shared memory goes away.
       for (int st = 0; st < SL::STAGES; ++st) {
         if (!((armed >> st) & 1u)) continue;
@@ -547,14 +627,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
         }
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    constexpr uint32_t idesc = make_idesc<BN, A_MN, B_MN>();
+  } else if (warp == 1 && rank == 0) {
+    // ------------------------------------------------------------------ MMA issuer (even CTA of a pair)
+    constexpr uint32_t idesc = make_idesc<TM, BN, A_MN, B_MN>();
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;
     Work w;
-    for (int i = 0; ok && get_work<BN>(p, i, w); ++i) {
+    for (int i = 0; ok && get_work<TM, BN>(p, i, bid, G, w); ++i) {
       const int buf = i & 1;
       const uint32_t bphase = (uint32_t)(i >> 1) & 1u;
       ok = mbar_wait(tempty_bar(buf), bphase ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA);
@@ -572,12 +652,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
           const uint64_t bdesc = make_smem_desc<B_MN>(sb);
 #pragma unroll
           for (int kk = 0; kk < BK / UMMA_K; ++kk) {
-            umma_bf16(d_tmem, adesc + (uint64_t)((kk * desc_k_advance<A_MN>()) >> 4),
+            umma_bf16<CTA2>(d_tmem, adesc + (uint64_t)((kk * desc_k_advance<A_MN>()) >> 4),
                       bdesc + (uint64_t)((kk * desc_k_advance<B_MN>()) >> 4), idesc,
                       (kb > 0 || kk > 0) ? 1u : 0u);
           }
-          umma_commit(empty_bar(stage));                      // frees the stage when the MMAs retire
-          if (kb == w.kblocks - 1) umma_commit(tfull_bar(buf));   // accumulator complete
+          umma_commit<CTA2>(empty_bar(stage));                      // frees the stage when the MMAs retire
+          if (kb == w.kblocks - 1) umma_commit<CTA2>(tfull_bar(buf));   // accumulator complete
         }
         __syncwarp();
         if (++stage == SL::STAGES) { stage = 0; phase ^= 1u; }
@@ -592,7 +672,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
     // done by the memory system, nothing is read back), the last slice prefetches the carry
     // with TMA loads, adds its own partial and writes the final result.
     const int quarter = warp & 3;
-    const uint32_t stg = smem_base + SL::STG_OFFSET + (uint32_t)quarter * 8192u;
+    constexpr uint32_t NB = SL::STG_BUFS;
+    const uint32_t stg = smem_base + SL::STG_OFFSET + (uint32_t)quarter * (NB * 4096u);
     const uint32_t row_off = (uint32_t)lane * 128u;
     const uint32_t swz = (uint32_t)(lane & 7);
     const bool out_sliced = (p.mode == MODE_COLS) || (p.mode == MODE_ROWS);
@@ -601,7 +682,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
     uint32_t n_cload = 0;   // carry boxes loaded by this warp
     bool ok = true;
     Work w;
-    for (int i = 0; ok && get_work<BN>(p, i, w); ++i) {
+    for (int i = 0; ok && get_work<TM, BN>(p, i, bid, G, w); ++i) {
+      w.a_row += (int)rank * BM;
+      w.row0 += (int)rank * BM;
       const int buf = i & 1;
       const uint32_t bphase = (uint32_t)(i >> 1) & 1u;
       ok = mbar_wait(tfull_bar(buf), bphase, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE);
@@ -613,8 +696,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
       if (p.tma_epilogue && p.mode == MODE_RED && lane == 0) {
         // The carry of this CTA's next tile is touched one main loop from now: have it in L2 by then.
         Work nx;
-        if (get_work<BN>(p, i + 1, nx) && nx.carry_in)
-          tma_prefetch_l2_3d(&p.carry_pf_map, nx.col0, nx.row0 + quarter * 32, 0);
+        if (get_work<TM, BN>(p, i + 1, bid, G, nx) && nx.carry_in)
+          tma_prefetch_l2_3d(&p.carry_pf_map, nx.col0, nx.row0 + (int)rank * BM + quarter * 32, 0);
       }
       if (!p.tma_epilogue) {
         // direct stores from registers (used when the epilogue also reads a second tensor)
@@ -646,9 +729,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
         const int r_in = w.a_row + quarter * 32;
         // One staged box: wait until the buffer's previous box has been read, fill it, hand it to TMA.
         auto stage_begin = [&]() -> uint32_t {
-          if (lane == 0) bulk_wait_read_1();
+          if (lane == 0) bulk_wait_read<NB - 1>();
           __syncwarp();
-          return stg + (n_store & 1u) * 4096u;
+          return stg + (n_store % NB) * 4096u;
         };
         auto stage_issue = [&](const CUtensorMap *map, uint32_t src, int col_in, bool reduce) {
           fence_proxy_async();
@@ -691,29 +774,29 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
           }
         } else if (w.carry_in) {
           // last slice: carry (prefetched by TMA, one box ahead) + accumulator -> bias/act -> out
-          const uint32_t cbar = bar_base + 8u * (2 * SL::STAGES + 5 + quarter * 2);
+          const uint32_t cbar = bar_base + 8u * (2 * SL::STAGES + 5 + quarter * NB);
           int nchunks = (w.col_end - w.col0 + 31) / 32;
           if (nchunks > BN / 32) nchunks = BN / 32;
           auto issue_load = [&](int c) {
             if (lane == 0) {
-              const uint32_t b = n_cload & 1u;
+              const uint32_t b = n_cload % NB;
               mbar_expect_tx(cbar + 8u * b, 4096u);
               tma_load_3d(stg + b * 4096u, &p.carry_map, cbar + 8u * b, w.col0 + c * 32, wrow0, 0);
             }
             ++n_cload;
           };
           const uint32_t first = n_cload;
-          issue_load(0);
+          for (int c = 0; c < (int)NB - 1 && c < nchunks; ++c) issue_load(c);
 #pragma unroll 1
           for (int c = 0; c < nchunks; ++c) {
-            if (c + 1 < nchunks) issue_load(c + 1);
+            if (c + (int)NB - 1 < nchunks) issue_load(c + (int)NB - 1);
             uint32_t v[32];
             tmem_ld_x32(taddr + (uint32_t)(c * 32), v);
             tmem_ld_wait();
             const uint32_t n = first + (uint32_t)c;
-            ok = mbar_wait(cbar + 8u * (n & 1u), (n >> 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE);
+            ok = mbar_wait(cbar + 8u * (n % NB), (n / NB) & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE);
             if (!ok) break;
-            const uint32_t src = stg + (n & 1u) * 4096u + row_off;
+            const uint32_t src = stg + (n % NB) * 4096u + row_off;
             const int cbase = w.col0 + c * 32;
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
@@ -836,7 +919,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(buf));
+      if (lane == 0) {
+        if (CTA2 && rank != 0) mbar_arrive_remote(tempty_bar(buf), 0);   // the even CTA's MMA thread waits on it
+        else mbar_arrive(tempty_bar(buf));
+      }
     }
     // Nothing this warp handed to TMA may still be reading shared memory (or be in flight) at exit.
     if (lane == 0) bulk_wait_all();
@@ -845,9 +931,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
 
   tc_fence_before();
   __syncthreads();
+  if (CTA2) cluster_sync_all();   // neither CTA of a pair leaves while the other may still touch its memory
   if (warp == 2) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, SL::TMEM_COLS);
+    tmem_dealloc<CTA2>(tmem_base, SL::TMEM_COLS);
   }
 }
 
