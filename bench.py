@@ -35,7 +35,11 @@ UNIT = "TFLOP/s"
 
 # DRAM bytes per launch of the dominant kernel from the committed ncu capture
 # (profiles/gemm_kernel_split_sweep.md): dram__bytes_read.sum + dram__bytes_write.sum.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    ("fwd", 8, "out"): 4005381632 + 262917120,
+    ("dx", 8, "out"): 5712420864 + 4002958592,
+    ("dw", 8, "out"): 4608154880 + 128154112,
+}
 
 
 def peaks():
@@ -184,6 +188,7 @@ def run_reference(args):
 def config_dict(args):
     return {"workload": WORKLOAD["name"], "M": WORKLOAD["M"], "N": WORKLOAD["N"], "K": WORKLOAD["K"],
             "k_split": args.k_split, "split_dim": args.split, "act": "none", "accumulate": "fp32 (TMEM)",
+            "carry": "fp32 running sum in the workspace (exact)",
             "l2": "inputs larger than L2 (X, W, dY, outputs total 1.07 GB per step)",
             "parallelism": "replicas only" if args.gpus > 1 else "single GPU"}
 
@@ -227,20 +232,20 @@ def run_ours(args):
     h_dw = torch.empty(N * K, dtype=torch.bfloat16).pin_memory()
     h_db = torch.empty(N, dtype=torch.float32).pin_memory()
 
-    def workspace(kk, sp):
-        _, a = P.osdp_split_linear_workspace_bytes(M, N, K, kk, sp, P.ACT_NONE, P.OP_LINEAR_FWD)
-        _, b = P.osdp_split_linear_workspace_bytes(M, N, K, kk, sp, P.ACT_NONE, P.OP_LINEAR_BWD)
+    def workspace(kk, sp, fl=0):
+        _, a = P.osdp_split_linear_workspace_bytes(M, N, K, kk, sp, P.ACT_NONE, P.OP_LINEAR_FWD, fl)
+        _, b = P.osdp_split_linear_workspace_bytes(M, N, K, kk, sp, P.ACT_NONE, P.OP_LINEAR_BWD, fl)
         return max(a, b)
 
     ws_bytes = workspace(k, split)
     ws = P.new_workspace(ws_bytes, dev)
     stream = torch.cuda.current_stream()
 
-    def fwd(kk=k, sp=split, w=ws):
-        P.osdp_split_linear_fwd(x, w_flat, 0, None, M, N, K, kk, sp, P.ACT_NONE, out, None, w, check=True)
+    def fwd(kk=k, sp=split, w=ws, fl=0):
+        P.osdp_split_linear_fwd(x, w_flat, 0, None, M, N, K, kk, sp, P.ACT_NONE, out, None, w, check=True, flags=fl)
 
-    def bwd_dx(kk=k, sp=split, w=ws):
-        P.osdp_split_linear_bwd(dy, x, w_flat, 0, None, M, N, K, kk, sp, P.ACT_NONE, dx, None, 0, P.DTYPE_BF16, 0,
+    def bwd_dx(kk=k, sp=split, w=ws, fl=0):
+        P.osdp_split_linear_bwd(dy, x, w_flat, 0, None, M, N, K, kk, sp, P.ACT_NONE, dx, None, 0, P.DTYPE_BF16, fl,
                                 None, w, check=True)
 
     def bwd_dw(kk=k, sp=split, w=ws):
@@ -251,8 +256,8 @@ def run_ours(args):
         P.osdp_split_linear_bwd(dy, x, w_flat, 0, None, M, N, K, kk, sp, P.ACT_NONE, None, None, 0, P.DTYPE_BF16, 0,
                                 db, w, check=True)
 
-    def step(kk=k, sp=split, w=ws):
-        fwd(kk, sp, w); bwd_dx(kk, sp, w); bwd_dw(kk, sp, w); bwd_db(kk, sp, w)
+    def step(kk=k, sp=split, w=ws, fl=0):
+        fwd(kk, sp, w, fl); bwd_dx(kk, sp, w, fl); bwd_dw(kk, sp, w); bwd_db(kk, sp, w)
 
     launches_per_step = 5     # fwd GEMM, dX GEMM, dW GEMM, column-sum partial + final
 
@@ -308,16 +313,28 @@ def run_ours(args):
         raise SystemExit("device status %d/%d after the timed region" % (rc, st))
 
     # ---- overhead versus the unsplit layer and the other split dimension, same process
+    # The configurations are run round-robin (one timed step each per round) so that clock and
+    # power drift over the measurement hits all of them alike; medians are reported.
     sweep = {}
     if rank == 0 and not args.no_sweep:
-        for kk, sp, label in ((1, P.SPLIT_OUT, "k1"), (k, P.SPLIT_OUT, "k%d_out" % k), (k, P.SPLIT_RED, "k%d_red" % k)):
-            nbytes = workspace(kk, sp)
-            w2 = ws if nbytes <= ws_bytes else P.new_workspace(nbytes, dev)
-            ms = timed(lambda: step(kk, sp, w2), max(args.steps // 2, 3), 3) / max(args.steps // 2, 3)
-            sweep[label] = {"ms_per_step": ms, "tflops": fl / ms / 1e9, "staging_bytes": nbytes}
-            del w2
+        cfgs = [(1, P.SPLIT_OUT, 0, "k1"), (k, P.SPLIT_OUT, 0, "k%d_out" % k), (k, P.SPLIT_RED, 0, "k%d_red" % k),
+                (k, P.SPLIT_OUT, P.FLAG_CARRY_BF16, "k%d_out_bf16_running_sum" % k),
+                (k, P.SPLIT_RED, P.FLAG_CARRY_BF16, "k%d_red_bf16_running_sum" % k)]
+        need = max(workspace(kk, sp, f) for kk, sp, f, _ in cfgs)
+        w2 = ws if need <= ws_bytes else P.new_workspace(need, dev)
+        times = {label: [] for _, _, _, label in cfgs}
+        for rnd in range(2 + max(args.steps // 2, 5)):
+            for kk, sp, f, label in cfgs:
+                a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+                a.record(stream); step(kk, sp, w2, f); b.record(stream); torch.cuda.synchronize()
+                if rnd >= 2:
+                    times[label].append(a.elapsed_time(b))
+        for kk, sp, f, label in cfgs:
+            ms = sorted(times[label])[len(times[label]) // 2]
+            sweep[label] = {"ms_per_step": ms, "tflops": fl / ms / 1e9, "staging_bytes": workspace(kk, sp, f)}
         for label in list(sweep):
             sweep[label]["overhead_vs_k1"] = sweep[label]["ms_per_step"] / sweep["k1"]["ms_per_step"] - 1.0
+        del w2
     if world > 1:
         barrier()
 

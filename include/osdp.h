@@ -77,6 +77,14 @@ extern "C" {
 
 #define OSDP_MAX_SPLIT 1024
 
+/* flags (bitwise or) */
+#define OSDP_FLAG_ACCUMULATE_DW 1   /* backward: dW += instead of dW = */
+#define OSDP_FLAG_CARRY_BF16 2      /* summed output: keep the running sum in the bf16 output buffer itself
+                                     * (slice 0 stores, later slices add in bf16) instead of an fp32 carry in the
+                                     * workspace: no carry memory, half the carry traffic, one extra bf16 rounding
+                                     * per slice (relative Frobenius error about 1.1e-3 * sqrt(1 + (k+1)/2)).
+                                     * Only without activation and without z_save. */
+
 int osdp_version(void);
 const char *osdp_status_string(int status);
 /* The cudaError_t (as int) of the most recent failed CUDA call made by this library on the
@@ -90,18 +98,20 @@ int osdp_slice_range(int64_t D, int k_split, int slice_idx, int64_t *begin, int6
 
 /* Exact scratch bytes a call with these arguments uses (the "staging" figure).  For the linear
  * ops (M,N,K) are the layer's; for the MLP ops pass M = tokens, N = ffn, K = hidden.
- * The query assumes every optional output (dx, dbias, ...) is requested. */
+ * The query assumes every optional output (dx, dbias, ...) is requested.  `flags` as for the call
+ * (OSDP_FLAG_CARRY_BF16 removes the fp32 carry). */
 int osdp_split_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int k_split, int split_dim,
-                                      int act, int op, size_t *bytes);
+                                      int act, int op, int flags, size_t *bytes);
 
 /* Forward of all k slices in slice-major order (Section 3.3 steps 1-3).
  *   x [M,K] bf16; bias [N] fp32 or NULL; out [M,N] bf16 = act(X W^T + bias);
  *   z_save [M,N] bf16 or NULL: receives the pre-activation (what the backward needs when act != NONE).
- * OUT: slice s writes columns R_s of out.  RED: partial products are summed (fp32 carry in ws);
- * bias and activation are applied once, after the last slice. */
+ * OUT: slice s writes columns R_s of out.  RED: partial products are summed (fp32 carry in ws, or
+ * in `out` itself with OSDP_FLAG_CARRY_BF16); bias and activation are applied once.
+ * flags: 0 or OSDP_FLAG_CARRY_BF16. */
 int osdp_split_linear_fwd(const void *x, const void *w_flat, int64_t w_offset, const float *bias,
                           int64_t M, int64_t N, int64_t K, int k_split, int split_dim, int act,
-                          void *out, void *z_save, void *ws, size_t ws_bytes, void *stream);
+                          int flags, void *out, void *z_save, void *ws, size_t ws_bytes, void *stream);
 
 /* One slice of the forward (Section 3.3 step 2, "the computation of each slice is executed
  * sequentially"): lets a caller put other work between slices.  Slices must be issued in
@@ -109,19 +119,20 @@ int osdp_split_linear_fwd(const void *x, const void *w_flat, int64_t w_offset, c
  * starts the carry and slice k-1 writes `out`. */
 int osdp_split_linear_fwd_slice(const void *x, const void *w_flat, int64_t w_offset, const float *bias,
                                 int64_t M, int64_t N, int64_t K, int k_split, int split_dim, int act,
-                                int slice_idx, void *out, void *z_save, void *ws, size_t ws_bytes,
-                                void *stream);
+                                int flags, int slice_idx, void *out, void *z_save, void *ws,
+                                size_t ws_bytes, void *stream);
 
 /* Backward of all k slices in slice-major order.
  *   dy [M,N] bf16; x [M,K] bf16; z_saved [M,N] bf16 (pre-activation; required iff act != NONE);
  *   dx [M,K] bf16 or NULL; dw_flat + dw_offset: dW [N,K] in dw_dtype (bf16 or fp32), NULL to skip;
- *   accumulate: 0 dW = ..., 1 dW += ...; dbias [N] fp32 or NULL (always overwritten).
+ *   flags: OSDP_FLAG_ACCUMULATE_DW (dW += ... instead of dW = ...), OSDP_FLAG_CARRY_BF16 (dX's running
+ *   sum in dx itself under OUT split); dbias [N] fp32 or NULL (always overwritten).
  * OUT: dW[R_s,:], db[R_s] per slice, dX = sum over slices (fp32 carry in ws).
  * RED: dX[:,C_s], dW[:,C_s] per slice. */
 int osdp_split_linear_bwd(const void *dy, const void *x, const void *w_flat, int64_t w_offset,
                           const void *z_saved, int64_t M, int64_t N, int64_t K, int k_split,
                           int split_dim, int act, void *dx, void *dw_flat, int64_t dw_offset,
-                          int dw_dtype, int accumulate, float *dbias, void *ws, size_t ws_bytes,
+                          int dw_dtype, int flags, float *dbias, void *ws, size_t ws_bytes,
                           void *stream);
 
 /* One slice of the backward; same ordering rule as osdp_split_linear_fwd_slice.  Under RED
@@ -129,7 +140,7 @@ int osdp_split_linear_bwd(const void *dy, const void *x, const void *w_flat, int
 int osdp_split_linear_bwd_slice(const void *dy, const void *x, const void *w_flat, int64_t w_offset,
                                 const void *z_saved, int64_t M, int64_t N, int64_t K, int k_split,
                                 int split_dim, int act, int slice_idx, void *dx, void *dw_flat,
-                                int64_t dw_offset, int dw_dtype, int accumulate, float *dbias,
+                                int64_t dw_offset, int dw_dtype, int flags, float *dbias,
                                 void *ws, size_t ws_bytes, void *stream);
 
 /* Transformer MLP block split along the ffn dimension (first layer OUT-split + activation,
@@ -140,8 +151,8 @@ int osdp_split_linear_bwd_slice(const void *dy, const void *x, const void *w_fla
  * z1_save [M,ffn] bf16 or NULL receives the first layer's pre-activation for the backward. */
 int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const float *b1,
                        int64_t off_w2, const float *b2, int64_t M, int64_t hidden, int64_t ffn,
-                       int k_split, int act, void *out, void *z1_save, void *ws, size_t ws_bytes,
-                       void *stream);
+                       int k_split, int act, int flags, void *out, void *z1_save, void *ws,
+                       size_t ws_bytes, void *stream);
 
 /* Backward of the split MLP block, slice by slice, from the saved pre-activation z1_saved
  * [M,ffn] bf16:  dA_s = dY W2[:,F_s]; dZ_s = dA_s (.) act'(Z1_s); dW2[:,F_s] = dY^T act(Z1_s);
@@ -150,7 +161,7 @@ int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const 
 int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_t off_w1,
                        int64_t off_w2, const void *z1_saved, int64_t M, int64_t hidden, int64_t ffn,
                        int k_split, int act, void *dx, void *dw_flat, int64_t dw_off_w1,
-                       int64_t dw_off_w2, int dw_dtype, int accumulate, float *db1, float *db2,
+                       int64_t dw_off_w2, int dw_dtype, int flags, float *db1, float *db2,
                        void *ws, size_t ws_bytes, void *stream);
 
 /* Synchronises `stream`, copies the device status word at the start of `ws` to *status

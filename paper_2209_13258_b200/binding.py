@@ -16,6 +16,7 @@ SPLIT_OUT, SPLIT_RED = 0, 1
 ACT_NONE, ACT_GELU_TANH, ACT_GELU_ERF = 0, 1, 2
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 OP_LINEAR_FWD, OP_LINEAR_BWD, OP_MLP_FWD, OP_MLP_BWD = 0, 1, 2, 3
+FLAG_ACCUMULATE_DW, FLAG_CARRY_BF16 = 1, 2
 
 EXPORTS = [
     "osdp_version", "osdp_status_string", "osdp_last_cuda_error", "osdp_slice_range",
@@ -55,14 +56,14 @@ def lib():
         L.osdp_status_string.argtypes = [ci]
         L.osdp_last_cuda_error.restype = ci
         L.osdp_slice_range.argtypes = [i64, ci, ci, ctypes.POINTER(i64), ctypes.POINTER(i64)]
-        L.osdp_split_linear_workspace_bytes.argtypes = [i64, i64, i64, ci, ci, ci, ci, ctypes.POINTER(sz)]
-        fwd = [vp, vp, i64, vp, i64, i64, i64, ci, ci, ci]
+        L.osdp_split_linear_workspace_bytes.argtypes = [i64, i64, i64, ci, ci, ci, ci, ci, ctypes.POINTER(sz)]
+        fwd = [vp, vp, i64, vp, i64, i64, i64, ci, ci, ci, ci]
         L.osdp_split_linear_fwd.argtypes = fwd + [vp, vp, vp, sz, vp]
         L.osdp_split_linear_fwd_slice.argtypes = fwd + [ci, vp, vp, vp, sz, vp]
         bwd = [vp, vp, vp, i64, vp, i64, i64, i64, ci, ci, ci]
         L.osdp_split_linear_bwd.argtypes = bwd + [vp, vp, i64, ci, ci, vp, vp, sz, vp]
         L.osdp_split_linear_bwd_slice.argtypes = bwd + [ci, vp, vp, i64, ci, ci, vp, vp, sz, vp]
-        L.osdp_split_mlp_fwd.argtypes = [vp, vp, i64, vp, i64, vp, i64, i64, i64, ci, ci, vp, vp, vp, sz, vp]
+        L.osdp_split_mlp_fwd.argtypes = [vp, vp, i64, vp, i64, vp, i64, i64, i64, ci, ci, ci, vp, vp, vp, sz, vp]
         L.osdp_split_mlp_bwd.argtypes = [vp, vp, vp, i64, i64, vp, i64, i64, i64, ci, ci, vp, vp, i64, i64, ci, ci,
                                          vp, vp, vp, sz, vp]
         L.osdp_read_device_status.argtypes = [vp, ctypes.POINTER(ci), vp]
@@ -125,11 +126,11 @@ def osdp_slice_range(D, k_split, slice_idx):
     return rc, b.value, e.value
 
 
-def osdp_split_linear_workspace_bytes(M, N, K, k_split, split_dim, act, op):
+def osdp_split_linear_workspace_bytes(M, N, K, k_split, split_dim, act, op, flags=0):
     """Returns (status, bytes)."""
     n = ctypes.c_size_t()
     rc = lib().osdp_split_linear_workspace_bytes(int(M), int(N), int(K), int(k_split), int(split_dim), int(act),
-                                                 int(op), ctypes.byref(n))
+                                                 int(op), int(flags), ctypes.byref(n))
     return rc, n.value
 
 
@@ -140,58 +141,58 @@ def new_workspace(nbytes: int, device="cuda"):
 
 
 def osdp_split_linear_fwd(x, w_flat, w_offset, bias, M, N, K, k_split, split_dim, act, out, z_save, ws,
-                          stream=None, check=False):
+                          stream=None, check=False, flags=0):
     wp, wn = _ws(ws)
     rc = lib().osdp_split_linear_fwd(_ptr(x), _ptr(w_flat), int(w_offset), _ptr(bias), int(M), int(N), int(K),
-                                     int(k_split), int(split_dim), int(act), _ptr(out), _ptr(z_save), wp, wn,
-                                     _stream(stream))
+                                     int(k_split), int(split_dim), int(act), int(flags), _ptr(out), _ptr(z_save),
+                                     wp, wn, _stream(stream))
     return _ret(rc, check, "osdp_split_linear_fwd")
 
 
 def osdp_split_linear_fwd_slice(x, w_flat, w_offset, bias, M, N, K, k_split, split_dim, act, slice_idx, out,
-                                z_save, ws, stream=None, check=False):
+                                z_save, ws, stream=None, check=False, flags=0):
     wp, wn = _ws(ws)
     rc = lib().osdp_split_linear_fwd_slice(_ptr(x), _ptr(w_flat), int(w_offset), _ptr(bias), int(M), int(N), int(K),
-                                           int(k_split), int(split_dim), int(act), int(slice_idx), _ptr(out),
-                                           _ptr(z_save), wp, wn, _stream(stream))
+                                           int(k_split), int(split_dim), int(act), int(flags), int(slice_idx),
+                                           _ptr(out), _ptr(z_save), wp, wn, _stream(stream))
     return _ret(rc, check, "osdp_split_linear_fwd_slice")
 
 
 def osdp_split_linear_bwd(dy, x, w_flat, w_offset, z_saved, M, N, K, k_split, split_dim, act, dx, dw_flat,
-                          dw_offset, dw_dtype, accumulate, dbias, ws, stream=None, check=False):
+                          dw_offset, dw_dtype, flags, dbias, ws, stream=None, check=False):
     wp, wn = _ws(ws)
     rc = lib().osdp_split_linear_bwd(_ptr(dy), _ptr(x), _ptr(w_flat), int(w_offset), _ptr(z_saved), int(M), int(N),
                                      int(K), int(k_split), int(split_dim), int(act), _ptr(dx), _ptr(dw_flat),
-                                     int(dw_offset), int(dw_dtype), int(accumulate), _ptr(dbias), wp, wn,
+                                     int(dw_offset), int(dw_dtype), int(flags), _ptr(dbias), wp, wn,
                                      _stream(stream))
     return _ret(rc, check, "osdp_split_linear_bwd")
 
 
 def osdp_split_linear_bwd_slice(dy, x, w_flat, w_offset, z_saved, M, N, K, k_split, split_dim, act, slice_idx, dx,
-                                dw_flat, dw_offset, dw_dtype, accumulate, dbias, ws, stream=None, check=False):
+                                dw_flat, dw_offset, dw_dtype, flags, dbias, ws, stream=None, check=False):
     wp, wn = _ws(ws)
     rc = lib().osdp_split_linear_bwd_slice(_ptr(dy), _ptr(x), _ptr(w_flat), int(w_offset), _ptr(z_saved), int(M),
                                            int(N), int(K), int(k_split), int(split_dim), int(act), int(slice_idx),
-                                           _ptr(dx), _ptr(dw_flat), int(dw_offset), int(dw_dtype), int(accumulate),
+                                           _ptr(dx), _ptr(dw_flat), int(dw_offset), int(dw_dtype), int(flags),
                                            _ptr(dbias), wp, wn, _stream(stream))
     return _ret(rc, check, "osdp_split_linear_bwd_slice")
 
 
 def osdp_split_mlp_fwd(x, w_flat, off_w1, b1, off_w2, b2, M, hidden, ffn, k_split, act, out, z1_save, ws,
-                       stream=None, check=False):
+                       stream=None, check=False, flags=0):
     wp, wn = _ws(ws)
     rc = lib().osdp_split_mlp_fwd(_ptr(x), _ptr(w_flat), int(off_w1), _ptr(b1), int(off_w2), _ptr(b2), int(M),
-                                  int(hidden), int(ffn), int(k_split), int(act), _ptr(out), _ptr(z1_save), wp, wn,
-                                  _stream(stream))
+                                  int(hidden), int(ffn), int(k_split), int(act), int(flags), _ptr(out),
+                                  _ptr(z1_save), wp, wn, _stream(stream))
     return _ret(rc, check, "osdp_split_mlp_fwd")
 
 
 def osdp_split_mlp_bwd(dy, x, w_flat, off_w1, off_w2, z1_saved, M, hidden, ffn, k_split, act, dx, dw_flat,
-                       dw_off_w1, dw_off_w2, dw_dtype, accumulate, db1, db2, ws, stream=None, check=False):
+                       dw_off_w1, dw_off_w2, dw_dtype, flags, db1, db2, ws, stream=None, check=False):
     wp, wn = _ws(ws)
     rc = lib().osdp_split_mlp_bwd(_ptr(dy), _ptr(x), _ptr(w_flat), int(off_w1), int(off_w2), _ptr(z1_saved), int(M),
                                   int(hidden), int(ffn), int(k_split), int(act), _ptr(dx), _ptr(dw_flat),
-                                  int(dw_off_w1), int(dw_off_w2), int(dw_dtype), int(accumulate), _ptr(db1),
+                                  int(dw_off_w1), int(dw_off_w2), int(dw_dtype), int(flags), _ptr(db1),
                                   _ptr(db2), wp, wn, _stream(stream))
     return _ret(rc, check, "osdp_split_mlp_bwd")
 

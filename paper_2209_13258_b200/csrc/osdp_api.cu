@@ -94,7 +94,8 @@ struct WsPlan {
   size_t total;
 };
 
-int plan_workspace(int64_t M, int64_t N, int64_t K, int k, int split_dim, int act, int op, WsPlan *w) {
+int plan_workspace(int64_t M, int64_t N, int64_t K, int k, int split_dim, int act, int op, int flags, WsPlan *w) {
+  const bool fp32_carry = !(flags & OSDP_FLAG_CARRY_BF16);
   memset(w, 0, sizeof(*w));
   if (M <= 0 || N <= 0 || K <= 0) return OSDP_ERR_BAD_SHAPE;
   if (k == 0) k = 1;
@@ -112,13 +113,13 @@ int plan_workspace(int64_t M, int64_t N, int64_t K, int k, int split_dim, int ac
       if (split_dim != OSDP_SPLIT_OUT && split_dim != OSDP_SPLIT_RED) return OSDP_ERR_BAD_SPLIT;
       rc = slice_len(split_dim == OSDP_SPLIT_OUT ? N : K, k, &L);
       if (rc) return rc;
-      if (split_dim == OSDP_SPLIT_RED && k > 1) take((size_t)M * N * 4, &w->carry_off, &w->carry_bytes);
+      if (split_dim == OSDP_SPLIT_RED && k > 1 && fp32_carry) take((size_t)M * N * 4, &w->carry_off, &w->carry_bytes);
       break;
     case OSDP_OP_LINEAR_BWD:
       if (split_dim != OSDP_SPLIT_OUT && split_dim != OSDP_SPLIT_RED) return OSDP_ERR_BAD_SPLIT;
       rc = slice_len(split_dim == OSDP_SPLIT_OUT ? N : K, k, &L);
       if (rc) return rc;
-      if (split_dim == OSDP_SPLIT_OUT && k > 1) take((size_t)M * K * 4, &w->carry_off, &w->carry_bytes);
+      if (split_dim == OSDP_SPLIT_OUT && k > 1 && fp32_carry) take((size_t)M * K * 4, &w->carry_off, &w->carry_bytes);
       if (act != OSDP_ACT_NONE)
         take((size_t)M * (split_dim == OSDP_SPLIT_OUT ? L : N) * 2, &w->stage0_off, &w->stage0_bytes);
       take(chunks * (size_t)N * 4, &w->part_off, &w->part_bytes);
@@ -126,13 +127,13 @@ int plan_workspace(int64_t M, int64_t N, int64_t K, int k, int split_dim, int ac
     case OSDP_OP_MLP_FWD:   // N = ffn, K = hidden
       rc = slice_len(N, k, &L);
       if (rc) return rc;
-      if (k > 1) take((size_t)M * K * 4, &w->carry_off, &w->carry_bytes);
+      if (k > 1 && fp32_carry) take((size_t)M * K * 4, &w->carry_off, &w->carry_bytes);
       take((size_t)M * L * 2, &w->stage0_off, &w->stage0_bytes);
       break;
     case OSDP_OP_MLP_BWD:
       rc = slice_len(N, k, &L);
       if (rc) return rc;
-      if (k > 1) take((size_t)M * K * 4, &w->carry_off, &w->carry_bytes);
+      if (k > 1 && fp32_carry) take((size_t)M * K * 4, &w->carry_off, &w->carry_bytes);
       take((size_t)M * L * 2, &w->stage0_off, &w->stage0_bytes);
       take((size_t)M * L * 2, &w->stage1_off, &w->stage1_bytes);
       take(chunks * (size_t)(L > K ? L : K) * 4, &w->part_off, &w->part_bytes);
@@ -165,6 +166,7 @@ struct GemmCall {
   int k_total, s_begin, s_end;
   int64_t bn_P, bn_Q;   // extents that choose the tile width (the unsplit operator's, so k never changes it)
   Epilogue epi;
+  int carry_bf16;   // MODE_RED: running sum in `out` (bf16) instead of the fp32 carry buffer
   int *status;
 };
 
@@ -356,6 +358,7 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   p.mode = c.mode; p.L = (int)c.L; p.k_total = c.k_total; p.s_begin = c.s_begin; p.s_end = c.s_end;
   p.epi = c.epi;
   p.status = c.status;
+  p.carry_bf16 = (c.mode == MODE_RED && c.k_total > 1) ? c.carry_bf16 : 0;
   // Outputs leave through TMA unless the epilogue has to read a second tensor element-wise.
   p.tma_epilogue = (c.epi.gz == nullptr) ? 1 : 0;
   if (p.tma_epilogue) {
@@ -367,7 +370,7 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
                             nullptr);
       if (rc) return rc;
     }
-    if (c.mode == MODE_RED && c.k_total > 1) {
+    if (c.mode == MODE_RED && c.k_total > 1 && !p.carry_bf16) {
       CUtensorMap unused;
       rc = make_output_maps(c.epi.carry, true, c.P, c.Q, c.epi.ld_carry, MODE_NONE, c.L, 1, &unused, &p.carry_map,
                             nullptr);
@@ -456,10 +459,20 @@ int check_ws(const void *ws, size_t ws_bytes, const WsPlan &plan) {
   return OSDP_OK;
 }
 
+int check_flags(int flags, int allowed, int act, const void *z_save) {
+  if (flags & ~allowed) return OSDP_ERR_UNSUPPORTED;
+  if ((flags & OSDP_FLAG_CARRY_BF16) && (act != OSDP_ACT_NONE || z_save)) return OSDP_ERR_UNSUPPORTED;
+  return OSDP_OK;
+}
+
 int fwd_impl(const void *x, const void *w_flat, int64_t w_offset, const float *bias, int64_t M, int64_t N, int64_t K,
-             int k, int split_dim, int act, int s_begin, int s_end, bool single, void *out, void *z_save, void *ws,
-             size_t ws_bytes, void *stream) {
+             int k, int split_dim, int act, int flags, int s_begin, int s_end, bool single, void *out, void *z_save,
+             void *ws, size_t ws_bytes, void *stream) {
   if (!x || !w_flat || !out) return OSDP_ERR_NULL_POINTER;
+  {
+    const int frc = check_flags(flags, OSDP_FLAG_CARRY_BF16, act, z_save);
+    if (frc) return frc;
+  }
   int64_t L = 0;
   int rc = check_common(M, N, K, k, split_dim, act, &L);
   if (rc) return rc;
@@ -475,7 +488,7 @@ int fwd_impl(const void *x, const void *w_flat, int64_t w_offset, const float *b
   if (!aligned16(x) || !aligned16(w_flat) || !aligned16(out) || !aligned16(z_save) || !aligned16(bias))
     return OSDP_ERR_ALIGNMENT;
   WsPlan plan;
-  rc = plan_workspace(M, N, K, k, split_dim, act, OSDP_OP_LINEAR_FWD, &plan);
+  rc = plan_workspace(M, N, K, k, split_dim, act, OSDP_OP_LINEAR_FWD, flags, &plan);
   if (rc) return rc;
   rc = check_ws(ws, ws_bytes, plan);
   if (rc) return rc;
@@ -496,15 +509,19 @@ int fwd_impl(const void *x, const void *w_flat, int64_t w_offset, const float *b
   c.epi.act = act;
   c.epi.carry = reinterpret_cast<float *>(static_cast<char *>(ws) + plan.carry_off);
   c.epi.ld_carry = N;
+  c.carry_bf16 = (flags & OSDP_FLAG_CARRY_BF16) ? 1 : 0;
   c.status = static_cast<int *>(ws);
   return launch_gemm(c, static_cast<cudaStream_t>(stream));
 }
 
 int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset, const void *z_saved, int64_t M,
              int64_t N, int64_t K, int k, int split_dim, int act, int s_begin, int s_end, bool single, void *dx,
-             void *dw_flat, int64_t dw_offset, int dw_dtype, int accumulate, float *dbias, void *ws, size_t ws_bytes,
+             void *dw_flat, int64_t dw_offset, int dw_dtype, int flags, float *dbias, void *ws, size_t ws_bytes,
              void *stream_) {
   if (!dy || !x || !w_flat) return OSDP_ERR_NULL_POINTER;
+  // the bf16 running sum concerns dX only, which has neither bias nor activation of its own
+  if (flags & ~(OSDP_FLAG_ACCUMULATE_DW | OSDP_FLAG_CARRY_BF16)) return OSDP_ERR_UNSUPPORTED;
+  const int accumulate = (flags & OSDP_FLAG_ACCUMULATE_DW) ? 1 : 0;
   int64_t L = 0;
   int rc = check_common(M, N, K, k, split_dim, act, &L);
   if (rc) return rc;
@@ -523,7 +540,7 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
       !aligned16(dw_flat) || !aligned16(dbias))
     return OSDP_ERR_ALIGNMENT;
   WsPlan plan;
-  rc = plan_workspace(M, N, K, k, split_dim, act, OSDP_OP_LINEAR_BWD, &plan);
+  rc = plan_workspace(M, N, K, k, split_dim, act, OSDP_OP_LINEAR_BWD, flags, &plan);
   if (rc) return rc;
   rc = check_ws(ws, ws_bytes, plan);
   if (rc) return rc;
@@ -553,6 +570,7 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
     c.epi = plain_epilogue(dx, K, 0);
     c.epi.carry = carry;
     c.epi.ld_carry = K;
+    c.carry_bf16 = (flags & OSDP_FLAG_CARRY_BF16) ? 1 : 0;
     c.status = status;
     return launch_gemm(c, stream);
   };
@@ -651,50 +669,52 @@ int osdp_slice_range(int64_t D, int k_split, int slice_idx, int64_t *begin, int6
 }
 
 int osdp_split_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int k_split, int split_dim, int act, int op,
-                                      size_t *bytes) {
+                                      int flags, size_t *bytes) {
   if (!bytes) return OSDP_ERR_NULL_POINTER;
   if (act != OSDP_ACT_NONE && act != OSDP_ACT_GELU_TANH && act != OSDP_ACT_GELU_ERF) return OSDP_ERR_UNSUPPORTED;
+  if (flags & ~(OSDP_FLAG_ACCUMULATE_DW | OSDP_FLAG_CARRY_BF16)) return OSDP_ERR_UNSUPPORTED;
   WsPlan plan;
-  int rc = plan_workspace(M, N, K, k_split, split_dim, act, op, &plan);
+  int rc = plan_workspace(M, N, K, k_split, split_dim, act, op, flags, &plan);
   if (rc) return rc;
   *bytes = plan.total;
   return OSDP_OK;
 }
 
 int osdp_split_linear_fwd(const void *x, const void *w_flat, int64_t w_offset, const float *bias, int64_t M,
-                          int64_t N, int64_t K, int k_split, int split_dim, int act, void *out, void *z_save,
-                          void *ws, size_t ws_bytes, void *stream) {
-  return fwd_impl(x, w_flat, w_offset, bias, M, N, K, k_split, split_dim, act, 0, 0, false, out, z_save, ws, ws_bytes,
-                  stream);
+                          int64_t N, int64_t K, int k_split, int split_dim, int act, int flags, void *out,
+                          void *z_save, void *ws, size_t ws_bytes, void *stream) {
+  return fwd_impl(x, w_flat, w_offset, bias, M, N, K, k_split, split_dim, act, flags, 0, 0, false, out, z_save, ws,
+                  ws_bytes, stream);
 }
 
 int osdp_split_linear_fwd_slice(const void *x, const void *w_flat, int64_t w_offset, const float *bias, int64_t M,
-                                int64_t N, int64_t K, int k_split, int split_dim, int act, int slice_idx, void *out,
-                                void *z_save, void *ws, size_t ws_bytes, void *stream) {
-  return fwd_impl(x, w_flat, w_offset, bias, M, N, K, k_split, split_dim, act, slice_idx, 0, true, out, z_save, ws,
-                  ws_bytes, stream);
+                                int64_t N, int64_t K, int k_split, int split_dim, int act, int flags, int slice_idx,
+                                void *out, void *z_save, void *ws, size_t ws_bytes, void *stream) {
+  return fwd_impl(x, w_flat, w_offset, bias, M, N, K, k_split, split_dim, act, flags, slice_idx, 0, true, out, z_save,
+                  ws, ws_bytes, stream);
 }
 
 int osdp_split_linear_bwd(const void *dy, const void *x, const void *w_flat, int64_t w_offset, const void *z_saved,
                           int64_t M, int64_t N, int64_t K, int k_split, int split_dim, int act, void *dx,
-                          void *dw_flat, int64_t dw_offset, int dw_dtype, int accumulate, float *dbias, void *ws,
+                          void *dw_flat, int64_t dw_offset, int dw_dtype, int flags, float *dbias, void *ws,
                           size_t ws_bytes, void *stream) {
   return bwd_impl(dy, x, w_flat, w_offset, z_saved, M, N, K, k_split, split_dim, act, 0, 0, false, dx, dw_flat,
-                  dw_offset, dw_dtype, accumulate, dbias, ws, ws_bytes, stream);
+                  dw_offset, dw_dtype, flags, dbias, ws, ws_bytes, stream);
 }
 
 int osdp_split_linear_bwd_slice(const void *dy, const void *x, const void *w_flat, int64_t w_offset,
                                 const void *z_saved, int64_t M, int64_t N, int64_t K, int k_split, int split_dim,
                                 int act, int slice_idx, void *dx, void *dw_flat, int64_t dw_offset, int dw_dtype,
-                                int accumulate, float *dbias, void *ws, size_t ws_bytes, void *stream) {
+                                int flags, float *dbias, void *ws, size_t ws_bytes, void *stream) {
   return bwd_impl(dy, x, w_flat, w_offset, z_saved, M, N, K, k_split, split_dim, act, slice_idx, 0, true, dx, dw_flat,
-                  dw_offset, dw_dtype, accumulate, dbias, ws, ws_bytes, stream);
+                  dw_offset, dw_dtype, flags, dbias, ws, ws_bytes, stream);
 }
 
 int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const float *b1, int64_t off_w2,
-                       const float *b2, int64_t M, int64_t hidden, int64_t ffn, int k_split, int act, void *out,
-                       void *z1_save, void *ws, size_t ws_bytes, void *stream_) {
+                       const float *b2, int64_t M, int64_t hidden, int64_t ffn, int k_split, int act, int flags,
+                       void *out, void *z1_save, void *ws, size_t ws_bytes, void *stream_) {
   if (!x || !w_flat || !out) return OSDP_ERR_NULL_POINTER;
+  if (flags & ~OSDP_FLAG_CARRY_BF16) return OSDP_ERR_UNSUPPORTED;   // the second layer has no activation: allowed
   int64_t L = 0;
   int rc = check_common(M, ffn, hidden, k_split, OSDP_SPLIT_OUT, act, &L);
   if (rc) return rc;
@@ -704,7 +724,7 @@ int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const 
       !aligned16(b2))
     return OSDP_ERR_ALIGNMENT;
   WsPlan plan;
-  rc = plan_workspace(M, ffn, hidden, k, OSDP_SPLIT_OUT, act, OSDP_OP_MLP_FWD, &plan);
+  rc = plan_workspace(M, ffn, hidden, k, OSDP_SPLIT_OUT, act, OSDP_OP_MLP_FWD, flags, &plan);
   if (rc) return rc;
   rc = check_ws(ws, ws_bytes, plan);
   if (rc) return rc;
@@ -746,6 +766,7 @@ int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const 
     c.epi.bias = b2;
     c.epi.carry = carry;
     c.epi.ld_carry = hidden;
+    c.carry_bf16 = (flags & OSDP_FLAG_CARRY_BF16) ? 1 : 0;
     c.status = status;
     rc = launch_gemm(c, stream);
     if (rc) return rc;
@@ -755,9 +776,11 @@ int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const 
 
 int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_t off_w1, int64_t off_w2,
                        const void *z1_saved, int64_t M, int64_t hidden, int64_t ffn, int k_split, int act, void *dx,
-                       void *dw_flat, int64_t dw_off_w1, int64_t dw_off_w2, int dw_dtype, int accumulate, float *db1,
+                       void *dw_flat, int64_t dw_off_w1, int64_t dw_off_w2, int dw_dtype, int flags, float *db1,
                        float *db2, void *ws, size_t ws_bytes, void *stream_) {
   if (!dy || !x || !w_flat || !z1_saved) return OSDP_ERR_NULL_POINTER;
+  if (flags & ~(OSDP_FLAG_ACCUMULATE_DW | OSDP_FLAG_CARRY_BF16)) return OSDP_ERR_UNSUPPORTED;
+  const int accumulate = (flags & OSDP_FLAG_ACCUMULATE_DW) ? 1 : 0;
   int64_t L = 0;
   int rc = check_common(M, ffn, hidden, k_split, OSDP_SPLIT_OUT, act, &L);
   if (rc) return rc;
@@ -770,7 +793,7 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
       !aligned16(dw_flat) || !aligned16(db1) || !aligned16(db2))
     return OSDP_ERR_ALIGNMENT;
   WsPlan plan;
-  rc = plan_workspace(M, ffn, hidden, k, OSDP_SPLIT_OUT, act, OSDP_OP_MLP_BWD, &plan);
+  rc = plan_workspace(M, ffn, hidden, k, OSDP_SPLIT_OUT, act, OSDP_OP_MLP_BWD, flags, &plan);
   if (rc) return rc;
   rc = check_ws(ws, ws_bytes, plan);
   if (rc) return rc;
@@ -847,6 +870,7 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
       c.epi = plain_epilogue(dx, hidden, 0);
       c.epi.carry = carry;
       c.epi.ld_carry = hidden;
+      c.carry_bf16 = (flags & OSDP_FLAG_CARRY_BF16) ? 1 : 0;
       c.status = status;
       rc = launch_gemm(c, stream);
       if (rc) return rc;

@@ -68,6 +68,7 @@ struct GemmParams {
   CUtensorMap out_main, out_tail, z_main, z_tail, carry_map;
   CUtensorMap carry_pf_map;  // same tensor as carry_map, unswizzled box of 32 rows x BN columns, for L2 prefetch
   int out_sc_mul;
+  int carry_bf16;            // MODE_RED: the running sum is kept in `out` itself, in bf16 (no fp32 carry buffer)
   int tma_epilogue;          // 1: outputs leave through shared-memory staging + TMA; 0: direct stores
   Epilogue epi;
   int *status;               // device status word or null
@@ -386,8 +387,8 @@ __device__ __forceinline__ bool get_work(const GemmParams &p, int i, int bid, in
   w.col_end = col_base + cols;
   const int red = (p.mode == MODE_RED) ? min(p.L, p.R - s * p.L) : p.R;
   w.kblocks = ceil_div(red, BK);
-  w.carry_in = (p.mode == MODE_RED) && (s > 0);
-  w.carry_out = (p.mode == MODE_RED) && (s < p.k_total - 1);
+  w.carry_in = (p.mode == MODE_RED) && !p.carry_bf16 && (s > 0);
+  w.carry_out = (p.mode == MODE_RED) && !p.carry_bf16 && (s < p.k_total - 1);
   return true;
 }
 
@@ -749,13 +750,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
           }
           ++n_store;
         };
-        if (w.carry_out || (w.carry_in && w.first_of_slice)) {
+        // bf16 running sum kept in the output itself: slice 0 stores, every later slice reduce-adds.
+        const bool inplace_add = p.carry_bf16 && p.mode == MODE_RED && w.s > 0;
+        const bool skip_bias = p.carry_bf16 && p.mode == MODE_RED && w.s > 0;   // bias enters once, with slice 0
+        if (w.first_of_slice && (w.carry_in || inplace_add)) {
           // Slice boundary: everything this warp sent for the previous slice must have landed
           // before the same addresses are added to (or read) again.
-          if (w.first_of_slice && w.carry_in) {
-            if (lane == 0) bulk_wait_all();
-            __syncwarp();
-          }
+          if (lane == 0) bulk_wait_all();
+          __syncwarp();
         }
         if (w.carry_out) {
           // fp32 partial -> carry, 32 columns (128 bytes per row) per box
@@ -867,7 +869,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
               for (int j = 0; j < 32; ++j) { v[j] = lo[j]; v[32 + j] = hi[j]; }
             }
             uint4 packed[8];
-            if (p.epi.bias) {
+            if (p.epi.bias && !skip_bias) {
 #pragma unroll
               for (int g = 0; g < 8; ++g) {
                 if (cbase + g * 8 < w.col_end) {
@@ -913,7 +915,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
 #pragma unroll
             for (int g = 0; g < 8; ++g)
               st_shared_v4(dst + row_off + (((uint32_t)g ^ swz) << 4), packed[g].x, packed[g].y, packed[g].z, packed[g].w);
-            stage_issue(omap, dst, w.b_col + c * 64, p.epi.accumulate != 0);
+            stage_issue(omap, dst, w.b_col + c * 64, p.epi.accumulate != 0 || inplace_add);
           }
         }
       }

@@ -1,0 +1,159 @@
+"""Command-line runs of the split-linear path on synthetic tensors (device-side random data).
+
+    python -m paper_2209_13258_b200.sweep case M N K k split        one fwd+bwd (twice), for profilers
+    python -m paper_2209_13258_b200.sweep linear M N K [ks]         time vs slice granularity, both split dims
+    python -m paper_2209_13258_b200.sweep mlp M hidden ffn [ks]     MLP block split along ffn: time and staging
+
+The `linear` and `mlp` modes reproduce in kind the paper's Figure 7 (time and memory of an operator
+against slice granularity) for this single-GPU path: TFLOP/s, overhead versus k = 1, staging bytes.
+Timing: CUDA events on the current stream, median of `iters` runs after warm-up.
+"""
+from __future__ import annotations
+
+import json
+import sys
+
+import torch
+
+from . import binding as P
+
+
+def _time_interleaved(fns, rounds=12, warm=2):
+    """Median time (ms) of each callable.  The callables are run round-robin, one timed run each
+    per round, so that clock / power drift over the measurement hits every configuration alike."""
+    for _ in range(warm):
+        for fn in fns:
+            fn()
+    torch.cuda.synchronize()
+    ts = [[] for _ in fns]
+    for _ in range(rounds):
+        for i, fn in enumerate(fns):
+            a = torch.cuda.Event(enable_timing=True)
+            b = torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            ts[i].append(a.elapsed_time(b))
+    return [sorted(t)[len(t) // 2] for t in ts]
+
+
+def _linear_tensors(M, N, K):
+    dev = "cuda"
+    x = torch.randn(M, K, device=dev).bfloat16()
+    w = (torch.randn(N, K, device=dev) * 0.02).bfloat16()
+    dy = torch.randn(M, N, device=dev).bfloat16()
+    out = torch.empty(M, N, device=dev, dtype=torch.bfloat16)
+    dx = torch.empty(M, K, device=dev, dtype=torch.bfloat16)
+    dw = torch.empty(N, K, device=dev, dtype=torch.bfloat16)
+    db = torch.empty(N, device=dev, dtype=torch.float32)
+    return x, w, dy, out, dx, dw, db
+
+
+def _ws_linear(M, N, K, k, split, flags=0):
+    _, a = P.osdp_split_linear_workspace_bytes(M, N, K, k, split, 0, P.OP_LINEAR_FWD, flags)
+    _, b = P.osdp_split_linear_workspace_bytes(M, N, K, k, split, 0, P.OP_LINEAR_BWD, flags)
+    return max(a, b)
+
+
+def run_case(M, N, K, k, split):
+    x, w, dy, out, dx, dw, db = _linear_tensors(M, N, K)
+    ws = P.new_workspace(_ws_linear(M, N, K, k, split))
+    for _ in range(2):
+        P.osdp_split_linear_fwd(x, w, 0, None, M, N, K, k, split, 0, out, None, ws, check=True)
+        P.osdp_split_linear_bwd(dy, x, w, 0, None, M, N, K, k, split, 0, dx, dw, 0, 0, 0, None, ws, check=True)
+        torch.cuda.synchronize()
+    print("device status", P.osdp_read_device_status(ws))
+
+
+def sweep_linear(M, N, K, ks):
+    x, w, dy, out, dx, dw, db = _linear_tensors(M, N, K)
+    flops = 3 * 2.0 * M * N * K
+    cfgs = []
+    for k in ks:
+        for split, name in ((P.SPLIT_OUT, "out"), (P.SPLIT_RED, "red")):
+            if k == 1 and split == P.SPLIT_RED:
+                continue
+            if P.osdp_slice_range(N if split == P.SPLIT_OUT else K, k, 0)[0] != 0:
+                continue
+            cfgs.append((k, split, name, 0, _ws_linear(M, N, K, k, split)))
+            if k > 1:   # the summed output carried in bf16 in the output buffer instead of fp32 in the workspace
+                cfgs.append((k, split, name, P.FLAG_CARRY_BF16, _ws_linear(M, N, K, k, split, P.FLAG_CARRY_BF16)))
+    ws = P.new_workspace(max(c[4] for c in cfgs))     # one workspace, large enough for every configuration
+    fns = []
+    for k, split, name, fl, _ in cfgs:
+        fns.append(lambda k=k, split=split, fl=fl: P.osdp_split_linear_fwd(
+            x, w, 0, None, M, N, K, k, split, 0, out, None, ws, check=True, flags=fl))
+        fns.append(lambda k=k, split=split, fl=fl: P.osdp_split_linear_bwd(
+            dy, x, w, 0, None, M, N, K, k, split, 0, dx, dw, 0, 0, fl, db, ws, check=True))
+    ts = _time_interleaved(fns)
+    rows = []
+    base = ts[0] + ts[1]
+    for i, (k, split, name, fl, nbytes) in enumerate(cfgs):
+        tf, tb = ts[2 * i], ts[2 * i + 1]
+        t = tf + tb
+        rows.append({"k": k, "split": name, "carry": "bf16" if fl else "fp32", "fwd_ms": tf, "bwd_ms": tb, "ms": t,
+                     "tflops": flops / t / 1e9, "overhead_vs_k1": t / base - 1.0, "staging_bytes": nbytes})
+        print(json.dumps(rows[-1]), flush=True)
+    return rows
+
+
+def sweep_mlp(M, H, F, ks):
+    dev = "cuda"
+    x = torch.randn(M, H, device=dev).bfloat16()
+    dy = torch.randn(M, H, device=dev).bfloat16()
+    wf = (torch.randn(2 * F * H, device=dev) * 0.02).bfloat16()
+    b1 = torch.zeros(F, device=dev)
+    b2 = torch.zeros(H, device=dev)
+    out = torch.empty(M, H, device=dev, dtype=torch.bfloat16)
+    z1 = torch.empty(M, F, device=dev, dtype=torch.bfloat16)
+    dx = torch.empty(M, H, device=dev, dtype=torch.bfloat16)
+    dwf = torch.empty(2 * F * H, device=dev, dtype=torch.bfloat16)
+    db1 = torch.empty(F, device=dev)
+    db2 = torch.empty(H, device=dev)
+    flops = 2 * 3 * 2.0 * M * H * F
+    cfgs = []
+    for k in ks:
+        if P.osdp_slice_range(F, k, 0)[0] != 0:
+            continue
+        _, n1 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, 1, P.OP_MLP_FWD)
+        _, n2 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, 1, P.OP_MLP_BWD)
+        cfgs.append((k, n1, n2))
+    ws = P.new_workspace(max(max(c[1], c[2]) for c in cfgs))
+    fns = []
+    for k, _, _ in cfgs:
+        fns.append(lambda k=k: P.osdp_split_mlp_fwd(x, wf, 0, b1, F * H, b2, M, H, F, k, 1, out, z1, ws, check=True))
+        fns.append(lambda k=k: P.osdp_split_mlp_bwd(dy, x, wf, 0, F * H, z1, M, H, F, k, 1, dx, dwf, 0, F * H, 0, 0,
+                                                    db1, db2, ws, check=True))
+    ts = _time_interleaved(fns)
+    rows = []
+    base = ts[0] + ts[1]
+    for i, (k, n1, n2) in enumerate(cfgs):
+        tf, tb = ts[2 * i], ts[2 * i + 1]
+        t = tf + tb
+        rows.append({"k": k, "fwd_ms": tf, "bwd_ms": tb, "ms": t, "tflops": flops / t / 1e9,
+                     "overhead_vs_k1": t / base - 1.0, "staging_fwd_bytes": n1, "staging_bwd_bytes": n2})
+        print(json.dumps(rows[-1]), flush=True)
+    return rows
+
+
+def main(argv):
+    if len(argv) < 2:
+        print(__doc__)
+        return 2
+    mode = argv[1]
+    ks = [int(v) for v in argv[5].split(",")] if len(argv) > 5 and mode != "case" else [1, 2, 4, 8, 16, 32]
+    if mode == "case":
+        run_case(*[int(v) for v in argv[2:7]])
+    elif mode == "linear":
+        sweep_linear(int(argv[2]), int(argv[3]), int(argv[4]), ks)
+    elif mode == "mlp":
+        sweep_mlp(int(argv[2]), int(argv[3]), int(argv[4]), ks)
+    else:
+        print(__doc__)
+        return 2
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main(sys.argv))

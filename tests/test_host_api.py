@@ -60,6 +60,12 @@ def test_workspace_plan():
     assert f(1) == 256 + 8192 * 32768 * 2
     for k in (2, 4, 8, 16):
         assert f(k) == 256 + carry + 8192 * (32768 // k) * 2
+    assert q(8, 1, 0, P.OP_LINEAR_FWD) != (0, 256)
+    assert P.osdp_split_linear_workspace_bytes(M, N, K, 8, 1, 0, P.OP_LINEAR_FWD, P.FLAG_CARRY_BF16) == (0, 256)
+    assert P.osdp_split_linear_workspace_bytes(M, N, K, 8, 0, 0, P.OP_LINEAR_BWD, P.FLAG_CARRY_BF16) == (0, 256 + part)
+    assert P.osdp_split_linear_workspace_bytes(8192, 32768, 8192, 8, 0, 1, P.OP_MLP_FWD, P.FLAG_CARRY_BF16) == (
+        0, 256 + 8192 * 4096 * 2)
+    assert P.osdp_split_linear_workspace_bytes(8, 8, 8, 1, 0, 0, 0, 16)[0] == 6
     assert P.osdp_split_linear_workspace_bytes(8, 8, 8, 1, 0, 0, 9)[0] == 6
     assert P.osdp_split_linear_workspace_bytes(8, 8, 8, 1, 0, 7, 0)[0] == 6
     assert P.osdp_split_linear_workspace_bytes(8, 16, 8, 3, 0, 0, 0)[0] == 3
@@ -77,7 +83,7 @@ def _fwd(**kw):
 
 def _bwd(**kw):
     a = dict(dy=A, x=A, w_flat=A, w_offset=0, z_saved=None, M=64, N=64, K=64, k_split=2, split_dim=0, act=0,
-             dx=A, dw_flat=A, dw_offset=0, dw_dtype=1, accumulate=0, dbias=A, ws=(A, 1 << 30), stream=0)
+             dx=A, dw_flat=A, dw_offset=0, dw_dtype=1, flags=0, dbias=A, ws=(A, 1 << 30), stream=0)
     a.update(kw)
     return P.osdp_split_linear_bwd(**a)
 
@@ -91,6 +97,10 @@ def test_forward_argument_checks():
     assert _fwd(k_split=-1) == 3 and _fwd(k_split=9) == 3 and _fwd(split_dim=2) == 3
     assert _fwd(act=3) == 6
     assert _fwd(split_dim=1, ws=(A, 256)) == 5          # the carry does not fit
+    assert _fwd(split_dim=1, ws=(A, 256), flags=P.FLAG_CARRY_BF16) in (0, 7)   # bf16 running sum: no carry needed
+    assert _fwd(flags=P.FLAG_CARRY_BF16, act=1) == 6    # the bf16 running sum excludes an activation ...
+    assert _fwd(flags=P.FLAG_CARRY_BF16, z_save=A) == 6  # ... and a saved pre-activation
+    assert _fwd(flags=4) == 6 and _fwd(flags=P.FLAG_ACCUMULATE_DW) == 6
     assert P.osdp_split_linear_fwd_slice(A, A, 0, None, 64, 64, 64, 2, 0, 0, 2, A, None, (A, 1 << 20), stream=0) == 3
     # a well-formed call gets past the checks and fails only because there is no device / fake pointers
     if not _cuda():
@@ -104,6 +114,9 @@ def test_backward_argument_checks():
     assert _bwd(dw_offset=12) == 4 and _bwd(dx=A + 4) == 4 and _bwd(dbias=A + 4) == 4
     assert _bwd(k_split=9) == 3
     assert _bwd(ws=(A, 1024)) == 5
+    assert _bwd(flags=8) == 6
+    # with the bf16 running sum the backward needs only the column-sum partials
+    assert _bwd(ws=(A, 256 + 64 * 4), flags=P.FLAG_CARRY_BF16) in (0, 7)
     assert P.osdp_split_linear_bwd_slice(A, A, A, 0, None, 64, 64, 64, 2, 0, 0, -1, A, A, 0, 1, 0, A, (A, 1 << 20),
                                          stream=0) == 3
 
@@ -115,7 +128,7 @@ def test_mlp_argument_checks():
     assert f(x=None) == 1 and f(off_w2=3) == 4 and f(k_split=64) == 3 and f(ws=(A, 256)) == 5 and f(ffn=100) == 4
     b = lambda **kw: P.osdp_split_mlp_bwd(**dict(dict(dy=A, x=A, w_flat=A, off_w1=0, off_w2=64 * 256, z1_saved=A,
                                                       M=32, hidden=64, ffn=256, k_split=4, act=1, dx=A, dw_flat=A,
-                                                      dw_off_w1=0, dw_off_w2=64 * 256, dw_dtype=1, accumulate=0,
+                                                      dw_off_w1=0, dw_off_w2=64 * 256, dw_dtype=1, flags=0,
                                                       db1=A, db2=A, ws=(A, 1 << 30), stream=0), **kw))
     assert b(z1_saved=None) == 1 and b(dw_dtype=5) == 6 and b(dw_off_w1=4) == 4 and b(ws=(A, 4096)) == 5
 
