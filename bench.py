@@ -33,12 +33,12 @@ WORKLOAD = {"name": "split sweep GEMM M=16384 N=K=8192 bf16", "M": 16384, "N": 8
 METRIC = "split-linear fwd+bwd TFLOP/s"
 UNIT = "TFLOP/s"
 
-# DRAM bytes per launch of the dominant kernel from the committed ncu capture
-# (profiles/gemm_kernel_split_sweep.md): dram__bytes_read.sum + dram__bytes_write.sum.
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture of this
+# very command at full size, summarised in profiles/bench_split_sweep_k8_launch_list.md.
 NCU_TRAFFIC_BYTES = {
-    ("fwd", 8, "out"): 4005381632 + 262917120,
-    ("dx", 8, "out"): 5712420864 + 4002958592,
-    ("dw", 8, "out"): 4608154880 + 128154112,
+    ("fwd", 8, "out"): 3969529856 + 262909696,
+    ("dx", 8, "out"): 5697532160 + 4002740224,
+    ("dw", 8, "out"): 4107251968 + 127880448,
 }
 
 
