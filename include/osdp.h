@@ -169,6 +169,13 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
  * clears it.  Every device-side wait in this library is bounded; none can hang the GPU. */
 int osdp_read_device_status(void *ws, int *status, void *stream);
 
+/* Diagnostic for the failure-detection path (no counterpart in the paper): launches one warp that
+ * waits, with the bounded wait every kernel of this library uses, on a barrier nothing signals.
+ * After `limit_us` microseconds (1 .. 1 000 000) the wait gives up, the status word at the start of
+ * `ws` is set, and the kernel returns; osdp_read_device_status then reports
+ * OSDP_ERR_DEVICE_TIMEOUT.  The GPU context stays usable.  Asynchronous on `stream`. */
+int osdp_debug_wait_probe(void *ws, int64_t limit_us, void *stream);
+
 /* Bias gradient for callers that cannot allocate.  (The paper has no counterpart: it is an
  * addition for users of this library.)
  *

@@ -22,7 +22,7 @@ EXPORTS = [
     "osdp_version", "osdp_status_string", "osdp_last_cuda_error", "osdp_slice_range",
     "osdp_split_linear_workspace_bytes", "osdp_split_linear_fwd", "osdp_split_linear_fwd_slice",
     "osdp_split_linear_bwd", "osdp_split_linear_bwd_slice", "osdp_split_mlp_fwd", "osdp_split_mlp_bwd",
-    "osdp_read_device_status", "osdp_bias_grad_noalloc",
+    "osdp_read_device_status", "osdp_bias_grad_noalloc", "osdp_debug_wait_probe",
 ]
 
 _lib = None
@@ -68,6 +68,7 @@ def lib():
                                          vp, vp, vp, sz, vp]
         L.osdp_read_device_status.argtypes = [vp, ctypes.POINTER(ci), vp]
         L.osdp_bias_grad_noalloc.argtypes = [vp, i64, i64, vp, vp]
+        L.osdp_debug_wait_probe.argtypes = [vp, i64, vp]
         for name in EXPORTS:
             getattr(L, name)
             if name not in ("osdp_status_string",):
@@ -211,3 +212,11 @@ def osdp_bias_grad_noalloc(dy, M, N, dbias, stream=None, check=False):
     not touch the allocator).  Limit ceil(M/1024) * N <= 2**20; calls on one GPU must not overlap."""
     rc = lib().osdp_bias_grad_noalloc(_ptr(dy), int(M), int(N), _ptr(dbias), _stream(stream))
     return _ret(rc, check, "osdp_bias_grad_noalloc")
+
+
+def osdp_debug_wait_probe(ws, limit_us, stream=None, check=False):
+    """Launches the bounded-wait diagnostic: a wait that nothing satisfies ends after limit_us with the
+    device status word set (read it with osdp_read_device_status)."""
+    wp, _ = _ws(ws)
+    rc = lib().osdp_debug_wait_probe(wp, int(limit_us), _stream(stream))
+    return _ret(rc, check, "osdp_debug_wait_probe")

@@ -879,6 +879,16 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
   return OSDP_OK;
 }
 
+int osdp_debug_wait_probe(void *ws, int64_t limit_us, void *stream_) {
+  if (!ws) return OSDP_ERR_NULL_POINTER;
+  if (limit_us < 1 || limit_us > 1000000) return OSDP_ERR_BAD_SHAPE;
+  wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream_)>>>(static_cast<int *>(ws),
+                                                                    (unsigned long long)limit_us * 1000ull);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  return OSDP_OK;
+}
+
 int osdp_read_device_status(void *ws, int *status, void *stream_) {
   if (!ws || !status) return OSDP_ERR_NULL_POINTER;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);

@@ -107,7 +107,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false when the CTA is unwinding (this wait or another one ran out).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                          int *status, int code) {
+                                          int *status, int code, unsigned long long limit_ns = WAIT_LIMIT_NS) {
   if (mbar_try_wait(bar, parity)) return true;
   uint32_t polls = 0;
   unsigned long long t0 = 0;
@@ -118,7 +118,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       unsigned long long now = globaltimer_ns();
       if (t0 == 0) {
         t0 = now;
-      } else if (now - t0 > WAIT_LIMIT_NS) {
+      } else if (now - t0 > limit_ns) {
         *abort_flag = 1;
         if (status) atomicCAS(status, 0, code);
         return false;
@@ -938,6 +938,21 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
     tc_fence_after();
     tmem_dealloc<CTA2>(tmem_base, SL::TMEM_COLS);
   }
+}
+
+// Diagnostic: one warp waits, with the same bounded wait the GEMM uses, on a barrier that nothing
+// ever signals.  The wait gives up after limit_ns, records STATUS_TIMEOUT_PROBE and the kernel returns.
+enum : int { STATUS_TIMEOUT_PROBE = 199 };
+__global__ void wait_probe_kernel(int *status, unsigned long long limit_ns) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    fence_barrier_init();
+  }
+  __syncthreads();
+  mbar_wait(smem_u32(&bar), 0, &abort_flag, status, STATUS_TIMEOUT_PROBE, limit_ns);
 }
 
 }  // namespace osdp

@@ -361,3 +361,23 @@ def test_config4_wide_layer_k8(P):
     # and the second, split along the reduction dim
     check_large_linear(P, 8192, 32768, 8192, 8, 0, 0.01, 40)
     check_large_linear(P, 8192, 8192, 32768, 8, 1, 0.01, 41)
+
+
+# ---------------------------------------------------------------------------------------------
+# failure detection without a fault: a wait that nothing satisfies ends with a status, not a hang
+
+def test_bounded_wait_reports_timeout_and_context_stays_usable(P):
+    import time
+    ws = P.new_workspace(4096)
+    assert P.osdp_read_device_status(ws) == (0, 0)
+    t0 = time.perf_counter()
+    P.osdp_debug_wait_probe(ws, 20000, check=True)        # 20 ms limit
+    rc, st = P.osdp_read_device_status(ws)
+    dt = time.perf_counter() - t0
+    assert rc == 0 and st == 8                            # OSDP_ERR_DEVICE_TIMEOUT
+    assert 0.015 < dt < 2.0
+    assert P.osdp_read_device_status(ws) == (0, 0)        # the status word was cleared
+    # the context is intact: a normal call still works and matches the oracle
+    c = inputs.linear_case(128, 256, 64, layer=13)
+    compare(run_linear(P, c, 2, P.SPLIT_OUT), oracle_linear(c, 0, 2, oracle.SPLIT_OUT), 0)
+    assert P.osdp_debug_wait_probe(ws, 0) == 2 and P.osdp_debug_wait_probe(None, 10) == 1
