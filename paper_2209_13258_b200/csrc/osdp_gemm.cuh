@@ -561,8 +561,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
   const bool a_mid = A_MN ? (p.mode == MODE_ROWS) : (p.mode == MODE_RED);   // slice cuts A's contiguous dim
   const bool b_mid = B_MN ? (p.mode == MODE_COLS) : (p.mode == MODE_RED);
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+  // With both operands MN-major a stage takes four to six copies; two warps then walk the ring in
+  // lock step (warp 0 arms the stage's barrier and loads A, warp 3 loads B) so that two threads issue
+  // them in parallel.  Otherwise warp 0 does it all (measured: the split costs 1-2 % there).
+  constexpr bool SPLIT_PRODUCER = A_MN && B_MN;
+  if (warp == 0 || (SPLIT_PRODUCER && warp == 3)) {
+    // ------------------------------------------------------------------ TMA producer(s)
+    const bool load_a = (warp == 0);
+    const bool load_b = SPLIT_PRODUCER ? (warp == 3) : true;
     int stage = 0;
     uint32_t phase = 0;
     uint32_t armed = 0, armed_phase = 0;   // per-stage bookkeeping for the unwind path
@@ -583,13 +589,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
           const uint32_t sa = smem_base + stage * SL::STAGE_BYTES;
           const uint32_t sb = sa + SL::A_BYTES;
           const uint32_t fb = full_bar(stage);
-          if (!CTA2 || rank == 0) mbar_expect_tx(fb, SL::STAGE_BYTES * (CTA2 ? 2 : 1));
+          if (load_a && (!CTA2 || rank == 0)) mbar_expect_tx(fb, SL::STAGE_BYTES * (CTA2 ? 2 : 1));
           const int kc = kb * BK;
           auto tma_load = [&](uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2) {
             if (CTA2) tma_load_3d_pair(dst, map, fb, c0, c1, c2);
             else tma_load_3d(dst, map, fb, c0, c1, c2);
           };
-          if (A_MN) {
+          if (!load_a) {
+          } else if (A_MN) {
 #pragma unroll
             for (int j = 0; j < BM / 64; ++j) {
               const int in = w.a_row + j * 64;
@@ -600,7 +607,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
             if (a_mid) tma_load(sa, amap, kc, a_sc, w.a_row);
             else tma_load(sa, amap, kc, w.a_row, a_sc);
           }
-          if (B_MN) {
+          if (!load_b) {
+          } else if (B_MN) {
 #pragma unroll
             for (int j = 0; j < BNL / 64; ++j) {
               const int in = w.b_col + j * 64;
@@ -618,7 +626,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
         if (++stage == SL::STAGES) { stage = 0; phase ^= 1u; }
       }
     }
-    if (!ok && rank == 0) {
+    if (!ok && rank == 0 && load_a) {
       // Unwinding: let the copies already issued land before the CTA's shared memory goes away.
       for (int st = 0; st < SL::STAGES; ++st) {
         if (!((armed >> st) & 1u)) continue;
