@@ -338,15 +338,52 @@ def run_ours(args):
     if world > 1:
         barrier()
 
-    # ---- end to end: pinned host inputs copied in, results copied out, every step
-    def e2e_step():
-        x.copy_(h_x, non_blocking=True); dy.copy_(h_dy, non_blocking=True)
-        step()
-        h_out.copy_(out, non_blocking=True); h_dx.copy_(dx, non_blocking=True)
-        h_dw.copy_(dw_flat, non_blocking=True); h_db.copy_(db, non_blocking=True)
+    # ---- end to end: every step copies its inputs in from pinned host memory and all its results
+    # out to pinned host memory.  Three streams (copy-in, compute, copy-out) and two sets of device
+    # buffers, so that step i+1's inputs arrive and step i-1's results leave while step i computes.
+    # The library calls are the same C-ABI calls, issued on the compute stream.
+    s_in, s_cmp, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    bufs = []
+    for _ in range(2):
+        bufs.append({"x": torch.empty_like(x), "dy": torch.empty_like(dy), "out": torch.empty_like(out),
+                     "dx": torch.empty_like(dx), "dw": torch.empty_like(dw_flat), "db": torch.empty_like(db),
+                     "in_done": torch.cuda.Event(), "cmp_done": torch.cuda.Event(), "out_done": torch.cuda.Event()})
+    ws_e2e = [ws, P.new_workspace(ws_bytes, dev)]
 
-    e2e_steps = max(min(args.steps, 10), 1)
-    ms_e2e = max_over_ranks(timed(e2e_step, e2e_steps, 1), world, dev)
+    def e2e_run(n):
+        for i in range(n):
+            b = bufs[i % 2]
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(b["cmp_done"])          # the step that last read these inputs has finished
+                b["x"].copy_(h_x, non_blocking=True); b["dy"].copy_(h_dy, non_blocking=True)
+                b["in_done"].record(s_in)
+            with torch.cuda.stream(s_cmp):
+                s_cmp.wait_event(b["in_done"])
+                s_cmp.wait_event(b["out_done"])         # its previous results have been copied out
+                w = ws_e2e[i % 2]
+                P.osdp_split_linear_fwd(b["x"], w_flat, 0, None, M, N, K, k, split, P.ACT_NONE, b["out"], None, w,
+                                        check=True)
+                P.osdp_split_linear_bwd(b["dy"], b["x"], w_flat, 0, None, M, N, K, k, split, P.ACT_NONE, b["dx"],
+                                        b["dw"], 0, P.DTYPE_BF16, 0, b["db"], w, check=True)
+                b["cmp_done"].record(s_cmp)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(b["cmp_done"])
+                h_out.copy_(b["out"], non_blocking=True); h_dx.copy_(b["dx"], non_blocking=True)
+                h_dw.copy_(b["dw"], non_blocking=True); h_db.copy_(b["db"], non_blocking=True)
+                b["out_done"].record(s_out)
+
+    e2e_steps = max(min(args.steps, 10), 2)
+    e2e_run(2)
+    barrier()
+    t0 = time.perf_counter()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(s_in)
+    e2e_run(e2e_steps)
+    for st in (s_in, s_cmp):
+        s_out.wait_stream(st)
+    e1.record(s_out)
+    barrier()
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev)
     e2e_value = aggregate_value(fl, e2e_steps, world, ms_e2e)
     h2d = (h_x.numel() + h_dy.numel()) * 2
     d2h = (h_out.numel() + h_dx.numel() + h_dw.numel()) * 2 + h_db.numel() * 4
@@ -387,7 +424,9 @@ def run_ours(args):
         "sweep": sweep, "staging_bytes": ws_bytes,
         "roofline": roofline, "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": ms_e2e / e2e_steps},
+                "ms_per_step": ms_e2e / e2e_steps,
+                "how": "pinned host -> device copies, C-ABI fwd+bwd, device -> pinned host copies, every step; "
+                       "copy-in / compute / copy-out on three streams over two buffer sets"},
         "gpu_launches": launches_per_step * args.steps,
         "clocks": sampler.summary() if sampler else None,
     }

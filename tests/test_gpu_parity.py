@@ -381,3 +381,66 @@ def test_bounded_wait_reports_timeout_and_context_stays_usable(P):
     c = inputs.linear_case(128, 256, 64, layer=13)
     compare(run_linear(P, c, 2, P.SPLIT_OUT), oracle_linear(c, 0, 2, oracle.SPLIT_OUT), 0)
     assert P.osdp_debug_wait_probe(ws, 0) == 2 and P.osdp_debug_wait_probe(None, 10) == 1
+
+
+# ---------------------------------------------------------------------------------------------
+# config 4 as the chained MLP block (hidden 8192, ffn 32768, tokens 4 x 2048), k = 8 along ffn:
+# sampled token rows (Y, dX) and sampled ffn units (dW1 rows, dW2 columns, db1) against the oracle
+
+def test_config4_mlp_chain_k8_sampled(P):
+    M, H, F, k = 8192, 8192, 32768, 8
+    c = inputs.mlp_case(M, H, F, w_std=0.01, bias_std=0.01, layer=42)
+    g = run_mlp(P, c, k, dw_fp32=False)
+    rng = np.random.default_rng(42)
+    L = F // k
+    rows = _sample_idx(M, [128, 256, M // 2], rng, extra=4)
+    _, y = oracle.mlp_fwd(c["x"][rows], c["w1"], c["b1"], c["w2"], c["b2"], oracle.ACT_GELU_TANH, k)
+    dX, _, _, _, _ = oracle.mlp_bwd(c["dy"][rows], c["x"][rows], c["w1"], c["b1"], c["w2"], oracle.ACT_GELU_TANH, k)
+    idx = torch.from_numpy(rows).cuda()
+    assert_close(to_f64(g["y"][idx]), y, "Y rows")
+    assert_close(to_f64(g["dx"][idx]), dX, "dX rows")
+    # gradients of the weights of sampled ffn units depend only on those units' rows of W1 / columns of W2
+    fu = _sample_idx(F, list(range(L, F, L)), rng, extra=4)
+    w1s = np.ascontiguousarray(c["w1"][fu]); w2s = np.ascontiguousarray(c["w2"][:, fu]); b1s = c["b1"][fu]
+    _, dW1, db1, dW2, _ = oracle.mlp_bwd(c["dy"], c["x"], w1s, b1s, w2s, oracle.ACT_GELU_TANH, None)
+    fidx = torch.from_numpy(fu).cuda()
+    assert_close(to_f64(g["dw1"][fidx]), dW1, "dW1 rows")
+    assert_close(to_f64(g["dw2"][:, fidx]), dW2, "dW2 columns")
+    assert_close(to_f64(g["db1"][fidx]), db1, "db1")
+    assert_close(to_f64(g["db2"]), inputs.bf16_bits_to_f32(c["dy"]).astype(np.float64).sum(axis=0), "db2",
+                 relf_tol=1e-5)
+
+
+# ---------------------------------------------------------------------------------------------
+# the calls are plain asynchronous launches: a captured CUDA graph replays them bit for bit
+
+def test_cuda_graph_replay_matches_eager(P):
+    c = inputs.linear_case(512, 1024, 512, bias_std=0.1, layer=14)
+    M, N, K = 512, 1024, 512
+    x, dy, wf, b = to_dev(c["x"]), to_dev(c["dy"]), to_dev(c["w_flat"]), to_dev(c["bias"])
+    _, n1 = P.osdp_split_linear_workspace_bytes(M, N, K, 4, 1, 0, P.OP_LINEAR_FWD)
+    _, n2 = P.osdp_split_linear_workspace_bytes(M, N, K, 4, 1, 0, P.OP_LINEAR_BWD)
+    ws = P.new_workspace(max(n1, n2))
+    outs = [torch.empty(M, N, dtype=torch.bfloat16, device="cuda"), torch.empty(M, K, dtype=torch.bfloat16, device="cuda"),
+            torch.empty(N * K, dtype=torch.float32, device="cuda"), torch.empty(N, dtype=torch.float32, device="cuda")]
+
+    def step():
+        P.osdp_split_linear_fwd(x, wf, 0, b, M, N, K, 4, P.SPLIT_RED, 0, outs[0], None, ws, check=True)
+        P.osdp_split_linear_bwd(dy, x, wf, 0, None, M, N, K, 4, P.SPLIT_RED, 0, outs[1], outs[2], 0, P.DTYPE_FP32, 0,
+                                outs[3], ws, check=True)
+
+    step()
+    torch.cuda.synchronize()
+    eager = [o.clone() for o in outs]
+    s = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(graph, stream=s):
+            step()
+    for o in outs:
+        o.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    for e, o in zip(eager, outs):
+        assert torch.equal(_bits(e), _bits(o))
+    assert P.osdp_read_device_status(ws) == (0, 0)
