@@ -1,6 +1,7 @@
 """Command-line runs of the split-linear path on synthetic tensors (device-side random data).
 
     python -m paper_2209_13258_b200.sweep case M N K k split        one fwd+bwd (twice), for profilers
+    python -m paper_2209_13258_b200.sweep case-mlp M hidden ffn k   one MLP-block fwd+bwd (twice), for profilers
     python -m paper_2209_13258_b200.sweep linear M N K [ks]         time vs slice granularity, both split dims
     python -m paper_2209_13258_b200.sweep mlp M hidden ffn [ks]     MLP block split along ffn: time and staging
 
@@ -66,6 +67,30 @@ def run_case(M, N, K, k, split):
     print("device status", P.osdp_read_device_status(ws))
 
 
+def run_case_mlp(M, H, F, k, flags=0):
+    dev = "cuda"
+    x = torch.randn(M, H, device=dev).bfloat16()
+    dy = torch.randn(M, H, device=dev).bfloat16()
+    wf = (torch.randn(2 * F * H, device=dev) * 0.02).bfloat16()
+    b1 = torch.zeros(F, device=dev)
+    b2 = torch.zeros(H, device=dev)
+    out = torch.empty(M, H, device=dev, dtype=torch.bfloat16)
+    z1 = torch.empty(M, F, device=dev, dtype=torch.bfloat16)
+    dx = torch.empty(M, H, device=dev, dtype=torch.bfloat16)
+    dwf = torch.empty(2 * F * H, device=dev, dtype=torch.bfloat16)
+    db1 = torch.empty(F, device=dev)
+    db2 = torch.empty(H, device=dev)
+    _, n1 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, 1, P.OP_MLP_FWD, flags)
+    _, n2 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, 1, P.OP_MLP_BWD, flags)
+    ws = P.new_workspace(max(n1, n2))
+    for _ in range(2):
+        P.osdp_split_mlp_fwd(x, wf, 0, b1, F * H, b2, M, H, F, k, 1, out, z1, ws, check=True, flags=flags)
+        P.osdp_split_mlp_bwd(dy, x, wf, 0, F * H, z1, M, H, F, k, 1, dx, dwf, 0, F * H, 0, flags, db1, db2, ws,
+                             check=True)
+        torch.cuda.synchronize()
+    print("device status", P.osdp_read_device_status(ws))
+
+
 def sweep_linear(M, N, K, ks):
     x, w, dy, out, dx, dw, db = _linear_tensors(M, N, K)
     flops = 3 * 2.0 * M * N * K
@@ -116,22 +141,25 @@ def sweep_mlp(M, H, F, ks):
     for k in ks:
         if P.osdp_slice_range(F, k, 0)[0] != 0:
             continue
-        _, n1 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, 1, P.OP_MLP_FWD)
-        _, n2 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, 1, P.OP_MLP_BWD)
-        cfgs.append((k, n1, n2))
+        for fl in ((0,) if k == 1 else (0, P.FLAG_CARRY_BF16)):
+            _, n1 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, 1, P.OP_MLP_FWD, fl)
+            _, n2 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, 1, P.OP_MLP_BWD, fl)
+            cfgs.append((k, n1, n2, fl))
     ws = P.new_workspace(max(max(c[1], c[2]) for c in cfgs))
     fns = []
-    for k, _, _ in cfgs:
-        fns.append(lambda k=k: P.osdp_split_mlp_fwd(x, wf, 0, b1, F * H, b2, M, H, F, k, 1, out, z1, ws, check=True))
-        fns.append(lambda k=k: P.osdp_split_mlp_bwd(dy, x, wf, 0, F * H, z1, M, H, F, k, 1, dx, dwf, 0, F * H, 0, 0,
-                                                    db1, db2, ws, check=True))
+    for k, _, _, fl in cfgs:
+        fns.append(lambda k=k, fl=fl: P.osdp_split_mlp_fwd(x, wf, 0, b1, F * H, b2, M, H, F, k, 1, out, z1, ws,
+                                                           check=True, flags=fl))
+        fns.append(lambda k=k, fl=fl: P.osdp_split_mlp_bwd(dy, x, wf, 0, F * H, z1, M, H, F, k, 1, dx, dwf, 0, F * H,
+                                                           0, fl, db1, db2, ws, check=True))
     ts = _time_interleaved(fns)
     rows = []
     base = ts[0] + ts[1]
-    for i, (k, n1, n2) in enumerate(cfgs):
+    for i, (k, n1, n2, fl) in enumerate(cfgs):
         tf, tb = ts[2 * i], ts[2 * i + 1]
         t = tf + tb
-        rows.append({"k": k, "fwd_ms": tf, "bwd_ms": tb, "ms": t, "tflops": flops / t / 1e9,
+        rows.append({"k": k, "carry": "bf16" if fl else "fp32", "fwd_ms": tf, "bwd_ms": tb, "ms": t,
+                     "tflops": flops / t / 1e9,
                      "overhead_vs_k1": t / base - 1.0, "staging_fwd_bytes": n1, "staging_bwd_bytes": n2})
         print(json.dumps(rows[-1]), flush=True)
     return rows
@@ -142,9 +170,11 @@ def main(argv):
         print(__doc__)
         return 2
     mode = argv[1]
-    ks = [int(v) for v in argv[5].split(",")] if len(argv) > 5 and mode != "case" else [1, 2, 4, 8, 16, 32]
+    ks = [int(v) for v in argv[5].split(",")] if len(argv) > 5 and not mode.startswith("case") else [1, 2, 4, 8, 16, 32]
     if mode == "case":
         run_case(*[int(v) for v in argv[2:7]])
+    elif mode == "case-mlp":
+        run_case_mlp(*[int(v) for v in argv[2:6]])
     elif mode == "linear":
         sweep_linear(int(argv[2]), int(argv[3]), int(argv[4]), ks)
     elif mode == "mlp":
