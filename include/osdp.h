@@ -81,8 +81,9 @@ extern "C" {
 #define OSDP_FLAG_ACCUMULATE_DW 1   /* backward: dW += instead of dW = */
 #define OSDP_FLAG_CARRY_BF16 2      /* summed output: keep the running sum in the bf16 output buffer itself
                                      * (slice 0 stores, later slices add in bf16) instead of an fp32 carry in the
-                                     * workspace: no carry memory, half the carry traffic, one extra bf16 rounding
-                                     * per slice (relative Frobenius error about 1.1e-3 * sqrt(1 + (k+1)/2)).
+                                     * workspace: no carry memory, half the carry traffic, two extra bf16 roundings
+                                     * per slice (partial and sum).  Measured relative Frobenius error about
+                                     * 1.8e-3 * sqrt(1 + (k+1)/2): within 5e-3 up to k = 8, beyond it for k >= 16.
                                      * Only without activation and without z_save. */
 
 int osdp_version(void);

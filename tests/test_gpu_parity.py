@@ -444,3 +444,42 @@ def test_cuda_graph_replay_matches_eager(P):
     for e, o in zip(eager, outs):
         assert torch.equal(_bits(e), _bits(o))
     assert P.osdp_read_device_status(ws) == (0, 0)
+
+
+# ---------------------------------------------------------------------------------------------
+# seeded random shapes / splits / activations / flags: every tile-shape variant of the kernel
+# (CTA pairs, single CTAs with 256-, 128- and 64-wide tiles), slices narrower than a tile, one-row
+# batches, ragged everything
+
+def _random_cases(n, seed):
+    rng = np.random.default_rng(seed)
+    cases = []
+    while len(cases) < n:
+        big = rng.random() < 0.25
+        M = int(rng.integers(1, 3000 if big else 600))
+        N = 8 * int(rng.integers(1, 400 if big else 90))
+        K = 8 * int(rng.integers(1, 300 if big else 90))
+        split = int(rng.integers(0, 2))
+        D = N if split == 0 else K
+        k = int(rng.choice([1, 2, 3, 4, 5, 7, 8, 12, 16, max(1, D // 8)]))
+        act = int(rng.choice([0, 0, 1, 2]))
+        flags = 2 if (act == 0 and 1 < k <= 8 and rng.random() < 0.3) else 0   # bf16 running sum: k <= 8 only
+        cases.append((M, N, K, k, split, act, flags))
+    return cases
+
+
+@pytest.mark.parametrize("chunk", range(4))
+def test_random_shapes_against_oracle(P, chunk):
+    for idx, (M, N, K, k, split, act, flags) in enumerate(_random_cases(40, 2209)[chunk * 10:(chunk + 1) * 10]):
+        if P.osdp_slice_range(N if split == 0 else K, k, 0)[0] != 0:
+            continue
+        c = inputs.linear_case(M, N, K, w_std=0.05, bias_std=0.2, w_offset=8 * (idx % 5), flat_pad=8,
+                               layer=100 + chunk * 10 + idx)
+        g = run_linear(P, c, k, split, act=act, flags=flags, dw_fp32=bool(idx % 2))
+        o = oracle_linear(c, act, k, split)
+        loose = 3e-2 * (2 * k) ** 0.5 if flags else 3e-2
+        try:
+            compare(g, o, act, y_abs_tol=loose if split == 1 else 3e-2, dx_abs_tol=loose if split == 0 else 3e-2)
+        except AssertionError as e:
+            raise AssertionError("case M=%d N=%d K=%d k=%d split=%d act=%d flags=%d: %s" % (
+                M, N, K, k, split, act, flags, e))
