@@ -85,6 +85,8 @@ extern "C" {
                                      * per slice (partial and sum).  Measured relative Frobenius error about
                                      * 1.8e-3 * sqrt(1 + (k+1)/2): within 5e-3 up to k = 8, beyond it for k >= 16.
                                      * Only without activation and without z_save. */
+#define OSDP_FLAG_RECOMPUTE 4       /* osdp_split_mlp_bwd: recompute the first layer's pre-activation slice by
+                                     * slice instead of reading z1_saved (activation checkpointing). */
 
 int osdp_version(void);
 const char *osdp_status_string(int status);
@@ -158,8 +160,14 @@ int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const 
 /* Backward of the split MLP block, slice by slice, from the saved pre-activation z1_saved
  * [M,ffn] bf16:  dA_s = dY W2[:,F_s]; dZ_s = dA_s (.) act'(Z1_s); dW2[:,F_s] = dY^T act(Z1_s);
  * dW1[F_s,:] = dZ_s^T X; db1[F_s] = colsum dZ_s; dX = sum_s dZ_s W1[F_s,:]; db2 = colsum dY.
- * dW1/dW2 land at dw_off_w1/dw_off_w2 of dw_flat (dw_dtype).  Slice-sized dZ_s and A_s live in ws. */
-int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_t off_w1,
+ * dW1/dW2 land at dw_off_w1/dw_off_w2 of dw_flat (dw_dtype).  Slice-sized dZ_s and A_s live in ws.
+ * With OSDP_FLAG_RECOMPUTE (the paper's Section 2.3 setting, activation checkpointing) z1_saved is
+ * not read (may be NULL): Z1_s = X W1[F_s,:]^T + b1[F_s] is recomputed per slice (one more GEMM,
+ * one more slice-sized buffer), so that no [M,ffn] activation exists between forward and backward.
+ * dX, dW1, db1 are bit-identical to the saved-activation path; dW2 = dY^T act(Z1_s) uses the
+ * activation of the unrounded pre-activation, as the forward did.  b1 [ffn] fp32 or NULL is only
+ * read then. */
+int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_t off_w1, const float *b1,
                        int64_t off_w2, const void *z1_saved, int64_t M, int64_t hidden, int64_t ffn,
                        int k_split, int act, void *dx, void *dw_flat, int64_t dw_off_w1,
                        int64_t dw_off_w2, int dw_dtype, int flags, float *db1, float *db2,

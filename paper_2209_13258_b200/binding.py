@@ -16,7 +16,7 @@ SPLIT_OUT, SPLIT_RED = 0, 1
 ACT_NONE, ACT_GELU_TANH, ACT_GELU_ERF = 0, 1, 2
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 OP_LINEAR_FWD, OP_LINEAR_BWD, OP_MLP_FWD, OP_MLP_BWD = 0, 1, 2, 3
-FLAG_ACCUMULATE_DW, FLAG_CARRY_BF16 = 1, 2
+FLAG_ACCUMULATE_DW, FLAG_CARRY_BF16, FLAG_RECOMPUTE = 1, 2, 4
 
 EXPORTS = [
     "osdp_version", "osdp_status_string", "osdp_last_cuda_error", "osdp_slice_range",
@@ -64,8 +64,8 @@ def lib():
         L.osdp_split_linear_bwd.argtypes = bwd + [vp, vp, i64, ci, ci, vp, vp, sz, vp]
         L.osdp_split_linear_bwd_slice.argtypes = bwd + [ci, vp, vp, i64, ci, ci, vp, vp, sz, vp]
         L.osdp_split_mlp_fwd.argtypes = [vp, vp, i64, vp, i64, vp, i64, i64, i64, ci, ci, ci, vp, vp, vp, sz, vp]
-        L.osdp_split_mlp_bwd.argtypes = [vp, vp, vp, i64, i64, vp, i64, i64, i64, ci, ci, vp, vp, i64, i64, ci, ci,
-                                         vp, vp, vp, sz, vp]
+        L.osdp_split_mlp_bwd.argtypes = [vp, vp, vp, i64, vp, i64, vp, i64, i64, i64, ci, ci, vp, vp, i64, i64, ci,
+                                         ci, vp, vp, vp, sz, vp]
         L.osdp_read_device_status.argtypes = [vp, ctypes.POINTER(ci), vp]
         L.osdp_bias_grad_noalloc.argtypes = [vp, i64, i64, vp, vp]
         L.osdp_debug_wait_probe.argtypes = [vp, i64, vp]
@@ -189,9 +189,11 @@ def osdp_split_mlp_fwd(x, w_flat, off_w1, b1, off_w2, b2, M, hidden, ffn, k_spli
 
 
 def osdp_split_mlp_bwd(dy, x, w_flat, off_w1, off_w2, z1_saved, M, hidden, ffn, k_split, act, dx, dw_flat,
-                       dw_off_w1, dw_off_w2, dw_dtype, flags, db1, db2, ws, stream=None, check=False):
+                       dw_off_w1, dw_off_w2, dw_dtype, flags, db1, db2, ws, stream=None, check=False, b1=None):
+    """b1 is only read with FLAG_RECOMPUTE (z1_saved may then be None)."""
     wp, wn = _ws(ws)
-    rc = lib().osdp_split_mlp_bwd(_ptr(dy), _ptr(x), _ptr(w_flat), int(off_w1), int(off_w2), _ptr(z1_saved), int(M),
+    rc = lib().osdp_split_mlp_bwd(_ptr(dy), _ptr(x), _ptr(w_flat), int(off_w1), _ptr(b1), int(off_w2),
+                                  _ptr(z1_saved), int(M),
                                   int(hidden), int(ffn), int(k_split), int(act), _ptr(dx), _ptr(dw_flat),
                                   int(dw_off_w1), int(dw_off_w2), int(dw_dtype), int(flags), _ptr(db1),
                                   _ptr(db2), wp, wn, _stream(stream))

@@ -90,6 +90,7 @@ struct WsPlan {
   size_t carry_off, carry_bytes;      // fp32 running sum of the summed output
   size_t stage0_off, stage0_bytes;    // bf16 slice staging (G_s, A_s)
   size_t stage1_off, stage1_bytes;    // second bf16 slice staging (dZ_s)
+  size_t stage2_off, stage2_bytes;    // third bf16 slice staging (recomputed Z1_s)
   size_t part_off, part_bytes;        // column-sum partials
   size_t total;
 };
@@ -136,6 +137,7 @@ int plan_workspace(int64_t M, int64_t N, int64_t K, int k, int split_dim, int ac
       if (k > 1 && fp32_carry) take((size_t)M * K * 4, &w->carry_off, &w->carry_bytes);
       take((size_t)M * L * 2, &w->stage0_off, &w->stage0_bytes);
       take((size_t)M * L * 2, &w->stage1_off, &w->stage1_bytes);
+      if (flags & OSDP_FLAG_RECOMPUTE) take((size_t)M * L * 2, &w->stage2_off, &w->stage2_bytes);
       take(chunks * (size_t)(L > K ? L : K) * 4, &w->part_off, &w->part_bytes);
       break;
     default:
@@ -672,7 +674,8 @@ int osdp_split_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int k_spl
                                       int flags, size_t *bytes) {
   if (!bytes) return OSDP_ERR_NULL_POINTER;
   if (act != OSDP_ACT_NONE && act != OSDP_ACT_GELU_TANH && act != OSDP_ACT_GELU_ERF) return OSDP_ERR_UNSUPPORTED;
-  if (flags & ~(OSDP_FLAG_ACCUMULATE_DW | OSDP_FLAG_CARRY_BF16)) return OSDP_ERR_UNSUPPORTED;
+  if (flags & ~(OSDP_FLAG_ACCUMULATE_DW | OSDP_FLAG_CARRY_BF16 | OSDP_FLAG_RECOMPUTE)) return OSDP_ERR_UNSUPPORTED;
+  if ((flags & OSDP_FLAG_RECOMPUTE) && op != OSDP_OP_MLP_BWD) return OSDP_ERR_UNSUPPORTED;
   WsPlan plan;
   int rc = plan_workspace(M, N, K, k_split, split_dim, act, op, flags, &plan);
   if (rc) return rc;
@@ -774,12 +777,14 @@ int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const 
   return OSDP_OK;
 }
 
-int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_t off_w1, int64_t off_w2,
-                       const void *z1_saved, int64_t M, int64_t hidden, int64_t ffn, int k_split, int act, void *dx,
-                       void *dw_flat, int64_t dw_off_w1, int64_t dw_off_w2, int dw_dtype, int flags, float *db1,
-                       float *db2, void *ws, size_t ws_bytes, void *stream_) {
-  if (!dy || !x || !w_flat || !z1_saved) return OSDP_ERR_NULL_POINTER;
-  if (flags & ~(OSDP_FLAG_ACCUMULATE_DW | OSDP_FLAG_CARRY_BF16)) return OSDP_ERR_UNSUPPORTED;
+int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_t off_w1, const float *b1,
+                       int64_t off_w2, const void *z1_saved, int64_t M, int64_t hidden, int64_t ffn, int k_split,
+                       int act, void *dx, void *dw_flat, int64_t dw_off_w1, int64_t dw_off_w2, int dw_dtype,
+                       int flags, float *db1, float *db2, void *ws, size_t ws_bytes, void *stream_) {
+  if (flags & ~(OSDP_FLAG_ACCUMULATE_DW | OSDP_FLAG_CARRY_BF16 | OSDP_FLAG_RECOMPUTE)) return OSDP_ERR_UNSUPPORTED;
+  const bool recompute = (flags & OSDP_FLAG_RECOMPUTE) != 0;
+  if (!dy || !x || !w_flat || (!recompute && !z1_saved)) return OSDP_ERR_NULL_POINTER;
+  if (!aligned16(b1)) return OSDP_ERR_ALIGNMENT;
   const int accumulate = (flags & OSDP_FLAG_ACCUMULATE_DW) ? 1 : 0;
   int64_t L = 0;
   int rc = check_common(M, ffn, hidden, k_split, OSDP_SPLIT_OUT, act, &L);
@@ -805,6 +810,7 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
   const __nv_bfloat16 *z1 = static_cast<const __nv_bfloat16 *>(z1_saved);
   __nv_bfloat16 *a_s = reinterpret_cast<__nv_bfloat16 *>(wsb + plan.stage0_off);
   __nv_bfloat16 *dz_s = reinterpret_cast<__nv_bfloat16 *>(wsb + plan.stage1_off);
+  __nv_bfloat16 *z1_s = reinterpret_cast<__nv_bfloat16 *>(wsb + plan.stage2_off);
   float *carry = reinterpret_cast<float *>(wsb + plan.carry_off);
   float *partial = reinterpret_cast<float *>(wsb + plan.part_off);
   int *status = static_cast<int *>(ws);
@@ -819,17 +825,33 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
     const int64_t lo = (int64_t)s * L;
     const int64_t ls = (lo + L < ffn ? lo + L : ffn) - lo;
     GemmCall c;
-    // dZ_s = (dY W2[:,F_s]) (.) act'(Z1_s);  A_s = act(Z1_s)
+    if (recompute) {
+      // Z1_s = X W1[F_s,:]^T + b1[F_s] (the forward's first GEMM again, same bits), A_s = act(Z1_s)
+      memset(&c, 0, sizeof(c));
+      c.a = Operand{x, hidden, M, hidden, false, false};
+      c.b = Operand{w1 + lo * hidden, hidden, ls, hidden, false, false};
+      c.P = M; c.Q = ls; c.R = hidden; c.bn_P = M; c.bn_Q = L;
+      c.mode = MODE_NONE; c.L = ls; c.k_total = 1; c.s_begin = 0; c.s_end = 1;
+      c.epi = plain_epilogue(a_s, L, 0);
+      c.epi.bias = b1 ? b1 + lo : nullptr;
+      c.epi.z_save = z1_s;
+      c.epi.ld_z = L;
+      c.epi.act = act;
+      c.status = status;
+      rc = launch_gemm(c, stream);
+      if (rc) return rc;
+    }
+    // dZ_s = (dY W2[:,F_s]) (.) act'(Z1_s);  A_s = act(Z1_s) unless it was just recomputed
     memset(&c, 0, sizeof(c));
     c.a = Operand{dy, hidden, M, hidden, false, false};
     c.b = Operand{w2 + lo, ls, hidden, ffn, true, false};
     c.P = M; c.Q = ls; c.R = hidden; c.bn_P = M; c.bn_Q = L;
     c.mode = MODE_NONE; c.L = ls; c.k_total = 1; c.s_begin = 0; c.s_end = 1;
     c.epi = plain_epilogue(dz_s, L, 0);
-    c.epi.gz = z1 + lo;
-    c.epi.ld_gz = ffn;
+    c.epi.gz = recompute ? z1_s : z1 + lo;
+    c.epi.ld_gz = recompute ? L : ffn;
     c.epi.gz_act = act;
-    c.epi.act_out = a_s;
+    c.epi.act_out = recompute ? nullptr : a_s;
     c.epi.ld_act_out = L;
     c.status = status;
     rc = launch_gemm(c, stream);

@@ -141,24 +141,25 @@ def sweep_mlp(M, H, F, ks):
     for k in ks:
         if P.osdp_slice_range(F, k, 0)[0] != 0:
             continue
-        for fl in ((0,) if k == 1 else (0, P.FLAG_CARRY_BF16)):
-            _, n1 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, 1, P.OP_MLP_FWD, fl)
+        for fl in ((0, P.FLAG_RECOMPUTE) if k == 1 else (0, P.FLAG_CARRY_BF16, P.FLAG_RECOMPUTE)):
+            _, n1 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, 1, P.OP_MLP_FWD, fl & P.FLAG_CARRY_BF16)
             _, n2 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, 1, P.OP_MLP_BWD, fl)
             cfgs.append((k, n1, n2, fl))
     ws = P.new_workspace(max(max(c[1], c[2]) for c in cfgs))
     fns = []
     for k, _, _, fl in cfgs:
         fns.append(lambda k=k, fl=fl: P.osdp_split_mlp_fwd(x, wf, 0, b1, F * H, b2, M, H, F, k, 1, out, z1, ws,
-                                                           check=True, flags=fl))
+                                                           check=True, flags=fl & P.FLAG_CARRY_BF16))
         fns.append(lambda k=k, fl=fl: P.osdp_split_mlp_bwd(dy, x, wf, 0, F * H, z1, M, H, F, k, 1, dx, dwf, 0, F * H,
-                                                           0, fl, db1, db2, ws, check=True))
+                                                           0, fl, db1, db2, ws, check=True, b1=b1))
     ts = _time_interleaved(fns)
     rows = []
     base = ts[0] + ts[1]
     for i, (k, n1, n2, fl) in enumerate(cfgs):
         tf, tb = ts[2 * i], ts[2 * i + 1]
         t = tf + tb
-        rows.append({"k": k, "carry": "bf16" if fl else "fp32", "fwd_ms": tf, "bwd_ms": tb, "ms": t,
+        rows.append({"k": k, "carry": "bf16" if fl & P.FLAG_CARRY_BF16 else "fp32",
+                     "recompute": bool(fl & P.FLAG_RECOMPUTE), "fwd_ms": tf, "bwd_ms": tb, "ms": t,
                      "tflops": flops / t / 1e9,
                      "overhead_vs_k1": t / base - 1.0, "staging_fwd_bytes": n1, "staging_bwd_bytes": n2})
         print(json.dumps(rows[-1]), flush=True)

@@ -232,7 +232,7 @@ def test_maximum_split_and_tiny_shapes(P):
 # ---------------------------------------------------------------------------------------------
 # config 2: transformer MLP block, hidden 1024, ffn 4096, tokens 8 x 512, split along ffn
 
-def run_mlp(P, c, k, act=1, dw_fp32=True, flags=0):
+def run_mlp(P, c, k, act=1, dw_fp32=True, flags=0, recompute=False):
     M, H, F = c["M"], c["hidden"], c["ffn"]
     x, dy, wf = to_dev(c["x"]), to_dev(c["dy"]), to_dev(c["w_flat"])
     b1, b2 = to_dev(c["b1"]), to_dev(c["b2"])
@@ -244,8 +244,17 @@ def run_mlp(P, c, k, act=1, dw_fp32=True, flags=0):
     ws = P.new_workspace(max(n1, n2))
     P.osdp_split_mlp_fwd(x, wf, c["off_w1"], b1, c["off_w2"], b2, M, H, F, k, act, out.t, z1.t, ws, check=True,
                          flags=flags)
-    P.osdp_split_mlp_bwd(dy, x, wf, c["off_w1"], c["off_w2"], z1.t, M, H, F, k, act, dx.t, dwf.t, c["off_w1"],
-                         c["off_w2"], P.DTYPE_FP32 if dw_fp32 else P.DTYPE_BF16, flags, db1.t, db2.t, ws, check=True)
+    if recompute:
+        # activation checkpointing: the backward gets no saved activation and recomputes it per slice
+        _, n2 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, act, P.OP_MLP_BWD, flags | P.FLAG_RECOMPUTE)
+        ws = P.new_workspace(max(n1, n2))
+        P.osdp_split_mlp_bwd(dy, x, wf, c["off_w1"], c["off_w2"], None, M, H, F, k, act, dx.t, dwf.t, c["off_w1"],
+                             c["off_w2"], P.DTYPE_FP32 if dw_fp32 else P.DTYPE_BF16, flags | P.FLAG_RECOMPUTE,
+                             db1.t, db2.t, ws, check=True, b1=b1)
+    else:
+        P.osdp_split_mlp_bwd(dy, x, wf, c["off_w1"], c["off_w2"], z1.t, M, H, F, k, act, dx.t, dwf.t, c["off_w1"],
+                             c["off_w2"], P.DTYPE_FP32 if dw_fp32 else P.DTYPE_BF16, flags, db1.t, db2.t, ws,
+                             check=True)
     rc, st = P.osdp_read_device_status(ws)
     assert rc == 0 and st == 0
     for g in (out, z1, dx, dwf, db1, db2):
@@ -269,6 +278,23 @@ def test_mlp_small_ragged(P, k, flags):
     _, y = oracle.mlp_fwd(c["x"], c["w1"], c["b1"], c["w2"], c["b2"], oracle.ACT_GELU_TANH, k)
     grads = oracle.mlp_bwd(c["dy"], c["x"], c["w1"], c["b1"], c["w2"], oracle.ACT_GELU_TANH, k)
     compare_mlp(g, (y,) + tuple(grads), summed_abs_tol=3e-2 * (2 * k) ** 0.5 if flags else 3e-2)
+
+
+@pytest.mark.parametrize("k", [1, 3, 4])
+def test_mlp_backward_with_recomputation(P, k):
+    c = inputs.mlp_case(300, 264, 520, w_std=0.08, layer=15)
+    saved = run_mlp(P, c, k)
+    recomputed = run_mlp(P, c, k, recompute=True)
+    _, y = oracle.mlp_fwd(c["x"], c["w1"], c["b1"], c["w2"], c["b2"], oracle.ACT_GELU_TANH, k)
+    grads = oracle.mlp_bwd(c["dy"], c["x"], c["w1"], c["b1"], c["w2"], oracle.ACT_GELU_TANH, k)
+    compare_mlp(recomputed, (y,) + tuple(grads))
+    # The recomputed pre-activation has the same bits as the saved one, so everything derived from
+    # it is bit-identical.  dW2 = dY^T act(Z1) is not: the recomputation applies the activation to
+    # the unrounded pre-activation, exactly as the forward did, the saved path to its bf16 rounding.
+    for name in ("dx", "dw1", "db1", "db2"):
+        assert torch.equal(_bits(saved[name]), _bits(recomputed[name])), name
+    assert_close(to_f64(recomputed["dw2"]), to_f64(saved["dw2"]), "dW2 saved vs recomputed")
+    assert recomputed["staging"][0] > 0
 
 
 def test_config2_mlp_block_all_k(P):

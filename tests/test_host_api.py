@@ -131,6 +131,12 @@ def test_mlp_argument_checks():
                                                       dw_off_w1=0, dw_off_w2=64 * 256, dw_dtype=1, flags=0,
                                                       db1=A, db2=A, ws=(A, 1 << 30), stream=0), **kw))
     assert b(z1_saved=None) == 1 and b(dw_dtype=5) == 6 and b(dw_off_w1=4) == 4 and b(ws=(A, 4096)) == 5
+    # with recomputation no saved activation is needed, but one more slice-sized buffer is
+    assert b(z1_saved=None, flags=P.FLAG_RECOMPUTE) in (0, 7)
+    assert b(flags=16) == 6 and b(flags=P.FLAG_RECOMPUTE, b1=A + 4) == 4
+    plain = P.osdp_split_linear_workspace_bytes(32, 256, 64, 4, 0, 1, P.OP_MLP_BWD)[1]
+    assert P.osdp_split_linear_workspace_bytes(32, 256, 64, 4, 0, 1, P.OP_MLP_BWD, P.FLAG_RECOMPUTE)[1] == plain + 32 * 64 * 2
+    assert P.osdp_split_linear_workspace_bytes(32, 256, 64, 4, 0, 1, P.OP_MLP_FWD, P.FLAG_RECOMPUTE)[0] == 6
 
 
 def _cuda():
