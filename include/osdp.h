@@ -10,9 +10,9 @@
  *
  * and k = k_split slices are taken along
  *      OSDP_SPLIT_OUT : the N rows of W (outputs Y, dW, db concatenate; dX is summed), or
- *      OSDP_SPLIT_RED : the K columns of W and X -- the paper's own wording ("the last
- *                       dimension of the input data and the first dimension of the operator
- *                       ... all computation results are summed") -- Y is summed; dX, dW concatenate.
+ *      OSDP_SPLIT_RED : the K columns of W and X.  This is the split Section 3.3 describes: the
+ *                       input is cut along its last dimension, the operator along the matching
+ *                       one, and the slice products are added up.  Y is summed; dX, dW concatenate.
  * Slices are visited in ascending order (slice-major).  A summed output is carried between
  * slices as an fp32 running sum in the caller's workspace.
  *
@@ -116,8 +116,8 @@ int osdp_split_linear_fwd(const void *x, const void *w_flat, int64_t w_offset, c
                           int64_t M, int64_t N, int64_t K, int k_split, int split_dim, int act,
                           int flags, void *out, void *z_save, void *ws, size_t ws_bytes, void *stream);
 
-/* One slice of the forward (Section 3.3 step 2, "the computation of each slice is executed
- * sequentially"): lets a caller put other work between slices.  Slices must be issued in
+/* One slice of the forward (Section 3.3 step 2: the slices are computed one after another):
+ * lets a caller put other work between slices.  Slices must be issued in
  * ascending order on one stream with the same arguments and workspace: under RED slice 0
  * starts the carry and slice k-1 writes `out`. */
 int osdp_split_linear_fwd_slice(const void *x, const void *w_flat, int64_t w_offset, const float *bias,

@@ -16,7 +16,8 @@
  *   OUT split: the N rows of W are cut into k row ranges R_s (outputs concatenate,
  *              dX is the sum over slices).
  *   RED split: the K columns of W and of X are cut into k column ranges C_s (this is
- *              the paper's own wording: last dim of the input, results summed).
+ *              the split Section 3.3 describes: the input is cut along its last dimension and the
+ *              slice products are added up).
  * The split routines are written as literal loops over slices on sub-matrix views;
  * they do not call the unsplit routines, so "split == unsplit" is a test, not an
  * identity by construction.
