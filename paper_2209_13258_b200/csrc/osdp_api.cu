@@ -294,7 +294,7 @@ int launch_variant(const GemmParams &p, int64_t units, int sms, cudaStream_t str
     if (CTA2) {
       cudaLaunchConfig_t q = {};
       q.gridDim = dim3(2 * sms, 1, 1);
-      q.blockDim = dim3(NUM_THREADS, 1, 1);
+      q.blockDim = dim3(SL::THREADS, 1, 1);
       q.dynamicSmemBytes = SL::TOTAL;
       cudaLaunchAttribute qa[1];
       qa[0].id = cudaLaunchAttributeClusterDimension;
@@ -313,7 +313,7 @@ int launch_variant(const GemmParams &p, int64_t units, int sms, cudaStream_t str
   if (n_units <= 0) return OSDP_OK;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(CTA2 ? 2 * n_units : n_units, 1, 1);
-  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.blockDim = dim3(SL::THREADS, 1, 1);
   cfg.dynamicSmemBytes = SL::TOTAL;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -335,6 +335,18 @@ int launch_bn(const GemmParams &p, bool a_mn, bool b_mn, int64_t units, int sms,
 
 inline int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
+// Work items (tiles, summed over the launch's slices for concatenated outputs) for a tile shape.
+int64_t count_items(const GemmCall &c, int tm, int bn) {
+  if (c.mode == MODE_RED) return cdiv(c.P, tm) * cdiv(c.Q, bn);
+  const int64_t rows_full = (c.mode == MODE_ROWS) ? c.L : c.P;
+  const int64_t cols_full = (c.mode == MODE_COLS) ? c.L : c.Q;
+  const int nsl = c.s_end - c.s_begin;
+  const int last = c.s_end - 1;
+  const int64_t rows_last = (c.mode == MODE_ROWS) ? ((c.P - last * c.L) < c.L ? (c.P - last * c.L) : c.L) : c.P;
+  const int64_t cols_last = (c.mode == MODE_COLS) ? ((c.Q - last * c.L) < c.L ? (c.Q - last * c.L) : c.L) : c.Q;
+  return (int64_t)(nsl - 1) * cdiv(rows_full, tm) * cdiv(cols_full, bn) + cdiv(rows_last, tm) * cdiv(cols_last, bn);
+}
+
 int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   int sms = 0;
   int rc = device_sms(&sms);
@@ -349,12 +361,26 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   if (pair || cdiv(c.bn_P, BM) * cdiv(c.bn_Q, 256) >= want) bn = 256;
   else if (cdiv(c.bn_P, BM) * cdiv(c.bn_Q, 128) >= want) bn = 128;
   const int tm = pair ? 2 * BM : BM;
+  // Widest tile, 256 x 512 per CTA pair: 25 % fewer operand bytes per flop (the main loop is bound by
+  // its operand feed), but the accumulators fill the tensor memory, so the epilogue no longer
+  // overlaps the next tile's main loop.  It pays off for long reductions and when it does not leave
+  // a ragged last wave.  Measured model, per tile and CTA pair: 256-wide 6.5 ns per reduction
+  // element (epilogue hidden), 512-wide 11.5 ns per element plus 5 us of exposed epilogue; time =
+  // rounds of the persistent schedule x tile time.  Both tiles produce the same bits per element
+  // (same k-block order), so the choice may differ between launches.  Summed outputs keep 256.
+  if (pair && c.mode != MODE_RED) {
+    const int64_t units = sms / 2;
+    const int64_t red_len = c.R;
+    const double t_n = (double)cdiv(count_items(c, 2 * BM, 256), units) * (6.5e-3 * (double)red_len) + 5.0;
+    const double t_w = (double)cdiv(count_items(c, 2 * BM, 512), units) * (11.5e-3 * (double)red_len + 5.0);
+    if (t_w < 0.97 * t_n) bn = 512;
+  }
 
   GemmParams p;
   memset(&p, 0, sizeof(p));
   rc = make_operand_maps(c.a, true, c.mode, c.L, c.k_total, BM, &p.a_main, &p.a_tail, &p.a_sc_mul);
   if (rc) return rc;
-  rc = make_operand_maps(c.b, false, c.mode, c.L, c.k_total, pair ? bn / 2 : bn, &p.b_main, &p.b_tail, &p.b_sc_mul);
+  rc = make_operand_maps(c.b, false, c.mode, c.L, c.k_total, pair ? 128 : bn, &p.b_main, &p.b_tail, &p.b_sc_mul);
   if (rc) return rc;
   p.P = (int)c.P; p.Q = (int)c.Q; p.R = (int)c.R;
   p.mode = c.mode; p.L = (int)c.L; p.k_total = c.k_total; p.s_begin = c.s_begin; p.s_end = c.s_end;
@@ -386,18 +412,8 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   }
 
   // Work items of this launch (one per scheduling unit and tile).
-  int64_t items;
-  if (c.mode == MODE_RED) {
-    items = cdiv(c.P, tm) * cdiv(c.Q, bn);
-  } else {
-    const int64_t rows_full = (c.mode == MODE_ROWS) ? c.L : c.P;
-    const int64_t cols_full = (c.mode == MODE_COLS) ? c.L : c.Q;
-    const int nsl = c.s_end - c.s_begin;
-    const int last = c.s_end - 1;
-    const int64_t rows_last = (c.mode == MODE_ROWS) ? ((c.P - last * c.L) < c.L ? (c.P - last * c.L) : c.L) : c.P;
-    const int64_t cols_last = (c.mode == MODE_COLS) ? ((c.Q - last * c.L) < c.L ? (c.Q - last * c.L) : c.L) : c.Q;
-    items = (int64_t)(nsl - 1) * cdiv(rows_full, tm) * cdiv(cols_full, bn) + cdiv(rows_last, tm) * cdiv(cols_last, bn);
-  }
+  const int64_t items = count_items(c, tm, bn);
+  if (pair && bn == 512) return launch_bn<512, true>(p, c.a.mn_major, c.b.mn_major, items, sms, stream);
   if (pair) return launch_bn<256, true>(p, c.a.mn_major, c.b.mn_major, items, sms, stream);
   switch (bn) {
     case 256: return launch_bn<256, false>(p, c.a.mn_major, c.b.mn_major, items, sms, stream);

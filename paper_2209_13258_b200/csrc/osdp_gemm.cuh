@@ -307,18 +307,30 @@ __device__ __forceinline__ constexpr uint32_t make_idesc() {
 template <int BN, bool CTA2>
 struct SmemLayout {
   static constexpr int BNL = CTA2 ? BN / 2 : BN;   // B rows held by one CTA (a pair splits B between its CTAs)
+  // A pair's tile is made of NG column groups of 256 (one tcgen05.mma each per k-step, sharing A);
+  // of each group a CTA holds GB_ROWS rows of B.
+  static constexpr int NG = (CTA2 && BN > 256) ? BN / 256 : 1;
+  static constexpr int GB_ROWS = CTA2 ? BNL / NG : BN;
+  static constexpr int UMMA_N = BN / NG;
+  // Accumulator sets in tensor memory (512 columns in all): two, so that the epilogue of a tile
+  // overlaps the next tile's main loop, unless one tile already needs all 512 columns.
+  static constexpr int NBUF = (BN > 256) ? 1 : 2;
+  // With a single accumulator set the epilogue is exposed: eight warps drain it (two per TMEM lane
+  // quarter, half of the columns each) instead of four.
+  static constexpr int EPI_WARPS = (BN > 256) ? 8 : 4;
+  static constexpr int THREADS = 128 + 32 * EPI_WARPS;
   static constexpr int A_BYTES = BM * BK * 2;
   static constexpr int B_BYTES = BNL * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   // Epilogue staging: STG_BUFS boxes of 4 KB per epilogue warp (boxes in flight to/from global memory).
-  static constexpr int STG_BUFS = 2;
-  static constexpr int STG_BYTES = 4 * STG_BUFS * 4096;
+  static constexpr int STG_BUFS = (BN > 256) ? 1 : 2;
+  static constexpr int STG_BYTES = EPI_WARPS * STG_BUFS * 4096;
   static constexpr int RING_BYTES = 229376 - STG_BYTES;
   static constexpr int STAGES = (RING_BYTES / STAGE_BYTES) > 8 ? 8 : (RING_BYTES / STAGE_BYTES);
   static constexpr int STG_OFFSET = STAGES * STAGE_BYTES;
   static constexpr int BAR_OFFSET = STG_OFFSET + STG_BYTES;
   static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;   // barriers + alignment slack
-  static constexpr int TMEM_COLS = 2 * BN;
+  static constexpr int TMEM_COLS = NBUF * BN;
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -501,7 +513,7 @@ __device__ __forceinline__ void epilogue8(const Epilogue &e, long long row, int 
 // runs its own epilogue.  Per CTA a stage is 32 KB instead of 48 KB (6 stages instead of 4) and
 // half as many B bytes cross from L2 to shared memory per flop.
 template <int BN, bool A_MN, bool B_MN, bool CTA2>
-__global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
+__global__ void __launch_bounds__((BN > 256) ? 384 : 256, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
   using SL = SmemLayout<BN, CTA2>;
   constexpr int TM = CTA2 ? 2 * BM : BM;
   constexpr int BNL = SL::BNL;
@@ -530,9 +542,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull_bar(b), 1);
-      mbar_init(tempty_bar(b), CTA2 ? 8 : 4);
+      mbar_init(tempty_bar(b), SL::EPI_WARPS * (CTA2 ? 2 : 1));
     }
-    for (int b = 0; b < 4 * SL::STG_BUFS; ++b) mbar_init(bar_base + 8u * (2 * SL::STAGES + 5 + b), 1);   // carry prefetch
+    for (int b = 0; b < SL::EPI_WARPS * SL::STG_BUFS; ++b) mbar_init(bar_base + 8u * (2 * SL::STAGES + 5 + b), 1);   // carry prefetch
     *abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&p.a_main);
@@ -576,7 +588,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
     Work w;
     for (int i = 0; ok && get_work<TM, BN>(p, i, bid, G, w); ++i) {
       w.a_row += (int)rank * BM;            // this CTA's rows of the pair's tile
-      w.b_col += (int)rank * BNL;           // ... and its half of the B tile
+      w.b_col += (int)rank * SL::GB_ROWS * (CTA2 ? 1 : 0);   // ... and its half of each 256-column group of B
       const bool tail = (w.s == p.k_total - 1);
       const CUtensorMap *amap = (a_sliced && !tail) ? &p.a_main : &p.a_tail;
       const CUtensorMap *bmap = (b_sliced && !tail) ? &p.b_main : &p.b_tail;
@@ -611,13 +623,18 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
           } else if (B_MN) {
 #pragma unroll
             for (int j = 0; j < BNL / 64; ++j) {
-              const int in = w.b_col + j * 64;
+              constexpr int CPG = SL::GB_ROWS / 64;   // 64-wide chunks per column group
+              const int in = w.b_col + (j / CPG) * 256 + (j % CPG) * 64;
               if (b_mid) tma_load(sb + j * (BK * 128), bmap, in, b_sc, kc);
               else tma_load(sb + j * (BK * 128), bmap, in, kc, b_sc);
             }
           } else {
-            if (b_mid) tma_load(sb, bmap, kc, b_sc, w.b_col);
-            else tma_load(sb, bmap, kc, w.b_col, b_sc);
+#pragma unroll
+            for (int g = 0; g < SL::NG; ++g) {
+              const int row = w.b_col + g * 256;
+              if (b_mid) tma_load(sb + g * (SL::GB_ROWS * 128), bmap, kc, b_sc, row);
+              else tma_load(sb + g * (SL::GB_ROWS * 128), bmap, kc, row, b_sc);
+            }
           }
         }
         armed |= 1u << stage;
@@ -638,14 +655,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
     }
   } else if (warp == 1 && rank == 0) {
     // ------------------------------------------------------------------ MMA issuer (even CTA of a pair)
-    constexpr uint32_t idesc = make_idesc<TM, BN, A_MN, B_MN>();
+    constexpr uint32_t idesc = make_idesc<TM, SL::UMMA_N, A_MN, B_MN>();
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;
     Work w;
     for (int i = 0; ok && get_work<TM, BN>(p, i, bid, G, w); ++i) {
-      const int buf = i & 1;
-      const uint32_t bphase = (uint32_t)(i >> 1) & 1u;
+      const int buf = i % SL::NBUF;
+      const uint32_t bphase = (uint32_t)(i / SL::NBUF) & 1u;
       ok = mbar_wait(tempty_bar(buf), bphase ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA);
       if (!ok) break;
       tc_fence_after();
@@ -661,9 +678,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
           const uint64_t bdesc = make_smem_desc<B_MN>(sb);
 #pragma unroll
           for (int kk = 0; kk < BK / UMMA_K; ++kk) {
-            umma_bf16<CTA2>(d_tmem, adesc + (uint64_t)((kk * desc_k_advance<A_MN>()) >> 4),
-                      bdesc + (uint64_t)((kk * desc_k_advance<B_MN>()) >> 4), idesc,
-                      (kb > 0 || kk > 0) ? 1u : 0u);
+#pragma unroll
+            for (int g = 0; g < SL::NG; ++g) {
+              umma_bf16<CTA2>(d_tmem + (uint32_t)(g * SL::UMMA_N),
+                              adesc + (uint64_t)((kk * desc_k_advance<A_MN>()) >> 4),
+                              bdesc + (uint64_t)((g * SL::GB_ROWS * 128 + kk * desc_k_advance<B_MN>()) >> 4), idesc,
+                              (kb > 0 || kk > 0) ? 1u : 0u);
+            }
           }
           umma_commit<CTA2>(empty_bar(stage));                      // frees the stage when the MMAs retire
           if (kb == w.kblocks - 1) umma_commit<CTA2>(tfull_bar(buf));   // accumulator complete
@@ -681,8 +702,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
     // done by the memory system, nothing is read back), the last slice prefetches the carry
     // with TMA loads, adds its own partial and writes the final result.
     const int quarter = warp & 3;
+    const int wg = (warp - 4) >> 2;                 // which share of the tile's columns this warp drains
+    constexpr int EG = SL::EPI_WARPS / 4;
     constexpr uint32_t NB = SL::STG_BUFS;
-    const uint32_t stg = smem_base + SL::STG_OFFSET + (uint32_t)quarter * (NB * 4096u);
+    const uint32_t stg = smem_base + SL::STG_OFFSET + (uint32_t)(warp - 4) * (NB * 4096u);
     const uint32_t row_off = (uint32_t)lane * 128u;
     const uint32_t swz = (uint32_t)(lane & 7);
     const bool out_sliced = (p.mode == MODE_COLS) || (p.mode == MODE_ROWS);
@@ -694,8 +717,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
     for (int i = 0; ok && get_work<TM, BN>(p, i, bid, G, w); ++i) {
       w.a_row += (int)rank * BM;
       w.row0 += (int)rank * BM;
-      const int buf = i & 1;
-      const uint32_t bphase = (uint32_t)(i >> 1) & 1u;
+      const int buf = i % SL::NBUF;
+      const uint32_t bphase = (uint32_t)(i / SL::NBUF) & 1u;
       ok = mbar_wait(tfull_bar(buf), bphase, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE);
       if (!ok) break;
       tc_fence_after();
@@ -711,7 +734,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
       if (!p.tma_epilogue) {
         // direct stores from registers (used when the epilogue also reads a second tensor)
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
+        for (int c = wg * (BN / 32 / EG); c < (wg + 1) * (BN / 32 / EG); ++c) {
           const int cbase = w.col0 + c * 32;
           if (cbase >= w.col_end) break;
           uint32_t v[32];
@@ -770,7 +793,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
         if (w.carry_out) {
           // fp32 partial -> carry, 32 columns (128 bytes per row) per box
 #pragma unroll 1
-          for (int c = 0; c < BN / 32; ++c) {
+          for (int c = wg * (BN / 32 / EG); c < (wg + 1) * (BN / 32 / EG); ++c) {
             const int cbase = w.col0 + c * 32;
             if (cbase >= w.col_end) break;
             uint32_t v[32];
@@ -784,7 +807,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
           }
         } else if (w.carry_in) {
           // last slice: carry (prefetched by TMA, one box ahead) + accumulator -> bias/act -> out
-          const uint32_t cbar = bar_base + 8u * (2 * SL::STAGES + 5 + quarter * NB);
+          // (summed outputs are never given the 512-wide tile, so here every warp owns all columns)
+          const uint32_t cbar = bar_base + 8u * (2 * SL::STAGES + 5 + (warp - 4) * NB);
           int nchunks = (w.col_end - w.col0 + 31) / 32;
           if (nchunks > BN / 32) nchunks = BN / 32;
           auto issue_load = [&](int c) {
@@ -828,7 +852,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
         } else if (p.epi.out_fp32) {
           // fp32 output, 32 columns per box; += is a reduce-add
 #pragma unroll 1
-          for (int c = 0; c < BN / 32; ++c) {
+          for (int c = wg * (BN / 32 / EG); c < (wg + 1) * (BN / 32 / EG); ++c) {
             const int cbase = w.col0 + c * 32;
             if (cbase >= w.col_end) break;
             uint32_t v[32];
@@ -864,7 +888,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
         } else {
           // bf16 output, 64 columns (128 bytes per row) per box
 #pragma unroll 1
-          for (int c = 0; c < (BN + 63) / 64; ++c) {
+          for (int c = wg * ((BN + 63) / 64 / EG); c < (wg + 1) * ((BN + 63) / 64 / EG); ++c) {
             const int cbase = w.col0 + c * 64;
             if (cbase >= w.col_end) break;
             uint32_t v[64];
