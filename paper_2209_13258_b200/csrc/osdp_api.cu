@@ -316,10 +316,14 @@ int launch_variant(const GemmParams &p, int64_t units, int sms, cudaStream_t str
   cfg.blockDim = dim3(SL::THREADS, 1, 1);
   cfg.dynamicSmemBytes = SL::TOTAL;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = CTA2 ? 2 : 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr; cfg.numAttrs = 1;
+  // the kernel's prologue may overlap the tail of the previous kernel on the stream (it waits with
+  // griddepcontrol.wait before touching global memory)
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 2;
   e = cudaLaunchKernelEx(&cfg, kernel, p);
   if (e != cudaSuccess) return cuda_fail(e);
   return OSDP_OK;

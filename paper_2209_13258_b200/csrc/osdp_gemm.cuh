@@ -535,6 +535,11 @@ __global__ void __launch_bounds__((BN > 256) ? 384 : 256, 1) gemm_kernel(const _
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
 
+  // Programmatic dependent launch: the next kernel on the stream may be scheduled as soon as this
+  // grid's CTAs retire and may run its own prologue; it touches global memory only after its
+  // griddepcontrol.wait (below), which returns once this grid has completed and flushed.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
   if (threadIdx.x == 0) {
     for (int st = 0; st < SL::STAGES; ++st) {
       mbar_init(full_bar(st), 1);
@@ -565,6 +570,9 @@ __global__ void __launch_bounds__((BN > 256) ? 384 : 256, 1) gemm_kernel(const _
   __syncthreads();
   if (CTA2) cluster_sync_all();   // the peer's barriers exist before anything is signalled across the pair
   tc_fence_after();
+  // Everything above touched only shared and tensor memory.  From here on the kernel reads and
+  // writes global memory that an earlier kernel on the stream may have produced or may still read.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const uint32_t tmem_base = *tmem_holder;
 
   // Which operand dimension the slice coordinate belongs to (fixed by mode and operand major).
