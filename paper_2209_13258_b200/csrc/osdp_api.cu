@@ -435,15 +435,36 @@ Epilogue plain_epilogue(void *out, int64_t ld, int fp32) {
   return e;
 }
 
+// Launch of a helper kernel that takes part in programmatic dependent launch like the GEMMs.
+template <typename... KArgs, typename... Args>
+int launch_aux(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return OSDP_OK;
+}
+
 int launch_colsum(const void *g, int64_t ld, int64_t M, int c0, int ncols, float *partial, float *out,
                   cudaStream_t stream) {
   const int chunks = (int)cdiv(M, COLSUM_ROWS_PER_CHUNK);
   dim3 grid((unsigned)cdiv(ncols, 64), (unsigned)chunks);
-  colsum_partial_kernel<<<grid, 256, 0, stream>>>((const __nv_bfloat16 *)g, ld, M, c0, ncols, partial, ncols);
-  colsum_final_kernel<<<(unsigned)cdiv(ncols, 256), 256, 0, stream>>>(partial, ncols, chunks, ncols, out + c0);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return cuda_fail(e);
-  return OSDP_OK;
+  if (chunks == 1)   // one chunk of rows: its sums are the result (same summation order as the two-pass form)
+    return launch_aux(colsum_partial_kernel, grid, dim3(256), stream, (const __nv_bfloat16 *)g, (long long)ld,
+                      (long long)M, c0, ncols, out + c0, ncols);
+  int rc = launch_aux(colsum_partial_kernel, grid, dim3(256), stream, (const __nv_bfloat16 *)g, (long long)ld,
+                      (long long)M, c0, ncols, partial, ncols);
+  if (rc) return rc;
+  return launch_aux(colsum_final_kernel, dim3((unsigned)cdiv(ncols, 256)), dim3(256), stream,
+                    (const float *)partial, ncols, chunks, ncols, out + c0);
 }
 
 int launch_act_backward(const void *dy, int64_t ld_dy, const void *z, int64_t ld_z, void *g, int64_t ld_g, int64_t M,
@@ -454,11 +475,9 @@ int launch_act_backward(const void *dy, int64_t ld_dy, const void *z, int64_t ld
   const int64_t total = M * (ncols / 8);
   int64_t blocks = cdiv(total, 256);
   if (blocks > (int64_t)sms * 16) blocks = (int64_t)sms * 16;
-  act_backward_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const __nv_bfloat16 *)dy, ld_dy, (const __nv_bfloat16 *)z,
-                                                           ld_z, (__nv_bfloat16 *)g, ld_g, M, c0, ncols, act);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return cuda_fail(e);
-  return OSDP_OK;
+  return launch_aux(act_backward_kernel, dim3((unsigned)blocks), dim3(256), stream, (const __nv_bfloat16 *)dy,
+                    (long long)ld_dy, (const __nv_bfloat16 *)z, (long long)ld_z, (__nv_bfloat16 *)g, (long long)ld_g,
+                    (long long)M, c0, ncols, act);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -14,6 +14,8 @@ __global__ void __launch_bounds__(256) act_backward_kernel(const __nv_bfloat16 *
                                                            const __nv_bfloat16 *__restrict__ z, long long ld_z,
                                                            __nv_bfloat16 *__restrict__ g, long long ld_g,
                                                            long long M, int c0, int ncols, int act) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // inputs may come from the previous kernel on the stream
   const int vec_per_row = ncols >> 3;
   const long long total = M * vec_per_row;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
@@ -35,6 +37,8 @@ __global__ void __launch_bounds__(256) colsum_partial_kernel(const __nv_bfloat16
                                                              long long M, int c0, int ncols,
                                                              float *__restrict__ partial, int ld_partial) {
   __shared__ float2 red[8][32];
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const int col = blockIdx.x * 64 + tx * 2;
   const long long r0 = (long long)blockIdx.y * COLSUM_ROWS_PER_CHUNK;
@@ -67,6 +71,8 @@ __global__ void __launch_bounds__(256) colsum_partial_kernel(const __nv_bfloat16
 // out[c0 + c] = sum over chunks (ascending) of partial[chunk, c].
 __global__ void __launch_bounds__(256) colsum_final_kernel(const float *__restrict__ partial, int ld_partial,
                                                            int nchunks, int ncols, float *__restrict__ out) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
   if (c >= ncols) return;
   float s = 0.f;
