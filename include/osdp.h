@@ -106,6 +106,16 @@ int osdp_slice_range(int64_t D, int k_split, int slice_idx, int64_t *begin, int6
 int osdp_split_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int k_split, int split_dim,
                                       int act, int op, int flags, size_t *bytes);
 
+/* Slice-granularity suggestion (the paper's Section 5 leaves "how to automatically suggest a
+ * desirable slice granularity" as future work; this is the memory half of that question).
+ * Returns in *k_split the smallest valid k in [1, max_k] for which the call's workspace
+ * (osdp_split_linear_workspace_bytes with the same arguments) is at most budget_bytes: splitting
+ * costs time (carry traffic, smaller launches), so the least splitting that fits is preferred.
+ * OSDP_ERR_WORKSPACE_TOO_SMALL if no k up to max_k fits (e.g. a k-independent fp32 carry alone
+ * exceeds the budget; OSDP_FLAG_CARRY_BF16 removes it).  Host-only arithmetic. */
+int osdp_suggest_granularity(int64_t M, int64_t N, int64_t K, int split_dim, int act, int op, int flags,
+                             size_t budget_bytes, int max_k, int *k_split);
+
 /* Forward of all k slices in slice-major order (Section 3.3 steps 1-3).
  *   x [M,K] bf16; bias [N] fp32 or NULL; out [M,N] bf16 = act(X W^T + bias);
  *   z_save [M,N] bf16 or NULL: receives the pre-activation (what the backward needs when act != NONE).

@@ -10,5 +10,5 @@ from .binding import (  # noqa: F401
     osdp_last_cuda_error, osdp_read_device_status, osdp_slice_range, osdp_split_linear_bwd,
     osdp_split_linear_bwd_slice, osdp_split_linear_fwd, osdp_split_linear_fwd_slice,
     osdp_split_linear_workspace_bytes, osdp_split_mlp_bwd, osdp_split_mlp_fwd, osdp_status_string,
-    osdp_version, new_workspace, osdp_bias_grad_noalloc, osdp_debug_wait_probe,
+    osdp_version, new_workspace, osdp_bias_grad_noalloc, osdp_debug_wait_probe, osdp_suggest_granularity,
 )

@@ -22,7 +22,7 @@ EXPORTS = [
     "osdp_version", "osdp_status_string", "osdp_last_cuda_error", "osdp_slice_range",
     "osdp_split_linear_workspace_bytes", "osdp_split_linear_fwd", "osdp_split_linear_fwd_slice",
     "osdp_split_linear_bwd", "osdp_split_linear_bwd_slice", "osdp_split_mlp_fwd", "osdp_split_mlp_bwd",
-    "osdp_read_device_status", "osdp_bias_grad_noalloc", "osdp_debug_wait_probe",
+    "osdp_read_device_status", "osdp_bias_grad_noalloc", "osdp_debug_wait_probe", "osdp_suggest_granularity",
 ]
 
 _lib = None
@@ -69,6 +69,7 @@ def lib():
         L.osdp_read_device_status.argtypes = [vp, ctypes.POINTER(ci), vp]
         L.osdp_bias_grad_noalloc.argtypes = [vp, i64, i64, vp, vp]
         L.osdp_debug_wait_probe.argtypes = [vp, i64, vp]
+        L.osdp_suggest_granularity.argtypes = [i64, i64, i64, ci, ci, ci, ci, sz, ci, ctypes.POINTER(ci)]
         for name in EXPORTS:
             getattr(L, name)
             if name not in ("osdp_status_string",):
@@ -222,3 +223,11 @@ def osdp_debug_wait_probe(ws, limit_us, stream=None, check=False):
     wp, _ = _ws(ws)
     rc = lib().osdp_debug_wait_probe(wp, int(limit_us), _stream(stream))
     return _ret(rc, check, "osdp_debug_wait_probe")
+
+
+def osdp_suggest_granularity(M, N, K, split_dim, act, op, flags, budget_bytes, max_k=64):
+    """Returns (status, k): the smallest valid k <= max_k whose workspace fits budget_bytes."""
+    k = ctypes.c_int(0)
+    rc = lib().osdp_suggest_granularity(int(M), int(N), int(K), int(split_dim), int(act), int(op), int(flags),
+                                        int(budget_bytes), int(max_k), ctypes.byref(k))
+    return rc, k.value

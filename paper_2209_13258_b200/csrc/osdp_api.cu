@@ -722,6 +722,25 @@ int osdp_split_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int k_spl
   return OSDP_OK;
 }
 
+int osdp_suggest_granularity(int64_t M, int64_t N, int64_t K, int split_dim, int act, int op, int flags,
+                             size_t budget_bytes, int max_k, int *k_split) {
+  if (!k_split) return OSDP_ERR_NULL_POINTER;
+  if (max_k < 1 || max_k > OSDP_MAX_SPLIT) return OSDP_ERR_BAD_SPLIT;
+  size_t bytes = 0;
+  int rc = osdp_split_linear_workspace_bytes(M, N, K, 1, split_dim, act, op, flags, &bytes);
+  if (rc) return rc;   // bad shape / op / flags: the same verdict as the call itself would give
+  for (int k = 1; k <= max_k; ++k) {
+    rc = osdp_split_linear_workspace_bytes(M, N, K, k, split_dim, act, op, flags, &bytes);
+    if (rc == OSDP_ERR_BAD_SPLIT) continue;   // this k would leave an empty slice
+    if (rc) return rc;
+    if (bytes <= budget_bytes) {
+      *k_split = k;
+      return OSDP_OK;
+    }
+  }
+  return OSDP_ERR_WORKSPACE_TOO_SMALL;
+}
+
 int osdp_split_linear_fwd(const void *x, const void *w_flat, int64_t w_offset, const float *bias, int64_t M,
                           int64_t N, int64_t K, int k_split, int split_dim, int act, int flags, void *out,
                           void *z_save, void *ws, size_t ws_bytes, void *stream) {

@@ -153,3 +153,23 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "HERE", str(tmp_path))
     with pytest.raises(OSError, match="no CPU fallback"):
         binding.lib()
+
+
+def test_suggest_granularity():
+    # MLP block hidden 8192 / ffn 32768 / 8192 tokens, forward: staging = fp32 carry (268 MB, k > 1) + A_s
+    M, H, F = 8192, 8192, 32768
+    ws = lambda k, fl=0: P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, 1, P.OP_MLP_FWD, fl)[1]
+    sug = lambda budget, fl=0, mk=64: P.osdp_suggest_granularity(M, F, H, 0, 1, P.OP_MLP_FWD, fl, budget, mk)
+    assert sug(ws(1)) == (0, 1)                      # the unsplit block fits: do not split
+    rc, k = sug(ws(1) - 1)                           # k = 2 needs as much as k = 1 (the carry appears): k = 3 fits
+    assert (rc, k) == (0, 3) and ws(2) > ws(1) - 1 >= ws(3)
+    rc, k = sug(350 << 20)
+    assert rc == 0 and ws(k) <= (350 << 20) and all(ws(j) > (350 << 20) for j in range(1, k) if ws(j))
+    assert sug(200 << 20)[0] == 5                    # the k-independent fp32 carry alone is 268 MB
+    rc, k = sug(200 << 20, P.FLAG_CARRY_BF16)        # the bf16 running sum removes it
+    assert rc == 0 and ws(k, P.FLAG_CARRY_BF16) <= (200 << 20)
+    assert sug(1 << 20, mk=8)[0] == 5
+    # k values that would leave an empty slice are skipped, not reported as errors
+    assert P.osdp_suggest_granularity(64, 40, 64, 0, 0, P.OP_LINEAR_BWD, 0, 1 << 30, 64) == (0, 1)
+    assert P.osdp_suggest_granularity(64, 40, 64, 0, 0, P.OP_LINEAR_BWD, 0, 1 << 30, 0)[0] == 3
+    assert P.osdp_suggest_granularity(0, 40, 64, 0, 0, P.OP_LINEAR_BWD, 0, 1 << 30, 8)[0] == 2
