@@ -205,6 +205,9 @@ def run_ours(args):
     rank, world, local = dist_setup(args.gpus)
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the split-linear path has no CPU fallback")
+    if rank == 0:
+        from paper_2209_13258_b200.build import build as build_osdp
+        build_osdp()          # no-op when the in-tree library is up to date
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     if world > 1:
