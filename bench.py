@@ -322,7 +322,9 @@ def run_ours(args):
     if rank == 0 and not args.no_sweep:
         cfgs = [(1, P.SPLIT_OUT, 0, "k1"), (k, P.SPLIT_OUT, 0, "k%d_out" % k), (k, P.SPLIT_RED, 0, "k%d_red" % k),
                 (k, P.SPLIT_OUT, P.FLAG_CARRY_BF16, "k%d_out_bf16_running_sum" % k),
-                (k, P.SPLIT_RED, P.FLAG_CARRY_BF16, "k%d_red_bf16_running_sum" % k)]
+                (k, P.SPLIT_RED, P.FLAG_CARRY_BF16, "k%d_red_bf16_running_sum" % k),
+                (k, P.SPLIT_OUT, P.FLAG_PAIR_SLICES, "k%d_out_paired_slices" % k),
+                (k, P.SPLIT_RED, P.FLAG_PAIR_SLICES, "k%d_red_paired_slices" % k)]
         need = max(workspace(kk, sp, f) for kk, sp, f, _ in cfgs)
         w2 = ws if need <= ws_bytes else P.new_workspace(need, dev)
         times = {label: [] for _, _, _, label in cfgs}

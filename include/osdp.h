@@ -85,6 +85,10 @@ extern "C" {
                                      * per slice (partial and sum).  Measured relative Frobenius error about
                                      * 1.8e-3 * sqrt(1 + (k+1)/2): within 5e-3 up to k = 8, beyond it for k >= 16.
                                      * Only without activation and without z_save. */
+#define OSDP_FLAG_PAIR_SLICES 8     /* summed output, all-slices calls only: a tile accumulates the products of two
+                                     * adjacent slices in one pass, so two slices are read at a time (what a
+                                     * double-buffered slice gather holds anyway) and the running sum is carried
+                                     * half as often.  Exact fp32, but not bit-identical to the unpaired result. */
 #define OSDP_FLAG_RECOMPUTE 4       /* osdp_split_mlp_bwd: recompute the first layer's pre-activation slice by
                                      * slice instead of reading z1_saved (activation checkpointing). */
 
@@ -121,7 +125,7 @@ int osdp_suggest_granularity(int64_t M, int64_t N, int64_t K, int split_dim, int
  *   z_save [M,N] bf16 or NULL: receives the pre-activation (what the backward needs when act != NONE).
  * OUT: slice s writes columns R_s of out.  RED: partial products are summed (fp32 carry in ws, or
  * in `out` itself with OSDP_FLAG_CARRY_BF16); bias and activation are applied once.
- * flags: 0 or OSDP_FLAG_CARRY_BF16. */
+ * flags: 0, OSDP_FLAG_CARRY_BF16, OSDP_FLAG_PAIR_SLICES. */
 int osdp_split_linear_fwd(const void *x, const void *w_flat, int64_t w_offset, const float *bias,
                           int64_t M, int64_t N, int64_t K, int k_split, int split_dim, int act,
                           int flags, void *out, void *z_save, void *ws, size_t ws_bytes, void *stream);
@@ -139,7 +143,8 @@ int osdp_split_linear_fwd_slice(const void *x, const void *w_flat, int64_t w_off
  *   dy [M,N] bf16; x [M,K] bf16; z_saved [M,N] bf16 (pre-activation; required iff act != NONE);
  *   dx [M,K] bf16 or NULL; dw_flat + dw_offset: dW [N,K] in dw_dtype (bf16 or fp32), NULL to skip;
  *   flags: OSDP_FLAG_ACCUMULATE_DW (dW += ... instead of dW = ...), OSDP_FLAG_CARRY_BF16 (dX's running
- *   sum in dx itself under OUT split); dbias [N] fp32 or NULL (always overwritten).
+ *   sum in dx itself under OUT split), OSDP_FLAG_PAIR_SLICES (dX under OUT split);
+ *   dbias [N] fp32 or NULL (always overwritten).
  * OUT: dW[R_s,:], db[R_s] per slice, dX = sum over slices (fp32 carry in ws).
  * RED: dX[:,C_s], dW[:,C_s] per slice. */
 int osdp_split_linear_bwd(const void *dy, const void *x, const void *w_flat, int64_t w_offset,

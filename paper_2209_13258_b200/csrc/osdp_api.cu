@@ -169,6 +169,7 @@ struct GemmCall {
   int64_t bn_P, bn_Q;   // extents that choose the tile width (the unsplit operator's, so k never changes it)
   Epilogue epi;
   int carry_bf16;   // MODE_RED: running sum in `out` (bf16) instead of the fp32 carry buffer
+  int pair_slices;  // MODE_RED: accumulate two adjacent slices per pass
   int *status;
 };
 
@@ -391,6 +392,7 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   p.epi = c.epi;
   p.status = c.status;
   p.carry_bf16 = (c.mode == MODE_RED && c.k_total > 1) ? c.carry_bf16 : 0;
+  p.red_group = (c.mode == MODE_RED && c.pair_slices && c.s_end - c.s_begin > 1) ? 2 : 1;
   // Outputs leave through TMA unless the epilogue has to read a second tensor element-wise.
   p.tma_epilogue = (c.epi.gz == nullptr) ? 1 : 0;
   if (p.tma_epilogue) {
@@ -502,6 +504,7 @@ int check_ws(const void *ws, size_t ws_bytes, const WsPlan &plan) {
 
 int check_flags(int flags, int allowed, int act, const void *z_save) {
   if (flags & ~allowed) return OSDP_ERR_UNSUPPORTED;
+  if ((flags & OSDP_FLAG_PAIR_SLICES) && (flags & OSDP_FLAG_CARRY_BF16)) return OSDP_ERR_UNSUPPORTED;
   if ((flags & OSDP_FLAG_CARRY_BF16) && (act != OSDP_ACT_NONE || z_save)) return OSDP_ERR_UNSUPPORTED;
   return OSDP_OK;
 }
@@ -511,7 +514,7 @@ int fwd_impl(const void *x, const void *w_flat, int64_t w_offset, const float *b
              void *ws, size_t ws_bytes, void *stream) {
   if (!x || !w_flat || !out) return OSDP_ERR_NULL_POINTER;
   {
-    const int frc = check_flags(flags, OSDP_FLAG_CARRY_BF16, act, z_save);
+    const int frc = check_flags(flags, OSDP_FLAG_CARRY_BF16 | (single ? 0 : OSDP_FLAG_PAIR_SLICES), act, z_save);
     if (frc) return frc;
   }
   int64_t L = 0;
@@ -551,6 +554,7 @@ int fwd_impl(const void *x, const void *w_flat, int64_t w_offset, const float *b
   c.epi.carry = reinterpret_cast<float *>(static_cast<char *>(ws) + plan.carry_off);
   c.epi.ld_carry = N;
   c.carry_bf16 = (flags & OSDP_FLAG_CARRY_BF16) ? 1 : 0;
+  c.pair_slices = (flags & OSDP_FLAG_PAIR_SLICES) ? 1 : 0;
   c.status = static_cast<int *>(ws);
   return launch_gemm(c, static_cast<cudaStream_t>(stream));
 }
@@ -561,7 +565,10 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
              void *stream_) {
   if (!dy || !x || !w_flat) return OSDP_ERR_NULL_POINTER;
   // the bf16 running sum concerns dX only, which has neither bias nor activation of its own
-  if (flags & ~(OSDP_FLAG_ACCUMULATE_DW | OSDP_FLAG_CARRY_BF16)) return OSDP_ERR_UNSUPPORTED;
+  if (flags & ~(OSDP_FLAG_ACCUMULATE_DW | OSDP_FLAG_CARRY_BF16 | (single ? 0 : OSDP_FLAG_PAIR_SLICES)))
+    return OSDP_ERR_UNSUPPORTED;
+  if ((flags & OSDP_FLAG_PAIR_SLICES) && ((flags & OSDP_FLAG_CARRY_BF16) || act != OSDP_ACT_NONE))
+    return OSDP_ERR_UNSUPPORTED;   // with an activation the backward runs slice by slice (staged G_s)
   const int accumulate = (flags & OSDP_FLAG_ACCUMULATE_DW) ? 1 : 0;
   int64_t L = 0;
   int rc = check_common(M, N, K, k, split_dim, act, &L);
@@ -612,6 +619,7 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
     c.epi.carry = carry;
     c.epi.ld_carry = K;
     c.carry_bf16 = (flags & OSDP_FLAG_CARRY_BF16) ? 1 : 0;
+    c.pair_slices = (flags & OSDP_FLAG_PAIR_SLICES) ? 1 : 0;
     c.status = status;
     return launch_gemm(c, stream);
   };
@@ -713,8 +721,10 @@ int osdp_split_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int k_spl
                                       int flags, size_t *bytes) {
   if (!bytes) return OSDP_ERR_NULL_POINTER;
   if (act != OSDP_ACT_NONE && act != OSDP_ACT_GELU_TANH && act != OSDP_ACT_GELU_ERF) return OSDP_ERR_UNSUPPORTED;
-  if (flags & ~(OSDP_FLAG_ACCUMULATE_DW | OSDP_FLAG_CARRY_BF16 | OSDP_FLAG_RECOMPUTE)) return OSDP_ERR_UNSUPPORTED;
+  if (flags & ~(OSDP_FLAG_ACCUMULATE_DW | OSDP_FLAG_CARRY_BF16 | OSDP_FLAG_RECOMPUTE | OSDP_FLAG_PAIR_SLICES))
+    return OSDP_ERR_UNSUPPORTED;
   if ((flags & OSDP_FLAG_RECOMPUTE) && op != OSDP_OP_MLP_BWD) return OSDP_ERR_UNSUPPORTED;
+  if ((flags & OSDP_FLAG_PAIR_SLICES) && op != OSDP_OP_LINEAR_FWD && op != OSDP_OP_LINEAR_BWD) return OSDP_ERR_UNSUPPORTED;
   WsPlan plan;
   int rc = plan_workspace(M, N, K, k_split, split_dim, act, op, flags, &plan);
   if (rc) return rc;

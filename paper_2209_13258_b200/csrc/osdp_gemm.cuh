@@ -68,6 +68,7 @@ struct GemmParams {
   CUtensorMap out_main, out_tail, z_main, z_tail, carry_map;
   CUtensorMap carry_pf_map;  // same tensor as carry_map, unswizzled box of 32 rows x BN columns, for L2 prefetch
   int out_sc_mul;
+  int red_group;             // MODE_RED: slices whose products a tile accumulates in one pass (1, or 2 = adjacent pairs)
   int carry_bf16;            // MODE_RED: the running sum is kept in `out` itself, in bf16 (no fp32 carry buffer)
   int tma_epilogue;          // 1: outputs leave through shared-memory staging + TMA; 0: direct stores
   Epilogue epi;
@@ -337,7 +338,8 @@ struct SmemLayout {
 // Tile schedule (identical in every warp role)
 
 struct Work {
-  int s;                     // slice
+  int s;                     // slice (MODE_RED with pairing: the first slice of the pair)
+  int s_count;               // slices accumulated in this pass (1, or 2 under MODE_RED pairing)
   int row0, row_end;         // output rows of the tile, clipped extent of the slice
   int col0, col_end;
   int kblocks;               // reduction blocks of this slice
@@ -358,15 +360,18 @@ __device__ __forceinline__ bool get_work(const GemmParams &p, int i, int bid, in
     const int tiles = ceil_div(p.P, TM) * ceil_div(p.Q, BN);
     if (bid >= tiles) return false;
     const int n_my = (tiles - bid + G - 1) / G;
+    const int grp = p.red_group > 1 ? p.red_group : 1;
     const int srel = i / n_my;
-    if (srel >= nsl) return false;
-    s = p.s_begin + srel;
+    if (srel >= ceil_div(nsl, grp)) return false;
+    s = p.s_begin + srel * grp;
+    w.s_count = min(grp, p.s_end - s);
     t = bid + (i - srel * n_my) * G;
     rows = p.P;
     cols = p.Q;
     w.first_of_slice = (i == srel * n_my);
   } else {
     w.first_of_slice = 0;
+    w.s_count = 1;
     const int rows_full = (p.mode == MODE_ROWS) ? p.L : p.P;
     const int cols_full = (p.mode == MODE_COLS) ? p.L : p.Q;
     const int t_full = ceil_div(rows_full, TM) * ceil_div(cols_full, BN);
@@ -397,10 +402,14 @@ __device__ __forceinline__ bool get_work(const GemmParams &p, int i, int bid, in
   w.col0 = col_base + w.b_col;
   w.row_end = row_base + rows;
   w.col_end = col_base + cols;
-  const int red = (p.mode == MODE_RED) ? min(p.L, p.R - s * p.L) : p.R;
-  w.kblocks = ceil_div(red, BK);
+  if (p.mode == MODE_RED) {
+    w.kblocks = 0;
+    for (int ss = s; ss < s + w.s_count; ++ss) w.kblocks += ceil_div(min(p.L, p.R - ss * p.L), BK);
+  } else {
+    w.kblocks = ceil_div(p.R, BK);
+  }
   w.carry_in = (p.mode == MODE_RED) && !p.carry_bf16 && (s > 0);
-  w.carry_out = (p.mode == MODE_RED) && !p.carry_bf16 && (s < p.k_total - 1);
+  w.carry_out = (p.mode == MODE_RED) && !p.carry_bf16 && (s + w.s_count - 1 < p.k_total - 1);
   return true;
 }
 
@@ -597,12 +606,15 @@ __global__ void __launch_bounds__((BN > 256) ? 384 : 256, 1) gemm_kernel(const _
     for (int i = 0; ok && get_work<TM, BN>(p, i, bid, G, w); ++i) {
       w.a_row += (int)rank * BM;            // this CTA's rows of the pair's tile
       w.b_col += (int)rank * SL::GB_ROWS * (CTA2 ? 1 : 0);   // ... and its half of each 256-column group of B
-      const bool tail = (w.s == p.k_total - 1);
+      for (int sl = 0; sl < w.s_count && ok; ++sl) {
+      const int ss = w.s + sl;               // the slice whose operand boxes are loaded now
+      const bool tail = (ss == p.k_total - 1);
       const CUtensorMap *amap = (a_sliced && !tail) ? &p.a_main : &p.a_tail;
       const CUtensorMap *bmap = (b_sliced && !tail) ? &p.b_main : &p.b_tail;
-      const int a_sc = (a_sliced && !tail) ? w.s * p.a_sc_mul : 0;
-      const int b_sc = (b_sliced && !tail) ? w.s * p.b_sc_mul : 0;
-      for (int kb = 0; kb < w.kblocks; ++kb) {
+      const int a_sc = (a_sliced && !tail) ? ss * p.a_sc_mul : 0;
+      const int b_sc = (b_sliced && !tail) ? ss * p.b_sc_mul : 0;
+      const int nkb = (p.mode == MODE_RED) ? ceil_div(min(p.L, p.R - ss * p.L), BK) : w.kblocks;
+      for (int kb = 0; kb < nkb; ++kb) {
         ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER);
         if (!ok) break;
         if (lane == 0) {
@@ -649,6 +661,7 @@ __global__ void __launch_bounds__((BN > 256) ? 384 : 256, 1) gemm_kernel(const _
         armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
         __syncwarp();
         if (++stage == SL::STAGES) { stage = 0; phase ^= 1u; }
+      }
       }
     }
     if (!ok && rank == 0 && load_a) {

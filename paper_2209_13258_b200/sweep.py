@@ -104,6 +104,8 @@ def sweep_linear(M, N, K, ks):
             cfgs.append((k, split, name, 0, _ws_linear(M, N, K, k, split)))
             if k > 1:   # the summed output carried in bf16 in the output buffer instead of fp32 in the workspace
                 cfgs.append((k, split, name, P.FLAG_CARRY_BF16, _ws_linear(M, N, K, k, split, P.FLAG_CARRY_BF16)))
+            if k > 2:   # exact fp32 carry, adjacent slices accumulated in pairs (two slices live)
+                cfgs.append((k, split, name, P.FLAG_PAIR_SLICES, _ws_linear(M, N, K, k, split, P.FLAG_PAIR_SLICES)))
     ws = P.new_workspace(max(c[4] for c in cfgs))     # one workspace, large enough for every configuration
     fns = []
     for k, split, name, fl, _ in cfgs:
@@ -117,7 +119,9 @@ def sweep_linear(M, N, K, ks):
     for i, (k, split, name, fl, nbytes) in enumerate(cfgs):
         tf, tb = ts[2 * i], ts[2 * i + 1]
         t = tf + tb
-        rows.append({"k": k, "split": name, "carry": "bf16" if fl else "fp32", "fwd_ms": tf, "bwd_ms": tb, "ms": t,
+        rows.append({"k": k, "split": name,
+                     "carry": {0: "fp32", P.FLAG_CARRY_BF16: "bf16", P.FLAG_PAIR_SLICES: "fp32-paired"}[fl],
+                     "fwd_ms": tf, "bwd_ms": tb, "ms": t,
                      "tflops": flops / t / 1e9, "overhead_vs_k1": t / base - 1.0, "staging_bytes": nbytes})
         print(json.dumps(rows[-1]), flush=True)
     return rows

@@ -172,6 +172,31 @@ def test_bf16_running_sum(P, shape, split):
 
 
 # ---------------------------------------------------------------------------------------------
+# adjacent slices accumulated in pairs (two slices live): exact fp32, half as many carried boundaries
+
+@pytest.mark.parametrize("shape", [(300, 520, 328), (1024, 2048, 1024), (2100, 2560, 2304)])
+@pytest.mark.parametrize("split", [0, 1])
+def test_paired_slices(P, shape, split):
+    M, N, K = shape
+    c = inputs.linear_case(M, N, K, w_std=0.05, bias_std=0.3, layer=16)
+    o = oracle_linear(c, 0)
+    for k in (2, 3, 5, 8):
+        if P.osdp_slice_range(N if split == 0 else K, k, 0)[0] != 0:
+            continue
+        g = run_linear(P, c, k, split, flags=P.FLAG_PAIR_SLICES)
+        compare(g, o, 0)
+        # concatenated outputs are untouched by the pairing
+        plain = run_linear(P, c, k, split)
+        for name in (("y", "dw", "db") if split == 0 else ("dx", "dw", "db")):
+            assert torch.equal(_bits(g[name]), _bits(plain[name])), name
+    # with an activation the forward's summed output still pairs (bias and activation after the last pair)
+    if split == 1:
+        ga = run_linear(P, c, 4, split, act=1, flags=0)
+        oa = oracle_linear(c, 1, 4, split)
+        compare(ga, oa, 1)
+
+
+# ---------------------------------------------------------------------------------------------
 # bit identity, per-slice calls, determinism
 
 def _bits(t):

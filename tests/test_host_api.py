@@ -101,6 +101,10 @@ def test_forward_argument_checks():
     assert _fwd(flags=P.FLAG_CARRY_BF16, act=1) == 6    # the bf16 running sum excludes an activation ...
     assert _fwd(flags=P.FLAG_CARRY_BF16, z_save=A) == 6  # ... and a saved pre-activation
     assert _fwd(flags=4) == 6 and _fwd(flags=P.FLAG_ACCUMULATE_DW) == 6
+    assert _fwd(split_dim=1, flags=P.FLAG_PAIR_SLICES) in (0, 7)
+    assert _fwd(split_dim=1, flags=P.FLAG_PAIR_SLICES | P.FLAG_CARRY_BF16) == 6
+    assert P.osdp_split_linear_fwd_slice(A, A, 0, None, 64, 64, 64, 2, 1, 0, 0, A, None, (A, 1 << 20), stream=0,
+                                         flags=P.FLAG_PAIR_SLICES) == 6
     assert P.osdp_split_linear_fwd_slice(A, A, 0, None, 64, 64, 64, 2, 0, 0, 2, A, None, (A, 1 << 20), stream=0) == 3
     # a well-formed call gets past the checks and fails only because there is no device / fake pointers
     if not _cuda():
@@ -114,7 +118,13 @@ def test_backward_argument_checks():
     assert _bwd(dw_offset=12) == 4 and _bwd(dx=A + 4) == 4 and _bwd(dbias=A + 4) == 4
     assert _bwd(k_split=9) == 3
     assert _bwd(ws=(A, 1024)) == 5
-    assert _bwd(flags=8) == 6
+    assert _bwd(flags=32) == 6
+    # pairing of adjacent slices: all-slices calls only, not together with the bf16 running sum or an activation
+    assert _bwd(flags=P.FLAG_PAIR_SLICES) in (0, 7)
+    assert _bwd(flags=P.FLAG_PAIR_SLICES | P.FLAG_CARRY_BF16) == 6
+    assert _bwd(flags=P.FLAG_PAIR_SLICES, act=1, z_saved=A) == 6
+    assert P.osdp_split_linear_bwd_slice(A, A, A, 0, None, 64, 64, 64, 2, 0, 0, 0, A, A, 0, 1, P.FLAG_PAIR_SLICES, A,
+                                         (A, 1 << 20), stream=0) == 6
     # with the bf16 running sum the backward needs only the column-sum partials
     assert _bwd(ws=(A, 256 + 64 * 4), flags=P.FLAG_CARRY_BF16) in (0, 7)
     assert P.osdp_split_linear_bwd_slice(A, A, A, 0, None, 64, 64, 64, 2, 0, 0, -1, A, A, 0, 1, 0, A, (A, 1 << 20),
