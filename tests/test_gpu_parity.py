@@ -534,3 +534,19 @@ def test_random_shapes_against_oracle(P, chunk):
         except AssertionError as e:
             raise AssertionError("case M=%d N=%d K=%d k=%d split=%d act=%d flags=%d: %s" % (
                 M, N, K, k, split, act, flags, e))
+
+
+# ---------------------------------------------------------------------------------------------
+# a shape for which the tile model picks the 256 x 512 tile (74 wide tiles = one round, reduction
+# 8192) in the GEMMs whose epilogues do more than store: bias + pre-activation save + GeLU (first
+# layer forward) and the activation backward that reads Z1 element-wise (MLP backward)
+
+def test_mlp_wide_tile_epilogues(P):
+    M, H, F = 512, 8192, 18944
+    c = inputs.mlp_case(M, H, F, w_std=0.01, bias_std=0.05, layer=17)
+    _, y = oracle.mlp_fwd(c["x"], c["w1"], c["b1"], c["w2"], c["b2"], oracle.ACT_GELU_TANH, None)
+    grads = oracle.mlp_bwd(c["dy"], c["x"], c["w1"], c["b1"], c["w2"], oracle.ACT_GELU_TANH, None)
+    g = run_mlp(P, c, 1, dw_fp32=False)
+    compare_mlp(g, (y,) + tuple(grads))
+    g2 = run_mlp(P, c, 2, dw_fp32=False, recompute=True)
+    compare_mlp(g2, (y,) + tuple(grads))
