@@ -373,7 +373,8 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   // element (epilogue hidden), 512-wide 11.5 ns per element plus 5 us of exposed epilogue; time =
   // rounds of the persistent schedule x tile time.  Both tiles produce the same bits per element
   // (same k-block order), so the choice may differ between launches.  Summed outputs keep 256.
-  if (pair && c.mode != MODE_RED) {
+  // So does the GEMM whose epilogue reads a second tensor element-wise (direct stores, slower: better hidden).
+  if (pair && c.mode != MODE_RED && c.epi.gz == nullptr) {
     const int64_t units = sms / 2;
     const int64_t red_len = c.R;
     const double t_n = (double)cdiv(count_items(c, 2 * BM, 256), units) * (6.5e-3 * (double)red_len) + 5.0;
