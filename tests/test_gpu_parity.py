@@ -538,8 +538,8 @@ def test_random_shapes_against_oracle(P, chunk):
 
 # ---------------------------------------------------------------------------------------------
 # a shape for which the tile model picks the 256 x 512 tile (74 wide tiles = one round, reduction
-# 8192) in the GEMMs whose epilogues do more than store: bias + pre-activation save + GeLU (first
-# layer forward) and the activation backward that reads Z1 element-wise (MLP backward)
+# 8192) in a GEMM whose epilogue does more than store: bias + pre-activation save + GeLU (first layer
+# forward, and its recomputation in the backward), next to 256-wide tiles in the same chain
 
 def test_mlp_wide_tile_epilogues(P):
     M, H, F = 512, 8192, 18944
