@@ -550,3 +550,18 @@ def test_mlp_wide_tile_epilogues(P):
     compare_mlp(g, (y,) + tuple(grads))
     g2 = run_mlp(P, c, 2, dw_fp32=False, recompute=True)
     compare_mlp(g2, (y,) + tuple(grads))
+
+
+# ---------------------------------------------------------------------------------------------
+# ragged extents on the 256 x 512 tile: 2000 x 4232 x 8200 makes the model pick it for the forward and
+# for dX (72 and 136 wide tiles); with k = 3 the slices (length 1416) end inside a 512-wide tile
+
+@pytest.mark.parametrize("k,split", [(1, 0), (3, 0), (3, 1)])
+def test_ragged_extents_on_the_wide_tile(P, k, split):
+    c = inputs.linear_case(2000, 4232, 8200, w_std=0.02, bias_std=0.1, w_offset=24, flat_pad=8, layer=18)
+    g = run_linear(P, c, k, split, dw_fp32=False)
+    compare(g, oracle_linear(c, 0), 0)
+    if k > 1:
+        g1 = run_linear(P, c, 1, split, dw_fp32=False)
+        for name in (("y", "dw", "db") if split == 0 else ("dx", "dw", "db")):
+            assert torch.equal(_bits(g[name]), _bits(g1[name])), name
