@@ -8,6 +8,9 @@
 #include <cuda_runtime.h>
 #include <string.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "osdp_aux.cuh"
 #include "osdp_gemm.cuh"
 
@@ -16,6 +19,10 @@ using namespace osdp;
 namespace {
 
 thread_local int g_last_cuda_error = 0;
+
+// One lock for the rare first-use set-up paths (driver entry point, per-device attributes); the hot
+// path only reads an atomic flag.
+std::mutex g_setup_mutex;
 
 int cuda_fail(cudaError_t e) {
   g_last_cuda_error = (int)e;
@@ -32,37 +39,36 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   CUtensorMapFloatOOBfill);
 
 int get_encode_fn(EncodeTiledFn *out) {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
+  static std::atomic<EncodeTiledFn> fn{nullptr};
+  EncodeTiledFn f = fn.load(std::memory_order_acquire);
+  if (!f) {
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
     void *p = nullptr;
     cudaDriverEntryPointQueryResult q;
     cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
     if (e != cudaSuccess) return cuda_fail(e);
     if (q != cudaDriverEntryPointSuccess || !p) return cuda_fail(cudaErrorNotSupported);
-    fn = (EncodeTiledFn)p;
+    f = (EncodeTiledFn)p;
+    fn.store(f, std::memory_order_release);
   }
-  *out = fn;
+  *out = f;
   return OSDP_OK;
 }
 
-struct DeviceInfo {
-  int sms;
-  bool attrs_set;
-};
-DeviceInfo g_dev[64];
+std::atomic<int> g_dev_sms[64];
 
 int device_sms(int *sms) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return cuda_fail(e);
   if (dev < 0 || dev >= 64) return cuda_fail(cudaErrorInvalidDevice);
-  if (g_dev[dev].sms == 0) {
-    int n = 0;
+  int n = g_dev_sms[dev].load(std::memory_order_relaxed);
+  if (n == 0) {
     e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return cuda_fail(e);
-    g_dev[dev].sms = n;
+    g_dev_sms[dev].store(n, std::memory_order_relaxed);
   }
-  *sms = g_dev[dev].sms;
+  *sms = n;
   return OSDP_OK;
 }
 
@@ -281,15 +287,16 @@ int make_output_maps(void *base, bool fp32, int64_t P, int64_t Q, int64_t ld, in
 // `units` = work items of the launch (tiles, summed over slices for concatenated outputs).
 template <int BN, bool A_MN, bool B_MN, bool CTA2>
 int launch_variant(const GemmParams &p, int64_t units, int sms, cudaStream_t stream) {
-  static bool attr_done[64] = {};
-  static int max_clusters[64] = {};
+  static std::atomic<bool> attr_done[64];
+  static std::atomic<int> max_clusters[64];
   using SL = SmemLayout<BN, CTA2>;
   auto kernel = gemm_kernel<BN, A_MN, B_MN, CTA2>;
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return cuda_fail(e);
   dev &= 63;
-  if (!attr_done[dev]) {
+  if (!attr_done[dev].load(std::memory_order_acquire)) {
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
     e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::TOTAL);
     if (e != cudaSuccess) return cuda_fail(e);
     if (CTA2) {
@@ -305,11 +312,11 @@ int launch_variant(const GemmParams &p, int64_t units, int sms, cudaStream_t str
       e = cudaOccupancyMaxActiveClusters(&n, kernel, &q);
       if (e != cudaSuccess) return cuda_fail(e);
       if (n < 1) return cuda_fail(cudaErrorLaunchOutOfResources);
-      max_clusters[dev] = n;
+      max_clusters[dev].store(n, std::memory_order_relaxed);
     }
-    attr_done[dev] = true;
+    attr_done[dev].store(true, std::memory_order_release);
   }
-  const int64_t cap = CTA2 ? max_clusters[dev] : sms;
+  const int64_t cap = CTA2 ? max_clusters[dev].load(std::memory_order_relaxed) : sms;
   const int n_units = (int)(units < cap ? units : cap);
   if (n_units <= 0) return OSDP_OK;
   cudaLaunchConfig_t cfg = {};
@@ -1019,23 +1026,23 @@ __device__ __align__(256) float g_noalloc_partials[OSDP_NOALLOC_MAX_PARTIALS];
 
 // In host code `g_noalloc_partials` is only a handle for the runtime, not a device address:
 // the address a kernel may use is looked up per device, once, with that device current.
-float *g_noalloc_ptr[64] = {};
-bool g_noalloc_ready[64] = {};
+std::atomic<float *> g_noalloc_ptr[64];
 
 int noalloc_scratch(float **ptr) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return cuda_fail(e);
   if (dev < 0 || dev >= 64) return cuda_fail(cudaErrorInvalidDevice);
-  if (!g_noalloc_ready[dev]) {
+  float *dp = g_noalloc_ptr[dev].load(std::memory_order_acquire);
+  if (!dp) {
     void *p = nullptr;
-    e = cudaGetSymbolAddress(&p, g_noalloc_partials);
+    e = cudaGetSymbolAddress(&p, g_noalloc_partials);   // with device `dev` current
     if (e != cudaSuccess) return cuda_fail(e);
     if (!p) return cuda_fail(cudaErrorInvalidSymbol);
-    g_noalloc_ptr[dev] = static_cast<float *>(p);
-    g_noalloc_ready[dev] = true;
+    dp = static_cast<float *>(p);
+    g_noalloc_ptr[dev].store(dp, std::memory_order_release);
   }
-  *ptr = g_noalloc_ptr[dev];
+  *ptr = dp;
   return OSDP_OK;
 }
 
