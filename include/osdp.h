@@ -161,6 +161,43 @@ int osdp_split_linear_bwd_slice(const void *dy, const void *x, const void *w_fla
                                 int64_t dw_offset, int dw_dtype, int flags, float *dbias,
                                 void *ws, size_t ws_bytes, void *stream);
 
+/* ---- Slices of a sharded operator (Section 3.3, last part: with zero-redundancy data parallelism
+ * only the slice being processed is gathered, so the gathered weights take size(W)/k instead of
+ * size(W)).  The caller (one process per GPU) keeps 1/world of every slice, all-gathers slice s
+ * into a staging buffer, runs the slice, and reduce-scatters the slice's weight gradient; the
+ * three entry points below are the per-GPU part of that loop.  They communicate nothing.
+ *
+ * Shard layout of slice `slice_idx` (host only, no GPU needed).  A gathered slice is a compact
+ * row-major matrix: OUT  W[R_s, :]  as [len(R_s), K], *ld = K;  RED  W[:, C_s]  as [N, len(C_s)],
+ * *ld = len(C_s).  *slice_elems = its element count; every rank holds *shard_elems contiguous
+ * elements of it (a multiple of 8; world * shard_elems >= slice_elems, the surplus is padding at
+ * the end of the gathered buffer); *shard_offset = where the rank's part of this slice starts in the
+ * rank's shard buffer (slices stored one after another).  slice_idx == k is allowed and returns
+ * the shard buffer's total length in *shard_offset.  Any output pointer may be NULL. */
+int osdp_zdp_shard_layout(int64_t N, int64_t K, int k_split, int split_dim, int world, int slice_idx,
+                          int64_t *slice_elems, int64_t *shard_elems, int64_t *shard_offset,
+                          int64_t *ld);
+
+/* osdp_split_linear_fwd_slice with the slice's weights given as the gathered compact matrix
+ * `w_slice` (device, bf16, 16-byte aligned, leading dimension ld_w >= the layout's *ld, a multiple of
+ * 8) instead of a window of the flat buffer.  Everything else (x, bias, out, z_save, workspace,
+ * ordering of the slices, flags 0 or OSDP_FLAG_CARRY_BF16) as in osdp_split_linear_fwd_slice;
+ * outputs are bit-identical to that call's. */
+int osdp_zdp_linear_fwd_slice(const void *x, const void *w_slice, int64_t ld_w, const float *bias,
+                              int64_t M, int64_t N, int64_t K, int k_split, int split_dim, int act,
+                              int flags, int slice_idx, void *out, void *z_save, void *ws,
+                              size_t ws_bytes, void *stream);
+
+/* osdp_split_linear_bwd_slice with gathered weights `w_slice` (as above) and the slice's weight
+ * gradient written to the compact matrix `dw_slice` (same shape as the gathered slice, leading
+ * dimension ld_dw, dtype dw_dtype; NULL to skip), ready to be reduce-scattered.  dx, dbias, z_saved,
+ * flags (OSDP_FLAG_ACCUMULATE_DW, OSDP_FLAG_CARRY_BF16) as in osdp_split_linear_bwd_slice. */
+int osdp_zdp_linear_bwd_slice(const void *dy, const void *x, const void *w_slice, int64_t ld_w,
+                              const void *z_saved, int64_t M, int64_t N, int64_t K, int k_split,
+                              int split_dim, int act, int slice_idx, void *dx, void *dw_slice,
+                              int64_t ld_dw, int dw_dtype, int flags, float *dbias, void *ws,
+                              size_t ws_bytes, void *stream);
+
 /* Transformer MLP block split along the ffn dimension (first layer OUT-split + activation,
  * second layer RED-split, Section 3.3 applied to both MatMuls of the block):
  *   out [M,hidden] = sum_s act(X W1[F_s,:]^T + b1[F_s]) W2[:,F_s]^T + b2, slice by slice.

@@ -23,6 +23,7 @@ EXPORTS = [
     "osdp_split_linear_workspace_bytes", "osdp_split_linear_fwd", "osdp_split_linear_fwd_slice",
     "osdp_split_linear_bwd", "osdp_split_linear_bwd_slice", "osdp_split_mlp_fwd", "osdp_split_mlp_bwd",
     "osdp_read_device_status", "osdp_bias_grad_noalloc", "osdp_debug_wait_probe", "osdp_suggest_granularity",
+    "osdp_zdp_shard_layout", "osdp_zdp_linear_fwd_slice", "osdp_zdp_linear_bwd_slice",
 ]
 
 _lib = None
@@ -70,6 +71,11 @@ def lib():
         L.osdp_bias_grad_noalloc.argtypes = [vp, i64, i64, vp, vp]
         L.osdp_debug_wait_probe.argtypes = [vp, i64, vp]
         L.osdp_suggest_granularity.argtypes = [i64, i64, i64, ci, ci, ci, ci, sz, ci, ctypes.POINTER(ci)]
+        p64 = ctypes.POINTER(i64)
+        L.osdp_zdp_shard_layout.argtypes = [i64, i64, ci, ci, ci, ci, p64, p64, p64, p64]
+        L.osdp_zdp_linear_fwd_slice.argtypes = [vp, vp, i64, vp, i64, i64, i64, ci, ci, ci, ci, ci, vp, vp, vp, sz, vp]
+        L.osdp_zdp_linear_bwd_slice.argtypes = [vp, vp, vp, i64, vp, i64, i64, i64, ci, ci, ci, ci, vp, vp, i64, ci,
+                                                ci, vp, vp, sz, vp]
         for name in EXPORTS:
             getattr(L, name)
             if name not in ("osdp_status_string",):
@@ -231,3 +237,30 @@ def osdp_suggest_granularity(M, N, K, split_dim, act, op, flags, budget_bytes, m
     rc = lib().osdp_suggest_granularity(int(M), int(N), int(K), int(split_dim), int(act), int(op), int(flags),
                                         int(budget_bytes), int(max_k), ctypes.byref(k))
     return rc, k.value
+
+
+def osdp_zdp_shard_layout(N, K, k_split, split_dim, world, slice_idx):
+    """Returns (status, slice_elems, shard_elems, shard_offset, ld) for one slice of a sharded operator."""
+    a, b, c, d = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
+    rc = lib().osdp_zdp_shard_layout(int(N), int(K), int(k_split), int(split_dim), int(world), int(slice_idx),
+                                     ctypes.byref(a), ctypes.byref(b), ctypes.byref(c), ctypes.byref(d))
+    return rc, a.value, b.value, c.value, d.value
+
+
+def osdp_zdp_linear_fwd_slice(x, w_slice, ld_w, bias, M, N, K, k_split, split_dim, act, slice_idx, out, z_save, ws,
+                              stream=None, check=False, flags=0):
+    wp, wn = _ws(ws)
+    rc = lib().osdp_zdp_linear_fwd_slice(_ptr(x), _ptr(w_slice), int(ld_w), _ptr(bias), int(M), int(N), int(K),
+                                         int(k_split), int(split_dim), int(act), int(flags), int(slice_idx),
+                                         _ptr(out), _ptr(z_save), wp, wn, _stream(stream))
+    return _ret(rc, check, "osdp_zdp_linear_fwd_slice")
+
+
+def osdp_zdp_linear_bwd_slice(dy, x, w_slice, ld_w, z_saved, M, N, K, k_split, split_dim, act, slice_idx, dx,
+                              dw_slice, ld_dw, dw_dtype, flags, dbias, ws, stream=None, check=False):
+    wp, wn = _ws(ws)
+    rc = lib().osdp_zdp_linear_bwd_slice(_ptr(dy), _ptr(x), _ptr(w_slice), int(ld_w), _ptr(z_saved), int(M), int(N),
+                                         int(K), int(k_split), int(split_dim), int(act), int(slice_idx), _ptr(dx),
+                                         _ptr(dw_slice), int(ld_dw), int(dw_dtype), int(flags), _ptr(dbias), wp, wn,
+                                         _stream(stream))
+    return _ret(rc, check, "osdp_zdp_linear_bwd_slice")

@@ -176,6 +176,7 @@ struct GemmCall {
   Epilogue epi;
   int carry_bf16;   // MODE_RED: running sum in `out` (bf16) instead of the fp32 carry buffer
   int pair_slices;  // MODE_RED: accumulate two adjacent slices per pass
+  int out_is_slice; // MODE_ROWS / MODE_COLS: `epi.out` is the slice's own compact matrix, not the whole output
   int *status;
 };
 
@@ -269,13 +270,13 @@ int make_operand_maps(const Operand &op, bool is_a, int mode, int64_t L, int k, 
 
 // Output-side maps: boxes of 32 rows x 128 bytes written by one epilogue warp.
 int make_output_maps(void *base, bool fp32, int64_t P, int64_t Q, int64_t ld, int mode, int64_t L, int k,
-                     CUtensorMap *main_map, CUtensorMap *tail_map, int *sc_mul) {
+                     CUtensorMap *main_map, CUtensorMap *tail_map, int *sc_mul, bool whole = true) {
   ViewSpec v;
   v.base = base; v.elem_bytes = fp32 ? 4 : 2;
   v.dt = fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
-  v.inner = Q; v.outer = P; v.ld = ld;
+  v.inner = Q; v.outer = P; v.ld = ld;   // whole == false: P x Q are the slice's own extents
   v.mid = (mode == MODE_COLS);
-  v.cut = (mode == MODE_COLS || mode == MODE_ROWS) && k > 1;
+  v.cut = (mode == MODE_COLS || mode == MODE_ROWS) && k > 1 && whole;
   v.L = L; v.k = k;
   v.box_inner = fp32 ? 32 : 64;
   v.box_outer = 32;
@@ -404,8 +405,18 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   // Outputs leave through TMA unless the epilogue has to read a second tensor element-wise.
   p.tma_epilogue = (c.epi.gz == nullptr) ? 1 : 0;
   if (p.tma_epilogue) {
-    rc = make_output_maps(c.epi.out, c.epi.out_fp32 != 0, c.P, c.Q, c.epi.ld_out, c.mode, c.L, c.k_total, &p.out_main,
-                          &p.out_tail, &p.out_sc_mul);
+    if (c.out_is_slice && c.k_total > 1 && (c.mode == MODE_ROWS || c.mode == MODE_COLS)) {
+      // the launch covers one slice and writes it as a compact matrix of the slice's extents
+      if (c.s_end - c.s_begin != 1 || c.epi.z_save) return OSDP_ERR_UNSUPPORTED;
+      const int64_t full = (c.mode == MODE_ROWS) ? c.P : c.Q;
+      const int64_t ls = (full - c.s_begin * c.L < c.L) ? full - c.s_begin * c.L : c.L;
+      rc = make_output_maps(c.epi.out, c.epi.out_fp32 != 0, c.mode == MODE_ROWS ? ls : c.P,
+                            c.mode == MODE_COLS ? ls : c.Q, c.epi.ld_out, c.mode, c.L, c.k_total, &p.out_main,
+                            &p.out_tail, &p.out_sc_mul, false);
+    } else {
+      rc = make_output_maps(c.epi.out, c.epi.out_fp32 != 0, c.P, c.Q, c.epi.ld_out, c.mode, c.L, c.k_total,
+                            &p.out_main, &p.out_tail, &p.out_sc_mul);
+    }
     if (rc) return rc;
     if (c.epi.z_save) {
       rc = make_output_maps(c.epi.z_save, false, c.P, c.Q, c.epi.ld_z, c.mode, c.L, c.k_total, &p.z_main, &p.z_tail,
@@ -517,9 +528,11 @@ int check_flags(int flags, int allowed, int act, const void *z_save) {
   return OSDP_OK;
 }
 
+// `ld_w_slice` > 0: `w_flat` + `w_offset` is not the whole operator but slice `s_begin` of it, gathered into
+// a compact matrix with that leading dimension ([slice rows, K] under OUT, [N, slice columns] under RED).
 int fwd_impl(const void *x, const void *w_flat, int64_t w_offset, const float *bias, int64_t M, int64_t N, int64_t K,
              int k, int split_dim, int act, int flags, int s_begin, int s_end, bool single, void *out, void *z_save,
-             void *ws, size_t ws_bytes, void *stream) {
+             void *ws, size_t ws_bytes, void *stream, int64_t ld_w_slice = 0) {
   if (!x || !w_flat || !out) return OSDP_ERR_NULL_POINTER;
   {
     const int frc = check_flags(flags, OSDP_FLAG_CARRY_BF16 | (single ? 0 : OSDP_FLAG_PAIR_SLICES), act, z_save);
@@ -550,6 +563,15 @@ int fwd_impl(const void *x, const void *w_flat, int64_t w_offset, const float *b
   memset(&c, 0, sizeof(c));
   c.a = Operand{x, K, M, K, false, true};
   c.b = Operand{w, K, N, K, false, true};
+  if (ld_w_slice > 0) {
+    if (!single) return OSDP_ERR_UNSUPPORTED;
+    if (ld_w_slice & 7) return OSDP_ERR_ALIGNMENT;
+    const int64_t D = (split_dim == OSDP_SPLIT_OUT) ? N : K;
+    const int64_t ls = (D - s_begin * L < L) ? D - s_begin * L : L;
+    if (ld_w_slice < (split_dim == OSDP_SPLIT_OUT ? K : ls)) return OSDP_ERR_BAD_SHAPE;
+    c.b = (split_dim == OSDP_SPLIT_OUT) ? Operand{w, K, ls, ld_w_slice, false, false}
+                                        : Operand{w, ls, N, ld_w_slice, false, false};
+  }
   c.P = M; c.Q = N; c.R = K;
   c.bn_P = M; c.bn_Q = N;
   c.mode = (k == 1) ? MODE_NONE : (split_dim == OSDP_SPLIT_OUT ? MODE_COLS : MODE_RED);
@@ -570,7 +592,9 @@ int fwd_impl(const void *x, const void *w_flat, int64_t w_offset, const float *b
 int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset, const void *z_saved, int64_t M,
              int64_t N, int64_t K, int k, int split_dim, int act, int s_begin, int s_end, bool single, void *dx,
              void *dw_flat, int64_t dw_offset, int dw_dtype, int flags, float *dbias, void *ws, size_t ws_bytes,
-             void *stream_) {
+             void *stream_, int64_t ld_w_slice = 0, int64_t ld_dw_slice = 0) {
+  // ld_w_slice > 0: W is slice `s_begin` gathered into a compact matrix (see fwd_impl);
+  // ld_dw_slice > 0: dW of the slice is written as a compact matrix of the same shape.
   if (!dy || !x || !w_flat) return OSDP_ERR_NULL_POINTER;
   // the bf16 running sum concerns dX only, which has neither bias nor activation of its own
   if (flags & ~(OSDP_FLAG_ACCUMULATE_DW | OSDP_FLAG_CARRY_BF16 | (single ? 0 : OSDP_FLAG_PAIR_SLICES)))
@@ -613,13 +637,22 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
     dw = (dw_dtype == OSDP_DTYPE_FP32) ? (void *)(static_cast<float *>(dw_flat) + dw_offset)
                                        : (void *)(static_cast<__nv_bfloat16 *>(dw_flat) + dw_offset);
   const bool out_split = (split_dim == OSDP_SPLIT_OUT);
-  const int mode_sum = (k == 1) ? MODE_NONE : MODE_RED;
+  const int64_t D = out_split ? N : K;
+  const int64_t ls0 = (D - s_begin * L < L) ? D - s_begin * L : L;   // extent of slice s_begin
+  if (ld_w_slice > 0 || ld_dw_slice > 0) {
+    if (!single) return OSDP_ERR_UNSUPPORTED;
+    if ((ld_w_slice & 7) || (ld_dw_slice & 7)) return OSDP_ERR_ALIGNMENT;
+    if (ld_w_slice > 0 && ld_w_slice < (out_split ? K : ls0)) return OSDP_ERR_BAD_SHAPE;
+    if (ld_dw_slice > 0 && ld_dw_slice < (out_split ? K : ls0)) return OSDP_ERR_BAD_SHAPE;
+  }
 
   auto dx_call = [&](const Operand &g, int sb, int se) {
     GemmCall c;
     memset(&c, 0, sizeof(c));
     c.a = g;                                        // G [M,N], reduction N contiguous
     c.b = Operand{w, K, N, K, true, true};          // W [N,K]: output dim K contiguous
+    if (ld_w_slice > 0)
+      c.b = out_split ? Operand{w, K, ls0, ld_w_slice, true, false} : Operand{w, ls0, N, ld_w_slice, true, false};
     c.P = M; c.Q = K; c.R = N; c.bn_P = M; c.bn_Q = K;
     c.mode = (k == 1) ? MODE_NONE : (out_split ? MODE_RED : MODE_COLS);
     c.L = L; c.k_total = k; c.s_begin = sb; c.s_end = se;
@@ -639,12 +672,12 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
     c.P = N; c.Q = K; c.R = M; c.bn_P = N; c.bn_Q = K;
     c.mode = (k == 1) ? MODE_NONE : (out_split ? MODE_ROWS : MODE_COLS);
     c.L = L; c.k_total = k; c.s_begin = sb; c.s_end = se;
-    c.epi = plain_epilogue(dw, K, dw_dtype == OSDP_DTYPE_FP32);
+    c.epi = plain_epilogue(dw, ld_dw_slice > 0 ? ld_dw_slice : K, dw_dtype == OSDP_DTYPE_FP32);
     c.epi.accumulate = accumulate;
+    c.out_is_slice = (ld_dw_slice > 0 && k > 1) ? 1 : 0;
     c.status = status;
     return launch_gemm(c, stream);
   };
-  (void)mode_sum;
 
   if (act == OSDP_ACT_NONE) {
     if (dx) { rc = dx_call(Operand{dy, N, M, N, false, true}, s_begin, s_end); if (rc) return rc; }
@@ -787,6 +820,52 @@ int osdp_split_linear_bwd_slice(const void *dy, const void *x, const void *w_fla
                                 int flags, float *dbias, void *ws, size_t ws_bytes, void *stream) {
   return bwd_impl(dy, x, w_flat, w_offset, z_saved, M, N, K, k_split, split_dim, act, slice_idx, 0, true, dx, dw_flat,
                   dw_offset, dw_dtype, flags, dbias, ws, ws_bytes, stream);
+}
+
+int osdp_zdp_shard_layout(int64_t N, int64_t K, int k_split, int split_dim, int world, int slice_idx,
+                          int64_t *slice_elems, int64_t *shard_elems, int64_t *shard_offset, int64_t *ld) {
+  if (N <= 0 || K <= 0) return OSDP_ERR_BAD_SHAPE;
+  if ((N & 7) || (K & 7)) return OSDP_ERR_ALIGNMENT;
+  if (split_dim != OSDP_SPLIT_OUT && split_dim != OSDP_SPLIT_RED) return OSDP_ERR_BAD_SPLIT;
+  if (world < 1 || world > 65536) return OSDP_ERR_BAD_SHAPE;
+  const bool out_split = (split_dim == OSDP_SPLIT_OUT);
+  const int64_t D = out_split ? N : K;
+  const int64_t other = out_split ? K : N;
+  int64_t L = 0;
+  int rc = slice_len(D, k_split, &L);
+  if (rc) return rc;
+  const int k = k_split == 0 ? 1 : k_split;
+  if (slice_idx < 0 || slice_idx > k) return OSDP_ERR_BAD_SPLIT;
+  int64_t off = 0, ls = 0, elems = 0, shard = 0;
+  for (int s = 0; s <= slice_idx; ++s) {
+    off += shard;
+    if (s == k) { ls = 0; elems = 0; shard = 0; break; }
+    ls = (D - s * L < L) ? D - s * L : L;
+    elems = ls * other;
+    shard = (elems + (int64_t)world * 8 - 1) / ((int64_t)world * 8) * 8;
+  }
+  if (slice_elems) *slice_elems = elems;
+  if (shard_elems) *shard_elems = shard;
+  if (shard_offset) *shard_offset = off;
+  if (ld) *ld = out_split ? K : ls;
+  return OSDP_OK;
+}
+
+int osdp_zdp_linear_fwd_slice(const void *x, const void *w_slice, int64_t ld_w, const float *bias, int64_t M,
+                              int64_t N, int64_t K, int k_split, int split_dim, int act, int flags, int slice_idx,
+                              void *out, void *z_save, void *ws, size_t ws_bytes, void *stream) {
+  if (ld_w <= 0) return OSDP_ERR_BAD_SHAPE;
+  return fwd_impl(x, w_slice, 0, bias, M, N, K, k_split, split_dim, act, flags, slice_idx, 0, true, out, z_save, ws,
+                  ws_bytes, stream, ld_w);
+}
+
+int osdp_zdp_linear_bwd_slice(const void *dy, const void *x, const void *w_slice, int64_t ld_w, const void *z_saved,
+                              int64_t M, int64_t N, int64_t K, int k_split, int split_dim, int act, int slice_idx,
+                              void *dx, void *dw_slice, int64_t ld_dw, int dw_dtype, int flags, float *dbias,
+                              void *ws, size_t ws_bytes, void *stream) {
+  if (ld_w <= 0 || (dw_slice && ld_dw <= 0)) return OSDP_ERR_BAD_SHAPE;
+  return bwd_impl(dy, x, w_slice, 0, z_saved, M, N, K, k_split, split_dim, act, slice_idx, 0, true, dx, dw_slice, 0,
+                  dw_dtype, flags, dbias, ws, ws_bytes, stream, ld_w, dw_slice ? ld_dw : 0);
 }
 
 int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const float *b1, int64_t off_w2,

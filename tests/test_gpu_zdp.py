@@ -1,0 +1,216 @@
+"""GPU parity of the sharded slice loop (Section 3.3 combined with zero-redundancy data parallelism):
+the per-slice entry points that read a gathered compact slice, and the loop around them with the
+ranks of a data-parallel group emulated one after another in this process (no kernel waits on
+another rank), checked against the fp64 oracle on the whole batch."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2209_13258_b200 import inputs
+from util import Guarded, assert_close, to_dev, to_f64
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def P():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2209_13258_b200 as pkg
+    pkg.lib()
+    return pkg
+
+
+def bits(t):
+    return t.view(torch.int32 if t.dtype == torch.float32 else torch.int16)
+
+
+SHAPES = [(256, 2048, 512, 4), (300, 520, 328, 3), (130, 392, 264, 5), (1024, 1024, 2048, 2)]
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("split", [0, 1])
+@pytest.mark.parametrize("act", [0, 1])
+def test_gathered_slice_entry_points_match_flat_buffer_ones_bit_for_bit(P, shape, split, act):
+    from paper_2209_13258_b200.zdp import ShardLayout
+    M, N, K, k = shape
+    D = N if split == 0 else K
+    if P.osdp_slice_range(D, k, 0)[0] != 0:
+        pytest.skip("invalid split")
+    c = inputs.linear_case(M, N, K, w_std=0.05, bias_std=0.2, w_offset=64, flat_pad=8)
+    x, dy, wf, b = to_dev(c["x"]), to_dev(c["dy"]), to_dev(c["w_flat"]), to_dev(c["bias"])
+    off = c["w_offset"]
+    W = wf[off:off + N * K].view(N, K)
+    lay = ShardLayout(N, K, k, split, 1)
+    _, n1 = P.osdp_split_linear_workspace_bytes(M, N, K, k, split, act, P.OP_LINEAR_FWD)
+    _, n2 = P.osdp_split_linear_workspace_bytes(M, N, K, k, split, act, P.OP_LINEAR_BWD)
+    res = {}
+    for staged in (False, True):
+        ws = P.new_workspace(max(n1, n2))
+        out, z, dx = Guarded((M, N), torch.bfloat16), Guarded((M, N), torch.bfloat16), Guarded((M, K), torch.bfloat16)
+        dwf = torch.zeros(wf.numel(), dtype=torch.float32, device="cuda")
+        db = Guarded((N,), torch.float32)
+        zs = z.t if act else None
+        dw_full = torch.zeros(N, K, dtype=torch.float32, device="cuda")
+        for s in range(k):
+            if staged:
+                wslice = Guarded((lay.slices[s][2],), torch.bfloat16)
+                wslice.t.copy_(lay.slice_matrix(W, s).contiguous().reshape(-1))
+                P.osdp_zdp_linear_fwd_slice(x, wslice.t, lay.slices[s][5], b, M, N, K, k, split, act, s, out.t, zs, ws,
+                                            check=True)
+                wslice.check()
+            else:
+                P.osdp_split_linear_fwd_slice(x, wf, off, b, M, N, K, k, split, act, s, out.t, zs, ws, check=True)
+        for s in range(k):
+            if staged:
+                bq, e, elems, _, _, ld = lay.slices[s]
+                wslice = lay.slice_matrix(W, s).contiguous()
+                dws = Guarded((elems,), torch.float32)
+                P.osdp_zdp_linear_bwd_slice(dy, x, wslice, ld, zs, M, N, K, k, split, act, s, dx.t, dws.t, ld,
+                                            P.DTYPE_FP32, 0, db.t, ws, check=True)
+                dws.check()
+                assert not bool(torch.isnan(dws.t).any()), "slice gradient not fully written"
+                lay.slice_matrix(dw_full, s).copy_(dws.t.view(-1, ld))
+            else:
+                P.osdp_split_linear_bwd_slice(dy, x, wf, off, zs, M, N, K, k, split, act, s, dx.t, dwf, off,
+                                              P.DTYPE_FP32, 0, db.t, ws, check=True)
+        if not staged:
+            dw_full = dwf[off:off + N * K].view(N, K).clone()
+        rc, st = P.osdp_read_device_status(ws)
+        assert rc == 0 and st == 0
+        for g in (out, dx, db) + ((z,) if act else ()):
+            g.check()
+        res[staged] = {"y": out.t.clone(), "dx": dx.t.clone(), "dw": dw_full, "db": db.t.clone()}
+    for name in ("y", "dx", "dw", "db"):
+        assert torch.equal(bits(res[True][name]), bits(res[False][name])), name
+
+
+def test_gathered_slice_argument_errors(P):
+    M, N, K, k = 128, 256, 128, 2
+    x = torch.zeros(M, K, dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros(N // k, K, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(M, N, dtype=torch.bfloat16, device="cuda")
+    _, n = P.osdp_split_linear_workspace_bytes(M, N, K, k, 0, 0, P.OP_LINEAR_BWD)
+    ws = P.new_workspace(n)
+    f = P.osdp_zdp_linear_fwd_slice
+    assert f(x, w, 0, None, M, N, K, k, 0, 0, 0, out, None, ws) == 2        # ld_w <= 0
+    assert f(x, w, K - 8, None, M, N, K, k, 0, 0, 0, out, None, ws) == 2    # ld_w below the slice's row length
+    assert f(x, w, K + 4, None, M, N, K, k, 0, 0, 0, out, None, ws) == 4    # ld_w not a multiple of 8
+    assert f(x, w, K, None, M, N, K, k, 0, 0, 2, out, None, ws) == 3        # slice index out of range
+    assert f(x, None, K, None, M, N, K, k, 0, 0, 0, out, None, ws) == 1
+    g = P.osdp_zdp_linear_bwd_slice
+    dw = torch.zeros(N // k, K, dtype=torch.float32, device="cuda")
+    assert g(out, x, w, K, None, M, N, K, k, 0, 0, 0, None, dw, 0, P.DTYPE_FP32, 0, None, ws) == 2
+    assert g(out, x, w, K, None, M, N, K, k, 0, 0, 0, None, dw, K - 8, P.DTYPE_FP32, 0, None, ws) == 2
+    assert g(out, x, w, K, None, M, N, K, k, 0, 0, 0, None, dw, K, P.DTYPE_FP32, P.FLAG_PAIR_SLICES, None, ws) == 6
+    assert g(out, x, w, K, None, M, N, K, k, 0, 0, 0, None, None, 0, P.DTYPE_FP32, 0, None, ws) == 0   # dW skipped
+
+
+class EmulatedComm:
+    """The loop's two collectives for `world` ranks that run one after another in this process:
+    all ranks' parameter shards are visible, and reduce-scatter adds the caller's contribution to
+    per-rank accumulators (the sum over ranks is complete once every rank has run)."""
+
+    def __init__(self, rank, world, param_shards, grad_acc):
+        self.rank, self.world = rank, world
+        self.param_shards, self.grad_acc = param_shards, grad_acc
+
+    def all_gather_slice(self, dst, shard_buf, off, n):
+        assert shard_buf.data_ptr() == self.param_shards[self.rank].data_ptr()
+        for q in range(self.world):
+            dst[q * n:(q + 1) * n].copy_(self.param_shards[q][off:off + n])
+
+    def reduce_scatter_slice(self, shard_buf, off, n, src):
+        for q in range(self.world):
+            self.grad_acc[q][off:off + n] += src[q * n:(q + 1) * n].double()
+        shard_buf[off:off + n].copy_(src[self.rank * n:(self.rank + 1) * n])   # this rank's own term only
+
+    def all_reduce(self, t):
+        raise NotImplementedError
+
+
+@pytest.mark.parametrize("world", [1, 2, 3])
+@pytest.mark.parametrize("split", [0, 1])
+@pytest.mark.parametrize("case", [(384, 520, 264, 3, 1), (512, 2048, 512, 4, 0), (300, 1024, 1024, 8, 1)])
+def test_slice_loop_over_emulated_ranks_matches_oracle(P, world, split, case):
+    from paper_2209_13258_b200.zdp import ShardLayout, ZdpSplitLinear
+    M, N, K, k, act = case
+    D = N if split == 0 else K
+    if P.osdp_slice_range(D, k, 0)[0] != 0:
+        pytest.skip("invalid split")
+    c = inputs.linear_case(M, N, K, w_std=0.05, bias_std=0.2)
+    W = to_dev(c["w_flat"])[c["w_offset"]:c["w_offset"] + N * K].view(N, K)
+    bias = to_dev(c["bias"])
+    lay = ShardLayout(N, K, k, split, world)
+    param_shards = [lay.shard_of(W, r) for r in range(world)]
+    grad_acc = [torch.zeros(lay.shard_total, dtype=torch.float64, device="cuda") for _ in range(world)]
+    y = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+    dx = torch.empty(M, K, dtype=torch.bfloat16, device="cuda")
+    db = torch.zeros(N, dtype=torch.float64, device="cuda")
+    x_all, dy_all = to_dev(c["x"]), to_dev(c["dy"])
+    stage_bytes = None
+    for r in range(world):
+        rows = torch.arange(r, M, world, device="cuda")               # this rank's tokens
+        comm = EmulatedComm(r, world, param_shards, grad_acc)
+        layer = ZdpSplitLinear(N, K, k, split, act=act, comm=comm)
+        layer.param_shard = param_shards[r]                            # the rank's own shard buffer
+        xr, dyr = x_all[rows].contiguous(), dy_all[rows].contiguous()
+        zr = torch.empty(rows.numel(), N, dtype=torch.bfloat16, device="cuda") if act else None
+        yr = layer.forward(xr, bias=bias, z_save=zr)
+        dbr = torch.empty(N, dtype=torch.float32, device="cuda")
+        dxr = layer.backward(dyr, xr, z_saved=zr, dbias=dbr)
+        torch.cuda.synchronize()
+        rc, st = P.osdp_read_device_status(layer._ws)
+        assert rc == 0 and st == 0
+        y[rows], dx[rows] = yr, dxr
+        db += dbr.double()
+        stage_bytes = layer.staging_bytes(rows.numel())
+        # the gathered weights never take more than two slices' worth
+        assert stage_bytes["weight_staging"] == 2 * 2 * world * max(sl[3] for sl in lay.slices)
+        assert stage_bytes["weight_staging"] <= 2 * 2 * (N * K // k + 8 * world + max(N, K) * 8)
+    dW = lay.unshard(grad_acc)
+    z, yo = oracle.linear_fwd(c["x"], c["w"], c["bias"], act, k, split)
+    dXo, dWo, dbo = oracle.linear_bwd(c["dy"], c["x"], c["w"], z, act, k, split)
+    assert_close(to_f64(y), yo, "Y")
+    assert_close(to_f64(dx), dXo, "dX")
+    assert_close(dW.cpu().numpy(), dWo, "dW (sum over ranks)")
+    assert_close(db.cpu().numpy(), dbo, "db (sum over ranks)")
+
+
+def test_slice_loop_on_a_one_rank_nccl_group(P):
+    """The product's own communicator (torch.distributed, NCCL) with world size 1: every collective
+    of the loop runs, on its own stream, and the result matches the oracle."""
+    import torch.distributed as dist
+    from paper_2209_13258_b200.zdp import ZdpSplitLinear
+    if dist.is_initialized():
+        pytest.skip("a process group already exists in this process")
+    M, N, K, k = 512, 1024, 512, 4
+    dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29753", rank=0, world_size=1)
+    try:
+        for split in (0, 1):
+            c = inputs.linear_case(M, N, K, w_std=0.05, bias_std=0.2)
+            W = to_dev(c["w_flat"])[c["w_offset"]:c["w_offset"] + N * K].view(N, K)
+            layer = ZdpSplitLinear(N, K, k, split, act=1)
+            layer.load_full_weight(W)
+            x, dy, bias = to_dev(c["x"]), to_dev(c["dy"]), to_dev(c["bias"])
+            z = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+            db = torch.empty(N, dtype=torch.float32, device="cuda")
+            for _ in range(2):   # twice: staging buffers and events are reused correctly
+                y = layer.forward(x, bias=bias, z_save=z)
+                dx = layer.backward(dy, x, z_saved=z, dbias=db)
+            torch.cuda.synchronize()
+            dW = layer.layout.unshard([layer.grad_shard])
+            zo, yo = oracle.linear_fwd(c["x"], c["w"], c["bias"], 1, k, split)
+            dXo, dWo, dbo = oracle.linear_bwd(c["dy"], c["x"], c["w"], zo, 1, k, split)
+            assert_close(to_f64(y), yo, "Y")
+            assert_close(to_f64(dx), dXo, "dX")
+            assert_close(to_f64(dW), dWo, "dW")
+            assert_close(to_f64(db), dbo, "db")
+            # accumulate=True adds a second identical gradient
+            layer.backward(dy, x, z_saved=z, dbias=db, accumulate=True)
+            torch.cuda.synchronize()
+            assert_close(to_f64(layer.layout.unshard([layer.grad_shard])), 2 * dWo, "dW accumulated")
+    finally:
+        dist.destroy_process_group()
