@@ -4,6 +4,9 @@
     python -m paper_2209_13258_b200.sweep case-mlp M hidden ffn k   one MLP-block fwd+bwd (twice), for profilers
     python -m paper_2209_13258_b200.sweep linear M N K [ks]         time vs slice granularity, both split dims
     python -m paper_2209_13258_b200.sweep mlp M hidden ffn [ks]     MLP block split along ffn: time and staging
+    python -m paper_2209_13258_b200.sweep zdp M N K [ks]            sharded slice loop (gather / compute /
+                                                                    reduce-scatter per slice) against the resident-
+                                                                    weight path; also under torchrun, M tokens per rank
 
 The `linear` and `mlp` modes reproduce in kind the paper's Figure 7 (time and memory of an operator
 against slice granularity) for this single-GPU path: TFLOP/s, overhead versus k = 1, staging bytes.
@@ -170,6 +173,66 @@ def sweep_mlp(M, H, F, ks):
     return rows
 
 
+def sweep_zdp(M, N, K, ks):
+    """Time and staging of the sharded slice loop per granularity.  Stand-alone it forms a one-rank NCCL
+    group (every collective still runs, as a device copy); under torchrun every rank works on M tokens."""
+    import os
+    import torch.distributed as dist
+    from .zdp import ZdpSplitLinear
+    own_group = not dist.is_initialized()
+    if own_group:
+        if "RANK" in os.environ:
+            torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+            dist.init_process_group("nccl")
+        else:
+            dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29755", rank=0, world_size=1)
+    rank, world = dist.get_rank(), dist.get_world_size()
+    x, w, dy, out, dx, _, db = _linear_tensors(M, N, K)
+    dw = torch.empty(N, K, device="cuda", dtype=torch.float32)
+    flops = 3 * 2.0 * M * N * K
+    cfgs, fns, layers = [], [], []
+    for k in ks:
+        for split, name in ((P.SPLIT_OUT, "out"), (P.SPLIT_RED, "red")):
+            if k == 1 and split == P.SPLIT_RED:
+                continue
+            if P.osdp_slice_range(N if split == P.SPLIT_OUT else K, k, 0)[0] != 0:
+                continue
+            cfgs.append((k, split, name))
+    ws = P.new_workspace(max(_ws_linear(M, N, K, k, split) for k, split, _ in cfgs))
+    for k, split, name in cfgs:
+        layer = ZdpSplitLinear(N, K, k, split, dw_dtype=P.DTYPE_FP32)
+        layer.load_full_weight(w)
+        layers.append(layer)
+
+        def resident(k=k, split=split):
+            P.osdp_split_linear_fwd(x, w, 0, None, M, N, K, k, split, 0, out, None, ws, check=True)
+            P.osdp_split_linear_bwd(dy, x, w, 0, None, M, N, K, k, split, 0, dx, dw, 0, P.DTYPE_FP32, 0, db, ws,
+                                    check=True)
+
+        def sharded(layer=layer):
+            layer.forward(x, out=out)
+            layer.backward(dy, x, dx=dx, dbias=db)
+        fns += [resident, sharded]
+    ts = _time_interleaved(fns, rounds=8)
+    tt = torch.tensor(ts, device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)     # a step is as slow as its slowest rank
+    ts = tt.tolist()
+    rows = []
+    for i, (k, split, name) in enumerate(cfgs):
+        st = layers[i].staging_bytes(M)
+        rows.append({"k": k, "split": name, "world": world, "resident_ms": ts[2 * i], "sharded_ms": ts[2 * i + 1],
+                     "sharded_tflops_all_ranks": world * flops / ts[2 * i + 1] / 1e9,
+                     "loop_overhead": ts[2 * i + 1] / ts[2 * i] - 1.0,
+                     "weight_staging_bytes": st["weight_staging"], "grad_staging_bytes": st["grad_staging"],
+                     "workspace_bytes": st["workspace"], "full_gather_bytes": N * K * 2, "full_grad_bytes": N * K * 4})
+        if rank == 0:
+            print(json.dumps(rows[-1]), flush=True)
+    if own_group:
+        dist.destroy_process_group()
+    return rows
+
+
 def main(argv):
     if len(argv) < 2:
         print(__doc__)
@@ -184,6 +247,8 @@ def main(argv):
         sweep_linear(int(argv[2]), int(argv[3]), int(argv[4]), ks)
     elif mode == "mlp":
         sweep_mlp(int(argv[2]), int(argv[3]), int(argv[4]), ks)
+    elif mode == "zdp":
+        sweep_zdp(int(argv[2]), int(argv[3]), int(argv[4]), ks)
     else:
         print(__doc__)
         return 2

@@ -116,9 +116,10 @@ class ZdpSplitLinear:
         self.grad_shard = torch.zeros(self.layout.shard_total, dtype=gdt, device=self.device)
         # Two staging buffers each for gathered weights and for weight gradients: slice s+1 is gathered
         # while slice s computes.  Their tails beyond a slice's elements are never written by the kernels.
-        self.w_stage = [torch.zeros(self.layout.stage_elems, dtype=torch.bfloat16, device=self.device) for _ in range(2)]
-        self.dw_stage = [torch.zeros(self.layout.stage_elems, dtype=gdt, device=self.device) for _ in range(2)]
+        self.w_stage = [torch.zeros(self.layout.stage_elems, dtype=torch.bfloat16, device=self.device) for _ in range(min(2, self.k))]
+        self.dw_stage = [torch.zeros(self.layout.stage_elems, dtype=gdt, device=self.device) for _ in range(min(2, self.k))]
         self.comm_stream = torch.cuda.Stream(device=self.device)
+        self.side_stream = torch.cuda.Stream(device=self.device)
         self._ws = None
         self._ws_key = None
 
@@ -134,8 +135,8 @@ class ZdpSplitLinear:
         _, b = B.osdp_split_linear_workspace_bytes(M, self.N, self.K, self.k, self.split_dim, self.act,
                                                    B.OP_LINEAR_BWD, self.flags & B.FLAG_CARRY_BF16)
         stage = sum(t.numel() * t.element_size() for t in self.w_stage + self.dw_stage)
-        return {"weight_staging": 2 * self.w_stage[0].numel() * 2,
-                "grad_staging": stage - 2 * self.w_stage[0].numel() * 2, "workspace": max(f, b)}
+        wbytes = len(self.w_stage) * self.w_stage[0].numel() * 2
+        return {"weight_staging": wbytes, "grad_staging": stage - wbytes, "workspace": max(f, b)}
 
     def _workspace(self, M):
         nbytes = self.staging_bytes(M)["workspace"]
@@ -145,17 +146,28 @@ class ZdpSplitLinear:
         return self._ws
 
     # -- the slice loops --------------------------------------------------------------------------
-    def _gather(self, s, free_event):
+    # Slices whose outputs are concatenated (forward under OUT, dW always, dX under RED) do not depend on
+    # one another, so consecutive ones are launched on two alternating streams: the next slice's CTAs
+    # take over the SMs that the current slice's last, partly filled wave leaves idle.  Slices of a summed
+    # output (forward under RED, dX under OUT) stay in order on the caller's stream.
+    def _gather(self, s, free_events):
         """Issues the all-gather of slice s into its staging buffer on the communication stream."""
         import torch
         _, _, _, shard, off, _ = self.layout.slices[s]
         with torch.cuda.stream(self.comm_stream):
-            if free_event is not None:
-                self.comm_stream.wait_event(free_event)     # the slice that last read this buffer is done
+            for ev in free_events:
+                self.comm_stream.wait_event(ev)             # the slice that last read this buffer is done
             self.comm.all_gather_slice(self.w_stage[s & 1], self.param_shard, off, shard)
             ready = torch.cuda.Event()
             ready.record(self.comm_stream)
         return ready
+
+    @staticmethod
+    def _mark(stream):
+        import torch
+        ev = torch.cuda.Event()
+        ev.record(stream)
+        return ev
 
     def forward(self, x, bias=None, out=None, z_save=None):
         import torch
@@ -165,17 +177,23 @@ class ZdpSplitLinear:
             out = torch.empty(M, self.N, dtype=torch.bfloat16, device=self.device)
         ws = self._workspace(M)
         self.comm_stream.wait_stream(cur)                   # shards may just have been updated on `cur`
-        done = [None, None]
-        ready = self._gather(0, None)
+        two = self.k > 1 and self.split_dim == B.SPLIT_OUT
+        lanes = [cur, self.side_stream] if two else [cur, cur]
+        if two:
+            self.side_stream.wait_stream(cur)
+        done = [[], []]
+        ready = self._gather(0, [])
         for s in range(self.k):
             nxt = self._gather(s + 1, done[(s + 1) & 1]) if s + 1 < self.k else None
-            cur.wait_event(ready)
+            st = lanes[s & 1]
+            st.wait_event(ready)
             B.osdp_zdp_linear_fwd_slice(x, self.w_stage[s & 1], self.layout.slices[s][5], bias, M, self.N, self.K,
-                                        self.k, self.split_dim, self.act, s, out, z_save, ws, stream=cur, check=True,
+                                        self.k, self.split_dim, self.act, s, out, z_save, ws, stream=st, check=True,
                                         flags=self.flags & B.FLAG_CARRY_BF16)
-            done[s & 1] = torch.cuda.Event()
-            done[s & 1].record(cur)
+            done[s & 1] = [self._mark(st)]
             ready = nxt
+        if two:
+            cur.wait_stream(self.side_stream)
         self.comm_stream.wait_stream(cur)
         return out
 
@@ -185,36 +203,57 @@ class ZdpSplitLinear:
         dbias (if given) is this rank's column sum; reduce it with comm.all_reduce where needed."""
         import torch
         M = x.shape[0]
-        cur = torch.cuda.current_stream(self.device)
+        cur, side = torch.cuda.current_stream(self.device), self.side_stream
         if need_dx and dx is None:
             dx = torch.empty(M, self.K, dtype=torch.bfloat16, device=self.device)
         ws = self._workspace(M)
         self.comm_stream.wait_stream(cur)
-        w_free = [None, None]
+        side.wait_stream(cur)
+        out_split = self.split_dim == B.SPLIT_OUT
+        # OUT: the dX chain on `cur`, the independent dW_s on `side` (not with an activation: its staged
+        # G_s in the workspace serves one stream).  RED: whole slices alternate between the two streams.
+        split_calls = self.k > 1 and out_split and self.act == B.ACT_NONE and need_dx
+        alternate = self.k > 1 and not out_split
+        flags = self.flags & B.FLAG_CARRY_BF16
+        w_free = [[], []]
         dw_free = [None, None]
         tmp = torch.empty_like(self.dw_stage[0][:max(sl[3] for sl in self.layout.slices)]) if accumulate else None
-        ready = self._gather(0, None)
+        ready = self._gather(0, [])
         for s in range(self.k):
+            b = s & 1
             nxt = self._gather(s + 1, w_free[(s + 1) & 1]) if s + 1 < self.k else None
             _, _, _, shard, off, ld = self.layout.slices[s]
-            cur.wait_event(ready)
-            if dw_free[s & 1] is not None:
-                cur.wait_event(dw_free[s & 1])              # the reduce-scatter that read this buffer is done
-            B.osdp_zdp_linear_bwd_slice(dy, x, self.w_stage[s & 1], ld, z_saved, M, self.N, self.K, self.k,
-                                        self.split_dim, self.act, s, dx if need_dx else None, self.dw_stage[s & 1],
-                                        ld, self.dw_dtype, self.flags & B.FLAG_CARRY_BF16, dbias, ws, stream=cur,
-                                        check=True)
-            w_free[s & 1] = torch.cuda.Event()
-            w_free[s & 1].record(cur)
+            args = (dy, x, self.w_stage[b], ld, z_saved, M, self.N, self.K, self.k, self.split_dim, self.act, s)
+            if split_calls:
+                cur.wait_event(ready)
+                B.osdp_zdp_linear_bwd_slice(*args, dx, None, 0, self.dw_dtype, flags, None, ws, stream=cur, check=True)
+                side.wait_event(ready)
+                if dw_free[b] is not None:
+                    side.wait_event(dw_free[b])             # the reduce-scatter that read this buffer is done
+                B.osdp_zdp_linear_bwd_slice(*args, None, self.dw_stage[b], ld, self.dw_dtype, 0, dbias, ws,
+                                            stream=side, check=True)
+                w_free[b] = [self._mark(cur), self._mark(side)]
+                dw_done = w_free[b][1]
+            else:
+                st = (cur, side)[b] if alternate else cur
+                if alternate and s == 1 and self.act != B.ACT_NONE:
+                    st.wait_event(w_free[0][0])             # slice 0 stages G for every later slice
+                st.wait_event(ready)
+                if dw_free[b] is not None:
+                    st.wait_event(dw_free[b])
+                B.osdp_zdp_linear_bwd_slice(*args, dx if need_dx else None, self.dw_stage[b], ld, self.dw_dtype,
+                                            flags, dbias, ws, stream=st, check=True)
+                w_free[b] = [self._mark(st)]
+                dw_done = w_free[b][0]
             with torch.cuda.stream(self.comm_stream):
-                self.comm_stream.wait_event(w_free[s & 1])
+                self.comm_stream.wait_event(dw_done)
                 if accumulate:
-                    self.comm.reduce_scatter_slice(tmp, 0, shard, self.dw_stage[s & 1])
+                    self.comm.reduce_scatter_slice(tmp, 0, shard, self.dw_stage[b])
                     self.grad_shard[off:off + shard].add_(tmp[:shard])
                 else:
-                    self.comm.reduce_scatter_slice(self.grad_shard, off, shard, self.dw_stage[s & 1])
-                dw_free[s & 1] = torch.cuda.Event()
-                dw_free[s & 1].record(self.comm_stream)
+                    self.comm.reduce_scatter_slice(self.grad_shard, off, shard, self.dw_stage[b])
+                dw_free[b] = self._mark(self.comm_stream)
             ready = nxt
+        cur.wait_stream(side)
         cur.wait_stream(self.comm_stream)                   # grad_shard is complete for whoever runs next on `cur`
         return dx
