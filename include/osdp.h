@@ -59,6 +59,7 @@ extern "C" {
 #define OSDP_ERR_CUDA 7               /* a CUDA call failed; see osdp_last_cuda_error */
 #define OSDP_ERR_DEVICE_TIMEOUT 8     /* a bounded device-side wait ran out (status word) */
 #define OSDP_ERR_EXCEEDS_STATIC_SCRATCH 9 /* osdp_bias_grad_noalloc: ceil(M/1024) * N too large */
+#define OSDP_ERR_SEARCH_LIMIT 10      /* osdp_plan_search: node budget spent; the plan returned is feasible, maybe not optimal */
 
 #define OSDP_SPLIT_OUT 0
 #define OSDP_SPLIT_RED 1
@@ -262,6 +263,38 @@ int osdp_debug_wait_probe(void *ws, int64_t limit_us, void *stream);
  * GPU (different streams, different threads) race on it: serialise them. */
 #define OSDP_NOALLOC_MAX_PARTIALS (1 << 20)
 int osdp_bias_grad_noalloc(const void *dy, int64_t M, int64_t N, float *dbias, void *stream);
+
+/* ---- Execution-plan search (host only; Section 3.1: problem formulation and cost model, Algorithm 1).
+ * An operator is five doubles {model, act, extra, S, gamma}: bytes of its model states (parameters and
+ * optimiser states), activation bytes per sample, other bytes, bytes of its parameters (what the
+ * collectives move), computation time per sample.  `ops` holds n of them back to back.  A mode is
+ * 0 (DP: states replicated, two collectives per step) or 1 (ZDP: states sharded over the `world` ranks,
+ * three collectives).  With N = world:
+ *   memory(p, b) = sum_i ( model_i or model_i / N ) + b * act_i + extra_i
+ *   time(p, b)   = sum_i ( 2 or 3 ) * (N - 1) * (alpha + S_i / N * beta) + b * gamma_i
+ * alpha = latency per communication step, beta = transfer time per byte; all values >= 0 and finite.
+ *
+ * osdp_plan_cost: memory and time of one given plan at batch size `batch`. */
+int osdp_plan_cost(const double *ops, int n, int world, double alpha, double beta, const uint8_t *modes,
+                   int batch, double *memory, double *time);
+
+/* osdp_plan_search: for b = 1, 2, ... the feasible plan (memory <= mem_limit) of least time; stops at the
+ * first b for which nothing fits or after max_batch (the paper's loop has no such cap; it keeps the loop
+ * finite when memory never runs out); returns the candidate with the least time per sample, time / b
+ * (the first such b on ties): modes[n], *batch, *time_per_sample.  *batch = 0 and *time_per_sample = +inf
+ * if nothing fits at b = 1.  The search is exact (depth-first with the memory and best-so-far prunings
+ * and a relaxation bound) unless it visits more than max_nodes nodes in one batch size (<= 0: 2e8), in
+ * which case it returns OSDP_ERR_SEARCH_LIMIT with the best feasible plan found.  nodes_visited may be
+ * NULL.  n <= 16384. */
+int osdp_plan_search(const double *ops, int n, int world, double alpha, double beta, double mem_limit,
+                     int max_batch, int64_t max_nodes, uint8_t *modes, int *batch,
+                     double *time_per_sample, int64_t *nodes_visited);
+
+/* Section 3.3, last paragraph: an operator cut into k slices is planned slice by slice (some slices DP,
+ * the others ZDP).  Writes k operators (5 doubles each) to `slices`: 1/k of every byte count, and
+ * gamma * (1 + overhead) / k, `overhead` being the measured relative cost of running the operator
+ * split k ways (> -1). */
+int osdp_plan_expand_slices(const double *op, int k, double overhead, double *slices);
 
 #ifdef __cplusplus
 }

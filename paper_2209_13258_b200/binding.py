@@ -24,6 +24,7 @@ EXPORTS = [
     "osdp_split_linear_bwd", "osdp_split_linear_bwd_slice", "osdp_split_mlp_fwd", "osdp_split_mlp_bwd",
     "osdp_read_device_status", "osdp_bias_grad_noalloc", "osdp_debug_wait_probe", "osdp_suggest_granularity",
     "osdp_zdp_shard_layout", "osdp_zdp_linear_fwd_slice", "osdp_zdp_linear_bwd_slice",
+    "osdp_plan_cost", "osdp_plan_search", "osdp_plan_expand_slices",
 ]
 
 _lib = None
@@ -76,6 +77,10 @@ def lib():
         L.osdp_zdp_linear_fwd_slice.argtypes = [vp, vp, i64, vp, i64, i64, i64, ci, ci, ci, ci, ci, vp, vp, vp, sz, vp]
         L.osdp_zdp_linear_bwd_slice.argtypes = [vp, vp, vp, i64, vp, i64, i64, i64, ci, ci, ci, ci, vp, vp, i64, ci,
                                                 ci, vp, vp, sz, vp]
+        pd, pu8, dbl = ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_uint8), ctypes.c_double
+        L.osdp_plan_cost.argtypes = [pd, ci, ci, dbl, dbl, pu8, ci, pd, pd]
+        L.osdp_plan_search.argtypes = [pd, ci, ci, dbl, dbl, dbl, ci, i64, pu8, ctypes.POINTER(ci), pd, p64]
+        L.osdp_plan_expand_slices.argtypes = [pd, ci, dbl, pd]
         for name in EXPORTS:
             getattr(L, name)
             if name not in ("osdp_status_string",):
@@ -264,3 +269,36 @@ def osdp_zdp_linear_bwd_slice(dy, x, w_slice, ld_w, z_saved, M, N, K, k_split, s
                                          _ptr(dw_slice), int(ld_dw), int(dw_dtype), int(flags), _ptr(dbias), wp, wn,
                                          _stream(stream))
     return _ret(rc, check, "osdp_zdp_linear_bwd_slice")
+
+
+def _ops_array(ops):
+    flat = [float(v) for op in ops for v in op]
+    if len(flat) != 5 * len(ops):
+        raise ValueError("an operator is (model, act, extra, S, gamma)")
+    return (ctypes.c_double * len(flat))(*flat)
+
+
+def osdp_plan_cost(ops, world, alpha, beta, modes, batch):
+    """Returns (status, memory, time) of one plan; ops = [(model, act, extra, S, gamma), ...], modes 0 DP / 1 ZDP."""
+    m, t = ctypes.c_double(), ctypes.c_double()
+    md = (ctypes.c_uint8 * len(ops))(*[int(v) for v in modes])
+    rc = lib().osdp_plan_cost(_ops_array(ops), len(ops), int(world), float(alpha), float(beta), md, int(batch),
+                              ctypes.byref(m), ctypes.byref(t))
+    return rc, m.value, t.value
+
+
+def osdp_plan_search(ops, world, alpha, beta, mem_limit, max_batch, max_nodes=0):
+    """Returns (status, modes, batch, time_per_sample, nodes_visited)."""
+    md = (ctypes.c_uint8 * len(ops))()
+    b, t, nodes = ctypes.c_int(), ctypes.c_double(), ctypes.c_int64()
+    rc = lib().osdp_plan_search(_ops_array(ops), len(ops), int(world), float(alpha), float(beta), float(mem_limit),
+                                int(max_batch), int(max_nodes), md, ctypes.byref(b), ctypes.byref(t),
+                                ctypes.byref(nodes))
+    return rc, tuple(md), b.value, t.value, nodes.value
+
+
+def osdp_plan_expand_slices(op, k, overhead=0.0):
+    """Returns (status, [k slice operators])."""
+    out = (ctypes.c_double * (5 * max(int(k), 1)))()
+    rc = lib().osdp_plan_expand_slices((ctypes.c_double * 5)(*[float(v) for v in op]), int(k), float(overhead), out)
+    return rc, [tuple(out[5 * s:5 * s + 5]) for s in range(max(int(k), 1))] if rc == 0 else []

@@ -7,7 +7,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libosdp.so")
-SOURCES = ["osdp_api.cu"]
+SOURCES = ["osdp_api.cu", "osdp_plan.cu"]
 HEADERS = ["osdp_gemm.cuh", "osdp_aux.cuh", os.path.join("..", "..", "include", "osdp.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -755,6 +755,7 @@ const char *osdp_status_string(int status) {
     case OSDP_ERR_CUDA: return "CUDA error";
     case OSDP_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
     case OSDP_ERR_EXCEEDS_STATIC_SCRATCH: return "problem larger than the library's built-in scratch";
+    case OSDP_ERR_SEARCH_LIMIT: return "plan search stopped at its node budget";
     default: return "unknown status";
   }
 }

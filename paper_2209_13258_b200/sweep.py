@@ -8,6 +8,11 @@
                                                                     reduce-scatter per slice) against the resident-
                                                                     weight path; also under torchrun, M tokens per rank
 
+    python -m paper_2209_13258_b200.sweep plan hidden layers tokens world mem_GB [ks]
+                                                                    execution plan (DP / ZDP per operator or per
+                                                                    slice, batch size) for a GPT-like stack of
+                                                                    linears, from compute times measured here
+
 The `linear` and `mlp` modes reproduce in kind the paper's Figure 7 (time and memory of an operator
 against slice granularity) for this single-GPU path: TFLOP/s, overhead versus k = 1, staging bytes.
 Timing: CUDA events on the current stream, median of `iters` runs after warm-up.
@@ -233,6 +238,52 @@ def sweep_zdp(M, N, K, ks):
     return rows
 
 
+def plan_from_measurements(hidden, layers, tokens, world, mem_gb, ks, alpha=10e-6, beta=1.0 / 770e9):
+    """Section 3.1 / Algorithm 1 fed with this GPU's kernel times: gamma_i of each linear of a GPT-like layer
+    (QKV, out-projection, the two MLP layers; `tokens` tokens per sample) is measured per slice granularity,
+    then the plan search runs on whole operators and on operators cut into k slices (Section 3.3, last
+    paragraph).  States: 16 bytes per parameter; wire: bf16 parameters; activations: the bf16 input and
+    output of each linear; alpha / beta default to 10 us per step and the 770 GB/s peer-copy figure."""
+    shapes = [("qkv", 3 * hidden, hidden), ("proj", hidden, hidden), ("fc1", 4 * hidden, hidden),
+              ("fc2", hidden, 4 * hidden)]
+    split_of = {"qkv": P.SPLIT_OUT, "proj": P.SPLIT_RED, "fc1": P.SPLIT_OUT, "fc2": P.SPLIT_RED}
+    gamma = {}
+    for name, N, K in shapes:
+        x, w, dy, out, dx, dw, db = _linear_tensors(tokens, N, K)
+        split = split_of[name]
+        valid = [k for k in ks if P.osdp_slice_range(N if split == P.SPLIT_OUT else K, k, 0)[0] == 0]
+        ws = P.new_workspace(max(_ws_linear(tokens, N, K, k, split) for k in valid))
+        fns = []
+        for k in valid:
+            def step(k=k):
+                P.osdp_split_linear_fwd(x, w, 0, None, tokens, N, K, k, split, 0, out, None, ws, check=True)
+                P.osdp_split_linear_bwd(dy, x, w, 0, None, tokens, N, K, k, split, 0, dx, dw, 0, 0, 0, db, ws,
+                                        check=True)
+            fns.append(step)
+        for k, t in zip(valid, _time_interleaved(fns)):
+            gamma[(name, k)] = t * 1e-3
+    limit = mem_gb * 1e9
+    rows = []
+    for k in ks:
+        if any((name, k) not in gamma for name, _, _ in shapes):
+            continue
+        ops = []
+        for _ in range(layers):
+            for name, N, K in shapes:
+                params = float(N * K)
+                op = (16.0 * params, 2.0 * tokens * (N + K), 0.0, 2.0 * params, gamma[(name, 1)])
+                rc, sl = P.osdp_plan_expand_slices(op, k, gamma[(name, k)] / gamma[(name, 1)] - 1.0)
+                ops += sl
+        rc, modes, b, t, nodes = P.osdp_plan_search(ops, world, alpha, beta, limit, 4096)
+        row = {"k": k, "status": rc, "operators": len(ops), "batch": b, "dp": modes.count(0) if b else 0,
+               "zdp": modes.count(1) if b else 0, "time_per_sample_ms": t * 1e3 if b else None,
+               "samples_per_s_per_gpu": 1.0 / t if b else 0.0, "nodes": nodes,
+               "gamma_ms": {name: gamma[(name, k)] * 1e3 for name, _, _ in shapes}}
+        rows.append(row)
+        print(json.dumps(row), flush=True)
+    return rows
+
+
 def main(argv):
     if len(argv) < 2:
         print(__doc__)
@@ -249,6 +300,9 @@ def main(argv):
         sweep_mlp(int(argv[2]), int(argv[3]), int(argv[4]), ks)
     elif mode == "zdp":
         sweep_zdp(int(argv[2]), int(argv[3]), int(argv[4]), ks)
+    elif mode == "plan":
+        ks = [int(v) for v in argv[7].split(",")] if len(argv) > 7 else [1, 2, 4, 8]
+        plan_from_measurements(int(argv[2]), int(argv[3]), int(argv[4]), int(argv[5]), float(argv[6]), ks)
     else:
         print(__doc__)
         return 2
