@@ -448,6 +448,19 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
       const cuuint32_t box[3] = {(cuuint32_t)bn, 32, 1};
       rc = encode3d(&p.carry_pf_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, c.epi.carry, dims, str, box, false);
       if (rc) return rc;
+      if (!c.epi.out_fp32) {
+        // the last slice's bf16 results leave as unswizzled boxes of 32 rows x 32 columns
+        const cuuint32_t box32[3] = {32, 32, 1};
+        const cuuint64_t so[2] = {(cuuint64_t)c.epi.ld_out * 2, (cuuint64_t)c.epi.ld_out * 2 * (cuuint64_t)c.P};
+        rc = encode3d(&p.out32_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, c.epi.out, dims, so, box32, false);
+        if (rc) return rc;
+        if (c.epi.z_save) {
+          const cuuint64_t sz[2] = {(cuuint64_t)c.epi.ld_z * 2, (cuuint64_t)c.epi.ld_z * 2 * (cuuint64_t)c.P};
+          rc = encode3d(&p.z32_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, c.epi.z_save, dims, sz, box32, false);
+          if (rc) return rc;
+        }
+      }
+
     }
   }
 

@@ -67,6 +67,7 @@ struct GemmParams {
   // Output-side maps (3-D, same slice-coordinate scheme): final output, saved pre-activation, fp32 carry.
   CUtensorMap out_main, out_tail, z_main, z_tail, carry_map;
   CUtensorMap carry_pf_map;  // same tensor as carry_map, unswizzled box of 32 rows x BN columns, for L2 prefetch
+  CUtensorMap out32_map, z32_map;   // summed output's last slice: bf16 out / z_save as unswizzled boxes of 32 x 32
   int out_sc_mul;
   int red_group;             // MODE_RED: slices whose products a tile accumulates in one pass (1, or 2 = adjacent pairs)
   int carry_bf16;            // MODE_RED: the running sum is kept in `out` itself, in bf16 (no fp32 carry buffer)
@@ -827,13 +828,18 @@ __global__ void __launch_bounds__((BN > 256) ? 384 : 256, 1) gemm_kernel(const _
             stage_issue(&p.carry_map, dst, cbase, w.carry_in != 0);
           }
         } else if (w.carry_in) {
-          // last slice: carry (prefetched by TMA, one box ahead) + accumulator -> bias/act -> out
-          // (summed outputs are never given the 512-wide tile, so here every warp owns all columns)
+          // Last slice: carry + accumulator -> bias/act -> out.  The carry box of the next 32 columns is
+          // fetched by TMA while this one is worked on; a box that has been read into registers is
+          // overwritten in place with the bf16 results (64 bytes per row; z_save in its second half) and
+          // leaves as a TMA store, so the buffer takes its next carry box once that store has read it.
+          // (Summed outputs are never given the 512-wide tile, so here every warp owns all columns.)
           const uint32_t cbar = bar_base + 8u * (2 * SL::STAGES + 5 + (warp - 4) * NB);
           int nchunks = (w.col_end - w.col0 + 31) / 32;
           if (nchunks > BN / 32) nchunks = BN / 32;
+          const bool staged_out = !p.epi.out_fp32;
           auto issue_load = [&](int c) {
             if (lane == 0) {
+              if (staged_out) bulk_wait_read<0>();   // the store that last left from this buffer
               const uint32_t b = n_cload % NB;
               mbar_expect_tx(cbar + 8u * b, 4096u);
               tma_load_3d(stg + b * 4096u, &p.carry_map, cbar + 8u * b, w.col0 + c * 32, wrow0, 0);
@@ -841,6 +847,8 @@ __global__ void __launch_bounds__((BN > 256) ? 384 : 256, 1) gemm_kernel(const _
             ++n_cload;
           };
           const uint32_t first = n_cload;
+          if (lane == 0) bulk_wait_read<0>();
+          __syncwarp();
           for (int c = 0; c < (int)NB - 1 && c < nchunks; ++c) issue_load(c);
 #pragma unroll 1
           for (int c = 0; c < nchunks; ++c) {
@@ -851,23 +859,71 @@ __global__ void __launch_bounds__((BN > 256) ? 384 : 256, 1) gemm_kernel(const _
             const uint32_t n = first + (uint32_t)c;
             ok = mbar_wait(cbar + 8u * (n % NB), (n / NB) & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE);
             if (!ok) break;
-            const uint32_t src = stg + (n % NB) * 4096u + row_off;
+            const uint32_t buf0 = stg + (n % NB) * 4096u;
+            const uint32_t src = buf0 + row_off;
             const int cbase = w.col0 + c * 32;
+            float f[32];
 #pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              const float4 c0 = ld_shared_f4(src + (((uint32_t)(2 * g) ^ swz) << 4));
-              const float4 c1 = ld_shared_f4(src + (((uint32_t)(2 * g + 1) ^ swz) << 4));
-              const int col = cbase + g * 8;
-              if (row < w.row_end && col < w.col_end) {
-                float f[8];
-                f[0] = __uint_as_float(v[g * 8 + 0]) + c0.x; f[1] = __uint_as_float(v[g * 8 + 1]) + c0.y;
-                f[2] = __uint_as_float(v[g * 8 + 2]) + c0.z; f[3] = __uint_as_float(v[g * 8 + 3]) + c0.w;
-                f[4] = __uint_as_float(v[g * 8 + 4]) + c1.x; f[5] = __uint_as_float(v[g * 8 + 5]) + c1.y;
-                f[6] = __uint_as_float(v[g * 8 + 6]) + c1.z; f[7] = __uint_as_float(v[g * 8 + 7]) + c1.w;
-                epilogue8(p.epi, row, col, f, 0, 0);
+            for (int g = 0; g < 8; ++g) {
+              const float4 cv = ld_shared_f4(src + (((uint32_t)g ^ swz) << 4));
+              f[4 * g + 0] = __uint_as_float(v[4 * g + 0]) + cv.x;
+              f[4 * g + 1] = __uint_as_float(v[4 * g + 1]) + cv.y;
+              f[4 * g + 2] = __uint_as_float(v[4 * g + 2]) + cv.z;
+              f[4 * g + 3] = __uint_as_float(v[4 * g + 3]) + cv.w;
+            }
+            if (!staged_out) {
+#pragma unroll
+              for (int g = 0; g < 4; ++g) {
+                const int col = cbase + g * 8;
+                if (row < w.row_end && col < w.col_end) {
+                  float e8[8];
+#pragma unroll
+                  for (int j = 0; j < 8; ++j) e8[j] = f[g * 8 + j];
+                  epilogue8(p.epi, row, col, e8, 0, 0);
+                }
+              }
+              __syncwarp();   // the buffer may be refilled once every lane has read it
+              continue;
+            }
+            if (p.epi.bias) {
+#pragma unroll
+              for (int g = 0; g < 8; ++g) {
+                if (cbase + g * 4 < w.col_end) {
+                  const float4 b0 = *reinterpret_cast<const float4 *>(p.epi.bias + cbase + g * 4);
+                  f[4 * g + 0] += b0.x; f[4 * g + 1] += b0.y; f[4 * g + 2] += b0.z; f[4 * g + 3] += b0.w;
+                }
               }
             }
-            __syncwarp();   // the buffer may be refilled once every lane has read it
+            __syncwarp();   // every lane has read its carry row: the box may now be overwritten
+            if (p.epi.z_save) {
+#pragma unroll
+              for (int g = 0; g < 4; ++g) {
+                float e8[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) e8[j] = f[g * 8 + j];
+                const uint4 pk = pack_bf16x8(e8);
+                st_shared_v4(buf0 + 2048u + (uint32_t)lane * 64u + (uint32_t)g * 16u, pk.x, pk.y, pk.z, pk.w);
+              }
+            }
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              float e8[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) e8[j] = f[g * 8 + j];
+              if (p.epi.act != ACT_NONE) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) e8[j] = gelu_f(e8[j], p.epi.act);
+              }
+              const uint4 pk = pack_bf16x8(e8);
+              st_shared_v4(buf0 + (uint32_t)lane * 64u + (uint32_t)g * 16u, pk.x, pk.y, pk.z, pk.w);
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_3d(&p.out32_map, buf0, w.b_col + c * 32, r_in, 0);
+              if (p.epi.z_save) tma_store_3d(&p.z32_map, buf0 + 2048u, w.b_col + c * 32, r_in, 0);
+              bulk_commit();
+            }
           }
           if (!ok) break;
         } else if (p.epi.out_fp32) {
