@@ -1,5 +1,9 @@
 """Slice loop of a sharded (zero-redundancy data parallel) split linear layer, one process per GPU.
 
+Section 3.3, last paragraph, is covered too: a slice may instead be kept in DP mode (replicated
+weights, gradient all-reduced), so that one operator runs partly replicated and partly sharded, as
+an execution plan from ``osdp_plan_search`` over the operator's slices prescribes.
+
 Section 3.3, last part: every rank keeps 1/world of each weight slice; slice s is all-gathered
 into a slice-sized staging buffer while slice s-1 computes, and the slice's weight gradient is
 reduce-scattered as soon as it exists, so the gathered weights (and gradients) live at
@@ -86,22 +90,27 @@ class DistComm:
         dist.reduce_scatter_tensor(shard_buf[off:off + n], src[:n * self.world], op=dist.ReduceOp.SUM,
                                    group=self.group)
 
-    def all_reduce(self, t):
+    def all_reduce(self, t, tag=None):
         import torch.distributed as dist
         dist.all_reduce(t, op=dist.ReduceOp.SUM, group=self.group)
 
 
-class ZdpSplitLinear:
-    """Y = act(X W^T + b) with W sharded over the ranks slice by slice; forward and backward gather one
-    slice at a time.  `comm` supplies rank, world and the two slice collectives (DistComm by default).
+DP, ZDP = 0, 1
 
-    param_shard : bf16 [layout.shard_total]   this rank's part of W (slice-major)
-    grad_shard  : dw_dtype, same length       this rank's part of sum over ranks of dW
+
+class ZdpSplitLinear:
+    """Y = act(X W^T + b) with W cut into k slices, each slice either sharded over the ranks (ZDP: gathered
+    for use, gradient reduce-scattered) or replicated (DP: resident, gradient all-reduced).  `comm` supplies
+    rank, world and the collectives (DistComm by default); `slice_modes` one mode per slice (default all ZDP).
+
+    param_shard : bf16   this rank's parts of the ZDP slices, one after another
+    grad_shard  : dw_dtype, same length: this rank's parts of sum over ranks of dW (ZDP slices)
+    dp_weight[s], dp_grad[s] : the compact matrices of DP slice s (whole, on every rank)
     Tokens are sharded by the caller: every rank passes its own X / dY rows.
     """
 
     def __init__(self, N, K, k_split, split_dim, act=B.ACT_NONE, dw_dtype=B.DTYPE_FP32, comm=None, device="cuda",
-                 flags=0):
+                 flags=0, slice_modes=None):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("ZdpSplitLinear needs a CUDA device: there is no CPU path")
@@ -110,14 +119,29 @@ class ZdpSplitLinear:
         self.flags = int(flags)
         self.layout = ShardLayout(N, K, k_split, split_dim, self.comm.world)
         self.k = self.layout.k
+        self.modes = [ZDP] * self.k if slice_modes is None else [int(m) for m in slice_modes]
+        if len(self.modes) != self.k or any(m not in (DP, ZDP) for m in self.modes):
+            raise ValueError("slice_modes needs one mode (0 = DP, 1 = ZDP) per slice")
         self.device = torch.device(device)
         gdt = torch.float32 if dw_dtype == B.DTYPE_FP32 else torch.bfloat16
-        self.param_shard = torch.zeros(self.layout.shard_total, dtype=torch.bfloat16, device=self.device)
-        self.grad_shard = torch.zeros(self.layout.shard_total, dtype=gdt, device=self.device)
-        # Two staging buffers each for gathered weights and for weight gradients: slice s+1 is gathered
-        # while slice s computes.  Their tails beyond a slice's elements are never written by the kernels.
-        self.w_stage = [torch.zeros(self.layout.stage_elems, dtype=torch.bfloat16, device=self.device) for _ in range(min(2, self.k))]
-        self.dw_stage = [torch.zeros(self.layout.stage_elems, dtype=gdt, device=self.device) for _ in range(min(2, self.k))]
+        self.zdp_slices = [s for s in range(self.k) if self.modes[s] == ZDP]
+        self._zord = {s: i for i, s in enumerate(self.zdp_slices)}
+        self._zoff, total = {}, 0                      # where slice s's part starts in this rank's shard buffers
+        for s in self.zdp_slices:
+            self._zoff[s] = total
+            total += self.layout.slices[s][3]
+        self.param_shard = torch.zeros(max(total, 8), dtype=torch.bfloat16, device=self.device)
+        self.grad_shard = torch.zeros(max(total, 8), dtype=gdt, device=self.device)
+        self.dp_weight = {s: torch.zeros(self.layout.slices[s][2], dtype=torch.bfloat16, device=self.device)
+                          for s in range(self.k) if self.modes[s] == DP}
+        self.dp_grad = {s: torch.zeros(self.layout.slices[s][2], dtype=gdt, device=self.device) for s in self.dp_weight}
+        # Two staging buffers each for gathered weights and for weight gradients: the next slice is gathered
+        # while this one computes.  Their tails beyond a slice's elements are never written by the kernels.
+        wst = max([self.layout.slices[s][3] for s in self.zdp_slices] + [0]) * self.comm.world
+        self.w_stage = [torch.zeros(wst, dtype=torch.bfloat16, device=self.device)
+                        for _ in range(min(2, len(self.zdp_slices)))]
+        self.dw_stage = [torch.zeros(self.layout.stage_elems, dtype=gdt, device=self.device)
+                         for _ in range(min(2, self.k))]
         self.comm_stream = torch.cuda.Stream(device=self.device)
         self.side_stream = torch.cuda.Stream(device=self.device)
         self._ws = None
@@ -125,18 +149,45 @@ class ZdpSplitLinear:
 
     # -- bookkeeping ------------------------------------------------------------------------------
     def load_full_weight(self, w_full):
-        """Keeps this rank's shards of a full [N, K] bf16 weight (initialisation / checkpoint load)."""
-        self.param_shard.copy_(self.layout.shard_of(w_full.to(self.device), self.comm.rank))
+        """Keeps this rank's part of a full [N, K] bf16 weight (initialisation / checkpoint load): the rank's
+        shard of every ZDP slice, the whole of every DP slice."""
+        w_full = w_full.to(self.device)
+        shard = self.layout.shard_of(w_full, self.comm.rank)
+        for s in self.zdp_slices:
+            _, _, _, n, off, _ = self.layout.slices[s]
+            self.param_shard[self._zoff[s]:self._zoff[s] + n].copy_(shard[off:off + n])
+        for s, t in self.dp_weight.items():
+            t.copy_(self.layout.slice_matrix(w_full, s).contiguous().reshape(-1))
+
+    def full_from_parts(self, shard_bufs, dp_parts):
+        """A full [N, K] tensor from all ranks' shard buffers (laid out like param_shard / grad_shard) and the
+        DP slices' compact tensors (checkpoint save; copies only)."""
+        import torch
+        ref = shard_bufs[0] if shard_bufs else next(iter(dp_parts.values()))
+        full = torch.empty(self.N, self.K, dtype=ref.dtype, device=ref.device)
+        for s, (b, e, elems, n, _, ld) in enumerate(self.layout.slices):
+            if self.modes[s] == ZDP:
+                o = self._zoff[s]
+                flat = torch.cat([sh[o:o + n] for sh in shard_bufs])[:elems]
+            else:
+                flat = dp_parts[s][:elems]
+            self.layout.slice_matrix(full, s).copy_(flat.reshape(-1, ld))
+        return full
 
     def staging_bytes(self, M):
-        """Bytes this layer holds besides its shards: weight and gradient staging plus the kernels' workspace."""
+        """Bytes this layer holds besides its weights and gradients: staging plus the kernels' workspace."""
         _, f = B.osdp_split_linear_workspace_bytes(M, self.N, self.K, self.k, self.split_dim, self.act,
                                                    B.OP_LINEAR_FWD, self.flags & B.FLAG_CARRY_BF16)
         _, b = B.osdp_split_linear_workspace_bytes(M, self.N, self.K, self.k, self.split_dim, self.act,
                                                    B.OP_LINEAR_BWD, self.flags & B.FLAG_CARRY_BF16)
-        stage = sum(t.numel() * t.element_size() for t in self.w_stage + self.dw_stage)
-        wbytes = len(self.w_stage) * self.w_stage[0].numel() * 2
-        return {"weight_staging": wbytes, "grad_staging": stage - wbytes, "workspace": max(f, b)}
+        nbytes = lambda ts: sum(t.numel() * t.element_size() for t in ts)
+        return {"weight_staging": nbytes(self.w_stage), "grad_staging": nbytes(self.dw_stage), "workspace": max(f, b)}
+
+    def state_bytes(self):
+        """Bytes of weights and gradients resident on this rank (shards of ZDP slices, whole DP slices)."""
+        nbytes = lambda ts: sum(t.numel() * t.element_size() for t in ts)
+        return {"weights": nbytes([self.param_shard] + list(self.dp_weight.values())),
+                "grads": nbytes([self.grad_shard] + list(self.dp_grad.values()))}
 
     def _workspace(self, M):
         nbytes = self.staging_bytes(M)["workspace"]
@@ -150,24 +201,45 @@ class ZdpSplitLinear:
     # one another, so consecutive ones are launched on two alternating streams: the next slice's CTAs
     # take over the SMs that the current slice's last, partly filled wave leaves idle.  Slices of a summed
     # output (forward under RED, dX under OUT) stay in order on the caller's stream.
-    def _gather(self, s, free_events):
-        """Issues the all-gather of slice s into its staging buffer on the communication stream."""
-        import torch
-        _, _, _, shard, off, _ = self.layout.slices[s]
-        with torch.cuda.stream(self.comm_stream):
-            for ev in free_events:
-                self.comm_stream.wait_event(ev)             # the slice that last read this buffer is done
-            self.comm.all_gather_slice(self.w_stage[s & 1], self.param_shard, off, shard)
-            ready = torch.cuda.Event()
-            ready.record(self.comm_stream)
-        return ready
-
     @staticmethod
     def _mark(stream):
         import torch
         ev = torch.cuda.Event()
         ev.record(stream)
         return ev
+
+    class _Gathers:
+        """Issues the all-gathers of the ZDP slices in order, one slice ahead of the slice in use."""
+
+        def __init__(self, layer):
+            self.layer, self.issued, self.ready = layer, 0, {}
+            self.free = [[], []]            # events after which weight staging buffer b may be overwritten
+
+        def ensure(self, upto):
+            import torch
+            L = self.layer
+            while self.issued <= upto and self.issued < len(L.zdp_slices):
+                s = L.zdp_slices[self.issued]
+                b = self.issued & 1
+                n = L.layout.slices[s][3]
+                with torch.cuda.stream(L.comm_stream):
+                    for ev in self.free[b]:
+                        L.comm_stream.wait_event(ev)        # the slice that last read this buffer is done
+                    L.comm.all_gather_slice(L.w_stage[b], L.param_shard, L._zoff[s], n)
+                    self.ready[s] = L._mark(L.comm_stream)
+                self.issued += 1
+
+        def weights(self, s, streams):
+            """The compact weight matrix of slice s, valid on `streams` (gathered one slice ahead for ZDP)."""
+            L = self.layer
+            if L.modes[s] == DP:
+                return L.dp_weight[s], None
+            i = L._zord[s]
+            self.ensure(i)
+            for st in streams:
+                st.wait_event(self.ready[s])
+            self.ensure(i + 1)                              # buffer (i + 1) & 1 was last read by ordinal i - 1
+            return L.w_stage[i & 1], i & 1
 
     def forward(self, x, bias=None, out=None, z_save=None):
         import torch
@@ -176,31 +248,31 @@ class ZdpSplitLinear:
         if out is None:
             out = torch.empty(M, self.N, dtype=torch.bfloat16, device=self.device)
         ws = self._workspace(M)
-        self.comm_stream.wait_stream(cur)                   # shards may just have been updated on `cur`
+        self.comm_stream.wait_stream(cur)                   # weights may just have been updated on `cur`
         two = self.k > 1 and self.split_dim == B.SPLIT_OUT
         lanes = [cur, self.side_stream] if two else [cur, cur]
         if two:
             self.side_stream.wait_stream(cur)
-        done = [[], []]
-        ready = self._gather(0, [])
+        g = self._Gathers(self)
+        g.ensure(0)
         for s in range(self.k):
-            nxt = self._gather(s + 1, done[(s + 1) & 1]) if s + 1 < self.k else None
             st = lanes[s & 1]
-            st.wait_event(ready)
-            B.osdp_zdp_linear_fwd_slice(x, self.w_stage[s & 1], self.layout.slices[s][5], bias, M, self.N, self.K,
-                                        self.k, self.split_dim, self.act, s, out, z_save, ws, stream=st, check=True,
+            w, b = g.weights(s, [st])
+            B.osdp_zdp_linear_fwd_slice(x, w, self.layout.slices[s][5], bias, M, self.N, self.K, self.k,
+                                        self.split_dim, self.act, s, out, z_save, ws, stream=st, check=True,
                                         flags=self.flags & B.FLAG_CARRY_BF16)
-            done[s & 1] = [self._mark(st)]
-            ready = nxt
+            if b is not None:
+                g.free[b] = [self._mark(st)]
         if two:
             cur.wait_stream(self.side_stream)
         self.comm_stream.wait_stream(cur)
         return out
 
     def backward(self, dy, x, z_saved=None, dx=None, dbias=None, need_dx=True, accumulate=False):
-        """Gathers W_s again (the second all-gather of ZDP), computes the slice's dX part, dW_s and db, and
-        reduce-scatters dW_s into grad_shard (sum over ranks; `accumulate` adds to what is there).
-        dbias (if given) is this rank's column sum; reduce it with comm.all_reduce where needed."""
+        """Per slice: W_s (gathered again for ZDP slices: the second all-gather of ZDP), the slice's dX part,
+        dW_s and db; then dW_s is reduce-scattered into grad_shard (ZDP) or all-reduced into dp_grad[s] (DP),
+        summed over ranks; `accumulate` adds to what is there.  dbias (if given) is this rank's column sum;
+        reduce it with comm.all_reduce where needed."""
         import torch
         M = x.shape[0]
         cur, side = torch.cuda.current_stream(self.device), self.side_stream
@@ -215,45 +287,59 @@ class ZdpSplitLinear:
         split_calls = self.k > 1 and out_split and self.act == B.ACT_NONE and need_dx
         alternate = self.k > 1 and not out_split
         flags = self.flags & B.FLAG_CARRY_BF16
-        w_free = [[], []]
+        g = self._Gathers(self)
+        g.ensure(0)
         dw_free = [None, None]
-        tmp = torch.empty_like(self.dw_stage[0][:max(sl[3] for sl in self.layout.slices)]) if accumulate else None
-        ready = self._gather(0, [])
+        first_done = None
         for s in range(self.k):
-            b = s & 1
-            nxt = self._gather(s + 1, w_free[(s + 1) & 1]) if s + 1 < self.k else None
-            _, _, _, shard, off, ld = self.layout.slices[s]
-            args = (dy, x, self.w_stage[b], ld, z_saved, M, self.N, self.K, self.k, self.split_dim, self.act, s)
+            _, _, elems, shard, _, ld = self.layout.slices[s]
+            zdp = self.modes[s] == ZDP
+            j = s & 1                                       # gradient staging buffer of this slice
+            direct = not zdp and not accumulate             # DP: the kernel writes dp_grad[s] itself
+            dw_dst = self.dp_grad[s] if direct else self.dw_stage[j]
             if split_calls:
-                cur.wait_event(ready)
+                w, b = g.weights(s, [cur, side])
+                args = (dy, x, w, ld, z_saved, M, self.N, self.K, self.k, self.split_dim, self.act, s)
                 B.osdp_zdp_linear_bwd_slice(*args, dx, None, 0, self.dw_dtype, flags, None, ws, stream=cur, check=True)
-                side.wait_event(ready)
-                if dw_free[b] is not None:
-                    side.wait_event(dw_free[b])             # the reduce-scatter that read this buffer is done
-                B.osdp_zdp_linear_bwd_slice(*args, None, self.dw_stage[b], ld, self.dw_dtype, 0, dbias, ws,
-                                            stream=side, check=True)
-                w_free[b] = [self._mark(cur), self._mark(side)]
-                dw_done = w_free[b][1]
+                if not direct and dw_free[j] is not None:
+                    side.wait_event(dw_free[j])             # the collective that read this buffer is done
+                B.osdp_zdp_linear_bwd_slice(*args, None, dw_dst, ld, self.dw_dtype, 0, dbias, ws, stream=side,
+                                            check=True)
+                done = [self._mark(cur), self._mark(side)]
+                dw_done = done[1]
             else:
-                st = (cur, side)[b] if alternate else cur
+                st = (cur, side)[s & 1] if alternate else cur
                 if alternate and s == 1 and self.act != B.ACT_NONE:
-                    st.wait_event(w_free[0][0])             # slice 0 stages G for every later slice
-                st.wait_event(ready)
-                if dw_free[b] is not None:
-                    st.wait_event(dw_free[b])
-                B.osdp_zdp_linear_bwd_slice(*args, dx if need_dx else None, self.dw_stage[b], ld, self.dw_dtype,
-                                            flags, dbias, ws, stream=st, check=True)
-                w_free[b] = [self._mark(st)]
-                dw_done = w_free[b][0]
+                    st.wait_event(first_done)               # slice 0 stages G for every later slice
+                w, b = g.weights(s, [st])
+                if not direct and dw_free[j] is not None:
+                    st.wait_event(dw_free[j])
+                B.osdp_zdp_linear_bwd_slice(dy, x, w, ld, z_saved, M, self.N, self.K, self.k, self.split_dim,
+                                            self.act, s, dx if need_dx else None, dw_dst, ld, self.dw_dtype, flags,
+                                            dbias, ws, stream=st, check=True)
+                done = [self._mark(st)]
+                dw_done = done[0]
+            if s == 0:
+                first_done = done[0]
+            if b is not None:
+                g.free[b] = done
             with torch.cuda.stream(self.comm_stream):
                 self.comm_stream.wait_event(dw_done)
-                if accumulate:
-                    self.comm.reduce_scatter_slice(tmp, 0, shard, self.dw_stage[b])
-                    self.grad_shard[off:off + shard].add_(tmp[:shard])
+                if zdp:
+                    o = self._zoff[s]
+                    if accumulate:
+                        tmp = torch.empty_like(self.dw_stage[j][:shard])
+                        self.comm.reduce_scatter_slice(tmp, 0, shard, self.dw_stage[j])
+                        self.grad_shard[o:o + shard].add_(tmp)
+                    else:
+                        self.comm.reduce_scatter_slice(self.grad_shard, o, shard, self.dw_stage[j])
+                elif direct:
+                    self.comm.all_reduce(self.dp_grad[s], tag=s)
                 else:
-                    self.comm.reduce_scatter_slice(self.grad_shard, off, shard, self.dw_stage[b])
-                dw_free[b] = self._mark(self.comm_stream)
-            ready = nxt
+                    self.comm.all_reduce(self.dw_stage[j][:elems], tag=s)
+                    self.dp_grad[s].add_(self.dw_stage[j][:elems])
+                if not direct:
+                    dw_free[j] = self._mark(self.comm_stream)
         cur.wait_stream(side)
-        cur.wait_stream(self.comm_stream)                   # grad_shard is complete for whoever runs next on `cur`
+        cur.wait_stream(self.comm_stream)                   # gradients are complete for whoever runs next on `cur`
         return dx

@@ -109,53 +109,49 @@ def test_gathered_slice_argument_errors(P):
 
 
 class EmulatedComm:
-    """The loop's two collectives for `world` ranks that run one after another in this process:
-    all ranks' parameter shards are visible, and reduce-scatter adds the caller's contribution to
-    per-rank accumulators (the sum over ranks is complete once every rank has run)."""
+    """The loop's collectives for `world` ranks that run one after another in this process: all ranks'
+    parameter shards are visible, and reduce-scatter / all-reduce add the caller's contribution to shared
+    fp64 accumulators (the sum over ranks is complete once every rank has run)."""
 
-    def __init__(self, rank, world, param_shards, grad_acc):
-        self.rank, self.world = rank, world
-        self.param_shards, self.grad_acc = param_shards, grad_acc
+    def __init__(self, rank, world, shared):
+        self.rank, self.world, self.shared = rank, world, shared
 
     def all_gather_slice(self, dst, shard_buf, off, n):
-        assert shard_buf.data_ptr() == self.param_shards[self.rank].data_ptr()
+        assert shard_buf.data_ptr() == self.shared["param"][self.rank].data_ptr()
         for q in range(self.world):
-            dst[q * n:(q + 1) * n].copy_(self.param_shards[q][off:off + n])
+            dst[q * n:(q + 1) * n].copy_(self.shared["param"][q][off:off + n])
 
     def reduce_scatter_slice(self, shard_buf, off, n, src):
         for q in range(self.world):
-            self.grad_acc[q][off:off + n] += src[q * n:(q + 1) * n].double()
+            self.shared["grad_acc"][q][off:off + n] += src[q * n:(q + 1) * n].double()
         shard_buf[off:off + n].copy_(src[self.rank * n:(self.rank + 1) * n])   # this rank's own term only
 
-    def all_reduce(self, t):
-        raise NotImplementedError
+    def all_reduce(self, t, tag=None):
+        acc = self.shared["dp_acc"]
+        acc[tag] = t.double().clone() if tag not in acc else acc[tag] + t.double()
 
 
-@pytest.mark.parametrize("world", [1, 2, 3])
-@pytest.mark.parametrize("split", [0, 1])
-@pytest.mark.parametrize("case", [(384, 520, 264, 3, 1), (512, 2048, 512, 4, 0), (300, 1024, 1024, 8, 1)])
-def test_slice_loop_over_emulated_ranks_matches_oracle(P, world, split, case):
-    from paper_2209_13258_b200.zdp import ShardLayout, ZdpSplitLinear
-    M, N, K, k, act = case
-    D = N if split == 0 else K
-    if P.osdp_slice_range(D, k, 0)[0] != 0:
-        pytest.skip("invalid split")
+def run_emulated_ranks(P, world, M, N, K, k, split, act, modes):
+    """Forward + backward of the slice loop for every emulated rank on its own token rows; returns the
+    assembled Y, dX, sum over ranks of dW and db, and the first rank's layer."""
+    from paper_2209_13258_b200.zdp import ZdpSplitLinear
     c = inputs.linear_case(M, N, K, w_std=0.05, bias_std=0.2)
     W = to_dev(c["w_flat"])[c["w_offset"]:c["w_offset"] + N * K].view(N, K)
     bias = to_dev(c["bias"])
-    lay = ShardLayout(N, K, k, split, world)
-    param_shards = [lay.shard_of(W, r) for r in range(world)]
-    grad_acc = [torch.zeros(lay.shard_total, dtype=torch.float64, device="cuda") for _ in range(world)]
+    shared = {"param": [None] * world, "grad_acc": [None] * world, "dp_acc": {}}
+    layers = []
+    for r in range(world):
+        layer = ZdpSplitLinear(N, K, k, split, act=act, comm=EmulatedComm(r, world, shared), slice_modes=modes)
+        layer.load_full_weight(W)
+        shared["param"][r] = layer.param_shard
+        shared["grad_acc"][r] = torch.zeros(layer.grad_shard.numel(), dtype=torch.float64, device="cuda")
+        layers.append(layer)
     y = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
     dx = torch.empty(M, K, dtype=torch.bfloat16, device="cuda")
     db = torch.zeros(N, dtype=torch.float64, device="cuda")
     x_all, dy_all = to_dev(c["x"]), to_dev(c["dy"])
-    stage_bytes = None
-    for r in range(world):
+    for r, layer in enumerate(layers):
         rows = torch.arange(r, M, world, device="cuda")               # this rank's tokens
-        comm = EmulatedComm(r, world, param_shards, grad_acc)
-        layer = ZdpSplitLinear(N, K, k, split, act=act, comm=comm)
-        layer.param_shard = param_shards[r]                            # the rank's own shard buffer
         xr, dyr = x_all[rows].contiguous(), dy_all[rows].contiguous()
         zr = torch.empty(rows.numel(), N, dtype=torch.bfloat16, device="cuda") if act else None
         yr = layer.forward(xr, bias=bias, z_save=zr)
@@ -166,17 +162,57 @@ def test_slice_loop_over_emulated_ranks_matches_oracle(P, world, split, case):
         assert rc == 0 and st == 0
         y[rows], dx[rows] = yr, dxr
         db += dbr.double()
-        stage_bytes = layer.staging_bytes(rows.numel())
-        # the gathered weights never take more than two slices' worth
-        assert stage_bytes["weight_staging"] == 2 * 2 * world * max(sl[3] for sl in lay.slices)
-        assert stage_bytes["weight_staging"] <= 2 * 2 * (N * K // k + 8 * world + max(N, K) * 8)
-    dW = lay.unshard(grad_acc)
+    dW = layers[0].full_from_parts(shared["grad_acc"], shared["dp_acc"])
+    return c, y, dx, dW, db, layers[0]
+
+
+def check_against_oracle(c, y, dx, dW, db, act, k, split):
     z, yo = oracle.linear_fwd(c["x"], c["w"], c["bias"], act, k, split)
     dXo, dWo, dbo = oracle.linear_bwd(c["dy"], c["x"], c["w"], z, act, k, split)
     assert_close(to_f64(y), yo, "Y")
     assert_close(to_f64(dx), dXo, "dX")
     assert_close(dW.cpu().numpy(), dWo, "dW (sum over ranks)")
     assert_close(db.cpu().numpy(), dbo, "db (sum over ranks)")
+
+
+@pytest.mark.parametrize("world", [1, 2, 3])
+@pytest.mark.parametrize("split", [0, 1])
+@pytest.mark.parametrize("case", [(384, 520, 264, 3, 1), (512, 2048, 512, 4, 0), (300, 1024, 1024, 8, 1)])
+def test_slice_loop_over_emulated_ranks_matches_oracle(P, world, split, case):
+    M, N, K, k, act = case
+    D = N if split == 0 else K
+    if P.osdp_slice_range(D, k, 0)[0] != 0:
+        pytest.skip("invalid split")
+    c, y, dx, dW, db, layer = run_emulated_ranks(P, world, M, N, K, k, split, act, None)
+    check_against_oracle(c, y, dx, dW, db, act, k, split)
+    # the gathered weights never take more than two slices' worth
+    st = layer.staging_bytes(M)
+    assert st["weight_staging"] == 2 * 2 * world * max(sl[3] for sl in layer.layout.slices)
+    assert st["weight_staging"] <= 2 * 2 * (N * K // k + 8 * world + max(N, K) * 8)
+    assert layer.state_bytes()["weights"] == 2 * layer.layout.shard_total
+
+
+MIXED = [((512, 2048, 512, 4, 0), [0, 1, 1, 0]), ((512, 2048, 512, 4, 0), [1, 0, 0, 0]),
+         ((384, 520, 264, 3, 1), [0, 0, 1]), ((300, 1024, 1024, 8, 1), [1, 0, 1, 1, 0, 0, 1, 0]),
+         ((256, 512, 512, 2, 0), [0, 0])]
+
+
+@pytest.mark.parametrize("world", [2, 3])
+@pytest.mark.parametrize("split", [0, 1])
+@pytest.mark.parametrize("case,modes", MIXED)
+def test_slices_in_mixed_dp_and_zdp_modes_match_oracle(P, world, split, case, modes):
+    """Section 3.3, last paragraph: some slices of one operator replicated (DP), the others sharded (ZDP)."""
+    M, N, K, k, act = case
+    D = N if split == 0 else K
+    if P.osdp_slice_range(D, k, 0)[0] != 0:
+        pytest.skip("invalid split")
+    c, y, dx, dW, db, layer = run_emulated_ranks(P, world, M, N, K, k, split, act, modes)
+    check_against_oracle(c, y, dx, dW, db, act, k, split)
+    # resident weights: whole DP slices plus 1/world of the ZDP slices (up to the 8-element padding)
+    dp_elems = sum(layer.layout.slices[s][2] for s in range(k) if modes[s] == 0)
+    zdp_shard = sum(layer.layout.slices[s][3] for s in range(k) if modes[s] == 1)
+    assert layer.state_bytes()["weights"] == 2 * (dp_elems + max(zdp_shard, 8))
+    assert len(layer.w_stage) == min(2, modes.count(1))
 
 
 def test_slice_loop_on_a_one_rank_nccl_group(P):
@@ -189,10 +225,10 @@ def test_slice_loop_on_a_one_rank_nccl_group(P):
     M, N, K, k = 512, 1024, 512, 4
     dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29753", rank=0, world_size=1)
     try:
-        for split in (0, 1):
+        for split, modes in ((0, None), (1, None), (0, [0, 1, 1, 0]), (1, [1, 0, 0, 1])):
             c = inputs.linear_case(M, N, K, w_std=0.05, bias_std=0.2)
             W = to_dev(c["w_flat"])[c["w_offset"]:c["w_offset"] + N * K].view(N, K)
-            layer = ZdpSplitLinear(N, K, k, split, act=1)
+            layer = ZdpSplitLinear(N, K, k, split, act=1, slice_modes=modes)
             layer.load_full_weight(W)
             x, dy, bias = to_dev(c["x"]), to_dev(c["dy"]), to_dev(c["bias"])
             z = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
@@ -201,7 +237,7 @@ def test_slice_loop_on_a_one_rank_nccl_group(P):
                 y = layer.forward(x, bias=bias, z_save=z)
                 dx = layer.backward(dy, x, z_saved=z, dbias=db)
             torch.cuda.synchronize()
-            dW = layer.layout.unshard([layer.grad_shard])
+            dW = layer.full_from_parts([layer.grad_shard], layer.dp_grad)
             zo, yo = oracle.linear_fwd(c["x"], c["w"], c["bias"], 1, k, split)
             dXo, dWo, dbo = oracle.linear_bwd(c["dy"], c["x"], c["w"], zo, 1, k, split)
             assert_close(to_f64(y), yo, "Y")
@@ -211,6 +247,6 @@ def test_slice_loop_on_a_one_rank_nccl_group(P):
             # accumulate=True adds a second identical gradient
             layer.backward(dy, x, z_saved=z, dbias=db, accumulate=True)
             torch.cuda.synchronize()
-            assert_close(to_f64(layer.layout.unshard([layer.grad_shard])), 2 * dWo, "dW accumulated")
+            assert_close(to_f64(layer.full_from_parts([layer.grad_shard], layer.dp_grad)), 2 * dWo, "dW accumulated")
     finally:
         dist.destroy_process_group()
