@@ -340,6 +340,48 @@ def run_ours(args):
         for label in list(sweep):
             sweep[label]["overhead_vs_k1"] = sweep[label]["ms_per_step"] / sweep["k1"]["ms_per_step"] - 1.0
         del w2
+
+    # ---- the transformer MLP block of the small model configuration (hidden 1024, ffn 4096, 8 x 512
+    # tokens, Linear -> GeLU -> Linear split along ffn, k = 1, 2, 4, 8): forward + backward, same round-robin
+    # timing.  Secondary figures; the headline above is the split-sweep operator.
+    mlp_block = {}
+    if rank == 0 and not args.no_sweep:
+        Mm, Hh, Ff = 4096, 1024, 4096
+        xm = torch.randn(Mm, Hh, device=dev).bfloat16()
+        dym = torch.randn(Mm, Hh, device=dev).bfloat16()
+        off1, off2 = 0, Ff * Hh
+        wfm = (torch.randn(2 * Ff * Hh, device=dev) * 0.02).bfloat16()
+        b1m = torch.zeros(Ff, device=dev); b2m = torch.zeros(Hh, device=dev)
+        outm = torch.empty(Mm, Hh, device=dev, dtype=torch.bfloat16); dxm = torch.empty_like(outm)
+        z1m = torch.empty(Mm, Ff, device=dev, dtype=torch.bfloat16)
+        dwm = torch.empty(2 * Ff * Hh, device=dev, dtype=torch.bfloat16)
+        db1m = torch.empty(Ff, device=dev); db2m = torch.empty(Hh, device=dev)
+        ks = (1, 2, 4, 8)
+        wsm = {}
+        for kk in ks:
+            n1 = P.osdp_split_linear_workspace_bytes(Mm, Ff, Hh, kk, P.SPLIT_OUT, P.ACT_GELU_TANH, P.OP_MLP_FWD)[1]
+            n2 = P.osdp_split_linear_workspace_bytes(Mm, Ff, Hh, kk, P.SPLIT_OUT, P.ACT_GELU_TANH, P.OP_MLP_BWD)[1]
+            wsm[kk] = (P.new_workspace(max(n1, n2), dev), max(n1, n2))
+
+        def mlp_step(kk):
+            P.osdp_split_mlp_fwd(xm, wfm, off1, b1m, off2, b2m, Mm, Hh, Ff, kk, P.ACT_GELU_TANH, outm, z1m, wsm[kk][0],
+                                 stream=stream, check=True)
+            P.osdp_split_mlp_bwd(dym, xm, wfm, off1, off2, z1m, Mm, Hh, Ff, kk, P.ACT_GELU_TANH, dxm, dwm, off1, off2,
+                                 P.DTYPE_BF16, 0, db1m, db2m, wsm[kk][0], stream=stream, check=True)
+        tm = {kk: [] for kk in ks}
+        for rnd in range(12):
+            for kk in ks:
+                a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+                a.record(stream); mlp_step(kk); b.record(stream); torch.cuda.synchronize()
+                if rnd >= 2:
+                    tm[kk].append(a.elapsed_time(b))
+        flm = 6 * 2.0 * Mm * Hh * Ff
+        for kk in ks:
+            ms = sorted(tm[kk])[len(tm[kk]) // 2]
+            mlp_block["k%d" % kk] = {"ms_per_step": ms, "tflops": flm / ms / 1e9, "staging_bytes": wsm[kk][1]}
+        for kk in ks:
+            mlp_block["k%d" % kk]["overhead_vs_k1"] = mlp_block["k%d" % kk]["ms_per_step"] / mlp_block["k1"]["ms_per_step"] - 1.0
+        del wsm
     if world > 1:
         barrier()
 
@@ -426,7 +468,7 @@ def run_ours(args):
         "frac_of_bf16_peak": {"measured_burst_1658": value / world / pk["bf16_tflops"],
                               "measured_sustained_1378": value / world / pk["bf16_tflops_sustained"],
                               "datasheet_2250": value / world / 2250.0},
-        "sweep": sweep, "staging_bytes": ws_bytes,
+        "sweep": sweep, "mlp_block_hidden1024_ffn4096_tokens4096": mlp_block, "staging_bytes": ws_bytes,
         "roofline": roofline, "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e / e2e_steps,
