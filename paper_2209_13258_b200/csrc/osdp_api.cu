@@ -417,9 +417,31 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   p.status = c.status;
   p.carry_bf16 = (c.mode == MODE_RED && c.k_total > 1) ? c.carry_bf16 : 0;
   p.red_group = (c.mode == MODE_RED && c.pair_slices && c.s_end - c.s_begin > 1) ? 2 : 1;
-  // Outputs leave through TMA unless the epilogue has to read a second tensor element-wise.
-  p.tma_epilogue = (c.epi.gz == nullptr) ? 1 : 0;
-  if (p.tma_epilogue) {
+  // Outputs leave through TMA.  The epilogue that reads a second tensor element-wise (gz) does too
+  // (its input arrives by TMA as well) when the launch is unsliced and writes bf16, which is how the MLP
+  // backward uses it; otherwise that epilogue falls back to direct stores from registers.
+  const bool gz_tma = c.epi.gz && c.mode == MODE_NONE && !c.epi.out_fp32 && !c.epi.accumulate && !c.epi.bias &&
+                      !c.epi.z_save && c.epi.act == ACT_NONE;
+  p.tma_epilogue = (c.epi.gz == nullptr || gz_tma) ? 1 : 0;
+  if (gz_tma) {
+    const cuuint64_t dims[3] = {(cuuint64_t)c.Q, (cuuint64_t)c.P, 1};
+    const cuuint32_t box32[3] = {32, 32, 1};
+    const cuuint64_t sg[2] = {(cuuint64_t)c.epi.ld_gz * 2, (cuuint64_t)c.epi.ld_gz * 2 * (cuuint64_t)c.P};
+    rc = encode3d(&p.gz32_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, c.epi.gz, dims, sg, box32, false);
+    if (rc) return rc;
+    const cuuint32_t boxpf[3] = {(cuuint32_t)bn, 32, 1};
+    rc = encode3d(&p.gz_pf_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, c.epi.gz, dims, sg, boxpf, false);
+    if (rc) return rc;
+    const cuuint64_t so[2] = {(cuuint64_t)c.epi.ld_out * 2, (cuuint64_t)c.epi.ld_out * 2 * (cuuint64_t)c.P};
+    rc = encode3d(&p.out32_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, c.epi.out, dims, so, box32, false);
+    if (rc) return rc;
+    if (c.epi.act_out) {
+      const cuuint64_t sa[2] = {(cuuint64_t)c.epi.ld_act_out * 2, (cuuint64_t)c.epi.ld_act_out * 2 * (cuuint64_t)c.P};
+      rc = encode3d(&p.z32_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, c.epi.act_out, dims, sa, box32, false);
+      if (rc) return rc;
+    }
+  }
+  if (p.tma_epilogue && !gz_tma) {
     if (c.out_is_slice && c.k_total > 1 && (c.mode == MODE_ROWS || c.mode == MODE_COLS)) {
       // the launch covers one slice and writes it as a compact matrix of the slice's extents
       if (c.s_end - c.s_begin != 1 || c.epi.z_save) return OSDP_ERR_UNSUPPORTED;

@@ -31,40 +31,44 @@ __global__ void __launch_bounds__(256) act_backward_kernel(const __nv_bfloat16 *
   }
 }
 
-// partial[chunk, c] = sum over the chunk's rows of g[row, c0 + c]; 64 columns per block.
-// Row order inside a chunk: lane ty sums rows ty, ty+8, ...; then lanes 0..7 are added in order.
+// partial[chunk, c] = sum over the chunk's rows of g[row, c0 + c]; 64 columns per block (c0, ncols
+// multiples of 8, g 16-byte aligned).  A thread owns 8 adjacent columns (one 16-byte load per row) and
+// every 32nd row of the chunk; row order inside a chunk: row lane ty sums rows ty, ty+32, ...; then the
+// 32 row lanes are added in ascending order.  The order never depends on how the operator is split.
 __global__ void __launch_bounds__(256) colsum_partial_kernel(const __nv_bfloat16 *__restrict__ g, long long ld,
                                                              long long M, int c0, int ncols,
                                                              float *__restrict__ partial, int ld_partial) {
-  __shared__ float2 red[8][32];
+  __shared__ float red[32][64 + 1];
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  const int col = blockIdx.x * 64 + tx * 2;
+  const int tx = threadIdx.x & 7, ty = threadIdx.x >> 3;
+  const int col = blockIdx.x * 64 + tx * 8;
   const long long r0 = (long long)blockIdx.y * COLSUM_ROWS_PER_CHUNK;
   const long long r1 = min(M, r0 + COLSUM_ROWS_PER_CHUNK);
-  float2 acc = make_float2(0.f, 0.f);
+  float acc[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) acc[j] = 0.f;
   if (col < ncols) {
     const __nv_bfloat16 *src = g + c0 + col;
-#pragma unroll 8
-    for (long long r = r0 + ty; r < r1; r += 8) {
-      const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162 *>(src + r * ld);
-      const float2 f = __bfloat1622float2(v);
-      acc.x += f.x;
-      acc.y += f.y;
+#pragma unroll 4
+    for (long long r = r0 + ty; r < r1; r += 32) {
+      float f[8];
+      unpack_bf16x8(*reinterpret_cast<const uint4 *>(src + r * ld), f);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[j] += f[j];
     }
   }
-  red[ty][tx] = acc;
-  __syncthreads();
-  if (ty == 0 && col < ncols) {
-    float2 s = red[0][tx];
 #pragma unroll
-    for (int t = 1; t < 8; ++t) {
-      s.x += red[t][tx].x;
-      s.y += red[t][tx].y;
+  for (int j = 0; j < 8; ++j) red[ty][tx * 8 + j] = acc[j];
+  __syncthreads();
+  if (threadIdx.x < 64) {
+    const int c = blockIdx.x * 64 + threadIdx.x;
+    if (c < ncols) {
+      float s = red[0][threadIdx.x];
+#pragma unroll
+      for (int t = 1; t < 32; ++t) s += red[t][threadIdx.x];
+      partial[(long long)blockIdx.y * ld_partial + c] = s;
     }
-    partial[(long long)blockIdx.y * ld_partial + col] = s.x;
-    partial[(long long)blockIdx.y * ld_partial + col + 1] = s.y;
   }
 }
 

@@ -67,7 +67,10 @@ struct GemmParams {
   // Output-side maps (3-D, same slice-coordinate scheme): final output, saved pre-activation, fp32 carry.
   CUtensorMap out_main, out_tail, z_main, z_tail, carry_map;
   CUtensorMap carry_pf_map;  // same tensor as carry_map, unswizzled box of 32 rows x BN columns, for L2 prefetch
-  CUtensorMap out32_map, z32_map;   // summed output's last slice: bf16 out / z_save as unswizzled boxes of 32 x 32
+  CUtensorMap out32_map, z32_map;   // bf16 out / second bf16 output (z_save, act_out) as unswizzled boxes of 32 x 32:
+                                    // the last slice of a summed output and the epilogue that reads gz
+  CUtensorMap gz32_map;             // the element-wise second input gz, same boxes
+  CUtensorMap gz_pf_map;            // gz as boxes of 32 rows x BN columns, for L2 prefetch
   int out_sc_mul;
   int red_group;             // MODE_RED: slices whose products a tile accumulates in one pass (1, or 2 = adjacent pairs)
   int carry_bf16;            // MODE_RED: the running sum is kept in `out` itself, in bf16 (no fp32 carry buffer)
@@ -439,6 +442,27 @@ __device__ __forceinline__ float gelu_grad_f(float x, int act) {
   }
   return 1.0f;
 }
+// act'(x) and act(x) together (they share the transcendental)
+__device__ __forceinline__ void gelu_grad_and_value_f(float x, int act, float &grad, float &value) {
+  if (act == ACT_GELU_TANH) {
+    const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
+    const float t = tanhf(u);
+    const float du = 0.7978845608028654f * (1.0f + 0.134145f * x * x);
+    const float h = 0.5f * (1.0f + t);
+    grad = h + 0.5f * x * (1.0f - t * t) * du;
+    value = x * h;
+    return;
+  }
+  if (act == ACT_GELU_ERF) {
+    const float Phi = 0.5f * (1.0f + erff(x * 0.7071067811865476f));
+    const float phi = 0.3989422804014327f * __expf(-0.5f * x * x);
+    grad = Phi + x * phi;
+    value = x * Phi;
+    return;
+  }
+  grad = 1.0f;
+  value = x;
+}
 __device__ __forceinline__ void unpack_bf16x8(const uint4 &u, float (&f)[8]) {
   const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
@@ -739,6 +763,8 @@ __global__ void __launch_bounds__((BN > 256) ? 384 : 256, 1) gemm_kernel(const _
     for (int i = 0; ok && get_work<TM, BN>(p, i, bid, G, w); ++i) {
       w.a_row += (int)rank * BM;
       w.row0 += (int)rank * BM;
+      if (i == 0 && p.tma_epilogue && p.epi.gz && lane == 0)   // this CTA's first tile: while its main loop runs
+        tma_prefetch_l2_3d(&p.gz_pf_map, w.b_col, w.a_row + quarter * 32, 0);
       const int buf = i % SL::NBUF;
       const uint32_t bphase = (uint32_t)(i / SL::NBUF) & 1u;
       ok = mbar_wait(tfull_bar(buf), bphase, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE);
@@ -752,6 +778,12 @@ __global__ void __launch_bounds__((BN > 256) ? 384 : 256, 1) gemm_kernel(const _
         Work nx;
         if (get_work<TM, BN>(p, i + 1, bid, G, nx) && nx.carry_in)
           tma_prefetch_l2_3d(&p.carry_pf_map, nx.col0, nx.row0 + (int)rank * BM + quarter * 32, 0);
+      }
+      if (p.tma_epilogue && p.epi.gz && lane == 0) {
+        // likewise the next tile's rows of gz
+        Work nx;
+        if (get_work<TM, BN>(p, i + 1, bid, G, nx))
+          tma_prefetch_l2_3d(&p.gz_pf_map, nx.b_col, nx.a_row + (int)rank * BM + quarter * 32, 0);
       }
       if (!p.tma_epilogue) {
         // direct stores from registers (used when the epilogue also reads a second tensor)
@@ -922,6 +954,69 @@ __global__ void __launch_bounds__((BN > 256) ? 384 : 256, 1) gemm_kernel(const _
             if (lane == 0) {
               tma_store_3d(&p.out32_map, buf0, w.b_col + c * 32, r_in, 0);
               if (p.epi.z_save) tma_store_3d(&p.z32_map, buf0 + 2048u, w.b_col + c * 32, r_in, 0);
+              bulk_commit();
+            }
+          }
+          if (!ok) break;
+        } else if (p.epi.gz) {
+          // out = acc (.) act'(gz), act_out = act(gz): the gz box of the next 32 columns is fetched by TMA
+          // while this one is worked on; the results overwrite the consumed box (act_out in the
+          // buffer's second half) and leave as TMA stores.  Unsliced launches only.
+          const uint32_t cbar = bar_base + 8u * (2 * SL::STAGES + 5 + (warp - 4) * NB);
+          int nchunks = (w.col_end - w.col0 + 31) / 32;
+          if (nchunks > BN / 32) nchunks = BN / 32;
+          auto issue_load = [&](int c) {
+            if (lane == 0) {
+              bulk_wait_read<0>();   // the stores that last left from this buffer
+              const uint32_t b = n_cload % NB;
+              mbar_expect_tx(cbar + 8u * b, 2048u);
+              tma_load_3d(stg + b * 4096u, &p.gz32_map, cbar + 8u * b, w.b_col + c * 32, r_in, 0);
+            }
+            ++n_cload;
+          };
+          const uint32_t first = n_cload;
+          for (int c = 0; c < (int)NB - 1 && c < nchunks; ++c) issue_load(c);
+#pragma unroll 1
+          for (int c = 0; c < nchunks; ++c) {
+            if (c + (int)NB - 1 < nchunks) issue_load(c + (int)NB - 1);
+            uint32_t v[32];
+            tmem_ld_x32(taddr + (uint32_t)(c * 32), v);
+            tmem_ld_wait();
+            const uint32_t n = first + (uint32_t)c;
+            ok = mbar_wait(cbar + 8u * (n % NB), (n / NB) & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE);
+            if (!ok) break;
+            const uint32_t buf0 = stg + (n % NB) * 4096u;
+            const uint32_t mine = buf0 + (uint32_t)lane * 64u;
+            float4 zq[4];
+#pragma unroll
+            for (int g = 0; g < 4; ++g) zq[g] = ld_shared_f4(mine + (uint32_t)g * 16u);
+            __syncwarp();   // every lane has read its row of gz: the box may now be overwritten
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              float z[8], f[8];
+              uint4 zb;
+              zb.x = __float_as_uint(zq[g].x); zb.y = __float_as_uint(zq[g].y);
+              zb.z = __float_as_uint(zq[g].z); zb.w = __float_as_uint(zq[g].w);
+              unpack_bf16x8(zb, z);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                float grad, val;
+                gelu_grad_and_value_f(z[j], p.epi.gz_act, grad, val);
+                f[j] = __uint_as_float(v[g * 8 + j]) * grad;
+                z[j] = val;
+              }
+              const uint4 pk = pack_bf16x8(f);
+              st_shared_v4(mine + (uint32_t)g * 16u, pk.x, pk.y, pk.z, pk.w);
+              if (p.epi.act_out) {
+                const uint4 pa = pack_bf16x8(z);
+                st_shared_v4(mine + 2048u + (uint32_t)g * 16u, pa.x, pa.y, pa.z, pa.w);
+              }
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_3d(&p.out32_map, buf0, w.b_col + c * 32, r_in, 0);
+              if (p.epi.act_out) tma_store_3d(&p.z32_map, buf0 + 2048u, w.b_col + c * 32, r_in, 0);
               bulk_commit();
             }
           }
