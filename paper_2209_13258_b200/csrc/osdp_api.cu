@@ -286,12 +286,12 @@ int make_output_maps(void *base, bool fp32, int64_t P, int64_t Q, int64_t ld, in
 
 // One kernel variant: sets its attributes once per device, sizes the grid and launches.
 // `units` = work items of the launch (tiles, summed over slices for concatenated outputs).
-template <int BN, bool A_MN, bool B_MN, bool CTA2>
+template <int BN, bool A_MN, bool B_MN, bool CTA2, bool HEAVY = false>
 int launch_variant(const GemmParams &p, int64_t units, int sms, cudaStream_t stream) {
   static std::atomic<bool> attr_done[64];
   static std::atomic<int> max_clusters[64];
-  using SL = SmemLayout<BN, CTA2>;
-  auto kernel = gemm_kernel<BN, A_MN, B_MN, CTA2>;
+  using SL = SmemLayout<BN, CTA2, HEAVY>;
+  auto kernel = gemm_kernel<BN, A_MN, B_MN, CTA2, HEAVY>;
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return cuda_fail(e);
@@ -339,7 +339,13 @@ int launch_variant(const GemmParams &p, int64_t units, int sms, cudaStream_t str
 }
 
 template <int BN, bool CTA2>
-int launch_bn(const GemmParams &p, bool a_mn, bool b_mn, int64_t units, int sms, cudaStream_t stream) {
+int launch_bn(const GemmParams &p, bool a_mn, bool b_mn, bool heavy, int64_t units, int sms, cudaStream_t stream) {
+  if constexpr (BN == 128 || BN == 256) {
+    // eight epilogue warps for epilogues with a transcendental per element (forward with activation,
+    // activation backward): only the operand layouts those launches use
+    if (heavy && !a_mn && !b_mn) return launch_variant<BN, false, false, CTA2, true>(p, units, sms, stream);
+    if (heavy && !a_mn && b_mn) return launch_variant<BN, false, true, CTA2, true>(p, units, sms, stream);
+  }
   if (!a_mn && !b_mn) return launch_variant<BN, false, false, CTA2>(p, units, sms, stream);
   if (!a_mn && b_mn) return launch_variant<BN, false, true, CTA2>(p, units, sms, stream);
   if (a_mn && b_mn) return launch_variant<BN, true, true, CTA2>(p, units, sms, stream);
@@ -488,12 +494,13 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
 
   // Work items of this launch (one per scheduling unit and tile).
   const int64_t items = count_items(c, tm, bn);
-  if (pair && bn == 512) return launch_bn<512, true>(p, c.a.mn_major, c.b.mn_major, items, sms, stream);
-  if (pair) return launch_bn<256, true>(p, c.a.mn_major, c.b.mn_major, items, sms, stream);
+  const bool heavy = (c.epi.act != ACT_NONE || gz_tma) && c.mode != MODE_RED && p.tma_epilogue;
+  if (pair && bn == 512) return launch_bn<512, true>(p, c.a.mn_major, c.b.mn_major, false, items, sms, stream);
+  if (pair) return launch_bn<256, true>(p, c.a.mn_major, c.b.mn_major, heavy, items, sms, stream);
   switch (bn) {
-    case 256: return launch_bn<256, false>(p, c.a.mn_major, c.b.mn_major, items, sms, stream);
-    case 128: return launch_bn<128, false>(p, c.a.mn_major, c.b.mn_major, items, sms, stream);
-    default: return launch_bn<64, false>(p, c.a.mn_major, c.b.mn_major, items, sms, stream);
+    case 256: return launch_bn<256, false>(p, c.a.mn_major, c.b.mn_major, heavy, items, sms, stream);
+    case 128: return launch_bn<128, false>(p, c.a.mn_major, c.b.mn_major, heavy, items, sms, stream);
+    default: return launch_bn<64, false>(p, c.a.mn_major, c.b.mn_major, heavy, items, sms, stream);
   }
 }
 

@@ -309,7 +309,7 @@ __device__ __forceinline__ constexpr uint32_t make_idesc() {
          ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(UM >> 4) << 24);
 }
 
-template <int BN, bool CTA2>
+template <int BN, bool CTA2, bool HEAVY = false>
 struct SmemLayout {
   static constexpr int BNL = CTA2 ? BN / 2 : BN;   // B rows held by one CTA (a pair splits B between its CTAs)
   // A pair's tile is made of NG column groups of 256 (one tcgen05.mma each per k-step, sharing A);
@@ -321,14 +321,16 @@ struct SmemLayout {
   // overlaps the next tile's main loop, unless one tile already needs all 512 columns.
   static constexpr int NBUF = (BN > 256) ? 1 : 2;
   // With a single accumulator set the epilogue is exposed: eight warps drain it (two per TMEM lane
-  // quarter, half of the columns each) instead of four.
-  static constexpr int EPI_WARPS = (BN > 256) ? 8 : 4;
+  // quarter, half of the columns each) instead of four.  HEAVY: the same eight warps for epilogues
+  // with a transcendental per element (activation, activation backward), which four warps, one per
+  // scheduler, cannot finish within a short main loop.
+  static constexpr int EPI_WARPS = (BN > 256 || HEAVY) ? 8 : 4;
   static constexpr int THREADS = 128 + 32 * EPI_WARPS;
   static constexpr int A_BYTES = BM * BK * 2;
   static constexpr int B_BYTES = BNL * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   // Epilogue staging: STG_BUFS boxes of 4 KB per epilogue warp (boxes in flight to/from global memory).
-  static constexpr int STG_BUFS = (BN > 256) ? 1 : 2;
+  static constexpr int STG_BUFS = (BN > 256 || HEAVY) ? 1 : 2;
   static constexpr int STG_BYTES = EPI_WARPS * STG_BUFS * 4096;
   static constexpr int RING_BYTES = 229376 - STG_BYTES;
   static constexpr int STAGES = (RING_BYTES / STAGE_BYTES) > 8 ? 8 : (RING_BYTES / STAGE_BYTES);
@@ -546,9 +548,9 @@ __device__ __forceinline__ void epilogue8(const Epilogue &e, long long row, int 
 // of the B tile (BN/2 rows), holds the accumulator of its 128 rows in its own tensor memory and
 // runs its own epilogue.  Per CTA a stage is 32 KB instead of 48 KB (6 stages instead of 4) and
 // half as many B bytes cross from L2 to shared memory per flop.
-template <int BN, bool A_MN, bool B_MN, bool CTA2>
-__global__ void __launch_bounds__((BN > 256) ? 384 : 256, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
-  using SL = SmemLayout<BN, CTA2>;
+template <int BN, bool A_MN, bool B_MN, bool CTA2, bool HEAVY = false>
+__global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
+  using SL = SmemLayout<BN, CTA2, HEAVY>;
   constexpr int TM = CTA2 ? 2 * BM : BM;
   constexpr int BNL = SL::BNL;
   const uint32_t rank = CTA2 ? cluster_ctarank() : 0u;
@@ -965,6 +967,8 @@ __global__ void __launch_bounds__((BN > 256) ? 384 : 256, 1) gemm_kernel(const _
           const uint32_t cbar = bar_base + 8u * (2 * SL::STAGES + 5 + (warp - 4) * NB);
           int nchunks = (w.col_end - w.col0 + 31) / 32;
           if (nchunks > BN / 32) nchunks = BN / 32;
+          const int c_lo = wg * (BN / 32 / EG);                       // this warp's share of the columns
+          const int c_hi = min((wg + 1) * (BN / 32 / EG), nchunks);
           auto issue_load = [&](int c) {
             if (lane == 0) {
               bulk_wait_read<0>();   // the stores that last left from this buffer
@@ -975,14 +979,14 @@ __global__ void __launch_bounds__((BN > 256) ? 384 : 256, 1) gemm_kernel(const _
             ++n_cload;
           };
           const uint32_t first = n_cload;
-          for (int c = 0; c < (int)NB - 1 && c < nchunks; ++c) issue_load(c);
+          for (int c = c_lo; c < c_lo + (int)NB - 1 && c < c_hi; ++c) issue_load(c);
 #pragma unroll 1
-          for (int c = 0; c < nchunks; ++c) {
-            if (c + (int)NB - 1 < nchunks) issue_load(c + (int)NB - 1);
+          for (int c = c_lo; c < c_hi; ++c) {
+            if (c + (int)NB - 1 < c_hi) issue_load(c + (int)NB - 1);
             uint32_t v[32];
             tmem_ld_x32(taddr + (uint32_t)(c * 32), v);
             tmem_ld_wait();
-            const uint32_t n = first + (uint32_t)c;
+            const uint32_t n = first + (uint32_t)(c - c_lo);
             ok = mbar_wait(cbar + 8u * (n % NB), (n / NB) & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE);
             if (!ok) break;
             const uint32_t buf0 = stg + (n % NB) * 4096u;
