@@ -36,9 +36,9 @@ UNIT = "TFLOP/s"
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture of this
 # very command at full size, summarised in profiles/bench_split_sweep_k8_launch_list.md.
 NCU_TRAFFIC_BYTES = {
-    ("fwd", 8, "out"): 2904284160 + 257555968,
-    ("dx", 8, "out"): 5648119808 + 4002051584,
-    ("dw", 8, "out"): 3386828032 + 120544768,
+    ("fwd", 8, "out"): 2711566336 + 255925504,
+    ("dx", 8, "out"): 5495490304 + 4003963648,
+    ("dw", 8, "out"): 2611305472 + 118412032,
 }
 
 
