@@ -71,13 +71,23 @@ def f32_to_bf16(x) -> np.ndarray:
     return out
 
 
+def e4m3_to_f64(bits) -> np.ndarray:
+    """Exact widening of fp8 e4m3 bit patterns (uint8) to fp64, via the C helper."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint8)
+    out = np.empty(bits.shape, dtype=np.float64)
+    lib().orc_e4m3_to_f64(bits.ctypes.data_as(ctypes.c_void_p), _p(out), ctypes.c_size_t(bits.size))
+    return out
+
+
 def as_f64(a) -> np.ndarray:
-    """uint16 arrays are bf16 bit patterns; anything else is a numeric array."""
+    """uint16 arrays are bf16 bit patterns, uint8 arrays fp8 e4m3 bit patterns; anything else is numeric."""
     if a is None:
         return None
     a = np.asarray(a)
     if a.dtype == np.uint16:
         return bf16_to_f64(a)
+    if a.dtype == np.uint8:
+        return e4m3_to_f64(a)
     return np.ascontiguousarray(a, dtype=np.float64)
 
 

@@ -78,6 +78,23 @@ void orc_f32_to_bf16(const float *in, uint16_t *out, size_t n)
     }
 }
 
+/* ---------------------------------------------------------------- fp8 (e4m3) -> fp64 */
+
+/* Exact widening of the 8-bit format with 1 sign, 4 exponent (bias 7) and 3 mantissa bits, the
+ * variant without infinities: exponent 15 with mantissa 7 is NaN, every other code is finite
+ * (largest 448); exponent 0 holds the subnormals m/8 * 2^-6. */
+void orc_e4m3_to_f64(const uint8_t *in, double *out, size_t n)
+{
+    for (size_t i = 0; i < n; ++i) {
+        const int sign = in[i] >> 7, e = (in[i] >> 3) & 15, m = in[i] & 7;
+        double v;
+        if (e == 15 && m == 7) v = NAN;
+        else if (e == 0) v = ldexp((double)m / 8.0, -6);
+        else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+        out[i] = sign ? -v : v;
+    }
+}
+
 /* ---------------------------------------------------------------- GeLU */
 
 static const double kSqrt2OverPi = 0.79788456080286535587989211986876;

@@ -85,6 +85,50 @@ def normal_f32(shape, std: float, stream: int, seed: int = BASE_SEED, mean: floa
     return (mean + std * normal_f64(n, stream, seed)).astype(np.float32).reshape(shape)
 
 
+def _e4m3_table() -> np.ndarray:
+    """Values of the 127 non-negative finite e4m3 codes 0x00..0x7E, ascending (code = index)."""
+    codes = np.arange(127)
+    e, m = codes >> 3, codes & 7
+    return np.where(e == 0, m / 8.0 * 2.0 ** -6, (1.0 + m / 8.0) * 2.0 ** (e.astype(np.float64) - 7.0))
+
+
+def f32_to_e4m3_bits(x: np.ndarray) -> np.ndarray:
+    """Round fp32 values to fp8 e4m3 (nearest, ties to the even code, magnitudes above 448 saturate to 448);
+    returns the uint8 bit patterns.  Table search: the nearest of the 127 finite magnitudes."""
+    x = np.ascontiguousarray(x, dtype=np.float32).astype(np.float64)
+    tab = _e4m3_table()
+    a = np.minimum(np.abs(x), 448.0)
+    lo = np.clip(np.searchsorted(tab, a, side="right") - 1, 0, 126)
+    hi = np.minimum(lo + 1, 126)
+    dlo, dhi = a - tab[lo], tab[hi] - a
+    pick_hi = (dhi < dlo) | ((dhi == dlo) & (hi % 2 == 0) & (hi != lo))
+    code = np.where(pick_hi, hi, lo).astype(np.uint8)
+    return code | (np.signbit(x).astype(np.uint8) << np.uint8(7))
+
+
+def normal_e4m3(shape, std: float, stream: int, seed: int = BASE_SEED):
+    """fp8 e4m3 bit patterns (uint8) of std * N(0,1) / scale and the per-tensor fp32 scale = max|x| / 448, so
+    that value = scale * e4m3(bits)."""
+    n = int(np.prod(shape))
+    z = (std * normal_f64(n, stream, seed)).astype(np.float32)
+    scale = np.float32(max(float(np.max(np.abs(z))), 1e-30) / 448.0)
+    return f32_to_e4m3_bits(z / scale).reshape(shape), float(scale)
+
+
+def linear_case_e4m3(M: int, N: int, K: int, *, x_std=1.0, w_std=0.02, dy_std=1.0, bias_std=0.0,
+                     layer: int = 0, seed: int = BASE_SEED, w_offset: int = 0, flat_pad: int = 0):
+    """linear_case with fp8 e4m3 operands: x, dy, w, w_flat are uint8 bit patterns with per-tensor scales
+    sx, sdy, sw (value = scale * e4m3(bits)); bias stays fp32."""
+    x, sx = normal_e4m3((M, K), x_std, stream_id(layer, STREAM_X), seed)
+    dy, sdy = normal_e4m3((M, N), dy_std, stream_id(layer, STREAM_DY), seed)
+    w, sw = normal_e4m3((N, K), w_std, stream_id(layer, STREAM_W), seed)
+    flat, _ = normal_e4m3((w_offset + N * K + flat_pad,), 1.0, stream_id(layer, 15), seed)
+    flat[w_offset:w_offset + N * K] = w.reshape(-1)
+    bias = normal_f32((N,), bias_std, stream_id(layer, STREAM_B), seed) if bias_std > 0.0 else np.zeros((N,), np.float32)
+    return {"x": x, "dy": dy, "w": w, "w_flat": flat, "w_offset": w_offset, "bias": bias, "sx": sx, "sdy": sdy,
+            "sw": sw, "M": M, "N": N, "K": K}
+
+
 def stream_id(layer: int, which: int) -> int:
     return 16 * layer + which
 

@@ -317,3 +317,36 @@ def test_slice_table_golden_file():
         assert [oracle.slice_range(D, k, s) for s in range(k)] == want
         n += 1
     assert n == 7
+
+
+# ---------------------------------------------------------------------------------------------
+# fp8 e4m3: the oracle's widening and the input generator's rounding, each against torch's own type
+
+def test_e4m3_widening_matches_torch_on_all_codes():
+    torch = pytest.importorskip("torch")
+    codes = np.arange(256, dtype=np.uint8)
+    mine = oracle.e4m3_to_f64(codes)
+    ref = torch.from_numpy(codes.copy()).view(torch.float8_e4m3fn).double().numpy()
+    assert np.array_equal(np.isnan(mine), np.isnan(ref)) and int(np.isnan(mine).sum()) == 2
+    ok = ~np.isnan(ref)
+    assert np.array_equal(mine[ok], ref[ok])
+    # landmarks of the format: largest value, smallest normal, smallest subnormal, signed zero
+    assert mine[0x7E] == 448.0 and mine[0x08] == 2.0 ** -6 and mine[0x01] == 2.0 ** -9
+    assert mine[0x80] == 0.0 and np.signbit(mine[0x80]) and mine[0x38] == 1.0
+
+
+def test_e4m3_rounding_of_the_input_generator_matches_torch():
+    torch = pytest.importorskip("torch")
+    from paper_2209_13258_b200 import inputs
+    rng = np.random.default_rng(11)
+    x = np.concatenate([rng.normal(0, 100, 200000), rng.normal(0, 1, 200000), rng.normal(0, 0.01, 200000),
+                        oracle.e4m3_to_f64(np.arange(0x7F, dtype=np.uint8)),                       # exact values
+                        (oracle.e4m3_to_f64(np.arange(0x7E, dtype=np.uint8)) +
+                         oracle.e4m3_to_f64(np.arange(1, 0x7F, dtype=np.uint8))) / 2]).astype(np.float32)  # ties
+    x = x[np.abs(x) <= 448.0]
+    mine = inputs.f32_to_e4m3_bits(x)
+    ref = torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    # -0 and +0 both stand for zero; everything else must be the same code
+    zero = (mine & 0x7F) == 0
+    assert np.array_equal(mine[~zero], ref[~zero]) and np.all((ref[zero] & 0x7F) == 0)
+    assert inputs.f32_to_e4m3_bits(np.array([1e6, -1e6], np.float32)).tolist() == [0x7E, 0xFE]   # saturation
