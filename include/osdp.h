@@ -162,6 +162,28 @@ int osdp_split_linear_bwd_slice(const void *dy, const void *x, const void *w_fla
                                 int64_t dw_offset, int dw_dtype, int flags, float *dbias,
                                 void *ws, size_t ws_bytes, void *stream);
 
+/* ---- fp8 (e4m3) operands.  The same split linear layer with X, W and dY stored as 8-bit floating point
+ * (1 sign, 4 exponent, 3 mantissa bits, no infinities; value = scale * e4m3(byte), one fp32 scale per
+ * tensor chosen by the caller).  The tensor cores multiply the e4m3 values exactly and accumulate in fp32;
+ * `scale` (= scale_x * scale_w) multiplies the accumulator before bias / activation.  The paper's method is
+ * agnostic of the number format; this variant runs the slices on tcgen05.mma.kind::f8f6f4 at twice the
+ * bf16 rate.  x8 [M,K], w8_flat (W [N,K] at ELEMENT = byte offset w_offset), out / z_save bf16 as before.
+ * N, K, w_offset and, for k > 1, the slice length ceil(D/k) rounded up to 8 must be multiples of 16
+ * (OSDP_ERR_ALIGNMENT otherwise).  Workspace: osdp_split_linear_workspace_bytes, same figures.
+ * flags as osdp_split_linear_fwd. */
+int osdp_split_linear_fwd_f8(const void *x8, const void *w8_flat, int64_t w_offset, float scale,
+                             const float *bias, int64_t M, int64_t N, int64_t K, int k_split,
+                             int split_dim, int act, int flags, void *out, void *z_save, void *ws,
+                             size_t ws_bytes, void *stream);
+
+/* Backward with fp8 operands: dX = scale_dx * (dY8 W8) in bf16, dW = scale_dw * (dY8^T X8) in dw_dtype
+ * (scale_dx = scale_dy * scale_w, scale_dw = scale_dy * scale_x).  No activation (dY itself is the fp8
+ * operand) and no bias gradient; everything else as osdp_split_linear_bwd. */
+int osdp_split_linear_bwd_f8(const void *dy8, const void *x8, const void *w8_flat, int64_t w_offset,
+                             float scale_dx, float scale_dw, int64_t M, int64_t N, int64_t K,
+                             int k_split, int split_dim, void *dx, void *dw_flat, int64_t dw_offset,
+                             int dw_dtype, int flags, void *ws, size_t ws_bytes, void *stream);
+
 /* ---- Slices of a sharded operator (Section 3.3, last part: with zero-redundancy data parallelism
  * only the slice being processed is gathered, so the gathered weights take size(W)/k instead of
  * size(W)).  The caller (one process per GPU) keeps 1/world of every slice, all-gathers slice s

@@ -25,6 +25,7 @@ EXPORTS = [
     "osdp_read_device_status", "osdp_bias_grad_noalloc", "osdp_debug_wait_probe", "osdp_suggest_granularity",
     "osdp_zdp_shard_layout", "osdp_zdp_linear_fwd_slice", "osdp_zdp_linear_bwd_slice",
     "osdp_plan_cost", "osdp_plan_search", "osdp_plan_expand_slices",
+    "osdp_split_linear_fwd_f8", "osdp_split_linear_bwd_f8",
 ]
 
 _lib = None
@@ -81,6 +82,10 @@ def lib():
         L.osdp_plan_cost.argtypes = [pd, ci, ci, dbl, dbl, pu8, ci, pd, pd]
         L.osdp_plan_search.argtypes = [pd, ci, ci, dbl, dbl, dbl, ci, i64, pu8, ctypes.POINTER(ci), pd, p64]
         L.osdp_plan_expand_slices.argtypes = [pd, ci, dbl, pd]
+        f32 = ctypes.c_float
+        L.osdp_split_linear_fwd_f8.argtypes = [vp, vp, i64, f32, vp, i64, i64, i64, ci, ci, ci, ci, vp, vp, vp, sz, vp]
+        L.osdp_split_linear_bwd_f8.argtypes = [vp, vp, vp, i64, f32, f32, i64, i64, i64, ci, ci, vp, vp, i64, ci, ci,
+                                               vp, sz, vp]
         for name in EXPORTS:
             getattr(L, name)
             if name not in ("osdp_status_string",):
@@ -302,3 +307,22 @@ def osdp_plan_expand_slices(op, k, overhead=0.0):
     out = (ctypes.c_double * (5 * max(int(k), 1)))()
     rc = lib().osdp_plan_expand_slices((ctypes.c_double * 5)(*[float(v) for v in op]), int(k), float(overhead), out)
     return rc, [tuple(out[5 * s:5 * s + 5]) for s in range(max(int(k), 1))] if rc == 0 else []
+
+
+def osdp_split_linear_fwd_f8(x8, w8_flat, w_offset, scale, bias, M, N, K, k_split, split_dim, act, out, z_save, ws,
+                             stream=None, check=False, flags=0):
+    wp, wn = _ws(ws)
+    rc = lib().osdp_split_linear_fwd_f8(_ptr(x8), _ptr(w8_flat), int(w_offset), float(scale), _ptr(bias), int(M),
+                                        int(N), int(K), int(k_split), int(split_dim), int(act), int(flags), _ptr(out),
+                                        _ptr(z_save), wp, wn, _stream(stream))
+    return _ret(rc, check, "osdp_split_linear_fwd_f8")
+
+
+def osdp_split_linear_bwd_f8(dy8, x8, w8_flat, w_offset, scale_dx, scale_dw, M, N, K, k_split, split_dim, dx, dw_flat,
+                             dw_offset, dw_dtype, flags, ws, stream=None, check=False):
+    wp, wn = _ws(ws)
+    rc = lib().osdp_split_linear_bwd_f8(_ptr(dy8), _ptr(x8), _ptr(w8_flat), int(w_offset), float(scale_dx),
+                                        float(scale_dw), int(M), int(N), int(K), int(k_split), int(split_dim),
+                                        _ptr(dx), _ptr(dw_flat), int(dw_offset), int(dw_dtype), int(flags), wp, wn,
+                                        _stream(stream))
+    return _ret(rc, check, "osdp_split_linear_bwd_f8")

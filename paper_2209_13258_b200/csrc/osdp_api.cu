@@ -9,6 +9,7 @@
 #include <string.h>
 
 #include <atomic>
+#include <cmath>
 #include <mutex>
 
 #include "osdp_aux.cuh"
@@ -177,6 +178,7 @@ struct GemmCall {
   int carry_bf16;   // MODE_RED: running sum in `out` (bf16) instead of the fp32 carry buffer
   int pair_slices;  // MODE_RED: accumulate two adjacent slices per pass
   int out_is_slice; // MODE_ROWS / MODE_COLS: `epi.out` is the slice's own compact matrix, not the whole output
+  int fp8;          // operands are fp8 e4m3 (1 byte per element) instead of bf16
   int *status;
 };
 
@@ -254,16 +256,17 @@ int make_sliced_maps(const ViewSpec &v, CUtensorMap *main_map, CUtensorMap *tail
 }
 
 int make_operand_maps(const Operand &op, bool is_a, int mode, int64_t L, int k, int tile_rows, CUtensorMap *main_map,
-                      CUtensorMap *tail_map, int *sc_mul) {
+                      CUtensorMap *tail_map, int *sc_mul, int eb = 2) {
   ViewSpec v;
-  v.base = op.base; v.elem_bytes = 2; v.dt = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+  v.base = op.base; v.elem_bytes = eb;
+  v.dt = (eb == 1) ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
   v.inner = op.inner; v.outer = op.outer; v.ld = op.ld;
   v.mid = op.mn_major ? (mode == (is_a ? MODE_ROWS : MODE_COLS)) : (mode == MODE_RED);
   const bool role_sliced = is_a ? (mode == MODE_ROWS || mode == MODE_RED) : (mode == MODE_COLS || mode == MODE_RED);
   v.cut = role_sliced && op.whole && k > 1;
   v.L = L; v.k = k;
-  v.box_inner = 64;
-  v.box_outer = op.mn_major ? (cuuint32_t)BK : (cuuint32_t)tile_rows;
+  v.box_inner = (cuuint32_t)(128 / eb);                                   // 128 bytes of the contiguous dimension
+  v.box_outer = op.mn_major ? (cuuint32_t)(128 / eb) : (cuuint32_t)tile_rows;   // MN-major: one k-block of rows
   *sc_mul = v.cut ? 1 : 0;
   return make_sliced_maps(v, main_map, tail_map);
 }
@@ -286,12 +289,12 @@ int make_output_maps(void *base, bool fp32, int64_t P, int64_t Q, int64_t ld, in
 
 // One kernel variant: sets its attributes once per device, sizes the grid and launches.
 // `units` = work items of the launch (tiles, summed over slices for concatenated outputs).
-template <int BN, bool A_MN, bool B_MN, bool CTA2, bool HEAVY = false>
+template <int BN, bool A_MN, bool B_MN, bool CTA2, bool HEAVY = false, int EB = 2>
 int launch_variant(const GemmParams &p, int64_t units, int sms, cudaStream_t stream) {
   static std::atomic<bool> attr_done[64];
   static std::atomic<int> max_clusters[64];
   using SL = SmemLayout<BN, CTA2, HEAVY>;
-  auto kernel = gemm_kernel<BN, A_MN, B_MN, CTA2, HEAVY>;
+  auto kernel = gemm_kernel<BN, A_MN, B_MN, CTA2, HEAVY, EB>;
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return cuda_fail(e);
@@ -340,6 +343,14 @@ int launch_variant(const GemmParams &p, int64_t units, int sms, cudaStream_t str
 
 template <int BN, bool CTA2>
 int launch_bn(const GemmParams &p, bool a_mn, bool b_mn, bool heavy, int64_t units, int sms, cudaStream_t stream) {
+  if (p.bk == 128) {   // fp8 operands: tiles from 128 columns up (an MN-major chunk is 128 wide)
+    if constexpr (BN >= 128) {
+      if (!a_mn && !b_mn) return launch_variant<BN, false, false, CTA2, false, 1>(p, units, sms, stream);
+      if (!a_mn && b_mn) return launch_variant<BN, false, true, CTA2, false, 1>(p, units, sms, stream);
+      if (a_mn && b_mn) return launch_variant<BN, true, true, CTA2, false, 1>(p, units, sms, stream);
+    }
+    return OSDP_ERR_UNSUPPORTED;
+  }
   if constexpr (BN == 128 || BN == 256) {
     // eight epilogue warps for epilogues with a transcendental per element (forward with activation,
     // activation backward): only the operand layouts those launches use
@@ -394,6 +405,8 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   const int64_t want = (int64_t)sms * 4 / 5;
   if (pair || cdiv(c.bn_P, BM) * cdiv(c.bn_Q, 256) >= want) bn = 256;
   else if (cdiv(c.bn_P, BM) * cdiv(c.bn_Q, 128) >= want) bn = 128;
+  const int eb = c.fp8 ? 1 : 2;
+  if (c.fp8 && bn < 128) bn = 128;
   const int tm = pair ? 2 * BM : BM;
   // Widest tile, 256 x 512 per CTA pair: 25 % fewer operand bytes per flop (the main loop is bound by
   // its operand feed), but the accumulators fill the tensor memory, so the epilogue no longer
@@ -405,21 +418,23 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   // So does the GEMM whose epilogue reads a second tensor element-wise (direct stores, slower: better hidden).
   if (pair && c.mode != MODE_RED && c.epi.gz == nullptr) {
     const int64_t units = sms / 2;
-    const int64_t red_len = c.R;
-    const double t_n = (double)cdiv(count_items(c, 2 * BM, 256), units) * (6.5e-3 * (double)red_len) + 5.0;
-    const double t_w = (double)cdiv(count_items(c, 2 * BM, 512), units) * (11.5e-3 * (double)red_len + 5.0);
+    const double red_len = (double)c.R * (c.fp8 ? 0.5 : 1.0);   // an fp8 k-step covers twice the elements
+    const double t_n = (double)cdiv(count_items(c, 2 * BM, 256), units) * (6.5e-3 * red_len) + 5.0;
+    const double t_w = (double)cdiv(count_items(c, 2 * BM, 512), units) * (11.5e-3 * red_len + 5.0);
     if (t_w < 0.97 * t_n) bn = 512;
   }
 
   GemmParams p;
   memset(&p, 0, sizeof(p));
-  rc = make_operand_maps(c.a, true, c.mode, c.L, c.k_total, BM, &p.a_main, &p.a_tail, &p.a_sc_mul);
+  rc = make_operand_maps(c.a, true, c.mode, c.L, c.k_total, BM, &p.a_main, &p.a_tail, &p.a_sc_mul, eb);
   if (rc) return rc;
-  rc = make_operand_maps(c.b, false, c.mode, c.L, c.k_total, pair ? 128 : bn, &p.b_main, &p.b_tail, &p.b_sc_mul);
+  rc = make_operand_maps(c.b, false, c.mode, c.L, c.k_total, pair ? 128 : bn, &p.b_main, &p.b_tail, &p.b_sc_mul, eb);
   if (rc) return rc;
+  p.bk = 128 / eb;
   p.P = (int)c.P; p.Q = (int)c.Q; p.R = (int)c.R;
   p.mode = c.mode; p.L = (int)c.L; p.k_total = c.k_total; p.s_begin = c.s_begin; p.s_end = c.s_end;
   p.epi = c.epi;
+  if (p.epi.scale == 0.0f) p.epi.scale = 1.0f;   // callers that zero-fill the call leave it unset
   p.status = c.status;
   p.carry_bf16 = (c.mode == MODE_RED && c.k_total > 1) ? c.carry_bf16 : 0;
   p.red_group = (c.mode == MODE_RED && c.pair_slices && c.s_end - c.s_begin > 1) ? 2 : 1;
@@ -494,7 +509,7 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
 
   // Work items of this launch (one per scheduling unit and tile).
   const int64_t items = count_items(c, tm, bn);
-  const bool heavy = (c.epi.act != ACT_NONE || gz_tma) && c.mode != MODE_RED && p.tma_epilogue;
+  const bool heavy = (c.epi.act != ACT_NONE || gz_tma) && c.mode != MODE_RED && p.tma_epilogue && !c.fp8;
   if (pair && bn == 512) return launch_bn<512, true>(p, c.a.mn_major, c.b.mn_major, false, items, sms, stream);
   if (pair) return launch_bn<256, true>(p, c.a.mn_major, c.b.mn_major, heavy, items, sms, stream);
   switch (bn) {
@@ -589,7 +604,8 @@ int check_flags(int flags, int allowed, int act, const void *z_save) {
 // a compact matrix with that leading dimension ([slice rows, K] under OUT, [N, slice columns] under RED).
 int fwd_impl(const void *x, const void *w_flat, int64_t w_offset, const float *bias, int64_t M, int64_t N, int64_t K,
              int k, int split_dim, int act, int flags, int s_begin, int s_end, bool single, void *out, void *z_save,
-             void *ws, size_t ws_bytes, void *stream, int64_t ld_w_slice = 0) {
+             void *ws, size_t ws_bytes, void *stream, int64_t ld_w_slice = 0, int fp8 = 0, float scale = 1.0f) {
+  // fp8: x and W are e4m3 bytes (16 elements per 16 bytes: extents, offset and slice length multiples of 16)
   if (!x || !w_flat || !out) return OSDP_ERR_NULL_POINTER;
   {
     const int frc = check_flags(flags, OSDP_FLAG_CARRY_BF16 | (single ? 0 : OSDP_FLAG_PAIR_SLICES), act, z_save);
@@ -607,6 +623,8 @@ int fwd_impl(const void *x, const void *w_flat, int64_t w_offset, const float *b
     s_end = k;
   }
   if (w_offset < 0 || (w_offset & 7)) return OSDP_ERR_ALIGNMENT;
+  if (fp8 && ((N & 15) || (K & 15) || (w_offset & 15) || (k > 1 && (L & 15)) || !std::isfinite(scale) || ld_w_slice > 0))
+    return (ld_w_slice > 0 || !std::isfinite(scale)) ? OSDP_ERR_UNSUPPORTED : OSDP_ERR_ALIGNMENT;
   if (!aligned16(x) || !aligned16(w_flat) || !aligned16(out) || !aligned16(z_save) || !aligned16(bias))
     return OSDP_ERR_ALIGNMENT;
   WsPlan plan;
@@ -615,9 +633,10 @@ int fwd_impl(const void *x, const void *w_flat, int64_t w_offset, const float *b
   rc = check_ws(ws, ws_bytes, plan);
   if (rc) return rc;
 
-  const __nv_bfloat16 *w = static_cast<const __nv_bfloat16 *>(w_flat) + w_offset;
+  const void *w = static_cast<const char *>(w_flat) + w_offset * (fp8 ? 1 : 2);
   GemmCall c;
   memset(&c, 0, sizeof(c));
+  c.fp8 = fp8;
   c.a = Operand{x, K, M, K, false, true};
   c.b = Operand{w, K, N, K, false, true};
   if (ld_w_slice > 0) {
@@ -634,6 +653,7 @@ int fwd_impl(const void *x, const void *w_flat, int64_t w_offset, const float *b
   c.mode = (k == 1) ? MODE_NONE : (split_dim == OSDP_SPLIT_OUT ? MODE_COLS : MODE_RED);
   c.L = L; c.k_total = k; c.s_begin = s_begin; c.s_end = s_end;
   c.epi = plain_epilogue(out, N, 0);
+  c.epi.scale = scale;
   c.epi.bias = bias;
   c.epi.z_save = static_cast<__nv_bfloat16 *>(z_save);
   c.epi.ld_z = N;
@@ -649,7 +669,9 @@ int fwd_impl(const void *x, const void *w_flat, int64_t w_offset, const float *b
 int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset, const void *z_saved, int64_t M,
              int64_t N, int64_t K, int k, int split_dim, int act, int s_begin, int s_end, bool single, void *dx,
              void *dw_flat, int64_t dw_offset, int dw_dtype, int flags, float *dbias, void *ws, size_t ws_bytes,
-             void *stream_, int64_t ld_w_slice = 0, int64_t ld_dw_slice = 0) {
+             void *stream_, int64_t ld_w_slice = 0, int64_t ld_dw_slice = 0, int fp8 = 0, float scale_dx = 1.0f,
+             float scale_dw = 1.0f) {
+  // fp8: dy, x and W are e4m3 bytes; no activation, no bias gradient (G = dY must itself be an fp8 operand)
   // ld_w_slice > 0: W is slice `s_begin` gathered into a compact matrix (see fwd_impl);
   // ld_dw_slice > 0: dW of the slice is written as a compact matrix of the same shape.
   if (!dy || !x || !w_flat) return OSDP_ERR_NULL_POINTER;
@@ -671,6 +693,12 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
     s_end = k;
   }
   if (act != OSDP_ACT_NONE && !z_saved) return OSDP_ERR_NULL_POINTER;
+  if (fp8) {
+    if (act != OSDP_ACT_NONE || dbias || ld_w_slice > 0 || ld_dw_slice > 0 || !std::isfinite(scale_dx) ||
+        !std::isfinite(scale_dw))
+      return OSDP_ERR_UNSUPPORTED;
+    if ((N & 15) || (K & 15) || (w_offset & 15) || (k > 1 && (L & 15))) return OSDP_ERR_ALIGNMENT;
+  }
   if (dw_dtype != OSDP_DTYPE_BF16 && dw_dtype != OSDP_DTYPE_FP32) return OSDP_ERR_UNSUPPORTED;
   if (w_offset < 0 || (w_offset & 7) || dw_offset < 0 || (dw_offset & 7)) return OSDP_ERR_ALIGNMENT;
   if (!aligned16(dy) || !aligned16(x) || !aligned16(w_flat) || !aligned16(z_saved) || !aligned16(dx) ||
@@ -684,7 +712,7 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
 
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   char *wsb = static_cast<char *>(ws);
-  const __nv_bfloat16 *w = static_cast<const __nv_bfloat16 *>(w_flat) + w_offset;
+  const void *w = static_cast<const char *>(w_flat) + w_offset * (fp8 ? 1 : 2);
   float *partial = reinterpret_cast<float *>(wsb + plan.part_off);
   float *carry = reinterpret_cast<float *>(wsb + plan.carry_off);
   __nv_bfloat16 *stage = reinterpret_cast<__nv_bfloat16 *>(wsb + plan.stage0_off);
@@ -706,6 +734,7 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
   auto dx_call = [&](const Operand &g, int sb, int se) {
     GemmCall c;
     memset(&c, 0, sizeof(c));
+    c.fp8 = fp8;
     c.a = g;                                        // G [M,N], reduction N contiguous
     c.b = Operand{w, K, N, K, true, true};          // W [N,K]: output dim K contiguous
     if (ld_w_slice > 0)
@@ -714,6 +743,7 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
     c.mode = (k == 1) ? MODE_NONE : (out_split ? MODE_RED : MODE_COLS);
     c.L = L; c.k_total = k; c.s_begin = sb; c.s_end = se;
     c.epi = plain_epilogue(dx, K, 0);
+    c.epi.scale = scale_dx;
     c.epi.carry = carry;
     c.epi.ld_carry = K;
     c.carry_bf16 = (flags & OSDP_FLAG_CARRY_BF16) ? 1 : 0;
@@ -724,12 +754,14 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
   auto dw_call = [&](const Operand &gt, int sb, int se) {
     GemmCall c;
     memset(&c, 0, sizeof(c));
+    c.fp8 = fp8;
     c.a = gt;                                       // G^T: output dim N contiguous in G
     c.b = Operand{x, K, M, K, true, true};          // X [M,K]: output dim K contiguous
     c.P = N; c.Q = K; c.R = M; c.bn_P = N; c.bn_Q = K;
     c.mode = (k == 1) ? MODE_NONE : (out_split ? MODE_ROWS : MODE_COLS);
     c.L = L; c.k_total = k; c.s_begin = sb; c.s_end = se;
     c.epi = plain_epilogue(dw, ld_dw_slice > 0 ? ld_dw_slice : K, dw_dtype == OSDP_DTYPE_FP32);
+    c.epi.scale = scale_dw;
     c.epi.accumulate = accumulate;
     c.out_is_slice = (ld_dw_slice > 0 && k > 1) ? 1 : 0;
     c.status = status;
@@ -878,6 +910,21 @@ int osdp_split_linear_bwd_slice(const void *dy, const void *x, const void *w_fla
                                 int flags, float *dbias, void *ws, size_t ws_bytes, void *stream) {
   return bwd_impl(dy, x, w_flat, w_offset, z_saved, M, N, K, k_split, split_dim, act, slice_idx, 0, true, dx, dw_flat,
                   dw_offset, dw_dtype, flags, dbias, ws, ws_bytes, stream);
+}
+
+int osdp_split_linear_fwd_f8(const void *x8, const void *w8_flat, int64_t w_offset, float scale, const float *bias,
+                             int64_t M, int64_t N, int64_t K, int k_split, int split_dim, int act, int flags,
+                             void *out, void *z_save, void *ws, size_t ws_bytes, void *stream) {
+  return fwd_impl(x8, w8_flat, w_offset, bias, M, N, K, k_split, split_dim, act, flags, 0, 0, false, out, z_save, ws,
+                  ws_bytes, stream, 0, 1, scale);
+}
+
+int osdp_split_linear_bwd_f8(const void *dy8, const void *x8, const void *w8_flat, int64_t w_offset, float scale_dx,
+                             float scale_dw, int64_t M, int64_t N, int64_t K, int k_split, int split_dim, void *dx,
+                             void *dw_flat, int64_t dw_offset, int dw_dtype, int flags, void *ws, size_t ws_bytes,
+                             void *stream) {
+  return bwd_impl(dy8, x8, w8_flat, w_offset, nullptr, M, N, K, k_split, split_dim, OSDP_ACT_NONE, 0, 0, false, dx,
+                  dw_flat, dw_offset, dw_dtype, flags, nullptr, ws, ws_bytes, stream, 0, 0, 1, scale_dx, scale_dw);
 }
 
 int osdp_zdp_shard_layout(int64_t N, int64_t K, int k_split, int split_dim, int world, int slice_idx,

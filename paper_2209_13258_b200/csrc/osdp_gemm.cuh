@@ -54,6 +54,7 @@ struct Epilogue {
   int gz_act;
   __nv_bfloat16 *act_out;    // [P,Q] or null: also write act(gz) here
   long long ld_act_out;
+  float scale;               // the accumulator is multiplied by this before anything else (fp8 operands' scales)
 };
 
 struct GemmParams {
@@ -75,6 +76,7 @@ struct GemmParams {
   int red_group;             // MODE_RED: slices whose products a tile accumulates in one pass (1, or 2 = adjacent pairs)
   int carry_bf16;            // MODE_RED: the running sum is kept in `out` itself, in bf16 (no fp32 carry buffer)
   int tma_epilogue;          // 1: outputs leave through shared-memory staging + TMA; 0: direct stores
+  int bk;                    // reduction elements per k-block: 128 / (bytes per operand element)
   Epilogue epi;
   int *status;               // device status word or null
 };
@@ -231,6 +233,24 @@ __device__ __forceinline__ void tc_fence_after() {
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
 template <bool CTA2>
+__device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                        uint32_t accumulate) {
+  if (CTA2)
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  else
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+template <bool CTA2>
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                           uint32_t accumulate) {
   if (CTA2)
@@ -278,6 +298,13 @@ __device__ __forceinline__ void tmem_ld_x32(uint32_t taddr, uint32_t (&v)[32]) {
 __device__ __forceinline__ void tmem_ld_wait() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+// Accumulator values times the product of the operands' scales (1 for bf16 operands: exact, skipped).
+__device__ __forceinline__ void scale_acc(uint32_t (&v)[32], float scale) {
+  if (scale != 1.0f) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * scale);
+  }
+}
 
 // ------------------------------------------------------------------------------------------------
 // Descriptors
@@ -286,9 +313,13 @@ __device__ __forceinline__ void tmem_ld_wait() {
 //  K-major tile  [rows][64 bf16]: rows are 128 B apart, groups of 8 rows 1024 B apart (SBO).
 //  MN-major tile [chunks of 64 MN][64 k-rows of 128 B]: 8 k-rows = 1024 B (SBO), MN chunks
 //  8192 B apart (LBO).
-template <bool MN_MAJOR>
+// EB = bytes per operand element (2: bf16, 1: fp8 e4m3).  A stage always holds 128 bytes of the
+// contiguous dimension per row, i.e. 128 / EB elements: 64 bf16 or 128 fp8 of the reduction for a K-major
+// tile (one k-block), 64 or 128 output rows/columns per chunk for an MN-major one; a k-block is
+// 128 / EB reduction elements, one tcgen05.mma covers 32 / EB of them (32 bytes of a K-major row).
+template <bool MN_MAJOR, int EB = 2>
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
-  constexpr uint64_t lbo = MN_MAJOR ? (uint64_t)((BK * 128) >> 4) : 1ull;
+  constexpr uint64_t lbo = MN_MAJOR ? (uint64_t)(((128 / EB) * 128) >> 4) : 1ull;
   constexpr uint64_t sbo = 1024 >> 4;
   uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
   d |= lbo << 16;
@@ -298,15 +329,16 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
   return d;
 }
 // Bytes the start address moves per UMMA_K step inside a stage.
-template <bool MN_MAJOR>
+template <bool MN_MAJOR, int EB = 2>
 __device__ __forceinline__ constexpr uint32_t desc_k_advance() {
-  return MN_MAJOR ? (UMMA_K * 128) : (UMMA_K * 2);
+  return MN_MAJOR ? ((32 / EB) * 128) : 32;
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = BN.
-template <int UM, int BN, bool A_MN, bool B_MN>
+// (operand format field: 1 = bf16 under kind::f16, 0 = e4m3 under kind::f8f6f4; accumulator fp32)
+template <int UM, int BN, bool A_MN, bool B_MN, int EB = 2>
 __device__ __forceinline__ constexpr uint32_t make_idesc() {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16) |
-         ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(UM >> 4) << 24);
+  return (1u << 4) | ((EB == 2 ? 1u : 0u) << 7) | ((EB == 2 ? 1u : 0u) << 10) | ((A_MN ? 1u : 0u) << 15) |
+         ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(UM >> 4) << 24);
 }
 
 template <int BN, bool CTA2, bool HEAVY = false>
@@ -326,8 +358,8 @@ struct SmemLayout {
   // scheduler, cannot finish within a short main loop.
   static constexpr int EPI_WARPS = (BN > 256 || HEAVY) ? 8 : 4;
   static constexpr int THREADS = 128 + 32 * EPI_WARPS;
-  static constexpr int A_BYTES = BM * BK * 2;
-  static constexpr int B_BYTES = BNL * BK * 2;
+  static constexpr int A_BYTES = BM * 128;    // 128 bytes of the contiguous dimension per row, whatever the type
+  static constexpr int B_BYTES = BNL * 128;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   // Epilogue staging: STG_BUFS boxes of 4 KB per epilogue warp (boxes in flight to/from global memory).
   static constexpr int STG_BUFS = (BN > 256 || HEAVY) ? 1 : 2;
@@ -410,9 +442,9 @@ __device__ __forceinline__ bool get_work(const GemmParams &p, int i, int bid, in
   w.col_end = col_base + cols;
   if (p.mode == MODE_RED) {
     w.kblocks = 0;
-    for (int ss = s; ss < s + w.s_count; ++ss) w.kblocks += ceil_div(min(p.L, p.R - ss * p.L), BK);
+    for (int ss = s; ss < s + w.s_count; ++ss) w.kblocks += ceil_div(min(p.L, p.R - ss * p.L), p.bk);
   } else {
-    w.kblocks = ceil_div(p.R, BK);
+    w.kblocks = ceil_div(p.R, p.bk);
   }
   w.carry_in = (p.mode == MODE_RED) && !p.carry_bf16 && (s > 0);
   w.carry_out = (p.mode == MODE_RED) && !p.carry_bf16 && (s + w.s_count - 1 < p.k_total - 1);
@@ -548,9 +580,11 @@ __device__ __forceinline__ void epilogue8(const Epilogue &e, long long row, int 
 // of the B tile (BN/2 rows), holds the accumulator of its 128 rows in its own tensor memory and
 // runs its own epilogue.  Per CTA a stage is 32 KB instead of 48 KB (6 stages instead of 4) and
 // half as many B bytes cross from L2 to shared memory per flop.
-template <int BN, bool A_MN, bool B_MN, bool CTA2, bool HEAVY = false>
+template <int BN, bool A_MN, bool B_MN, bool CTA2, bool HEAVY = false, int EB = 2>
 __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
   using SL = SmemLayout<BN, CTA2, HEAVY>;
+  constexpr int BKE = 128 / EB;   // reduction elements per k-block
+  constexpr int CW = 128 / EB;    // output rows / columns per 128-byte chunk of an MN-major operand
   constexpr int TM = CTA2 ? 2 * BM : BM;
   constexpr int BNL = SL::BNL;
   const uint32_t rank = CTA2 ? cluster_ctarank() : 0u;
@@ -640,7 +674,7 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
       const CUtensorMap *bmap = (b_sliced && !tail) ? &p.b_main : &p.b_tail;
       const int a_sc = (a_sliced && !tail) ? ss * p.a_sc_mul : 0;
       const int b_sc = (b_sliced && !tail) ? ss * p.b_sc_mul : 0;
-      const int nkb = (p.mode == MODE_RED) ? ceil_div(min(p.L, p.R - ss * p.L), BK) : w.kblocks;
+      const int nkb = (p.mode == MODE_RED) ? ceil_div(min(p.L, p.R - ss * p.L), BKE) : w.kblocks;
       for (int kb = 0; kb < nkb; ++kb) {
         ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER);
         if (!ok) break;
@@ -649,7 +683,7 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
           const uint32_t sb = sa + SL::A_BYTES;
           const uint32_t fb = full_bar(stage);
           if (load_a && (!CTA2 || rank == 0)) mbar_expect_tx(fb, SL::STAGE_BYTES * (CTA2 ? 2 : 1));
-          const int kc = kb * BK;
+          const int kc = kb * BKE;
           auto tma_load = [&](uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2) {
             if (CTA2) tma_load_3d_pair(dst, map, fb, c0, c1, c2);
             else tma_load_3d(dst, map, fb, c0, c1, c2);
@@ -657,10 +691,10 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
           if (!load_a) {
           } else if (A_MN) {
 #pragma unroll
-            for (int j = 0; j < BM / 64; ++j) {
-              const int in = w.a_row + j * 64;
-              if (a_mid) tma_load(sa + j * (BK * 128), amap, in, a_sc, kc);
-              else tma_load(sa + j * (BK * 128), amap, in, kc, a_sc);
+            for (int j = 0; j < BM / CW; ++j) {
+              const int in = w.a_row + j * CW;
+              if (a_mid) tma_load(sa + j * (BKE * 128), amap, in, a_sc, kc);
+              else tma_load(sa + j * (BKE * 128), amap, in, kc, a_sc);
             }
           } else {
             if (a_mid) tma_load(sa, amap, kc, a_sc, w.a_row);
@@ -669,11 +703,11 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
           if (!load_b) {
           } else if (B_MN) {
 #pragma unroll
-            for (int j = 0; j < BNL / 64; ++j) {
-              constexpr int CPG = SL::GB_ROWS / 64;   // 64-wide chunks per column group
-              const int in = w.b_col + (j / CPG) * 256 + (j % CPG) * 64;
-              if (b_mid) tma_load(sb + j * (BK * 128), bmap, in, b_sc, kc);
-              else tma_load(sb + j * (BK * 128), bmap, in, kc, b_sc);
+            for (int j = 0; j < (BNL + CW - 1) / CW; ++j) {
+              constexpr int CPG = (SL::GB_ROWS + CW - 1) / CW;   // chunks per column group
+              const int in = w.b_col + (j / CPG) * 256 + (j % CPG) * CW;
+              if (b_mid) tma_load(sb + j * (BKE * 128), bmap, in, b_sc, kc);
+              else tma_load(sb + j * (BKE * 128), bmap, in, kc, b_sc);
             }
           } else {
 #pragma unroll
@@ -703,7 +737,7 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
     }
   } else if (warp == 1 && rank == 0) {
     // ------------------------------------------------------------------ MMA issuer (even CTA of a pair)
-    constexpr uint32_t idesc = make_idesc<TM, SL::UMMA_N, A_MN, B_MN>();
+    constexpr uint32_t idesc = make_idesc<TM, SL::UMMA_N, A_MN, B_MN, EB>();
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;
@@ -722,16 +756,17 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
         if (lane == 0) {
           const uint32_t sa = smem_base + stage * SL::STAGE_BYTES;
           const uint32_t sb = sa + SL::A_BYTES;
-          const uint64_t adesc = make_smem_desc<A_MN>(sa);
-          const uint64_t bdesc = make_smem_desc<B_MN>(sb);
+          const uint64_t adesc = make_smem_desc<A_MN, EB>(sa);
+          const uint64_t bdesc = make_smem_desc<B_MN, EB>(sb);
 #pragma unroll
-          for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+          for (int kk = 0; kk < 4; ++kk) {   // four tcgen05.mma of 32 bytes of reduction each per k-block
 #pragma unroll
             for (int g = 0; g < SL::NG; ++g) {
-              umma_bf16<CTA2>(d_tmem + (uint32_t)(g * SL::UMMA_N),
-                              adesc + (uint64_t)((kk * desc_k_advance<A_MN>()) >> 4),
-                              bdesc + (uint64_t)((g * SL::GB_ROWS * 128 + kk * desc_k_advance<B_MN>()) >> 4), idesc,
-                              (kb > 0 || kk > 0) ? 1u : 0u);
+              const uint32_t d = d_tmem + (uint32_t)(g * SL::UMMA_N);
+              const uint64_t ad = adesc + (uint64_t)((kk * desc_k_advance<A_MN, EB>()) >> 4);
+              const uint64_t bd = bdesc + (uint64_t)((g * SL::GB_ROWS * 128 + kk * desc_k_advance<B_MN, EB>()) >> 4);
+              if (EB == 2) umma_bf16<CTA2>(d, ad, bd, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+              else umma_f8<CTA2>(d, ad, bd, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
             }
           }
           umma_commit<CTA2>(empty_bar(stage));                      // frees the stage when the MMAs retire
@@ -796,6 +831,7 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
           uint32_t v[32];
           tmem_ld_x32(taddr + (uint32_t)(c * 32), v);
           tmem_ld_wait();
+          scale_acc(v, p.epi.scale);
           if (row < w.row_end) {
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
@@ -855,6 +891,7 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
             uint32_t v[32];
             tmem_ld_x32(taddr + (uint32_t)(c * 32), v);
             tmem_ld_wait();
+            scale_acc(v, p.epi.scale);
             const uint32_t dst = stage_begin();
 #pragma unroll
             for (int j = 0; j < 8; ++j)
@@ -890,6 +927,7 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
             uint32_t v[32];
             tmem_ld_x32(taddr + (uint32_t)(c * 32), v);
             tmem_ld_wait();
+            scale_acc(v, p.epi.scale);
             const uint32_t n = first + (uint32_t)c;
             ok = mbar_wait(cbar + 8u * (n % NB), (n / NB) & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE);
             if (!ok) break;
@@ -986,6 +1024,7 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
             uint32_t v[32];
             tmem_ld_x32(taddr + (uint32_t)(c * 32), v);
             tmem_ld_wait();
+            scale_acc(v, p.epi.scale);
             const uint32_t n = first + (uint32_t)(c - c_lo);
             ok = mbar_wait(cbar + 8u * (n % NB), (n / NB) & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE);
             if (!ok) break;
@@ -1034,6 +1073,7 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
             uint32_t v[32];
             tmem_ld_x32(taddr + (uint32_t)(c * 32), v);
             tmem_ld_wait();
+            scale_acc(v, p.epi.scale);
             if (p.epi.bias) {
 #pragma unroll
               for (int g = 0; g < 4; ++g) {
@@ -1073,6 +1113,8 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
               tmem_ld_x32(taddr + (uint32_t)(c * 64), lo);
               if (BN >= 64) tmem_ld_x32(taddr + (uint32_t)(c * 64 + 32), hi);
               tmem_ld_wait();
+              scale_acc(lo, p.epi.scale);
+              if (BN >= 64) scale_acc(hi, p.epi.scale);
 #pragma unroll
               for (int j = 0; j < 32; ++j) { v[j] = lo[j]; v[32 + j] = hi[j]; }
             }
