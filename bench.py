@@ -382,6 +382,32 @@ def run_ours(args):
         for kk in ks:
             mlp_block["k%d" % kk]["overhead_vs_k1"] = mlp_block["k%d" % kk]["ms_per_step"] / mlp_block["k1"]["ms_per_step"] - 1.0
         del wsm
+    # ---- the same operator with fp8 (e4m3) operands, k = 1 and the headline split (secondary figures)
+    fp8 = {}
+    if rank == 0 and not args.no_sweep:
+        x8 = torch.randn(M, K, device=dev).to(torch.float8_e4m3fn).view(torch.uint8)
+        w8 = torch.randn(N * K, device=dev).to(torch.float8_e4m3fn).view(torch.uint8)
+        dy8 = torch.randn(M, N, device=dev).to(torch.float8_e4m3fn).view(torch.uint8)
+        need = max(workspace(1, P.SPLIT_OUT), workspace(k, P.SPLIT_OUT))
+        w8s = P.new_workspace(need, dev)
+
+        def f8_step(kk):
+            P.osdp_split_linear_fwd_f8(x8, w8, 0, 1.0, None, M, N, K, kk, P.SPLIT_OUT, 0, out, None, w8s, stream=stream,
+                                       check=True)
+            P.osdp_split_linear_bwd_f8(dy8, x8, w8, 0, 1.0, 1.0, M, N, K, kk, P.SPLIT_OUT, dx, dw_flat, 0,
+                                       P.DTYPE_BF16, 0, w8s, stream=stream, check=True)
+        t8 = {1: [], k: []}
+        for rnd in range(10):
+            for kk in t8:
+                a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+                a.record(stream); f8_step(kk); b.record(stream); torch.cuda.synchronize()
+                if rnd >= 2:
+                    t8[kk].append(a.elapsed_time(b))
+        for kk in t8:
+            ms = sorted(t8[kk])[len(t8[kk]) // 2]
+            fp8["k%d_out" % kk] = {"ms_per_step": ms, "tflops": fl / ms / 1e9,
+                                   "frac_of_2x_measured_bf16_burst": fl / ms / 1e9 / (2 * peaks()["bf16_tflops"])}
+        del w8s, x8, w8, dy8
     if world > 1:
         barrier()
 
@@ -468,7 +494,8 @@ def run_ours(args):
         "frac_of_bf16_peak": {"measured_burst_1658": value / world / pk["bf16_tflops"],
                               "measured_sustained_1378": value / world / pk["bf16_tflops_sustained"],
                               "datasheet_2250": value / world / 2250.0},
-        "sweep": sweep, "mlp_block_hidden1024_ffn4096_tokens4096": mlp_block, "staging_bytes": ws_bytes,
+        "sweep": sweep, "mlp_block_hidden1024_ffn4096_tokens4096": mlp_block,
+        "fp8_e4m3_operands": fp8, "staging_bytes": ws_bytes,
         "roofline": roofline, "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e / e2e_steps,

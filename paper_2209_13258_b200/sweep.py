@@ -3,6 +3,7 @@
     python -m paper_2209_13258_b200.sweep case M N K k split        one fwd+bwd (twice), for profilers
     python -m paper_2209_13258_b200.sweep case-mlp M hidden ffn k   one MLP-block fwd+bwd (twice), for profilers
     python -m paper_2209_13258_b200.sweep linear M N K [ks]         time vs slice granularity, both split dims
+    python -m paper_2209_13258_b200.sweep linear-f8 M N K [ks]      the same with fp8 (e4m3) operands
     python -m paper_2209_13258_b200.sweep mlp M hidden ffn [ks]     MLP block split along ffn: time and staging
     python -m paper_2209_13258_b200.sweep zdp M N K [ks]            sharded slice loop (gather / compute /
                                                                     reduce-scatter per slice) against the resident-
@@ -130,6 +131,43 @@ def sweep_linear(M, N, K, ks):
         rows.append({"k": k, "split": name,
                      "carry": {0: "fp32", P.FLAG_CARRY_BF16: "bf16", P.FLAG_PAIR_SLICES: "fp32-paired"}[fl],
                      "fwd_ms": tf, "bwd_ms": tb, "ms": t,
+                     "tflops": flops / t / 1e9, "overhead_vs_k1": t / base - 1.0, "staging_bytes": nbytes})
+        print(json.dumps(rows[-1]), flush=True)
+    return rows
+
+
+def sweep_linear_f8(M, N, K, ks):
+    """fp8 (e4m3) operands: forward + backward (dX, dW) per granularity and split dimension."""
+    dev = "cuda"
+    x8 = torch.randn(M, K, device=dev).to(torch.float8_e4m3fn).view(torch.uint8)
+    w8 = torch.randn(N, K, device=dev).to(torch.float8_e4m3fn).view(torch.uint8)
+    dy8 = torch.randn(M, N, device=dev).to(torch.float8_e4m3fn).view(torch.uint8)
+    out = torch.empty(M, N, device=dev, dtype=torch.bfloat16)
+    dx = torch.empty(M, K, device=dev, dtype=torch.bfloat16)
+    dw = torch.empty(N, K, device=dev, dtype=torch.bfloat16)
+    flops = 3 * 2.0 * M * N * K
+    cfgs = []
+    for k in ks:
+        for split, name in ((P.SPLIT_OUT, "out"), (P.SPLIT_RED, "red")):
+            if k == 1 and split == P.SPLIT_RED:
+                continue
+            rc, b, e = P.osdp_slice_range(N if split == P.SPLIT_OUT else K, k, 0)
+            if rc != 0 or (k > 1 and (e - b) % 16):
+                continue
+            cfgs.append((k, split, name, _ws_linear(M, N, K, k, split)))
+    ws = P.new_workspace(max(c[3] for c in cfgs))
+    fns = []
+    for k, split, name, _ in cfgs:
+        fns.append(lambda k=k, split=split: P.osdp_split_linear_fwd_f8(
+            x8, w8, 0, 1.0, None, M, N, K, k, split, 0, out, None, ws, check=True))
+        fns.append(lambda k=k, split=split: P.osdp_split_linear_bwd_f8(
+            dy8, x8, w8, 0, 1.0, 1.0, M, N, K, k, split, dx, dw, 0, P.DTYPE_BF16, 0, ws, check=True))
+    ts = _time_interleaved(fns)
+    rows = []
+    base = ts[0] + ts[1]
+    for i, (k, split, name, nbytes) in enumerate(cfgs):
+        t = ts[2 * i] + ts[2 * i + 1]
+        rows.append({"operands": "fp8 e4m3", "k": k, "split": name, "fwd_ms": ts[2 * i], "bwd_ms": ts[2 * i + 1], "ms": t,
                      "tflops": flops / t / 1e9, "overhead_vs_k1": t / base - 1.0, "staging_bytes": nbytes})
         print(json.dumps(rows[-1]), flush=True)
     return rows
@@ -296,6 +334,8 @@ def main(argv):
         run_case_mlp(*[int(v) for v in argv[2:6]])
     elif mode == "linear":
         sweep_linear(int(argv[2]), int(argv[3]), int(argv[4]), ks)
+    elif mode == "linear-f8":
+        sweep_linear_f8(int(argv[2]), int(argv[3]), int(argv[4]), ks)
     elif mode == "mlp":
         sweep_mlp(int(argv[2]), int(argv[3]), int(argv[4]), ks)
     elif mode == "zdp":
