@@ -2,6 +2,7 @@
 
     python -m paper_2209_13258_b200.sweep case M N K k split        one fwd+bwd (twice), for profilers
     python -m paper_2209_13258_b200.sweep case-mlp M hidden ffn k   one MLP-block fwd+bwd (twice), for profilers
+    python -m paper_2209_13258_b200.sweep case-f8 M N K k split     one fwd+bwd with fp8 operands (twice), for profilers
     python -m paper_2209_13258_b200.sweep linear M N K [ks]         time vs slice granularity, both split dims
     python -m paper_2209_13258_b200.sweep linear-f8 M N K [ks]      the same with fp8 (e4m3) operands
     python -m paper_2209_13258_b200.sweep mlp M hidden ffn [ks]     MLP block split along ffn: time and staging
@@ -72,6 +73,23 @@ def run_case(M, N, K, k, split):
     for _ in range(2):
         P.osdp_split_linear_fwd(x, w, 0, None, M, N, K, k, split, 0, out, None, ws, check=True)
         P.osdp_split_linear_bwd(dy, x, w, 0, None, M, N, K, k, split, 0, dx, dw, 0, 0, 0, None, ws, check=True)
+        torch.cuda.synchronize()
+    print("device status", P.osdp_read_device_status(ws))
+
+
+def run_case_f8(M, N, K, k, split):
+    dev = "cuda"
+    x8 = torch.randn(M, K, device=dev).to(torch.float8_e4m3fn).view(torch.uint8)
+    w8 = torch.randn(N, K, device=dev).to(torch.float8_e4m3fn).view(torch.uint8)
+    dy8 = torch.randn(M, N, device=dev).to(torch.float8_e4m3fn).view(torch.uint8)
+    out = torch.empty(M, N, device=dev, dtype=torch.bfloat16)
+    dx = torch.empty(M, K, device=dev, dtype=torch.bfloat16)
+    dw = torch.empty(N, K, device=dev, dtype=torch.bfloat16)
+    ws = P.new_workspace(_ws_linear(M, N, K, k, split))
+    for _ in range(2):
+        P.osdp_split_linear_fwd_f8(x8, w8, 0, 1.0, None, M, N, K, k, split, 0, out, None, ws, check=True)
+        P.osdp_split_linear_bwd_f8(dy8, x8, w8, 0, 1.0, 1.0, M, N, K, k, split, dx, dw, 0, P.DTYPE_BF16, 0, ws,
+                                   check=True)
         torch.cuda.synchronize()
     print("device status", P.osdp_read_device_status(ws))
 
@@ -330,6 +348,8 @@ def main(argv):
     ks = [int(v) for v in argv[5].split(",")] if len(argv) > 5 and not mode.startswith("case") else [1, 2, 4, 8, 16, 32]
     if mode == "case":
         run_case(*[int(v) for v in argv[2:7]])
+    elif mode == "case-f8":
+        run_case_f8(*[int(v) for v in argv[2:7]])
     elif mode == "case-mlp":
         run_case_mlp(*[int(v) for v in argv[2:6]])
     elif mode == "linear":
