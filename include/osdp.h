@@ -241,7 +241,12 @@ int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const 
  * one more slice-sized buffer), so that no [M,ffn] activation exists between forward and backward.
  * dX, dW1, db1 are bit-identical to the saved-activation path; dW2 = dY^T act(Z1_s) uses the
  * activation of the unrounded pre-activation, as the forward did.  b1 [ffn] fp32 or NULL is only
- * read then. */
+ * read then.
+ * When a slice's weight-gradient GEMMs are small (fewer 128 x 128 tiles than SMs) the call runs them
+ * on two streams of its own next to the dX GEMM: it forks from `stream` with an event and joins back
+ * into `stream` before the next slice, so the caller still sees one ordered call (a stream capture
+ * follows the fork).  The two streams and three events per device are created by the first such call;
+ * such calls on one device are serialised on the host while they enqueue. */
 int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_t off_w1, const float *b1,
                        int64_t off_w2, const void *z1_saved, int64_t M, int64_t hidden, int64_t ffn,
                        int k_split, int act, void *dx, void *dw_flat, int64_t dw_off_w1,

@@ -73,6 +73,42 @@ int device_sms(int *sms) {
   return OSDP_OK;
 }
 
+// Two internal streams and three events per device, created at the first call that wants them: small
+// independent launches of one call (the weight-gradient GEMMs of an MLP slice next to its dX GEMM) are
+// forked onto them from the caller's stream and joined back into it, so that they fill the SMs together.
+// The fork / join is plain event record + wait, which a stream capture follows into the side streams.
+struct SideStreams {
+  cudaStream_t s[2];
+  cudaEvent_t fork, join[2];
+};
+SideStreams g_side[64];
+std::atomic<bool> g_side_ready[64];
+std::mutex g_side_mutex;   // one call at a time enqueues a fork / join section (the events are shared)
+
+int side_streams(SideStreams **out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= 64) return cuda_fail(cudaErrorInvalidDevice);
+  if (!g_side_ready[dev].load(std::memory_order_acquire)) {
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    if (!g_side_ready[dev].load(std::memory_order_relaxed)) {
+      SideStreams &S = g_side[dev];
+      for (int i = 0; i < 2; ++i) {
+        e = cudaStreamCreateWithFlags(&S.s[i], cudaStreamNonBlocking);
+        if (e != cudaSuccess) return cuda_fail(e);
+        e = cudaEventCreateWithFlags(&S.join[i], cudaEventDisableTiming);
+        if (e != cudaSuccess) return cuda_fail(e);
+      }
+      e = cudaEventCreateWithFlags(&S.fork, cudaEventDisableTiming);
+      if (e != cudaSuccess) return cuda_fail(e);
+      g_side_ready[dev].store(true, std::memory_order_release);
+    }
+  }
+  *out = &g_side[dev];
+  return OSDP_OK;
+}
+
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -1081,6 +1117,13 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
   };
 
   if (db2) { rc = launch_colsum(dy, hidden, M, 0, (int)hidden, partial, db2, stream); if (rc) return rc; }
+  // Fork the slice's independent launches when its weight-gradient GEMMs are small (fewer 128 x 128 tiles
+  // than SMs): measured on B200, hidden 1024 / ffn 4096 / 4096 tokens at k = 8: 1.06 -> 0.84 ms; no
+  // effect, either way, on larger slices.
+  int sms = 0;
+  rc = device_sms(&sms);
+  if (rc) return rc;
+  const bool concurrent = dw_flat && cdiv(L, 128) * cdiv(hidden, 128) <= (int64_t)sms;
   for (int s = 0; s < k; ++s) {
     const int64_t lo = (int64_t)s * L;
     const int64_t ls = (lo + L < ffn ? lo + L : ffn) - lo;
@@ -1116,6 +1159,23 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
     c.status = status;
     rc = launch_gemm(c, stream);
     if (rc) return rc;
+    // The slice's three remaining GEMMs and its column sum depend only on what has been launched so far.
+    // Small ones (a few waves of tiles each) are forked onto the internal streams so that they share the
+    // SMs; large ones fill the GPU on their own and stay in order on the caller's stream.
+    SideStreams *side = nullptr;
+    std::unique_lock<std::mutex> side_lock;
+    cudaStream_t s_dw2 = stream, s_dw1 = stream;
+    if (concurrent) {
+      rc = side_streams(&side);
+      if (rc) return rc;
+      side_lock = std::unique_lock<std::mutex>(g_side_mutex);
+      cudaError_t e = cudaEventRecord(side->fork, stream);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(side->s[0], side->fork, 0);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(side->s[1], side->fork, 0);
+      if (e != cudaSuccess) return cuda_fail(e);
+      s_dw2 = side->s[0];
+      s_dw1 = side->s[1];
+    }
     if (dw_flat) {
       // dW2[:,F_s] = dY^T A_s
       memset(&c, 0, sizeof(c));
@@ -1126,7 +1186,7 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
       c.epi = plain_epilogue(dw_ptr(dw_off_w2 + lo), ffn, fp32);
       c.epi.accumulate = accumulate;
       c.status = status;
-      rc = launch_gemm(c, stream);
+      rc = launch_gemm(c, s_dw2);
       if (rc) return rc;
       // dW1[F_s,:] = dZ_s^T X
       memset(&c, 0, sizeof(c));
@@ -1137,10 +1197,10 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
       c.epi = plain_epilogue(dw_ptr(dw_off_w1 + lo * hidden), hidden, fp32);
       c.epi.accumulate = accumulate;
       c.status = status;
-      rc = launch_gemm(c, stream);
+      rc = launch_gemm(c, s_dw1);
       if (rc) return rc;
     }
-    if (db1) { rc = launch_colsum(dz_s, L, M, 0, (int)ls, partial, db1 + lo, stream); if (rc) return rc; }
+    if (db1) { rc = launch_colsum(dz_s, L, M, 0, (int)ls, partial, db1 + lo, s_dw1); if (rc) return rc; }
     if (dx) {
       // dX (+)= dZ_s W1[F_s,:]
       memset(&c, 0, sizeof(c));
@@ -1156,6 +1216,15 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
       c.status = status;
       rc = launch_gemm(c, stream);
       if (rc) return rc;
+    }
+    if (concurrent) {
+      // join: the next slice reuses the staging buffers these launches read
+      cudaError_t e = cudaSuccess;
+      for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+        e = cudaEventRecord(side->join[i], side->s[i]);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, side->join[i], 0);
+      }
+      if (e != cudaSuccess) return cuda_fail(e);
     }
   }
   return OSDP_OK;
