@@ -147,7 +147,10 @@ int osdp_split_linear_fwd_slice(const void *x, const void *w_flat, int64_t w_off
  *   sum in dx itself under OUT split), OSDP_FLAG_PAIR_SLICES (dX under OUT split);
  *   dbias [N] fp32 or NULL (always overwritten).
  * OUT: dW[R_s,:], db[R_s] per slice, dX = sum over slices (fp32 carry in ws).
- * RED: dX[:,C_s], dW[:,C_s] per slice. */
+ * RED: dX[:,C_s], dW[:,C_s] per slice.
+ * For a small operator without activation (fewer 128 x 128 output tiles than SMs in dX and in dW) the
+ * call runs dW and db on a stream of its own next to dX, forked from and joined back into `stream`
+ * (see osdp_split_mlp_bwd for the rules of these internal streams). */
 int osdp_split_linear_bwd(const void *dy, const void *x, const void *w_flat, int64_t w_offset,
                           const void *z_saved, int64_t M, int64_t N, int64_t K, int k_split,
                           int split_dim, int act, void *dx, void *dw_flat, int64_t dw_offset,

@@ -805,7 +805,29 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
   };
 
   if (act == OSDP_ACT_NONE) {
+    // dX, dW and db do not depend on one another.  A small operator (fewer 128 x 128 output tiles than SMs in
+    // both GEMMs) runs dW and db on an internal stream next to dX (fork from and join into `stream`).
+    SideStreams *side = nullptr;
+    std::unique_lock<std::mutex> side_lock;
+    cudaStream_t s_main = stream, s_side = stream;
+    {
+      int sms = 0;
+      rc = device_sms(&sms);
+      if (rc) return rc;
+      // (measured on B200, 256 x 2048 x 512 forward + backward: 42 -> 34 us at k = 1, 57 -> 46 us at k = 4)
+      if (dx && dw && cdiv(M, 128) * cdiv(K, 128) <= sms && cdiv(N, 128) * cdiv(K, 128) <= sms) {
+        rc = side_streams(&side);
+        if (rc) return rc;
+        side_lock = std::unique_lock<std::mutex>(g_side_mutex);
+        cudaError_t e = cudaEventRecord(side->fork, stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(side->s[0], side->fork, 0);
+        if (e != cudaSuccess) return cuda_fail(e);
+        s_side = side->s[0];
+      }
+    }
+    stream = s_main;
     if (dx) { rc = dx_call(Operand{dy, N, M, N, false, true}, s_begin, s_end); if (rc) return rc; }
+    stream = s_side;
     if (dw) { rc = dw_call(Operand{dy, N, M, N, true, true}, s_begin, s_end); if (rc) return rc; }
     if (dbias) {
       if (out_split) {
@@ -816,6 +838,12 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
         rc = launch_colsum(dy, N, M, 0, (int)N, partial, dbias, stream);
       }
       if (rc) return rc;
+    }
+    stream = s_main;
+    if (side) {
+      cudaError_t e = cudaEventRecord(side->join[0], side->s[0]);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, side->join[0], 0);
+      if (e != cudaSuccess) return cuda_fail(e);
     }
     return OSDP_OK;
   }
