@@ -417,12 +417,14 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   int sms = 0;
   int rc = device_sms(&sms);
   if (rc) return rc;
-  // Summed output with the exact carry and short slices (reduction length <= 512 per slice): one launch
-  // per slice.  The main loop of such a slice is shorter than its epilogue's carry traffic, and measured
-  // on B200 a launch boundary between slices is then faster than letting the CTAs drift across slices
-  // inside one launch (16384 x 8192 x 8192: k = 16 4.5 -> 3.9 ms, k = 32 7.8 -> 7.1 ms; no gain at
-  // k <= 8, a loss with the bf16 running sum).  Same arithmetic, same bits.
-  if (c.mode == MODE_RED && c.s_end - c.s_begin > 1 && !c.pair_slices && !c.carry_bf16 && c.L <= 512) {
+  // Summed output with the exact carry, short slices (reduction length <= 512 per slice) and many tiles
+  // per CTA pair (16 or more): one launch per slice.  The main loop of such a slice is shorter than its
+  // epilogue's carry traffic, and measured on B200 a launch boundary between slices is then faster than
+  // letting the CTAs drift across slices inside one launch (16384 x 8192 x 8192: k = 16 4.5 -> 3.9 ms,
+  // k = 32 7.8 -> 7.1 ms; no gain at k <= 8, a loss with the bf16 running sum, and a loss of 20 % on
+  // operators with only a few tiles per pair such as 8192 x 2048 x 2048).  Same arithmetic, same bits.
+  if (c.mode == MODE_RED && c.s_end - c.s_begin > 1 && !c.pair_slices && !c.carry_bf16 && c.L <= 512 &&
+      cdiv(c.P, 2 * BM) * cdiv(c.Q, 256) >= (int64_t)16 * (sms / 2)) {
     for (int s = c.s_begin; s < c.s_end; ++s) {
       GemmCall one = c;
       one.s_begin = s;
