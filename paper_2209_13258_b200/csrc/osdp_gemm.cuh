@@ -903,10 +903,11 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
           // fetched by TMA while this one is worked on; a box that has been read into registers is
           // overwritten in place with the bf16 results (64 bytes per row; z_save in its second half) and
           // leaves as a TMA store, so the buffer takes its next carry box once that store has read it.
-          // (Summed outputs are never given the 512-wide tile, so here every warp owns all columns.)
           const uint32_t cbar = bar_base + 8u * (2 * SL::STAGES + 5 + (warp - 4) * NB);
           int nchunks = (w.col_end - w.col0 + 31) / 32;
           if (nchunks > BN / 32) nchunks = BN / 32;
+          const int c_lo = wg * (BN / 32 / EG);                       // this warp's share of the columns
+          const int c_hi = min((wg + 1) * (BN / 32 / EG), nchunks);
           const bool staged_out = !p.epi.out_fp32;
           auto issue_load = [&](int c) {
             if (lane == 0) {
@@ -920,15 +921,15 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
           const uint32_t first = n_cload;
           if (lane == 0) bulk_wait_read<0>();
           __syncwarp();
-          for (int c = 0; c < (int)NB - 1 && c < nchunks; ++c) issue_load(c);
+          for (int c = c_lo; c < c_lo + (int)NB - 1 && c < c_hi; ++c) issue_load(c);
 #pragma unroll 1
-          for (int c = 0; c < nchunks; ++c) {
-            if (c + (int)NB - 1 < nchunks) issue_load(c + (int)NB - 1);
+          for (int c = c_lo; c < c_hi; ++c) {
+            if (c + (int)NB - 1 < c_hi) issue_load(c + (int)NB - 1);
             uint32_t v[32];
             tmem_ld_x32(taddr + (uint32_t)(c * 32), v);
             tmem_ld_wait();
             scale_acc(v, p.epi.scale);
-            const uint32_t n = first + (uint32_t)c;
+            const uint32_t n = first + (uint32_t)(c - c_lo);
             ok = mbar_wait(cbar + 8u * (n % NB), (n / NB) & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE);
             if (!ok) break;
             const uint32_t buf0 = stg + (n % NB) * 4096u;
