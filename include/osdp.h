@@ -224,6 +224,23 @@ int osdp_zdp_linear_bwd_slice(const void *dy, const void *x, const void *w_slice
                               int64_t ld_dw, int dw_dtype, int flags, float *dbias, void *ws,
                               size_t ws_bytes, void *stream);
 
+/* osdp_zdp_linear_bwd_slice with the reduce-scatter of the slice's weight gradient done by the GEMM's
+ * epilogue (compute step and collective in one kernel): instead of writing dW_s to a staging matrix, every
+ * 32-row box of it is reduce-added (TMA reduce-add, fp32 or bf16 per dw_dtype) directly into the buffer of the
+ * rank that owns those rows.  `dw_peers` is a HOST array of `world` (<= 8) DEVICE pointers; dw_peers[q] is
+ * where rank q keeps its part of this slice (shard_elems elements, the layout of osdp_zdp_shard_layout) -- this
+ * rank's own memory for q = rank, peer-mapped memory of the other GPUs otherwise (plain peer stores /
+ * reductions over NVLink; no multicast).  Every rank's call adds its term, so the buffers hold the sum over
+ * ranks once all ranks have finished the slice: zero them before the step and synchronise the ranks before
+ * reading them.  Needs the slice's row count (len R_s under OUT, N under RED) to be a multiple of 32 * world,
+ * else OSDP_ERR_UNSUPPORTED (use the staging form and a collective for that slice).  OSDP_FLAG_ACCUMULATE_DW
+ * is not accepted (the scatter always adds).  Everything else as osdp_zdp_linear_bwd_slice. */
+int osdp_zdp_linear_bwd_slice_scatter(const void *dy, const void *x, const void *w_slice, int64_t ld_w,
+                                      const void *z_saved, int64_t M, int64_t N, int64_t K, int k_split,
+                                      int split_dim, int act, int slice_idx, void *dx,
+                                      void *const *dw_peers, int world, int dw_dtype, int flags,
+                                      float *dbias, void *ws, size_t ws_bytes, void *stream);
+
 /* Transformer MLP block split along the ffn dimension (first layer OUT-split + activation,
  * second layer RED-split, Section 3.3 applied to both MatMuls of the block):
  *   out [M,hidden] = sum_s act(X W1[F_s,:]^T + b1[F_s]) W2[:,F_s]^T + b2, slice by slice.

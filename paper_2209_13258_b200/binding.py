@@ -25,7 +25,7 @@ EXPORTS = [
     "osdp_read_device_status", "osdp_bias_grad_noalloc", "osdp_debug_wait_probe", "osdp_suggest_granularity",
     "osdp_zdp_shard_layout", "osdp_zdp_linear_fwd_slice", "osdp_zdp_linear_bwd_slice",
     "osdp_plan_cost", "osdp_plan_search", "osdp_plan_expand_slices",
-    "osdp_split_linear_fwd_f8", "osdp_split_linear_bwd_f8",
+    "osdp_split_linear_fwd_f8", "osdp_split_linear_bwd_f8", "osdp_zdp_linear_bwd_slice_scatter",
 ]
 
 _lib = None
@@ -83,6 +83,8 @@ def lib():
         L.osdp_plan_search.argtypes = [pd, ci, ci, dbl, dbl, dbl, ci, i64, pu8, ctypes.POINTER(ci), pd, p64]
         L.osdp_plan_expand_slices.argtypes = [pd, ci, dbl, pd]
         f32 = ctypes.c_float
+        L.osdp_zdp_linear_bwd_slice_scatter.argtypes = [vp, vp, vp, i64, vp, i64, i64, i64, ci, ci, ci, ci, vp,
+                                                        ctypes.POINTER(vp), ci, ci, ci, vp, vp, sz, vp]
         L.osdp_split_linear_fwd_f8.argtypes = [vp, vp, i64, f32, vp, i64, i64, i64, ci, ci, ci, ci, vp, vp, vp, sz, vp]
         L.osdp_split_linear_bwd_f8.argtypes = [vp, vp, vp, i64, f32, f32, i64, i64, i64, ci, ci, vp, vp, i64, ci, ci,
                                                vp, sz, vp]
@@ -326,3 +328,15 @@ def osdp_split_linear_bwd_f8(dy8, x8, w8_flat, w_offset, scale_dx, scale_dw, M, 
                                         _ptr(dx), _ptr(dw_flat), int(dw_offset), int(dw_dtype), int(flags), wp, wn,
                                         _stream(stream))
     return _ret(rc, check, "osdp_split_linear_bwd_f8")
+
+
+def osdp_zdp_linear_bwd_slice_scatter(dy, x, w_slice, ld_w, z_saved, M, N, K, k_split, split_dim, act, slice_idx, dx,
+                                      dw_peers, dw_dtype, flags, dbias, ws, stream=None, check=False):
+    """dw_peers: one tensor (or raw device address) per rank: where that rank keeps its part of this slice."""
+    wp, wn = _ws(ws)
+    arr = (ctypes.c_void_p * len(dw_peers))(*[t if isinstance(t, int) else t.data_ptr() for t in dw_peers])
+    rc = lib().osdp_zdp_linear_bwd_slice_scatter(_ptr(dy), _ptr(x), _ptr(w_slice), int(ld_w), _ptr(z_saved), int(M),
+                                                 int(N), int(K), int(k_split), int(split_dim), int(act),
+                                                 int(slice_idx), _ptr(dx), arr, len(dw_peers), int(dw_dtype),
+                                                 int(flags), _ptr(dbias), wp, wn, _stream(stream))
+    return _ret(rc, check, "osdp_zdp_linear_bwd_slice_scatter")

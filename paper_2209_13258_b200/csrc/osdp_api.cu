@@ -215,6 +215,8 @@ struct GemmCall {
   int pair_slices;  // MODE_RED: accumulate two adjacent slices per pass
   int out_is_slice; // MODE_ROWS / MODE_COLS: `epi.out` is the slice's own compact matrix, not the whole output
   int fp8;          // operands are fp8 e4m3 (1 byte per element) instead of bf16
+  int n_peers;      // > 0: the output slice is reduce-added row block by row block into peer_out[0..n_peers)
+  void *peer_out[8];
   int *status;
 };
 
@@ -545,6 +547,28 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
     }
   }
 
+  if (c.n_peers > 0) {
+    // The epilogue scatters the (compact) output over the ranks' buffers, always as reduce-adds.
+    if (!p.tma_epilogue || c.mode == MODE_RED || c.n_peers > 8 || c.epi.gz || c.epi.z_save || c.epi.bias ||
+        c.epi.act != ACT_NONE || (c.k_total > 1 && (!c.out_is_slice || c.s_end - c.s_begin != 1)))
+      return OSDP_ERR_UNSUPPORTED;
+    const int64_t full_r = c.P, full_c = c.Q;
+    const int64_t ls = (c.k_total > 1) ? (((c.mode == MODE_ROWS ? full_r : full_c) - c.s_begin * c.L < c.L)
+                                              ? (c.mode == MODE_ROWS ? full_r : full_c) - c.s_begin * c.L : c.L) : 0;
+    const int64_t rows = (c.k_total > 1 && c.mode == MODE_ROWS) ? ls : full_r;
+    const int64_t cols = (c.k_total > 1 && c.mode == MODE_COLS) ? ls : full_c;
+    if (rows % c.n_peers || (rows / c.n_peers) % 32) return OSDP_ERR_UNSUPPORTED;
+    p.n_peers = c.n_peers;
+    p.rows_per_peer = (int)(rows / c.n_peers);
+    for (int q = 0; q < c.n_peers; ++q) {
+      if (!c.peer_out[q] || !aligned16(c.peer_out[q])) return c.peer_out[q] ? OSDP_ERR_ALIGNMENT : OSDP_ERR_NULL_POINTER;
+      CUtensorMap unused;
+      rc = make_output_maps(c.peer_out[q], c.epi.out_fp32 != 0, p.rows_per_peer, cols, cols, c.mode, c.L, c.k_total,
+                            &unused, &p.peer_out[q], nullptr, false);
+      if (rc) return rc;
+    }
+  }
+
   // Work items of this launch (one per scheduling unit and tile).
   const int64_t items = count_items(c, tm, bn);
   const bool heavy = (c.epi.act != ACT_NONE || gz_tma) && c.mode != MODE_RED && p.tma_epilogue && !c.fp8;
@@ -708,7 +732,9 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
              int64_t N, int64_t K, int k, int split_dim, int act, int s_begin, int s_end, bool single, void *dx,
              void *dw_flat, int64_t dw_offset, int dw_dtype, int flags, float *dbias, void *ws, size_t ws_bytes,
              void *stream_, int64_t ld_w_slice = 0, int64_t ld_dw_slice = 0, int fp8 = 0, float scale_dx = 1.0f,
-             float scale_dw = 1.0f) {
+             float scale_dw = 1.0f, void *const *dw_peers = nullptr, int n_peers = 0) {
+  // dw_peers: the slice's weight gradient is not written to dw_flat but reduce-added, row block by row block,
+  // into the n_peers ranks' buffers (the reduce-scatter of the slice done by the GEMM's epilogue)
   // fp8: dy, x and W are e4m3 bytes; no activation, no bias gradient (G = dY must itself be an fp8 operand)
   // ld_w_slice > 0: W is slice `s_begin` gathered into a compact matrix (see fwd_impl);
   // ld_dw_slice > 0: dW of the slice is written as a compact matrix of the same shape.
@@ -802,6 +828,10 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
     c.epi.scale = scale_dw;
     c.epi.accumulate = accumulate;
     c.out_is_slice = (ld_dw_slice > 0 && k > 1) ? 1 : 0;
+    if (n_peers > 0) {
+      c.n_peers = n_peers;
+      for (int q = 0; q < n_peers && q < 8; ++q) c.peer_out[q] = dw_peers[q];
+    }
     c.status = status;
     return launch_gemm(c, stream);
   };
@@ -1037,6 +1067,21 @@ int osdp_zdp_linear_bwd_slice(const void *dy, const void *x, const void *w_slice
   if (ld_w <= 0 || (dw_slice && ld_dw <= 0)) return OSDP_ERR_BAD_SHAPE;
   return bwd_impl(dy, x, w_slice, 0, z_saved, M, N, K, k_split, split_dim, act, slice_idx, 0, true, dx, dw_slice, 0,
                   dw_dtype, flags, dbias, ws, ws_bytes, stream, ld_w, dw_slice ? ld_dw : 0);
+}
+
+int osdp_zdp_linear_bwd_slice_scatter(const void *dy, const void *x, const void *w_slice, int64_t ld_w,
+                                      const void *z_saved, int64_t M, int64_t N, int64_t K, int k_split, int split_dim,
+                                      int act, int slice_idx, void *dx, void *const *dw_peers, int world, int dw_dtype,
+                                      int flags, float *dbias, void *ws, size_t ws_bytes, void *stream) {
+  if (ld_w <= 0) return OSDP_ERR_BAD_SHAPE;
+  if (!dw_peers) return OSDP_ERR_NULL_POINTER;
+  if (world < 1 || world > 8) return OSDP_ERR_UNSUPPORTED;
+  if (flags & OSDP_FLAG_ACCUMULATE_DW) return OSDP_ERR_UNSUPPORTED;   // the scatter always adds
+  int64_t ld = 0;
+  int rc = osdp_zdp_shard_layout(N, K, k_split, split_dim, world, slice_idx, nullptr, nullptr, nullptr, &ld);
+  if (rc) return rc;
+  return bwd_impl(dy, x, w_slice, 0, z_saved, M, N, K, k_split, split_dim, act, slice_idx, 0, true, dx, dw_peers[0], 0,
+                  dw_dtype, flags, dbias, ws, ws_bytes, stream, ld_w, ld, 0, 1.0f, 1.0f, dw_peers, world);
 }
 
 int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const float *b1, int64_t off_w2,

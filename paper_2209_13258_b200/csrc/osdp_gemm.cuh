@@ -72,6 +72,12 @@ struct GemmParams {
                                     // the last slice of a summed output and the epilogue that reads gz
   CUtensorMap gz32_map;             // the element-wise second input gz, same boxes
   CUtensorMap gz_pf_map;            // gz as boxes of 32 rows x BN columns, for L2 prefetch
+  // Output scattered over the ranks of a data-parallel group (a weight-gradient slice reduce-scattered by the
+  // epilogue itself): rank q owns rows [q * rows_per_peer, (q + 1) * rows_per_peer) of the slice's compact
+  // matrix; peer_out[q] maps that block in rank q's memory (its own, or a peer-mapped address) and every box
+  // is reduce-added there.  n_peers = 0: not used.
+  CUtensorMap peer_out[8];
+  int n_peers, rows_per_peer;
   int out_sc_mul;
   int red_group;             // MODE_RED: slices whose products a tile accumulates in one pass (1, or 2 = adjacent pairs)
   int carry_bf16;            // MODE_RED: the running sum is kept in `out` itself, in bf16 (no fp32 carry buffer)
@@ -861,7 +867,13 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
           fence_proxy_async();
           __syncwarp();
           if (lane == 0) {
-            if (out_mid && map != &p.carry_map) {
+            if (p.n_peers > 0 && (map == &p.out_main || map == &p.out_tail)) {
+              // the owner of this 32-row box (rows_per_peer is a multiple of 32, so a box has one owner)
+              const int q = r_in / p.rows_per_peer;
+              const int rl = r_in - q * p.rows_per_peer;
+              if (out_mid) tma_reduce_add_3d(&p.peer_out[q], src, col_in, 0, rl);
+              else tma_reduce_add_3d(&p.peer_out[q], src, col_in, rl, 0);
+            } else if (out_mid && map != &p.carry_map) {
               if (reduce) tma_reduce_add_3d(map, src, col_in, sc, r_in);
               else tma_store_3d(map, src, col_in, sc, r_in);
             } else {

@@ -251,7 +251,7 @@ def sweep_zdp(M, N, K, ks):
     x, w, dy, out, dx, _, db = _linear_tensors(M, N, K)
     dw = torch.empty(N, K, device="cuda", dtype=torch.float32)
     flops = 3 * 2.0 * M * N * K
-    cfgs, fns, layers = [], [], []
+    cfgs, fns, layers, fused_ok = [], [], [], True
     for k in ks:
         for split, name in ((P.SPLIT_OUT, "out"), (P.SPLIT_RED, "red")):
             if k == 1 and split == P.SPLIT_RED:
@@ -274,6 +274,21 @@ def sweep_zdp(M, N, K, ks):
             layer.forward(x, out=out)
             layer.backward(dy, x, dx=dx, dbias=db)
         fns += [resident, sharded]
+        # the same loop with the reduce-scatter done by the backward GEMM's epilogue (peer-mapped gradient shards)
+        try:
+            fl = ZdpSplitLinear(N, K, k, split, dw_dtype=P.DTYPE_FP32, fused_scatter=True) if fused_ok else None
+        except Exception:
+            fused_ok, fl = False, None
+        if fl is not None:
+            fl.load_full_weight(w)
+
+            def fused(fl=fl):
+                fl.forward(x, out=out)
+                fl.backward(dy, x, dx=dx, dbias=db)
+            fns.append(fused)
+        else:
+            fns.append(sharded)
+        layers[-1] = (layer, fl)
     ts = _time_interleaved(fns, rounds=8)
     tt = torch.tensor(ts, device="cuda", dtype=torch.float64)
     if world > 1:
@@ -281,10 +296,11 @@ def sweep_zdp(M, N, K, ks):
     ts = tt.tolist()
     rows = []
     for i, (k, split, name) in enumerate(cfgs):
-        st = layers[i].staging_bytes(M)
-        rows.append({"k": k, "split": name, "world": world, "resident_ms": ts[2 * i], "sharded_ms": ts[2 * i + 1],
-                     "sharded_tflops_all_ranks": world * flops / ts[2 * i + 1] / 1e9,
-                     "loop_overhead": ts[2 * i + 1] / ts[2 * i] - 1.0,
+        st = layers[i][0].staging_bytes(M)
+        rows.append({"k": k, "split": name, "world": world, "resident_ms": ts[3 * i], "sharded_ms": ts[3 * i + 1],
+                     "sharded_fused_scatter_ms": ts[3 * i + 2] if layers[i][1] is not None else None,
+                     "sharded_tflops_all_ranks": world * flops / ts[3 * i + 1] / 1e9,
+                     "loop_overhead": ts[3 * i + 1] / ts[3 * i] - 1.0,
                      "weight_staging_bytes": st["weight_staging"], "grad_staging_bytes": st["grad_staging"],
                      "workspace_bytes": st["workspace"], "full_gather_bytes": N * K * 2, "full_grad_bytes": N * K * 4})
         if rank == 0:

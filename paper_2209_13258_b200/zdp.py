@@ -94,6 +94,25 @@ class DistComm:
         import torch.distributed as dist
         dist.all_reduce(t, op=dist.ReduceOp.SUM, group=self.group)
 
+    def barrier(self):
+        import torch.distributed as dist
+        dist.barrier(group=self.group)
+
+    def peer_buffers(self, numel, dtype, device):
+        """One buffer of `numel` elements per rank, all addressable from this GPU: this rank's own and the
+        peer-mapped ones of the other ranks (torch symmetric memory over the group).  Returns the list indexed
+        by rank; entry [self.rank] is local memory."""
+        import torch.distributed as dist
+        try:
+            import torch.distributed._symmetric_memory as symm
+        except ImportError as e:   # pragma: no cover
+            raise RuntimeError("peer-mapped buffers need torch.distributed._symmetric_memory") from e
+        group = self.group if self.group is not None else dist.group.WORLD
+        local = symm.empty(int(numel), dtype=dtype, device=device)
+        handle = symm.rendezvous(local, group.group_name)
+        self._symm_keep = getattr(self, "_symm_keep", []) + [(local, handle)]
+        return [local if r == self.rank else handle.get_buffer(r, (int(numel),), dtype) for r in range(self.world)]
+
 
 DP, ZDP = 0, 1
 
@@ -110,7 +129,7 @@ class ZdpSplitLinear:
     """
 
     def __init__(self, N, K, k_split, split_dim, act=B.ACT_NONE, dw_dtype=B.DTYPE_FP32, comm=None, device="cuda",
-                 flags=0, slice_modes=None):
+                 flags=0, slice_modes=None, fused_scatter=False):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("ZdpSplitLinear needs a CUDA device: there is no CPU path")
@@ -131,7 +150,16 @@ class ZdpSplitLinear:
             self._zoff[s] = total
             total += self.layout.slices[s][3]
         self.param_shard = torch.zeros(max(total, 8), dtype=torch.bfloat16, device=self.device)
-        self.grad_shard = torch.zeros(max(total, 8), dtype=gdt, device=self.device)
+        # fused_scatter: the backward GEMM's epilogue reduce-adds each slice's dW straight into the owners'
+        # gradient shards, which therefore have to be addressable from every rank (comm.peer_buffers); the
+        # caller zeroes them (zero_grad) before the step and the ranks meet (comm.barrier) before reading them.
+        self.fused_scatter = bool(fused_scatter)
+        if self.fused_scatter:
+            self.peer_grad_shards = self.comm.peer_buffers(max(total, 8), gdt, self.device)
+            self.grad_shard = self.peer_grad_shards[self.comm.rank]
+            self.grad_shard.zero_()
+        else:
+            self.grad_shard = torch.zeros(max(total, 8), dtype=gdt, device=self.device)
         self.dp_weight = {s: torch.zeros(self.layout.slices[s][2], dtype=torch.bfloat16, device=self.device)
                           for s in range(self.k) if self.modes[s] == DP}
         self.dp_grad = {s: torch.zeros(self.layout.slices[s][2], dtype=gdt, device=self.device) for s in self.dp_weight}
@@ -140,8 +168,11 @@ class ZdpSplitLinear:
         wst = max([self.layout.slices[s][3] for s in self.zdp_slices] + [0]) * self.comm.world
         self.w_stage = [torch.zeros(wst, dtype=torch.bfloat16, device=self.device)
                         for _ in range(min(2, len(self.zdp_slices)))]
+        # (gradient staging only if some slice goes through a collective: not when the epilogue scatters them all)
+        need_dw_stage = any(self.modes[s] == ZDP and not self._scatter_ok(s) for s in range(self.k))
+        self._gdt = gdt
         self.dw_stage = [torch.zeros(self.layout.stage_elems, dtype=gdt, device=self.device)
-                         for _ in range(min(2, self.k))]
+                         for _ in range(min(2, self.k) if need_dw_stage else 0)]
         self.comm_stream = torch.cuda.Stream(device=self.device)
         self.side_stream = torch.cuda.Stream(device=self.device)
         self._ws = None
@@ -173,6 +204,17 @@ class ZdpSplitLinear:
                 flat = dp_parts[s][:elems]
             self.layout.slice_matrix(full, s).copy_(flat.reshape(-1, ld))
         return full
+
+    def zero_grad(self):
+        self.grad_shard.zero_()
+        for t in self.dp_grad.values():
+            t.zero_()
+
+    def _scatter_ok(self, s):
+        """Whether slice s can be reduce-scattered by the GEMM's epilogue (rows divisible by 32 * world)."""
+        b, e = self.layout.slices[s][0], self.layout.slices[s][1]
+        rows = (e - b) if self.split_dim == B.SPLIT_OUT else self.N
+        return self.fused_scatter and self.modes[s] == ZDP and rows % (32 * self.comm.world) == 0
 
     def staging_bytes(self, M):
         """Bytes this layer holds besides its weights and gradients: staging plus the kernels' workspace."""
@@ -295,7 +337,39 @@ class ZdpSplitLinear:
             _, _, elems, shard, _, ld = self.layout.slices[s]
             zdp = self.modes[s] == ZDP
             j = s & 1                                       # gradient staging buffer of this slice
+            if self._scatter_ok(s):
+                # the slice's dW goes from the GEMM's epilogue straight into the owners' shards (always added)
+                o = self._zoff[s]
+                peers = [int(t.data_ptr()) + o * t.element_size() for t in self.peer_grad_shards]
+                st = side if (self.k > 1 and out_split and self.act == B.ACT_NONE and need_dx) else \
+                    ((cur, side)[s & 1] if alternate else cur)
+                if alternate and s == 1 and self.act != B.ACT_NONE:
+                    st.wait_event(first_done)               # slice 0 stages G for every later slice
+                split_here = st is side and not alternate    # dX on `cur`, dW (+ db) on `side`
+                w, b = g.weights(s, [cur, st] if split_here else [st])
+                if split_here:
+                    B.osdp_zdp_linear_bwd_slice(dy, x, w, ld, z_saved, M, self.N, self.K, self.k, self.split_dim,
+                                                self.act, s, dx, None, 0, self.dw_dtype, flags, None, ws, stream=cur,
+                                                check=True)
+                    B.osdp_zdp_linear_bwd_slice_scatter(dy, x, w, ld, z_saved, M, self.N, self.K, self.k,
+                                                        self.split_dim, self.act, s, None, peers, self.dw_dtype, 0,
+                                                        dbias, ws, stream=st, check=True)
+                    done = [self._mark(cur), self._mark(st)]
+                else:
+                    B.osdp_zdp_linear_bwd_slice_scatter(dy, x, w, ld, z_saved, M, self.N, self.K, self.k,
+                                                        self.split_dim, self.act, s, dx if need_dx else None, peers,
+                                                        self.dw_dtype, flags, dbias, ws, stream=st, check=True)
+                    done = [self._mark(st)]
+                if s == 0:
+                    first_done = done[0]
+                if b is not None:
+                    g.free[b] = done
+                continue
             direct = not zdp and not accumulate             # DP: the kernel writes dp_grad[s] itself
+            if not direct and len(self.dw_stage) <= j:      # first use (a DP slice accumulating through staging)
+                import torch as _t
+                while len(self.dw_stage) <= j:
+                    self.dw_stage.append(_t.zeros(self.layout.stage_elems, dtype=self._gdt, device=self.device))
             dw_dst = self.dp_grad[s] if direct else self.dw_stage[j]
             if split_calls:
                 w, b = g.weights(s, [cur, side])

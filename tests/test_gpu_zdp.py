@@ -130,8 +130,18 @@ class EmulatedComm:
         acc = self.shared["dp_acc"]
         acc[tag] = t.double().clone() if tag not in acc else acc[tag] + t.double()
 
+    def barrier(self):
+        pass
 
-def run_emulated_ranks(P, world, M, N, K, k, split, act, modes):
+    def peer_buffers(self, numel, dtype, device):
+        # "peer" memory of the emulated ranks: one buffer per rank on this GPU, the same list for every rank
+        key = ("peer", numel, dtype)
+        if key not in self.shared:
+            self.shared[key] = [torch.zeros(numel, dtype=dtype, device=device) for _ in range(self.world)]
+        return self.shared[key]
+
+
+def run_emulated_ranks(P, world, M, N, K, k, split, act, modes, fused=False):
     """Forward + backward of the slice loop for every emulated rank on its own token rows; returns the
     assembled Y, dX, sum over ranks of dW and db, and the first rank's layer."""
     from paper_2209_13258_b200.zdp import ZdpSplitLinear
@@ -141,7 +151,8 @@ def run_emulated_ranks(P, world, M, N, K, k, split, act, modes):
     shared = {"param": [None] * world, "grad_acc": [None] * world, "dp_acc": {}}
     layers = []
     for r in range(world):
-        layer = ZdpSplitLinear(N, K, k, split, act=act, comm=EmulatedComm(r, world, shared), slice_modes=modes)
+        layer = ZdpSplitLinear(N, K, k, split, act=act, comm=EmulatedComm(r, world, shared), slice_modes=modes,
+                               fused_scatter=fused)
         layer.load_full_weight(W)
         shared["param"][r] = layer.param_shard
         shared["grad_acc"][r] = torch.zeros(layer.grad_shard.numel(), dtype=torch.float64, device="cuda")
@@ -162,7 +173,20 @@ def run_emulated_ranks(P, world, M, N, K, k, split, act, modes):
         assert rc == 0 and st == 0
         y[rows], dx[rows] = yr, dxr
         db += dbr.double()
-    dW = layers[0].full_from_parts(shared["grad_acc"], shared["dp_acc"])
+    if fused:
+        # slices scattered by the epilogue are complete in the ranks' own shards; the others came through the
+        # emulated collective and are complete in the fp64 accumulators
+        shards = []
+        for q, l in enumerate(layers):
+            t = shared["grad_acc"][q].clone()
+            for s in range(k):
+                if l._scatter_ok(s):
+                    n, o = l.layout.slices[s][3], l._zoff[s]
+                    t[o:o + n] = l.grad_shard[o:o + n].double()
+            shards.append(t)
+        dW = layers[0].full_from_parts(shards, shared["dp_acc"])
+    else:
+        dW = layers[0].full_from_parts(shared["grad_acc"], shared["dp_acc"])
     return c, y, dx, dW, db, layers[0]
 
 
@@ -190,6 +214,57 @@ def test_slice_loop_over_emulated_ranks_matches_oracle(P, world, split, case):
     assert st["weight_staging"] == 2 * 2 * world * max(sl[3] for sl in layer.layout.slices)
     assert st["weight_staging"] <= 2 * 2 * (N * K // k + 8 * world + max(N, K) * 8)
     assert layer.state_bytes()["weights"] == 2 * layer.layout.shard_total
+
+
+@pytest.mark.parametrize("world", [1, 2, 4])
+@pytest.mark.parametrize("split", [0, 1])
+@pytest.mark.parametrize("case,modes", [((512, 2048, 512, 4, 0), None), ((384, 1024, 1024, 8, 1), None),
+                                        ((512, 2048, 512, 4, 0), [0, 1, 1, 0]), ((256, 1024, 512, 1, 0), None),
+                                        ((300, 520, 264, 3, 1), None)])
+def test_reduce_scatter_fused_into_the_gemm_epilogue(P, world, split, case, modes):
+    """The backward GEMM's epilogue reduce-adds each slice's dW into the owning ranks' shards (peer buffers
+    emulated by one buffer per rank on this GPU); slices whose rows do not divide fall back to the collective."""
+    M, N, K, k, act = case
+    D = N if split == 0 else K
+    if P.osdp_slice_range(D, k, 0)[0] != 0:
+        pytest.skip("invalid split")
+    c, y, dx, dW, db, layer = run_emulated_ranks(P, world, M, N, K, k, split, act, modes, fused=True)
+    check_against_oracle(c, y, dx, dW, db, act, k, split)
+    rows = [(layer.layout.slices[s][1] - layer.layout.slices[s][0]) if split == 0 else N for s in range(k)]
+    expect = [layer.modes[s] == 1 and rows[s] % (32 * world) == 0 for s in range(k)]
+    assert [layer._scatter_ok(s) for s in range(k)] == expect
+    if (M, N, K) == (512, 2048, 512) and modes is None:
+        assert all(expect)          # this case really runs the fused path on every slice
+
+
+def test_fused_scatter_equals_staged_reduce_scatter_for_one_rank(P):
+    """world = 1: the epilogue's scatter into the rank's own shard gives the bits of the staged path."""
+    M, N, K, k = 512, 2048, 512, 4
+    for split in (0, 1):
+        res = []
+        for fused in (False, True):
+            c, y, dx, dW, db, layer = run_emulated_ranks(P, 1, M, N, K, k, split, 0, None, fused=fused)
+            res.append(dW)
+        assert torch.equal(res[0], res[1])
+
+
+def test_scatter_argument_errors(P):
+    M, N, K, k = 128, 256, 128, 2
+    x = torch.zeros(M, K, dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros(N // k, K, dtype=torch.bfloat16, device="cuda")
+    dy = torch.zeros(M, N, dtype=torch.bfloat16, device="cuda")
+    _, n = P.osdp_split_linear_workspace_bytes(M, N, K, k, 0, 0, P.OP_LINEAR_BWD)
+    ws = P.new_workspace(n)
+    g = P.osdp_zdp_linear_bwd_slice_scatter
+    sh = [torch.zeros(N // k * K // 2, dtype=torch.float32, device="cuda") for _ in range(2)]
+    assert g(dy, x, w, K, None, M, N, K, k, 0, 0, 0, None, sh, P.DTYPE_FP32, 0, None, ws) == 0
+    assert g(dy, x, w, K, None, M, N, K, k, 0, 0, 0, None, sh, P.DTYPE_FP32, P.FLAG_ACCUMULATE_DW, None, ws) == 6
+    sh3 = sh + [sh[0]]
+    assert g(dy, x, w, K, None, M, N, K, k, 0, 0, 0, None, sh3, P.DTYPE_FP32, 0, None, ws) == 6     # 128 rows / 3 ranks
+    sh8 = [sh[0]] * 8
+    assert g(dy, x, w, K, None, M, N, K, k, 0, 0, 0, None, sh8, P.DTYPE_FP32, 0, None, ws) == 6     # 16 rows per rank
+    assert g(dy, x, w, K, None, M, N, K, k, 0, 0, 0, None, [sh[0]] * 9, P.DTYPE_FP32, 0, None, ws) == 6
+    assert g(dy, x, w, K, None, M, N, K, k, 0, 0, 0, None, [sh[0], 0], P.DTYPE_FP32, 0, None, ws) == 1
 
 
 MIXED = [((512, 2048, 512, 4, 0), [0, 1, 1, 0]), ((512, 2048, 512, 4, 0), [1, 0, 0, 0]),
@@ -248,5 +323,28 @@ def test_slice_loop_on_a_one_rank_nccl_group(P):
             layer.backward(dy, x, z_saved=z, dbias=db, accumulate=True)
             torch.cuda.synchronize()
             assert_close(to_f64(layer.full_from_parts([layer.grad_shard], layer.dp_grad)), 2 * dWo, "dW accumulated")
+        # the epilogue's scatter into a shard allocated as symmetric memory (one rank: its own buffer)
+        try:
+            layer = ZdpSplitLinear(N, K, k, 0, act=0, fused_scatter=True)
+        except Exception as e:   # symmetric memory not available in this build / on this machine
+            print("symmetric memory unavailable:", repr(e)[:200])
+            layer = None
+        if layer is not None:
+            c = inputs.linear_case(M, N, K, w_std=0.05)
+            W = to_dev(c["w_flat"])[c["w_offset"]:c["w_offset"] + N * K].view(N, K)
+            layer.load_full_weight(W)
+            x, dy = to_dev(c["x"]), to_dev(c["dy"])
+            assert all(layer._scatter_ok(s) for s in range(k))
+            for _ in range(2):
+                layer.zero_grad()
+                y = layer.forward(x)
+                dx = layer.backward(dy, x)
+                layer.comm.barrier()
+            torch.cuda.synchronize()
+            zo, yo = oracle.linear_fwd(c["x"], c["w"], None, 0, k, 0)
+            dXo, dWo, _ = oracle.linear_bwd(c["dy"], c["x"], c["w"], zo, 0, k, 0)
+            assert_close(to_f64(y), yo, "Y")
+            assert_close(to_f64(dx), dXo, "dX")
+            assert_close(to_f64(layer.full_from_parts([layer.grad_shard], {})), dWo, "dW scattered by the epilogue")
     finally:
         dist.destroy_process_group()
