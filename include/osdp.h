@@ -241,6 +241,28 @@ int osdp_zdp_linear_bwd_slice_scatter(const void *dy, const void *x, const void 
                                       void *const *dw_peers, int world, int dw_dtype, int flags,
                                       float *dbias, void *ws, size_t ws_bytes, void *stream);
 
+/* One slice of the split MLP block (below) of a sharded operator pair: W1[F_s,:] and W2[:,F_s] are given as
+ * the gathered compact matrices w1_slice [len F_s, hidden] (contiguous rows) and w2_slice [hidden, len F_s]
+ * (leading dimension ld_w2 >= len F_s, a multiple of 8).  b1 [ffn], z1_save [M,ffn], out, workspace, flags and
+ * the ordering of the slices as in osdp_split_mlp_fwd, whose per-slice work this is, bit for bit. */
+int osdp_zdp_mlp_fwd_slice(const void *x, const void *w1_slice, const void *w2_slice, int64_t ld_w2,
+                           const float *b1, const float *b2, int64_t M, int64_t hidden, int64_t ffn,
+                           int k_split, int act, int flags, int slice_idx, void *out, void *z1_save,
+                           void *ws, size_t ws_bytes, void *stream);
+
+/* One slice of osdp_split_mlp_bwd with gathered compact weights.  The slice's weight gradients go either
+ * to compact matrices dw1_slice [len F_s, hidden] and dw2_slice [hidden, len F_s] (leading dimension
+ * ld_dw2), both or neither, ready for a reduce-scatter; or, when dw1_peers / dw2_peers (HOST arrays of `world`
+ * DEVICE pointers, both or neither) are given, straight into the owning ranks' shards from the GEMMs'
+ * epilogues, as in osdp_zdp_linear_bwd_slice_scatter (row counts len F_s and hidden must both be multiples
+ * of 32 * world).  db1 [ffn] receives the slice's part, db2 [hidden] is written by slice 0. */
+int osdp_zdp_mlp_bwd_slice(const void *dy, const void *x, const void *w1_slice, const void *w2_slice,
+                           int64_t ld_w2, const float *b1, const void *z1_saved, int64_t M, int64_t hidden,
+                           int64_t ffn, int k_split, int act, int slice_idx, void *dx, void *dw1_slice,
+                           void *dw2_slice, int64_t ld_dw2, void *const *dw1_peers, void *const *dw2_peers,
+                           int world, int dw_dtype, int flags, float *db1, float *db2, void *ws,
+                           size_t ws_bytes, void *stream);
+
 /* Transformer MLP block split along the ffn dimension (first layer OUT-split + activation,
  * second layer RED-split, Section 3.3 applied to both MatMuls of the block):
  *   out [M,hidden] = sum_s act(X W1[F_s,:]^T + b1[F_s]) W2[:,F_s]^T + b2, slice by slice.

@@ -14,4 +14,5 @@ from .binding import (  # noqa: F401
     osdp_zdp_shard_layout, osdp_zdp_linear_fwd_slice, osdp_zdp_linear_bwd_slice,
     osdp_plan_cost, osdp_plan_search, osdp_plan_expand_slices,
     osdp_split_linear_fwd_f8, osdp_split_linear_bwd_f8, osdp_zdp_linear_bwd_slice_scatter,
+    osdp_zdp_mlp_fwd_slice, osdp_zdp_mlp_bwd_slice,
 )

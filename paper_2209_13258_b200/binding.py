@@ -26,6 +26,7 @@ EXPORTS = [
     "osdp_zdp_shard_layout", "osdp_zdp_linear_fwd_slice", "osdp_zdp_linear_bwd_slice",
     "osdp_plan_cost", "osdp_plan_search", "osdp_plan_expand_slices",
     "osdp_split_linear_fwd_f8", "osdp_split_linear_bwd_f8", "osdp_zdp_linear_bwd_slice_scatter",
+    "osdp_zdp_mlp_fwd_slice", "osdp_zdp_mlp_bwd_slice",
 ]
 
 _lib = None
@@ -83,6 +84,10 @@ def lib():
         L.osdp_plan_search.argtypes = [pd, ci, ci, dbl, dbl, dbl, ci, i64, pu8, ctypes.POINTER(ci), pd, p64]
         L.osdp_plan_expand_slices.argtypes = [pd, ci, dbl, pd]
         f32 = ctypes.c_float
+        pvp = ctypes.POINTER(vp)
+        L.osdp_zdp_mlp_fwd_slice.argtypes = [vp, vp, vp, i64, vp, vp, i64, i64, i64, ci, ci, ci, ci, vp, vp, vp, sz, vp]
+        L.osdp_zdp_mlp_bwd_slice.argtypes = [vp, vp, vp, vp, i64, vp, vp, i64, i64, i64, ci, ci, ci, vp, vp, vp, i64,
+                                             pvp, pvp, ci, ci, ci, vp, vp, vp, sz, vp]
         L.osdp_zdp_linear_bwd_slice_scatter.argtypes = [vp, vp, vp, i64, vp, i64, i64, i64, ci, ci, ci, ci, vp,
                                                         ctypes.POINTER(vp), ci, ci, ci, vp, vp, sz, vp]
         L.osdp_split_linear_fwd_f8.argtypes = [vp, vp, i64, f32, vp, i64, i64, i64, ci, ci, ci, ci, vp, vp, vp, sz, vp]
@@ -340,3 +345,32 @@ def osdp_zdp_linear_bwd_slice_scatter(dy, x, w_slice, ld_w, z_saved, M, N, K, k_
                                                  int(slice_idx), _ptr(dx), arr, len(dw_peers), int(dw_dtype),
                                                  int(flags), _ptr(dbias), wp, wn, _stream(stream))
     return _ret(rc, check, "osdp_zdp_linear_bwd_slice_scatter")
+
+
+def _ptr_array(ts):
+    if ts is None:
+        return None
+    return (ctypes.c_void_p * len(ts))(*[t if isinstance(t, int) else t.data_ptr() for t in ts])
+
+
+def osdp_zdp_mlp_fwd_slice(x, w1_slice, w2_slice, ld_w2, b1, b2, M, hidden, ffn, k_split, act, slice_idx, out, z1_save,
+                           ws, stream=None, check=False, flags=0):
+    wp, wn = _ws(ws)
+    rc = lib().osdp_zdp_mlp_fwd_slice(_ptr(x), _ptr(w1_slice), _ptr(w2_slice), int(ld_w2), _ptr(b1), _ptr(b2), int(M),
+                                      int(hidden), int(ffn), int(k_split), int(act), int(flags), int(slice_idx),
+                                      _ptr(out), _ptr(z1_save), wp, wn, _stream(stream))
+    return _ret(rc, check, "osdp_zdp_mlp_fwd_slice")
+
+
+def osdp_zdp_mlp_bwd_slice(dy, x, w1_slice, w2_slice, ld_w2, b1, z1_saved, M, hidden, ffn, k_split, act, slice_idx, dx,
+                           dw1_slice, dw2_slice, ld_dw2, dw1_peers, dw2_peers, dw_dtype, flags, db1, db2, ws,
+                           stream=None, check=False):
+    """dw1_peers / dw2_peers: None, or one tensor (or device address) per rank for the epilogue's scatter."""
+    wp, wn = _ws(ws)
+    world = len(dw1_peers) if dw1_peers is not None else 0
+    rc = lib().osdp_zdp_mlp_bwd_slice(_ptr(dy), _ptr(x), _ptr(w1_slice), _ptr(w2_slice), int(ld_w2), _ptr(b1),
+                                      _ptr(z1_saved), int(M), int(hidden), int(ffn), int(k_split), int(act),
+                                      int(slice_idx), _ptr(dx), _ptr(dw1_slice), _ptr(dw2_slice), int(ld_dw2),
+                                      _ptr_array(dw1_peers), _ptr_array(dw2_peers), world, int(dw_dtype), int(flags),
+                                      _ptr(db1), _ptr(db2), wp, wn, _stream(stream))
+    return _ret(rc, check, "osdp_zdp_mlp_bwd_slice")

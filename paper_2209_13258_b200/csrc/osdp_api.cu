@@ -1084,9 +1084,20 @@ int osdp_zdp_linear_bwd_slice_scatter(const void *dy, const void *x, const void 
                   dw_dtype, flags, dbias, ws, ws_bytes, stream, ld_w, ld, 0, 1.0f, 1.0f, dw_peers, world);
 }
 
-int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const float *b1, int64_t off_w2,
-                       const float *b2, int64_t M, int64_t hidden, int64_t ffn, int k_split, int act, int flags,
-                       void *out, void *z1_save, void *ws, size_t ws_bytes, void *stream_) {
+// One slice of a sharded MLP block given as gathered compact matrices (and where its weight gradients go).
+struct MlpSlice {
+  int idx;                    // the slice; the call covers this slice only
+  const void *w1, *w2;        // W1[F_s,:] as [len F_s, hidden] (contiguous rows), W2[:,F_s] as [hidden, len F_s]
+  int64_t ld_w2;
+  void *dw1, *dw2;            // same shapes, dw_dtype; or the ranks' buffers for the epilogue's reduce-scatter
+  int64_t ld_dw2;
+  void *const *dw1_peers, *const *dw2_peers;
+  int world;
+};
+
+static int mlp_fwd_impl(const void *x, const void *w_flat, int64_t off_w1, const float *b1, int64_t off_w2,
+                        const float *b2, int64_t M, int64_t hidden, int64_t ffn, int k_split, int act, int flags,
+                        void *out, void *z1_save, void *ws, size_t ws_bytes, void *stream_, const MlpSlice *cs) {
   if (!x || !w_flat || !out) return OSDP_ERR_NULL_POINTER;
   if (flags & ~OSDP_FLAG_CARRY_BF16) return OSDP_ERR_UNSUPPORTED;   // the second layer has no activation: allowed
   int64_t L = 0;
@@ -1111,14 +1122,15 @@ int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const 
   float *carry = reinterpret_cast<float *>(wsb + plan.carry_off);
   int *status = static_cast<int *>(ws);
 
-  for (int s = 0; s < k; ++s) {
+  if (cs && (cs->idx < 0 || cs->idx >= k)) return OSDP_ERR_BAD_SPLIT;
+  for (int s = cs ? cs->idx : 0; s < (cs ? cs->idx + 1 : k); ++s) {
     const int64_t lo = (int64_t)s * L;
     const int64_t ls = (lo + L < ffn ? lo + L : ffn) - lo;
     // A_s = act(X W1[F_s,:]^T + b1[F_s])
     GemmCall c;
     memset(&c, 0, sizeof(c));
     c.a = Operand{x, hidden, M, hidden, false, false};
-    c.b = Operand{w1 + lo * hidden, hidden, ls, hidden, false, false};
+    c.b = Operand{cs ? static_cast<const __nv_bfloat16 *>(cs->w1) : w1 + lo * hidden, hidden, ls, hidden, false, false};
     c.P = M; c.Q = ls; c.R = hidden; c.bn_P = M; c.bn_Q = L;
     c.mode = MODE_NONE; c.L = ls; c.k_total = 1; c.s_begin = 0; c.s_end = 1;
     c.epi = plain_epilogue(a_s, L, 0);
@@ -1132,7 +1144,7 @@ int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const 
     // Y (+)= A_s W2[:,F_s]^T ; + b2 after the last slice
     memset(&c, 0, sizeof(c));
     c.a = Operand{a_s, ls, M, L, false, false};
-    c.b = Operand{w2, ffn, hidden, ffn, false, true};
+    c.b = cs ? Operand{cs->w2, ls, hidden, cs->ld_w2, false, false} : Operand{w2, ffn, hidden, ffn, false, true};
     c.P = M; c.Q = hidden; c.R = ffn; c.bn_P = M; c.bn_Q = hidden;
     c.mode = (k == 1) ? MODE_NONE : MODE_RED;
     c.L = L; c.k_total = k; c.s_begin = s; c.s_end = s + 1;
@@ -1148,10 +1160,11 @@ int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const 
   return OSDP_OK;
 }
 
-int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_t off_w1, const float *b1,
-                       int64_t off_w2, const void *z1_saved, int64_t M, int64_t hidden, int64_t ffn, int k_split,
-                       int act, void *dx, void *dw_flat, int64_t dw_off_w1, int64_t dw_off_w2, int dw_dtype,
-                       int flags, float *db1, float *db2, void *ws, size_t ws_bytes, void *stream_) {
+static int mlp_bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t off_w1, const float *b1,
+                        int64_t off_w2, const void *z1_saved, int64_t M, int64_t hidden, int64_t ffn, int k_split,
+                        int act, void *dx, void *dw_flat, int64_t dw_off_w1, int64_t dw_off_w2, int dw_dtype,
+                        int flags, float *db1, float *db2, void *ws, size_t ws_bytes, void *stream_,
+                        const MlpSlice *cs) {
   if (flags & ~(OSDP_FLAG_ACCUMULATE_DW | OSDP_FLAG_CARRY_BF16 | OSDP_FLAG_RECOMPUTE)) return OSDP_ERR_UNSUPPORTED;
   const bool recompute = (flags & OSDP_FLAG_RECOMPUTE) != 0;
   if (!dy || !x || !w_flat || (!recompute && !z1_saved)) return OSDP_ERR_NULL_POINTER;
@@ -1191,7 +1204,11 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
     return fp32 ? (void *)(static_cast<float *>(dw_flat) + off) : (void *)(static_cast<__nv_bfloat16 *>(dw_flat) + off);
   };
 
-  if (db2) { rc = launch_colsum(dy, hidden, M, 0, (int)hidden, partial, db2, stream); if (rc) return rc; }
+  if (cs && (cs->idx < 0 || cs->idx >= k)) return OSDP_ERR_BAD_SPLIT;
+  if (db2 && (!cs || cs->idx == 0)) {
+    rc = launch_colsum(dy, hidden, M, 0, (int)hidden, partial, db2, stream);
+    if (rc) return rc;
+  }
   // Fork the slice's independent launches when its weight-gradient GEMMs are small (fewer 128 x 128 tiles
   // than SMs): measured on B200, hidden 1024 / ffn 4096 / 4096 tokens at k = 8: 1.06 -> 0.84 ms; no
   // effect, either way, on larger slices.
@@ -1199,15 +1216,18 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
   rc = device_sms(&sms);
   if (rc) return rc;
   const bool concurrent = dw_flat && cdiv(L, 128) * cdiv(hidden, 128) <= (int64_t)sms;
-  for (int s = 0; s < k; ++s) {
+  for (int s = cs ? cs->idx : 0; s < (cs ? cs->idx + 1 : k); ++s) {
     const int64_t lo = (int64_t)s * L;
     const int64_t ls = (lo + L < ffn ? lo + L : ffn) - lo;
+    const __nv_bfloat16 *w1s = cs ? static_cast<const __nv_bfloat16 *>(cs->w1) : w1 + lo * hidden;   // [ls, hidden]
+    const __nv_bfloat16 *w2s = cs ? static_cast<const __nv_bfloat16 *>(cs->w2) : w2 + lo;            // [hidden, ls]
+    const int64_t ld_w2s = cs ? cs->ld_w2 : ffn;
     GemmCall c;
     if (recompute) {
       // Z1_s = X W1[F_s,:]^T + b1[F_s] (the forward's first GEMM again, same bits), A_s = act(Z1_s)
       memset(&c, 0, sizeof(c));
       c.a = Operand{x, hidden, M, hidden, false, false};
-      c.b = Operand{w1 + lo * hidden, hidden, ls, hidden, false, false};
+      c.b = Operand{w1s, hidden, ls, hidden, false, false};
       c.P = M; c.Q = ls; c.R = hidden; c.bn_P = M; c.bn_Q = L;
       c.mode = MODE_NONE; c.L = ls; c.k_total = 1; c.s_begin = 0; c.s_end = 1;
       c.epi = plain_epilogue(a_s, L, 0);
@@ -1222,7 +1242,7 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
     // dZ_s = (dY W2[:,F_s]) (.) act'(Z1_s);  A_s = act(Z1_s) unless it was just recomputed
     memset(&c, 0, sizeof(c));
     c.a = Operand{dy, hidden, M, hidden, false, false};
-    c.b = Operand{w2 + lo, ls, hidden, ffn, true, false};
+    c.b = Operand{w2s, ls, hidden, ld_w2s, true, false};
     c.P = M; c.Q = ls; c.R = hidden; c.bn_P = M; c.bn_Q = L;
     c.mode = MODE_NONE; c.L = ls; c.k_total = 1; c.s_begin = 0; c.s_end = 1;
     c.epi = plain_epilogue(dz_s, L, 0);
@@ -1258,8 +1278,13 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
       c.b = Operand{a_s, ls, M, L, true, false};
       c.P = hidden; c.Q = ls; c.R = M; c.bn_P = hidden; c.bn_Q = L;
       c.mode = MODE_NONE; c.L = ls; c.k_total = 1; c.s_begin = 0; c.s_end = 1;
-      c.epi = plain_epilogue(dw_ptr(dw_off_w2 + lo), ffn, fp32);
+      c.epi = cs ? plain_epilogue(cs->dw2_peers ? cs->dw2_peers[0] : cs->dw2, cs->ld_dw2, fp32)
+                 : plain_epilogue(dw_ptr(dw_off_w2 + lo), ffn, fp32);
       c.epi.accumulate = accumulate;
+      if (cs && cs->dw2_peers) {
+        c.n_peers = cs->world;
+        for (int q = 0; q < cs->world && q < 8; ++q) c.peer_out[q] = cs->dw2_peers[q];
+      }
       c.status = status;
       rc = launch_gemm(c, s_dw2);
       if (rc) return rc;
@@ -1269,8 +1294,13 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
       c.b = Operand{x, hidden, M, hidden, true, false};
       c.P = ls; c.Q = hidden; c.R = M; c.bn_P = L; c.bn_Q = hidden;
       c.mode = MODE_NONE; c.L = ls; c.k_total = 1; c.s_begin = 0; c.s_end = 1;
-      c.epi = plain_epilogue(dw_ptr(dw_off_w1 + lo * hidden), hidden, fp32);
+      c.epi = cs ? plain_epilogue(cs->dw1_peers ? cs->dw1_peers[0] : cs->dw1, hidden, fp32)
+                 : plain_epilogue(dw_ptr(dw_off_w1 + lo * hidden), hidden, fp32);
       c.epi.accumulate = accumulate;
+      if (cs && cs->dw1_peers) {
+        c.n_peers = cs->world;
+        for (int q = 0; q < cs->world && q < 8; ++q) c.peer_out[q] = cs->dw1_peers[q];
+      }
       c.status = status;
       rc = launch_gemm(c, s_dw1);
       if (rc) return rc;
@@ -1280,7 +1310,7 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
       // dX (+)= dZ_s W1[F_s,:]
       memset(&c, 0, sizeof(c));
       c.a = Operand{dz_s, ls, M, L, false, false};
-      c.b = Operand{w1, hidden, ffn, hidden, true, true};
+      c.b = cs ? Operand{w1s, hidden, ls, hidden, true, false} : Operand{w1, hidden, ffn, hidden, true, true};
       c.P = M; c.Q = hidden; c.R = ffn; c.bn_P = M; c.bn_Q = hidden;
       c.mode = (k == 1) ? MODE_NONE : MODE_RED;
       c.L = L; c.k_total = k; c.s_begin = s; c.s_end = s + 1;
@@ -1303,6 +1333,66 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
     }
   }
   return OSDP_OK;
+}
+
+int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const float *b1, int64_t off_w2,
+                       const float *b2, int64_t M, int64_t hidden, int64_t ffn, int k_split, int act, int flags,
+                       void *out, void *z1_save, void *ws, size_t ws_bytes, void *stream) {
+  return mlp_fwd_impl(x, w_flat, off_w1, b1, off_w2, b2, M, hidden, ffn, k_split, act, flags, out, z1_save, ws,
+                      ws_bytes, stream, nullptr);
+}
+
+int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_t off_w1, const float *b1,
+                       int64_t off_w2, const void *z1_saved, int64_t M, int64_t hidden, int64_t ffn, int k_split,
+                       int act, void *dx, void *dw_flat, int64_t dw_off_w1, int64_t dw_off_w2, int dw_dtype,
+                       int flags, float *db1, float *db2, void *ws, size_t ws_bytes, void *stream) {
+  return mlp_bwd_impl(dy, x, w_flat, off_w1, b1, off_w2, z1_saved, M, hidden, ffn, k_split, act, dx, dw_flat,
+                      dw_off_w1, dw_off_w2, dw_dtype, flags, db1, db2, ws, ws_bytes, stream, nullptr);
+}
+
+int osdp_zdp_mlp_fwd_slice(const void *x, const void *w1_slice, const void *w2_slice, int64_t ld_w2, const float *b1,
+                           const float *b2, int64_t M, int64_t hidden, int64_t ffn, int k_split, int act, int flags,
+                           int slice_idx, void *out, void *z1_save, void *ws, size_t ws_bytes, void *stream) {
+  if (!w1_slice || !w2_slice) return OSDP_ERR_NULL_POINTER;
+  if (ld_w2 <= 0 || (ld_w2 & 7)) return ld_w2 <= 0 ? OSDP_ERR_BAD_SHAPE : OSDP_ERR_ALIGNMENT;
+  if (!aligned16(w1_slice) || !aligned16(w2_slice)) return OSDP_ERR_ALIGNMENT;
+  MlpSlice cs;
+  memset(&cs, 0, sizeof(cs));
+  cs.idx = slice_idx; cs.w1 = w1_slice; cs.w2 = w2_slice; cs.ld_w2 = ld_w2;
+  return mlp_fwd_impl(x, w1_slice, 0, b1, 0, b2, M, hidden, ffn, k_split, act, flags, out, z1_save, ws, ws_bytes,
+                      stream, &cs);
+}
+
+int osdp_zdp_mlp_bwd_slice(const void *dy, const void *x, const void *w1_slice, const void *w2_slice, int64_t ld_w2,
+                           const float *b1, const void *z1_saved, int64_t M, int64_t hidden, int64_t ffn,
+                           int k_split, int act, int slice_idx, void *dx, void *dw1_slice, void *dw2_slice,
+                           int64_t ld_dw2, void *const *dw1_peers, void *const *dw2_peers, int world, int dw_dtype,
+                           int flags, float *db1, float *db2, void *ws, size_t ws_bytes, void *stream) {
+  if (!w1_slice || !w2_slice) return OSDP_ERR_NULL_POINTER;
+  if (ld_w2 <= 0 || (ld_w2 & 7)) return ld_w2 <= 0 ? OSDP_ERR_BAD_SHAPE : OSDP_ERR_ALIGNMENT;
+  if (!aligned16(w1_slice) || !aligned16(w2_slice) || !aligned16(dw1_slice) || !aligned16(dw2_slice))
+    return OSDP_ERR_ALIGNMENT;
+  const bool scatter = dw1_peers || dw2_peers;
+  if (scatter && (!dw1_peers || !dw2_peers)) return OSDP_ERR_NULL_POINTER;
+  if (scatter && (world < 1 || world > 8 || (flags & OSDP_FLAG_ACCUMULATE_DW))) return OSDP_ERR_UNSUPPORTED;
+  const bool want_dw = scatter || (dw1_slice && dw2_slice);
+  if (!scatter && ((dw1_slice != nullptr) != (dw2_slice != nullptr))) return OSDP_ERR_NULL_POINTER;
+  if (want_dw && !scatter && (ld_dw2 <= 0 || (ld_dw2 & 7))) return ld_dw2 <= 0 ? OSDP_ERR_BAD_SHAPE : OSDP_ERR_ALIGNMENT;
+  MlpSlice cs;
+  memset(&cs, 0, sizeof(cs));
+  cs.idx = slice_idx; cs.w1 = w1_slice; cs.w2 = w2_slice; cs.ld_w2 = ld_w2;
+  cs.dw1 = dw1_slice; cs.dw2 = dw2_slice; cs.ld_dw2 = ld_dw2;
+  cs.dw1_peers = dw1_peers; cs.dw2_peers = dw2_peers; cs.world = world;
+  if (scatter) {   // the compact dW2_s is [hidden, len F_s]: its leading dimension is the slice length
+    int64_t b = 0, e = 0;
+    int rc = osdp_slice_range(ffn, k_split, slice_idx, &b, &e);
+    if (rc) return rc;
+    cs.ld_dw2 = e - b;
+  }
+  // dw_flat only says whether weight gradients are wanted; the slice's own matrices are in `cs`
+  return mlp_bwd_impl(dy, x, w1_slice, 0, b1, 0, z1_saved, M, hidden, ffn, k_split, act, dx,
+                      want_dw ? const_cast<void *>(w1_slice) : nullptr, 0, 0, dw_dtype, flags, db1, db2, ws, ws_bytes,
+                      stream, &cs);
 }
 
 int osdp_debug_wait_probe(void *ws, int64_t limit_us, void *stream_) {

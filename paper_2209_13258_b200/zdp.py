@@ -417,3 +417,159 @@ class ZdpSplitLinear:
         cur.wait_stream(side)
         cur.wait_stream(self.comm_stream)                   # gradients are complete for whoever runs next on `cur`
         return dx
+
+
+class ZdpSplitMLP:
+    """Linear -> activation -> Linear with both weights sharded over the ranks, split along ffn (first layer OUT,
+    second layer RED) and gathered slice by slice: only W1[F_s,:] and W2[:,F_s] of the slice in use (and of the
+    next one, being gathered) exist in full; the slice's dW1 and dW2 are reduce-scattered as soon as they
+    exist, by a collective from slice-sized staging or, with fused_scatter, by the GEMMs' epilogues.
+
+    param_shard[0/1], grad_shard[0/1]: this rank's parts of W1 [ffn, hidden] / W2 [hidden, ffn] and of the summed
+    gradients, slice after slice (ShardLayout of each).
+    """
+
+    def __init__(self, hidden, ffn, k_split, act=B.ACT_GELU_TANH, dw_dtype=B.DTYPE_FP32, comm=None, device="cuda",
+                 flags=0, fused_scatter=False):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("ZdpSplitMLP needs a CUDA device: there is no CPU path")
+        self.comm = comm if comm is not None else DistComm()
+        self.hidden, self.ffn, self.act, self.dw_dtype, self.flags = int(hidden), int(ffn), int(act), int(dw_dtype), int(flags)
+        world = self.comm.world
+        self.layouts = [ShardLayout(ffn, hidden, k_split, B.SPLIT_OUT, world),
+                        ShardLayout(hidden, ffn, k_split, B.SPLIT_RED, world)]
+        self.k = self.layouts[0].k
+        self.device = torch.device(device)
+        gdt = torch.float32 if dw_dtype == B.DTYPE_FP32 else torch.bfloat16
+        self.param_shard = [torch.zeros(l.shard_total, dtype=torch.bfloat16, device=self.device) for l in self.layouts]
+        self.fused_scatter = bool(fused_scatter)
+        if self.fused_scatter:
+            self.peer_grad_shards = [self.comm.peer_buffers(l.shard_total, gdt, self.device) for l in self.layouts]
+            self.grad_shard = [p[self.comm.rank] for p in self.peer_grad_shards]
+            for t in self.grad_shard:
+                t.zero_()
+        else:
+            self.grad_shard = [torch.zeros(l.shard_total, dtype=gdt, device=self.device) for l in self.layouts]
+        nb = min(2, self.k)
+        self.w_stage = [[torch.zeros(l.stage_elems, dtype=torch.bfloat16, device=self.device) for _ in range(nb)]
+                        for l in self.layouts]
+        need = any(not self._scatter_ok(s) for s in range(self.k))
+        self.dw_stage = [[torch.zeros(l.stage_elems, dtype=gdt, device=self.device) for _ in range(nb if need else 0)]
+                         for l in self.layouts]
+        self.comm_stream = torch.cuda.Stream(device=self.device)
+        self._ws = None
+
+    def _scatter_ok(self, s):
+        ls = self.layouts[0].slices[s][1] - self.layouts[0].slices[s][0]
+        m = 32 * self.comm.world
+        return self.fused_scatter and ls % m == 0 and self.hidden % m == 0
+
+    def load_full_weights(self, w1_full, w2_full):
+        for i, w in enumerate((w1_full, w2_full)):
+            self.param_shard[i].copy_(self.layouts[i].shard_of(w.to(self.device), self.comm.rank))
+
+    def zero_grad(self):
+        for t in self.grad_shard:
+            t.zero_()
+
+    def staging_bytes(self, M):
+        nbytes = lambda ts: sum(t.numel() * t.element_size() for t in ts)
+        _, f = B.osdp_split_linear_workspace_bytes(M, self.ffn, self.hidden, self.k, B.SPLIT_OUT, self.act, B.OP_MLP_FWD,
+                                                   self.flags & B.FLAG_CARRY_BF16)
+        _, b = B.osdp_split_linear_workspace_bytes(M, self.ffn, self.hidden, self.k, B.SPLIT_OUT, self.act, B.OP_MLP_BWD,
+                                                   self.flags & (B.FLAG_CARRY_BF16 | B.FLAG_RECOMPUTE))
+        return {"weight_staging": nbytes(self.w_stage[0] + self.w_stage[1]),
+                "grad_staging": nbytes(self.dw_stage[0] + self.dw_stage[1]), "workspace": max(f, b)}
+
+    def _workspace(self, M):
+        n = self.staging_bytes(M)["workspace"]
+        if self._ws is None or self._ws.numel() != max(n, 256):
+            self._ws = B.new_workspace(n, device=self.device)
+        return self._ws
+
+    def _gather(self, s, free_events):
+        """Both weights of slice s into staging buffer s & 1, on the communication stream."""
+        import torch
+        with torch.cuda.stream(self.comm_stream):
+            for ev in free_events:
+                self.comm_stream.wait_event(ev)
+            for i, l in enumerate(self.layouts):
+                _, _, _, n, off, _ = l.slices[s]
+                self.comm.all_gather_slice(self.w_stage[i][s & 1], self.param_shard[i], off, n)
+            ev = torch.cuda.Event()
+            ev.record(self.comm_stream)
+        return ev
+
+    def forward(self, x, b1=None, b2=None, out=None, z1_save=None):
+        import torch
+        M = x.shape[0]
+        cur = torch.cuda.current_stream(self.device)
+        if out is None:
+            out = torch.empty(M, self.hidden, dtype=torch.bfloat16, device=self.device)
+        ws = self._workspace(M)
+        self.comm_stream.wait_stream(cur)
+        free = [[], []]
+        ready = self._gather(0, [])
+        for s in range(self.k):
+            nxt = self._gather(s + 1, free[(s + 1) & 1]) if s + 1 < self.k else None
+            cur.wait_event(ready)
+            B.osdp_zdp_mlp_fwd_slice(x, self.w_stage[0][s & 1], self.w_stage[1][s & 1], self.layouts[1].slices[s][5], b1,
+                                     b2, M, self.hidden, self.ffn, self.k, self.act, s, out, z1_save, ws, stream=cur,
+                                     check=True, flags=self.flags & B.FLAG_CARRY_BF16)
+            ev = torch.cuda.Event()
+            ev.record(cur)
+            free[s & 1] = [ev]
+            ready = nxt
+        self.comm_stream.wait_stream(cur)
+        return out
+
+    def backward(self, dy, x, z1_saved=None, b1=None, dx=None, db1=None, db2=None):
+        """z1_saved None: the pre-activation is recomputed per slice (needs b1).  Gradients of the weights are
+        summed over ranks into grad_shard (with fused_scatter they add to what is there: zero_grad first)."""
+        import torch
+        M = x.shape[0]
+        cur = torch.cuda.current_stream(self.device)
+        if dx is None:
+            dx = torch.empty(M, self.hidden, dtype=torch.bfloat16, device=self.device)
+        flags = (self.flags & B.FLAG_CARRY_BF16) | (B.FLAG_RECOMPUTE if z1_saved is None else 0)
+        if flags & B.FLAG_RECOMPUTE:
+            self.flags |= B.FLAG_RECOMPUTE          # the workspace plan has one more slice-sized buffer
+        ws = self._workspace(M)
+        self.comm_stream.wait_stream(cur)
+        w_free, dw_free = [[], []], [None, None]
+        ready = self._gather(0, [])
+        for s in range(self.k):
+            nxt = self._gather(s + 1, w_free[(s + 1) & 1]) if s + 1 < self.k else None
+            j = s & 1
+            cur.wait_event(ready)
+            ld2 = self.layouts[1].slices[s][5]
+            args = (dy, x, self.w_stage[0][j], self.w_stage[1][j], ld2, b1, z1_saved, M, self.hidden, self.ffn, self.k,
+                    self.act, s, dx)
+            if self._scatter_ok(s):
+                peers = []
+                for i, l in enumerate(self.layouts):
+                    off = l.slices[s][4]
+                    peers.append([int(t.data_ptr()) + off * t.element_size() for t in self.peer_grad_shards[i]])
+                B.osdp_zdp_mlp_bwd_slice(*args, None, None, 0, peers[0], peers[1], self.dw_dtype, flags, db1, db2, ws,
+                                         stream=cur, check=True)
+                done = torch.cuda.Event()
+                done.record(cur)
+            else:
+                if dw_free[j] is not None:
+                    cur.wait_event(dw_free[j])              # the collectives that read these buffers are done
+                B.osdp_zdp_mlp_bwd_slice(*args, self.dw_stage[0][j], self.dw_stage[1][j], ld2, None, None,
+                                         self.dw_dtype, flags, db1, db2, ws, stream=cur, check=True)
+                done = torch.cuda.Event()
+                done.record(cur)
+                with torch.cuda.stream(self.comm_stream):
+                    self.comm_stream.wait_event(done)
+                    for i, l in enumerate(self.layouts):
+                        _, _, _, n, off, _ = l.slices[s]
+                        self.comm.reduce_scatter_slice(self.grad_shard[i], off, n, self.dw_stage[i][j])
+                    dw_free[j] = torch.cuda.Event()
+                    dw_free[j].record(self.comm_stream)
+            w_free[j] = [done]
+            ready = nxt
+        cur.wait_stream(self.comm_stream)
+        return dx
