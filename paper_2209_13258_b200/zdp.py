@@ -102,7 +102,10 @@ class DistComm:
         """One buffer of `numel` elements per rank, all addressable from this GPU: this rank's own and the
         peer-mapped ones of the other ranks (torch symmetric memory over the group).  Returns the list indexed
         by rank; entry [self.rank] is local memory."""
+        import os
         import torch.distributed as dist
+        # plain peer mappings are all that is needed: no NVLink multicast object is bound to these buffers
+        os.environ.setdefault("TORCH_SYMM_MEM_DISABLE_MULTICAST", "1")
         try:
             import torch.distributed._symmetric_memory as symm
         except ImportError as e:   # pragma: no cover
