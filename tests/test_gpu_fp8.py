@@ -130,3 +130,17 @@ def test_fp8_argument_errors(P):
     assert f(x, w, 0, float("inf"), None, M, N, K, 1, 0, 0, out, None, ws) == 6
     assert f(x, None, 0, 1.0, None, M, N, K, 1, 0, 0, out, None, ws) == 1
     assert f(x, w, 0, 1.0, None, M, N, K, 1, 0, 0, out, None, ws) == 0
+
+
+@pytest.mark.parametrize("flags", [2, 8])
+@pytest.mark.parametrize("split", [0, 1])
+def test_fp8_summed_outputs_with_bf16_running_sum_and_paired_slices(P, flags, split):
+    """The carry modes of the bf16 path apply unchanged to fp8 operands (flag 2: bf16 running sum, 8: pairs)."""
+    M, N, K, k = 384, 1024, 1024, 4
+    c = inputs.linear_case_e4m3(M, N, K, w_std=0.05, w_offset=16, flat_pad=16, layer=8)
+    g = run_f8(P, c, k, split, act=0, flags=flags)
+    o = oracle_f8(c, 0, k, split)
+    tol = 3e-2 * (2 * k) ** 0.5 if flags == 2 else 3e-2     # the bf16 running sum rounds once more per slice
+    assert_close(to_f64(g["y"]), o["y"], "Y", abs_tol=tol)
+    assert_close(to_f64(g["dx"]), o["dx"], "dX", abs_tol=tol)
+    assert_close(to_f64(g["dw"]), o["dw"], "dW")

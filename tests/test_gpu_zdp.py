@@ -141,7 +141,7 @@ class EmulatedComm:
         return self.shared[key]
 
 
-def run_emulated_ranks(P, world, M, N, K, k, split, act, modes, fused=False):
+def run_emulated_ranks(P, world, M, N, K, k, split, act, modes, fused=False, dw_dtype=None):
     """Forward + backward of the slice loop for every emulated rank on its own token rows; returns the
     assembled Y, dX, sum over ranks of dW and db, and the first rank's layer."""
     from paper_2209_13258_b200.zdp import ZdpSplitLinear
@@ -152,7 +152,7 @@ def run_emulated_ranks(P, world, M, N, K, k, split, act, modes, fused=False):
     layers = []
     for r in range(world):
         layer = ZdpSplitLinear(N, K, k, split, act=act, comm=EmulatedComm(r, world, shared), slice_modes=modes,
-                               fused_scatter=fused)
+                               fused_scatter=fused, dw_dtype=P.DTYPE_FP32 if dw_dtype is None else dw_dtype)
         layer.load_full_weight(W)
         shared["param"][r] = layer.param_shard
         shared["grad_acc"][r] = torch.zeros(layer.grad_shard.numel(), dtype=torch.float64, device="cuda")
@@ -235,6 +235,15 @@ def test_reduce_scatter_fused_into_the_gemm_epilogue(P, world, split, case, mode
     assert [layer._scatter_ok(s) for s in range(k)] == expect
     if (M, N, K) == (512, 2048, 512) and modes is None:
         assert all(expect)          # this case really runs the fused path on every slice
+
+
+@pytest.mark.parametrize("world", [2, 4])
+def test_fused_scatter_with_bf16_gradients(P, world):
+    """bf16 gradient shards: the epilogue's reduce-add is a bf16 addition per rank's term."""
+    M, N, K, k = 512, 2048, 512, 4
+    c, y, dx, dW, db, layer = run_emulated_ranks(P, world, M, N, K, k, 0, 0, None, fused=True, dw_dtype=P.DTYPE_BF16)
+    assert all(layer._scatter_ok(s) for s in range(k)) and layer.grad_shard.dtype == torch.bfloat16
+    check_against_oracle(c, y, dx, dW, db, 0, k, 0)
 
 
 def test_fused_scatter_equals_staged_reduce_scatter_for_one_rank(P):
