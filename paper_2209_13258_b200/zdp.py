@@ -310,7 +310,7 @@ class ZdpSplitLinear:
                 g.free[b] = [self._mark(st)]
         if two:
             cur.wait_stream(self.side_stream)
-        self.comm_stream.wait_stream(cur)
+        cur.wait_stream(self.comm_stream)                   # join (also what a stream capture needs)
         return out
 
     def backward(self, dy, x, z_saved=None, dx=None, dbias=None, need_dx=True, accumulate=False):
@@ -524,7 +524,7 @@ class ZdpSplitMLP:
             ev.record(cur)
             free[s & 1] = [ev]
             ready = nxt
-        self.comm_stream.wait_stream(cur)
+        cur.wait_stream(self.comm_stream)                   # join (also what a stream capture needs)
         return out
 
     def backward(self, dy, x, z1_saved=None, b1=None, dx=None, db1=None, db2=None):

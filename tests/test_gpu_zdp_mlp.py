@@ -186,3 +186,52 @@ def test_mlp_slice_loop_over_emulated_ranks_matches_oracle(P, world, fused, shap
     # gathered weights: two slices' worth of each matrix
     per = sum(max(sl[3] for sl in lay.slices) for lay in layers[0].layouts) * world * 2
     assert st["weight_staging"] == (2 if k > 1 else 1) * per
+
+
+def test_sharded_loop_replays_from_a_cuda_graph(P):
+    """The whole loop (gathers on the communication stream, slice kernels, reduce-scatters or epilogue scatter)
+    is plain stream work with fork / join events: captured once on a one-rank NCCL group, the replay gives the
+    bits of the eager run."""
+    import torch.distributed as dist
+    from paper_2209_13258_b200.zdp import ZdpSplitMLP
+    if dist.is_initialized():
+        pytest.skip("a process group already exists in this process")
+    M, H, F, k = 512, 512, 2048, 4
+    dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29761", rank=0, world_size=1)
+    try:
+        c = inputs.mlp_case(M, H, F, w_std=0.05, bias_std=0.1, layer=9)
+        wf = to_dev(c["w_flat"])
+        x, dy, b1, b2 = to_dev(c["x"]), to_dev(c["dy"]), to_dev(c["b1"]), to_dev(c["b2"])
+        out = torch.empty(M, H, dtype=torch.bfloat16, device="cuda")
+        dx = torch.empty(M, H, dtype=torch.bfloat16, device="cuda")
+        z1 = torch.empty(M, F, dtype=torch.bfloat16, device="cuda")
+        for fused in (False, True):
+            try:
+                layer = ZdpSplitMLP(H, F, k, fused_scatter=fused)
+            except Exception as e:   # symmetric memory not available
+                print("skipping the fused form:", repr(e)[:200])
+                continue
+            layer.load_full_weights(wf[c["off_w1"]:c["off_w1"] + F * H].view(F, H),
+                                    wf[c["off_w2"]:c["off_w2"] + H * F].view(H, F))
+
+            def step():
+                layer.zero_grad()
+                layer.forward(x, b1, b2, out=out, z1_save=z1)
+                layer.backward(dy, x, z1_saved=z1, dx=dx)
+            step()
+            torch.cuda.synchronize()
+            ref = (out.clone(), dx.clone(), layer.grad_shard[0].clone(), layer.grad_shard[1].clone())
+            g, s = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+            with torch.cuda.stream(s):
+                with torch.cuda.graph(g, stream=s):
+                    step()
+            out.zero_(); dx.zero_()
+            for _ in range(2):
+                g.replay()
+            torch.cuda.synchronize()
+            for a, b in zip((out, dx, layer.grad_shard[0], layer.grad_shard[1]), ref):
+                assert torch.equal(bits(a), bits(b))
+            _, yo = oracle.mlp_fwd(c["x"], c["w1"], c["b1"], c["w2"], c["b2"], oracle.ACT_GELU_TANH, k)
+            assert_close(to_f64(out), yo, "Y")
+    finally:
+        dist.destroy_process_group()
