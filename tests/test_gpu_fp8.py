@@ -144,3 +144,22 @@ def test_fp8_summed_outputs_with_bf16_running_sum_and_paired_slices(P, flags, sp
     assert_close(to_f64(g["y"]), o["y"], "Y", abs_tol=tol)
     assert_close(to_f64(g["dx"]), o["dx"], "dX", abs_tol=tol)
     assert_close(to_f64(g["dw"]), o["dw"], "dW")
+
+
+@pytest.mark.parametrize("chunk", range(2))
+def test_fp8_random_shapes_against_oracle(P, chunk):
+    import random
+    rng = random.Random(5000 + chunk)
+    done = 0
+    while done < 10:
+        M = rng.choice([64, 130, 256, 300, 513, 1000])
+        N, K = 16 * rng.randint(1, 110), 16 * rng.randint(1, 110)
+        k, split = rng.choice([1, 2, 3, 4, 8]), rng.choice([0, 1])
+        rc, b, e = P.osdp_slice_range(N if split == 0 else K, k, 0)
+        if rc != 0 or (k > 1 and (e - b) % 16):
+            continue
+        act = rng.choice([0, 1])
+        c = inputs.linear_case_e4m3(M, N, K, w_std=0.05, bias_std=0.2, w_offset=16 * rng.randint(0, 9), flat_pad=16,
+                                    layer=70 + done)
+        compare(run_f8(P, c, k, split, act), oracle_f8(c, act, k, split), act)
+        done += 1

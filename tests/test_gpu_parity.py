@@ -565,3 +565,27 @@ def test_ragged_extents_on_the_wide_tile(P, k, split):
         g1 = run_linear(P, c, 1, split, dw_fp32=False)
         for name in (("y", "dw", "db") if split == 0 else ("dx", "dw", "db")):
             assert torch.equal(_bits(g[name]), _bits(g1[name])), name
+
+
+# ---------------------------------------------------------------------------------------------
+# seeded random MLP blocks: ragged extents, both GeLU forms, saved and recomputed pre-activation, both dW types
+
+@pytest.mark.parametrize("chunk", range(2))
+def test_random_mlp_blocks_against_oracle(P, chunk):
+    import random
+    rng = random.Random(4000 + chunk)
+    done = 0
+    while done < 8:
+        M = rng.choice([64, 130, 256, 300, 513, 1000])
+        H = 8 * rng.randint(1, 120)
+        F = 8 * rng.randint(2, 300)
+        k = rng.choice([1, 2, 3, 4, 5, 8])
+        if P.osdp_slice_range(F, k, 0)[0] != 0:
+            continue
+        act = rng.choice([1, 2])
+        c = inputs.mlp_case(M, H, F, w_std=0.05, bias_std=0.1, layer=30 + done)
+        g = run_mlp(P, c, k, act=act, dw_fp32=rng.random() < 0.5, recompute=rng.random() < 0.4)
+        _, y = oracle.mlp_fwd(c["x"], c["w1"], c["b1"], c["w2"], c["b2"], act, k)
+        grads = oracle.mlp_bwd(c["dy"], c["x"], c["w1"], c["b1"], c["w2"], act, k)
+        compare_mlp(g, (y,) + tuple(grads))
+        done += 1
