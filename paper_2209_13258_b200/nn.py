@@ -1,0 +1,115 @@
+"""torch.nn front end of the split linear layer: a module whose forward and backward are the library's
+calls (Section 3.3: the operator is processed as k sequential slices), so that a model can swap an
+``nn.Linear`` for it the way the paper's wrapper replaces FSDP's.
+
+Only argument marshalling and autograd bookkeeping happen here; every product, sum and activation runs in
+the CUDA kernels behind ``osdp_split_linear_fwd`` / ``osdp_split_linear_bwd``.  CUDA only: there is no CPU path.
+"""
+from __future__ import annotations
+
+import torch
+
+from . import binding as B
+
+
+class _SplitLinearFn(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, x, weight, bias, layer):
+        M = x.numel() // layer.in_features
+        x2 = x.reshape(M, layer.in_features)
+        if not x2.is_contiguous():
+            x2 = x2.contiguous()
+        N, K, k = layer.out_features, layer.in_features, layer.k_split
+        out = torch.empty(M, N, dtype=torch.bfloat16, device=x.device)
+        need_z = layer.act != B.ACT_NONE and (x.requires_grad or weight.requires_grad)
+        z = torch.empty(M, N, dtype=torch.bfloat16, device=x.device) if need_z else None
+        ws = layer._workspace(M)
+        # the parameter is read in place from the flat buffer it lives in (element offset of the view)
+        B.osdp_split_linear_fwd(x2, layer.flat, layer.w_offset, bias, M, N, K, k, layer.split_dim, layer.act, out, z, ws,
+                                check=True, flags=layer.flags)
+        ctx.layer, ctx.M = layer, M
+        ctx.save_for_backward(x2, z if z is not None else torch.empty(0, device=x.device), weight)
+        ctx.x_shape = x.shape
+        ctx.has_bias = bias is not None
+        return out.reshape(*x.shape[:-1], N)
+
+    @staticmethod
+    def backward(ctx, dy):
+        layer, M = ctx.layer, ctx.M
+        x2, z, weight = ctx.saved_tensors
+        N, K, k = layer.out_features, layer.in_features, layer.k_split
+        dy2 = dy.reshape(M, N)
+        if not dy2.is_contiguous():
+            dy2 = dy2.contiguous()
+        need_dx, need_dw, need_db = ctx.needs_input_grad[0], ctx.needs_input_grad[1], ctx.has_bias and ctx.needs_input_grad[2]
+        dx = torch.empty(M, K, dtype=torch.bfloat16, device=dy.device) if need_dx else None
+        dw = torch.empty(N, K, dtype=torch.bfloat16, device=dy.device) if need_dw else None
+        db = torch.empty(N, dtype=torch.float32, device=dy.device) if need_db else None
+        ws = layer._workspace(M)
+        B.osdp_split_linear_bwd(dy2, x2, layer.flat, layer.w_offset, z if z.numel() else None, M, N, K, k,
+                                layer.split_dim, layer.act, dx, dw, 0, B.DTYPE_BF16, layer.flags & B.FLAG_CARRY_BF16,
+                                db, ws, check=True)
+        return (dx.reshape(ctx.x_shape) if need_dx else None), dw, db, None
+
+
+class SplitLinear(torch.nn.Module):
+    """y = act(x W^T + b), computed as `k_split` sequential slices of W along `split_dim`
+    (SPLIT_OUT: rows of W, SPLIT_RED: columns of W and x).  bf16 activations and weight, fp32 bias.
+
+    `flat` (optional): a 1-D bf16 parameter buffer that already holds W [out_features, in_features] row-major
+    at element offset `w_offset` (a multiple of 8); the module's `weight` is then a view of it and nothing is
+    copied, which is how a flat-parameter wrapper stores its layers.  Without it the module owns its buffer.
+    """
+
+    def __init__(self, in_features, out_features, bias=True, k_split=1, split_dim=B.SPLIT_OUT, act=B.ACT_NONE,
+                 flags=0, flat=None, w_offset=0, device="cuda"):
+        super().__init__()
+        if in_features % 8 or out_features % 8:
+            raise ValueError("in_features and out_features must be multiples of 8")
+        self.in_features, self.out_features = int(in_features), int(out_features)
+        self.k_split, self.split_dim, self.act, self.flags = int(k_split), int(split_dim), int(act), int(flags)
+        n = self.in_features * self.out_features
+        if flat is None:
+            w = torch.empty(n, dtype=torch.bfloat16, device=device)
+            torch.nn.init.normal_(w, std=0.02)
+            self.flat_param = torch.nn.Parameter(w)
+            self._flat_owner, self.w_offset = None, 0
+        else:
+            if flat.dtype != torch.bfloat16 or flat.dim() != 1 or w_offset % 8 or w_offset + n > flat.numel():
+                raise ValueError("flat must be a 1-D bf16 buffer holding W at a multiple-of-8 element offset")
+            self.flat_param = None
+            self._flat_owner, self.w_offset = flat, int(w_offset)
+        self.bias = torch.nn.Parameter(torch.zeros(self.out_features, dtype=torch.float32, device=device)) if bias else None
+        self._ws = None
+        rc, _ = B.osdp_split_linear_workspace_bytes(1, self.out_features, self.in_features, self.k_split, self.split_dim,
+                                                    self.act, B.OP_LINEAR_FWD, self.flags)
+        if rc:
+            raise B.OsdpError(rc, "SplitLinear")
+
+    @property
+    def flat(self):
+        return self.flat_param if self._flat_owner is None else self._flat_owner
+
+    @property
+    def weight(self):
+        n = self.in_features * self.out_features
+        return self.flat[self.w_offset:self.w_offset + n].view(self.out_features, self.in_features)
+
+    def _workspace(self, M):
+        need = 0
+        for op in (B.OP_LINEAR_FWD, B.OP_LINEAR_BWD):
+            rc, n = B.osdp_split_linear_workspace_bytes(M, self.out_features, self.in_features, self.k_split,
+                                                        self.split_dim, self.act, op, self.flags)
+            if rc:
+                raise B.OsdpError(rc, "osdp_split_linear_workspace_bytes")
+            need = max(need, n)
+        if self._ws is None or self._ws.numel() < need or self._ws.device != self.flat.device:
+            self._ws = B.new_workspace(need, device=self.flat.device)
+        return self._ws
+
+    def forward(self, x):
+        if not x.is_cuda:
+            raise RuntimeError("SplitLinear runs on CUDA only: there is no CPU path")
+        if x.dtype != torch.bfloat16:
+            raise TypeError("SplitLinear takes bf16 activations")
+        return _SplitLinearFn.apply(x, self.weight, self.bias, self)
