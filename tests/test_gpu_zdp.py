@@ -307,7 +307,10 @@ def test_slice_loop_on_a_one_rank_nccl_group(P):
     if dist.is_initialized():
         pytest.skip("a process group already exists in this process")
     M, N, K, k = 512, 1024, 512, 4
-    dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29753", rank=0, world_size=1)
+    try:
+        dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29753", rank=0, world_size=1)
+    except Exception as e:   # no usable loopback / port on this machine: nothing of the library is at fault
+        pytest.skip("cannot form a one-rank NCCL group here: %r" % (e,))
     try:
         for split, modes in ((0, None), (1, None), (0, [0, 1, 1, 0]), (1, [1, 0, 0, 1])):
             c = inputs.linear_case(M, N, K, w_std=0.05, bias_std=0.2)

@@ -197,7 +197,10 @@ def test_sharded_loop_replays_from_a_cuda_graph(P):
     if dist.is_initialized():
         pytest.skip("a process group already exists in this process")
     M, H, F, k = 512, 512, 2048, 4
-    dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29761", rank=0, world_size=1)
+    try:
+        dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29761", rank=0, world_size=1)
+    except Exception as e:   # no usable loopback / port on this machine: nothing of the library is at fault
+        pytest.skip("cannot form a one-rank NCCL group here: %r" % (e,))
     try:
         c = inputs.mlp_case(M, H, F, w_std=0.05, bias_std=0.1, layer=9)
         wf = to_dev(c["w_flat"])
