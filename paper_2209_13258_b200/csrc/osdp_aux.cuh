@@ -25,8 +25,10 @@ __global__ void __launch_bounds__(256) act_backward_kernel(const __nv_bfloat16 *
     float a[8], b[8];
     unpack_bf16x8(*reinterpret_cast<const uint4 *>(dy + m * ld_dy + c0 + j), a);
     unpack_bf16x8(*reinterpret_cast<const uint4 *>(z + m * ld_z + c0 + j), b);
+    float grad[8];
+    gelu_grad_array(b, grad, act);
 #pragma unroll
-    for (int t = 0; t < 8; ++t) a[t] *= gelu_grad_f(b[t], act);
+    for (int t = 0; t < 8; ++t) a[t] *= grad[t];
     *reinterpret_cast<uint4 *>(g + m * ld_g + j) = pack_bf16x8(a);
   }
 }

@@ -460,10 +460,17 @@ __device__ __forceinline__ bool get_work(const GemmParams &p, int i, int bid, in
 // ------------------------------------------------------------------------------------------------
 // Epilogue arithmetic on 8 consecutive columns of one row
 
+// tanh on the special-function unit (tanh.approx.f32: about 2^-11 relative error, far inside the bf16
+// rounding of everything that is computed from it here); the library call costs tens of instructions.
+__device__ __forceinline__ float tanh_fast(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ float gelu_f(float x, int act) {
   if (act == ACT_GELU_TANH) {
     const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
-    return 0.5f * x * (1.0f + tanhf(u));
+    return 0.5f * x * (1.0f + tanh_fast(u));
   }
   if (act == ACT_GELU_ERF) return 0.5f * x * (1.0f + erff(x * 0.7071067811865476f));
   return x;
@@ -471,7 +478,7 @@ __device__ __forceinline__ float gelu_f(float x, int act) {
 __device__ __forceinline__ float gelu_grad_f(float x, int act) {
   if (act == ACT_GELU_TANH) {
     const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
-    const float t = tanhf(u);
+    const float t = tanh_fast(u);
     const float du = 0.7978845608028654f * (1.0f + 0.134145f * x * x);
     return 0.5f * (1.0f + t) + 0.5f * x * (1.0f - t * t) * du;
   }
@@ -486,7 +493,7 @@ __device__ __forceinline__ float gelu_grad_f(float x, int act) {
 __device__ __forceinline__ void gelu_grad_and_value_f(float x, int act, float &grad, float &value) {
   if (act == ACT_GELU_TANH) {
     const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
-    const float t = tanhf(u);
+    const float t = tanh_fast(u);
     const float du = 0.7978845608028654f * (1.0f + 0.134145f * x * x);
     const float h = 0.5f * (1.0f + t);
     grad = h + 0.5f * x * (1.0f - t * t) * du;
@@ -502,6 +509,45 @@ __device__ __forceinline__ void gelu_grad_and_value_f(float x, int act, float &g
   }
   grad = 1.0f;
   value = x;
+}
+// The same over small arrays, with the choice of the activation outside the element loop: the loop body is
+// then straight-line code whose N independent chains the compiler interleaves (with the choice inside, every
+// element was a branchy sequence executed one after another: about 180 cycles per element).
+template <int N>
+__device__ __forceinline__ void gelu_array(float (&f)[N], int act) {
+  if (act == ACT_GELU_TANH) {
+#pragma unroll
+    for (int j = 0; j < N; ++j) f[j] = gelu_f(f[j], ACT_GELU_TANH);
+  } else if (act == ACT_GELU_ERF) {
+#pragma unroll
+    for (int j = 0; j < N; ++j) f[j] = gelu_f(f[j], ACT_GELU_ERF);
+  }
+}
+template <int N>
+__device__ __forceinline__ void gelu_grad_array(const float (&x)[N], float (&grad)[N], int act) {
+  if (act == ACT_GELU_TANH) {
+#pragma unroll
+    for (int j = 0; j < N; ++j) grad[j] = gelu_grad_f(x[j], ACT_GELU_TANH);
+  } else if (act == ACT_GELU_ERF) {
+#pragma unroll
+    for (int j = 0; j < N; ++j) grad[j] = gelu_grad_f(x[j], ACT_GELU_ERF);
+  } else {
+#pragma unroll
+    for (int j = 0; j < N; ++j) grad[j] = 1.0f;
+  }
+}
+template <int N>
+__device__ __forceinline__ void gelu_grad_and_value_array(float (&x)[N], float (&grad)[N], int act) {   // x <- act(x)
+  if (act == ACT_GELU_TANH) {
+#pragma unroll
+    for (int j = 0; j < N; ++j) gelu_grad_and_value_f(x[j], ACT_GELU_TANH, grad[j], x[j]);
+  } else if (act == ACT_GELU_ERF) {
+#pragma unroll
+    for (int j = 0; j < N; ++j) gelu_grad_and_value_f(x[j], ACT_GELU_ERF, grad[j], x[j]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < N; ++j) grad[j] = 1.0f;
+  }
 }
 __device__ __forceinline__ void unpack_bf16x8(const uint4 &u, float (&f)[8]) {
   const uint32_t w[4] = {u.x, u.y, u.z, u.w};
@@ -542,20 +588,15 @@ __device__ __forceinline__ void epilogue8(const Epilogue &e, long long row, int 
     f[4] += b1.x; f[5] += b1.y; f[6] += b1.z; f[7] += b1.w;
   }
   if (e.z_save) *reinterpret_cast<uint4 *>(e.z_save + row * e.ld_z + col) = pack_bf16x8(f);
-  if (e.act != ACT_NONE) {
-#pragma unroll
-    for (int j = 0; j < 8; ++j) f[j] = gelu_f(f[j], e.act);
-  }
+  gelu_array(f, e.act);
   if (e.gz) {
     float z[8];
     unpack_bf16x8(*reinterpret_cast<const uint4 *>(e.gz + row * e.ld_gz + col), z);
+    float grad[8];
+    gelu_grad_and_value_array(z, grad, e.gz_act);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) f[j] *= gelu_grad_f(z[j], e.gz_act);
-    if (e.act_out) {
-#pragma unroll
-      for (int j = 0; j < 8; ++j) z[j] = gelu_f(z[j], e.gz_act);
-      *reinterpret_cast<uint4 *>(e.act_out + row * e.ld_act_out + col) = pack_bf16x8(z);
-    }
+    for (int j = 0; j < 8; ++j) f[j] *= grad[j];
+    if (e.act_out) *reinterpret_cast<uint4 *>(e.act_out + row * e.ld_act_out + col) = pack_bf16x8(z);
   }
   if (e.out_fp32) {
     float4 *o = reinterpret_cast<float4 *>(reinterpret_cast<float *>(e.out) + row * e.ld_out + col);
@@ -995,10 +1036,7 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
               float e8[8];
 #pragma unroll
               for (int j = 0; j < 8; ++j) e8[j] = f[g * 8 + j];
-              if (p.epi.act != ACT_NONE) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) e8[j] = gelu_f(e8[j], p.epi.act);
-              }
+              gelu_array(e8, p.epi.act);
               const uint4 pk = pack_bf16x8(e8);
               st_shared_v4(buf0 + (uint32_t)lane * 64u + (uint32_t)g * 16u, pk.x, pk.y, pk.z, pk.w);
             }
@@ -1054,13 +1092,9 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
               zb.x = __float_as_uint(zq[g].x); zb.y = __float_as_uint(zq[g].y);
               zb.z = __float_as_uint(zq[g].z); zb.w = __float_as_uint(zq[g].w);
               unpack_bf16x8(zb, z);
+              gelu_grad_and_value_array(z, f, p.epi.gz_act);   // f = act'(z), z = act(z)
 #pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                float grad, val;
-                gelu_grad_and_value_f(z[j], p.epi.gz_act, grad, val);
-                f[j] = __uint_as_float(v[g * 8 + j]) * grad;
-                z[j] = val;
-              }
+              for (int j = 0; j < 8; ++j) f[j] *= __uint_as_float(v[g * 8 + j]);
               const uint4 pk = pack_bf16x8(f);
               st_shared_v4(mine + (uint32_t)g * 16u, pk.x, pk.y, pk.z, pk.w);
               if (p.epi.act_out) {
@@ -1105,8 +1139,12 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
               }
             }
             if (p.epi.act != ACT_NONE) {
+              float a32[32];
 #pragma unroll
-              for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(gelu_f(__uint_as_float(v[j]), p.epi.act));
+              for (int j = 0; j < 32; ++j) a32[j] = __uint_as_float(v[j]);
+              gelu_array(a32, p.epi.act);
+#pragma unroll
+              for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(a32[j]);
             }
             const uint32_t dst = stage_begin();
 #pragma unroll
@@ -1168,10 +1206,7 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
               float f[8];
 #pragma unroll
               for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[g * 8 + j]);
-              if (p.epi.act != ACT_NONE) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) f[j] = gelu_f(f[j], p.epi.act);
-              }
+              gelu_array(f, p.epi.act);
               packed[g] = pack_bf16x8(f);
             }
             const uint32_t dst = stage_begin();
