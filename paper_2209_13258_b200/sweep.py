@@ -3,6 +3,8 @@
     python -m paper_2209_13258_b200.sweep case M N K k split        one fwd+bwd (twice), for profilers
     python -m paper_2209_13258_b200.sweep case-mlp M hidden ffn k   one MLP-block fwd+bwd (twice), for profilers
     python -m paper_2209_13258_b200.sweep case-f8 M N K k split     one fwd+bwd with fp8 operands (twice), for profilers
+    python -m paper_2209_13258_b200.sweep latency M N K k split     small operators: one fwd+bwd with a warm and with
+                                                                    a flushed L2 (median and best of 50 after 10 warm-ups)
     python -m paper_2209_13258_b200.sweep linear M N K [ks]         time vs slice granularity, both split dims
     python -m paper_2209_13258_b200.sweep linear-f8 M N K [ks]      the same with fp8 (e4m3) operands
     python -m paper_2209_13258_b200.sweep mlp M hidden ffn [ks]     MLP block split along ffn: time and staging
@@ -116,6 +118,49 @@ def run_case_mlp(M, H, F, k, flags=0):
                              check=True)
         torch.cuda.synchronize()
     print("device status", P.osdp_read_device_status(ws))
+
+
+def run_latency(M, N, K, k, split, iters=50, warm=10):
+    """Forward + backward of a small operator, timed one step at a time: with the operands left in L2 by the
+    previous step, and after the L2 has been flushed (a 256 MB buffer is overwritten between steps)."""
+    x, w, dy, out, dx, dw, db = _linear_tensors(M, N, K)
+    ws = P.new_workspace(_ws_linear(M, N, K, k, split))
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def step():
+        P.osdp_split_linear_fwd(x, w, 0, None, M, N, K, k, split, 0, out, None, ws, check=True)
+        P.osdp_split_linear_bwd(dy, x, w, 0, None, M, N, K, k, split, 0, dx, dw, 0, 0, 0, db, ws, check=True)
+    res = {}
+    for name, cold in (("warm_l2", False), ("cold_l2", True)):
+        ts = []
+        for i in range(warm + iters):
+            if cold:
+                flush.fill_(i & 255)
+            a = torch.cuda.Event(enable_timing=True)
+            b = torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record()
+            step()
+            b.record()
+            torch.cuda.synchronize()
+            if i >= warm:
+                ts.append(a.elapsed_time(b) * 1e3)
+        ts.sort()
+        res[name] = {"median_us": ts[len(ts) // 2], "best_us": ts[0]}
+    # several steps issued back to back (the host runs ahead): the device-side time of a step
+    torch.cuda.synchronize()
+    a = torch.cuda.Event(enable_timing=True)
+    b = torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(200):
+        step()
+    b.record()
+    torch.cuda.synchronize()
+    res["back_to_back_us"] = a.elapsed_time(b) * 1e3 / 200
+    res.update({"M": M, "N": N, "K": K, "k": k, "split": "out" if split == P.SPLIT_OUT else "red",
+                "flops": 3 * 2.0 * M * N * K, "bytes_min": 2 * 3 * (M * K + N * K + M * N)})
+    print(json.dumps(res), flush=True)
+    return res
 
 
 def sweep_linear(M, N, K, ks):
@@ -368,6 +413,8 @@ def main(argv):
         run_case_f8(*[int(v) for v in argv[2:7]])
     elif mode == "case-mlp":
         run_case_mlp(*[int(v) for v in argv[2:6]])
+    elif mode == "latency":
+        run_latency(*[int(v) for v in argv[2:7]])
     elif mode == "linear":
         sweep_linear(int(argv[2]), int(argv[3]), int(argv[4]), ks)
     elif mode == "linear-f8":

@@ -589,3 +589,37 @@ def test_random_mlp_blocks_against_oracle(P, chunk):
         grads = oracle.mlp_bwd(c["dy"], c["x"], c["w1"], c["b1"], c["w2"], act, k)
         compare_mlp(g, (y,) + tuple(grads))
         done += 1
+
+
+# ---------------------------------------------------------------------------------------------
+# the calls allocate nothing: staging is exactly the caller's workspace
+
+def test_calls_allocate_no_device_memory(P):
+    M, N, K, k = 512, 2048, 1024, 4
+    c = inputs.linear_case(M, N, K)
+    x, dy, wf = to_dev(c["x"]), to_dev(c["dy"]), to_dev(c["w_flat"])
+    out = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+    dx = torch.empty(M, K, dtype=torch.bfloat16, device="cuda")
+    dw = torch.empty(N * K, dtype=torch.float32, device="cuda")
+    db = torch.empty(N, dtype=torch.float32, device="cuda")
+    _, n1 = P.osdp_split_linear_workspace_bytes(M, N, K, k, 1, 0, P.OP_LINEAR_FWD)
+    _, n2 = P.osdp_split_linear_workspace_bytes(M, N, K, k, 0, 0, P.OP_LINEAR_BWD)
+    ws = P.new_workspace(max(n1, n2))
+
+    def step():
+        P.osdp_split_linear_fwd(x, wf, 0, None, M, N, K, k, 1, 0, out, None, ws, check=True)
+        P.osdp_split_linear_bwd(dy, x, wf, 0, None, M, N, K, k, 0, 0, dx, dw, 0, P.DTYPE_FP32, 0, db, ws, check=True)
+    step()                                   # first use: kernel attributes, internal streams
+    torch.cuda.synchronize()
+    torch.cuda.reset_peak_memory_stats()
+    before_alloc = torch.cuda.memory_allocated()
+    free_before, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert torch.cuda.max_memory_allocated() == before_alloc       # nothing through torch's allocator
+    assert free_after == free_before                                # and nothing behind its back
+    # the reported staging is what the call needs: one byte less is refused, nothing is launched
+    assert P.osdp_split_linear_bwd(dy, x, wf, 0, None, M, N, K, k, 0, 0, dx, dw, 0, P.DTYPE_FP32, 0, db,
+                                   (ws.data_ptr(), n2 - 1)) == 5
