@@ -5,6 +5,8 @@
     python -m paper_2209_13258_b200.sweep case-f8 M N K k split     one fwd+bwd with fp8 operands (twice), for profilers
     python -m paper_2209_13258_b200.sweep latency M N K k split     small operators: one fwd+bwd with a warm and with
                                                                     a flushed L2 (median and best of 50 after 10 warm-ups)
+    python -m paper_2209_13258_b200.sweep sustained M N K k split [seconds]   fwd+bwd back to back for >= `seconds`
+                                                                    (default 2): the power-limited figure
     python -m paper_2209_13258_b200.sweep linear M N K [ks]         time vs slice granularity, both split dims
     python -m paper_2209_13258_b200.sweep linear-f8 M N K [ks]      the same with fp8 (e4m3) operands
     python -m paper_2209_13258_b200.sweep mlp M hidden ffn [ks]     MLP block split along ffn: time and staging
@@ -161,6 +163,46 @@ def run_latency(M, N, K, k, split, iters=50, warm=10):
                 "flops": 3 * 2.0 * M * N * K, "bytes_min": 2 * 3 * (M * K + N * K + M * N)})
     print(json.dumps(res), flush=True)
     return res
+
+
+def run_sustained(M, N, K, k, split, seconds=2.0):
+    """Forward + backward issued back to back for at least `seconds`: the figure a long training loop sees
+    under the power cap, next to the median and best of 50 single steps."""
+    x, w, dy, out, dx, dw, db = _linear_tensors(M, N, K)
+    ws = P.new_workspace(_ws_linear(M, N, K, k, split))
+    flops = 3 * 2.0 * M * N * K
+
+    def step():
+        P.osdp_split_linear_fwd(x, w, 0, None, M, N, K, k, split, 0, out, None, ws, check=True)
+        P.osdp_split_linear_bwd(dy, x, w, 0, None, M, N, K, k, split, 0, dx, dw, 0, 0, 0, db, ws, check=True)
+    for _ in range(10):
+        step()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(50):
+        a = torch.cuda.Event(enable_timing=True)
+        b = torch.cuda.Event(enable_timing=True)
+        a.record()
+        step()
+        b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b))
+    ts.sort()
+    n = max(50, int(seconds * 1e3 / ts[len(ts) // 2]) + 1)
+    a = torch.cuda.Event(enable_timing=True)
+    b = torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(n):
+        step()
+    b.record()
+    torch.cuda.synchronize()
+    total = a.elapsed_time(b)
+    row = {"M": M, "N": N, "K": K, "k": k, "split": "out" if split == P.SPLIT_OUT else "red",
+           "median_ms": ts[len(ts) // 2], "best_ms": ts[0], "median_tflops": flops / ts[len(ts) // 2] / 1e9,
+           "best_tflops": flops / ts[0] / 1e9, "sustained_steps": n, "sustained_seconds": total / 1e3,
+           "sustained_ms": total / n, "sustained_tflops": flops * n / total / 1e9}
+    print(json.dumps(row), flush=True)
+    return row
 
 
 def sweep_linear(M, N, K, ks):
@@ -413,6 +455,8 @@ def main(argv):
         run_case_f8(*[int(v) for v in argv[2:7]])
     elif mode == "case-mlp":
         run_case_mlp(*[int(v) for v in argv[2:6]])
+    elif mode == "sustained":
+        run_sustained(*[int(v) for v in argv[2:7]], seconds=float(argv[7]) if len(argv) > 7 else 2.0)
     elif mode == "latency":
         run_latency(*[int(v) for v in argv[2:7]])
     elif mode == "linear":
