@@ -483,6 +483,17 @@ def run_ours(args):
                 "peak_kind": "%s, %s" % (peak_kind, pk["source"]),
                 "frac_of_burst_peak": achieved / pk["bf16_tflops"],
                 "per_launch_ms": per_kernel_ms, "traffic": NCU_TRAFFIC_BYTES.get((dom, k, args.split))}
+    # Both floors of that launch: tensor time of its flops, and HBM time of its algorithmic bytes (operands once per
+    # slice that re-reads them, plus 2 x 4 bytes x (k - 1) per element of a summed output for the fp32 carry).
+    carried = (dom == "dx" and args.split == "out") or (dom == "fwd" and args.split == "red")
+    alg_bytes = {"fwd": 2.0 * ((k if args.split == "out" else 1) * M * K + N * K + M * N),
+                 "dx": 2.0 * ((k if args.split == "red" else 1) * M * N + N * K + M * K),
+                 "dw": 2.0 * (M * N + N * K + M * K + (k - 1) * (M * K if args.split == "out" else M * N))}[dom]
+    if carried:
+        alg_bytes += 8.0 * (k - 1) * (M * K if dom == "dx" else M * N)
+    roofline["algorithmic_bytes"] = alg_bytes
+    roofline["tensor_floor_ms"] = gemm_flops / (pk[peak_kind] * 1e12) * 1e3
+    roofline["hbm_floor_ms"] = alg_bytes / (pk["hbm_gbs"] * 1e9) * 1e3
 
     # ---- CPU baseline: the oracle, as it stands, on a bounded sample of the same workload
     cpu = None
