@@ -231,8 +231,9 @@ int osdp_zdp_linear_bwd_slice(const void *dy, const void *x, const void *w_slice
  * where rank q keeps its part of this slice (shard_elems elements, the layout of osdp_zdp_shard_layout) -- this
  * rank's own memory for q = rank, peer-mapped memory of the other GPUs otherwise (plain peer stores /
  * reductions over NVLink; no multicast).  Every rank's call adds its term, so the buffers hold the sum over
- * ranks once all ranks have finished the slice: zero them before the step and synchronise the ranks before
- * reading them.  Needs the slice's row count (len R_s under OUT, N under RED) to be a multiple of 32 * world,
+ * ranks once all ranks have finished the slice: every rank zeroes its buffer, the ranks synchronise (nobody
+ * may add into a buffer its owner has not zeroed yet), the calls run, the ranks synchronise again, and only
+ * then are the buffers read.  Needs the slice's row count (len R_s under OUT, N under RED) to be a multiple of 32 * world,
  * else OSDP_ERR_UNSUPPORTED (use the staging form and a collective for that slice).  OSDP_FLAG_ACCUMULATE_DW
  * is not accepted (the scatter always adds).  Everything else as osdp_zdp_linear_bwd_slice. */
 int osdp_zdp_linear_bwd_slice_scatter(const void *dy, const void *x, const void *w_slice, int64_t ld_w,

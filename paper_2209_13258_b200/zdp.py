@@ -154,8 +154,9 @@ class ZdpSplitLinear:
             total += self.layout.slices[s][3]
         self.param_shard = torch.zeros(max(total, 8), dtype=torch.bfloat16, device=self.device)
         # fused_scatter: the backward GEMM's epilogue reduce-adds each slice's dW straight into the owners'
-        # gradient shards, which therefore have to be addressable from every rank (comm.peer_buffers); the
-        # caller zeroes them (zero_grad) before the step and the ranks meet (comm.barrier) before reading them.
+        # gradient shards, which therefore have to be addressable from every rank (comm.peer_buffers).  A step
+        # is then: zero_grad() on every rank; comm.barrier() (no rank may add into a shard that its owner has
+        # not zeroed yet); backward(); comm.barrier() (every rank's terms have arrived); read grad_shard.
         self.fused_scatter = bool(fused_scatter)
         if self.fused_scatter:
             self.peer_grad_shards = self.comm.peer_buffers(max(total, 8), gdt, self.device)
