@@ -76,3 +76,37 @@ def expand_slices(op, k, overhead=0.0):
     the measured relative time overhead of running the operator split k ways."""
     model, act, extra, S, gamma = op
     return [(model / k, act / k, extra / k, S / k, gamma * (1.0 + overhead) / k) for _ in range(k)]
+
+
+def search_granularity(ops, candidates, world, alpha, beta, mem_limit, max_batch):
+    """Section 3.3, last paragraph, with the slice granularity of every operator left free as well (the
+    paper takes it as given): candidates[i] lists the (k, overhead) pairs allowed for operator i.  For
+    each batch size of Algorithm 1 every combination of granularities is tried, each operator replaced by
+    its slices (expand_slices) and the slices planned one by one by the exhaustive inner loop.  Returns
+    (ks, dp_counts, b, time per sample, candidates_per_batch): ks[i] the granularity chosen for operator i,
+    dp_counts[i] how many of its slices run in DP; (None, None, 0, inf, []) if nothing fits at b = 1.
+    Tiny instances only: the work is prod_i |candidates[i]| * 2^(sum of k)."""
+    per_batch = []
+    for b in range(1, max_batch + 1):
+        best = None
+        for choice in itertools.product(*candidates):
+            expanded, owner = [], []
+            for i, (op, (k, overhead)) in enumerate(zip(ops, choice)):
+                expanded += expand_slices(op, k, overhead)
+                owner += [i] * k
+            t, modes = best_plan_for_batch(expanded, b, world, alpha, beta, mem_limit)
+            if modes is not None and (best is None or t < best[0]):
+                dp = [0] * len(ops)
+                for i, p in zip(owner, modes):
+                    dp[i] += 1 if p == DP else 0
+                best = (t, [k for k, _ in choice], dp)
+        if best is None:
+            break
+        per_batch.append((best[0] / b, best[1], best[2], b))
+    if not per_batch:
+        return None, None, 0, float("inf"), []
+    top = per_batch[0]
+    for c in per_batch[1:]:
+        if c[0] < top[0]:
+            top = c
+    return top[1], top[2], top[3], top[0], per_batch

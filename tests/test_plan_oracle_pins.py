@@ -112,3 +112,52 @@ def test_expand_slices_preserves_totals():
     assert OP.search([op], world, alpha, beta, limit, 1)[0] == (1,)
     assert sorted(OP.search(OP.expand_slices(op, 4), world, alpha, beta, limit, 1)[0]) == [0, 0, 0, 1]
     assert t_sliced < t_whole
+
+
+# ---- granularity left free (Section 3.3, last paragraph)
+
+def _granularity_golden():
+    rows = []
+    with open(os.path.join(os.path.dirname(__file__), "golden", "plan_granularity_example.txt")) as f:
+        for line in f:
+            if line.startswith("best"):
+                v = line.split()
+                rows.append((float(v[1]), int(v[2]), int(v[3]), int(v[4]), float(v[5])))
+    return rows
+
+
+def test_hand_worked_granularity_instance():
+    op = (8.0, 3.0, 0.0, 4.0, 10.0)
+    rows = _granularity_golden()
+    assert len(rows) == 2
+    for alpha, k, dp, b, t in rows:
+        ks, dps, bb, tt, _ = OP.search_granularity([op], [[(1, 0.0), (2, 0.02)]], 2, alpha, 1.0, 9.5, 8)
+        assert (ks, dps, bb) == ([k], [dp], b)
+        assert tt == pytest.approx(t, rel=1e-13)
+
+
+def test_one_whole_candidate_reduces_to_the_plain_search():
+    rng = random.Random(77)
+    for _ in range(20):
+        n = rng.randint(1, 6)
+        ops = [(rng.uniform(0, 100), rng.uniform(0, 9), rng.uniform(0, 3), rng.uniform(0, 50), rng.uniform(0.1, 2))
+               for _ in range(n)]
+        world, alpha, beta = rng.choice([2, 4, 8]), rng.uniform(0, 1), rng.uniform(0, 0.3)
+        limit = rng.uniform(0.5, 1.2) * OP.memory_cost(ops, [0] * n, 2, world)
+        modes, b, t, _ = OP.search(ops, world, alpha, beta, limit, 6)
+        ks, dps, b2, t2, _ = OP.search_granularity(ops, [[(1, 0.0)]] * n, world, alpha, beta, limit, 6)
+        assert b2 == b and t2 == t
+        if b:
+            assert ks == [1] * n and dps == [1 - m for m in modes]
+
+
+def test_more_candidates_never_cost_more_and_latency_decides():
+    op = (40.0, 2.0, 1.0, 20.0, 3.0)
+    ops = [op, op]
+    limit = OP.memory_cost(ops, [0, 1], 2, 4)            # room for one of the two in DP at b = 2, not both
+    for alpha in (0.0, 0.5, 5.0):
+        whole = OP.search_granularity(ops, [[(1, 0.0)]] * 2, 4, alpha, 0.1, limit, 3)
+        free = OP.search_granularity(ops, [[(1, 0.0), (2, 0.0), (4, 0.0)]] * 2, 4, alpha, 0.1, limit, 3)
+        assert free[3] <= whole[3] * (1 + 1e-15)
+    # without latency, finer slices cost nothing; with a large latency per step every extra slice is a loss
+    assert OP.search_granularity(ops, [[(1, 0.0), (4, 0.0)]] * 2, 4, 50.0, 0.1, limit, 3)[0] == [1, 1]
