@@ -366,6 +366,29 @@ int osdp_plan_search(const double *ops, int n, int world, double alpha, double b
  * split k ways (> -1). */
 int osdp_plan_expand_slices(const double *op, int k, double overhead, double *slices);
 
+/* osdp_plan_search with the slice granularity of every operator left free as well (the paper takes it as
+ * given and leaves its automatic choice open).  Operator i may be cut into cand_k[a] slices at a measured
+ * relative overhead cand_overhead[a] (> -1), a in [cand_begin[i], cand_begin[i+1]); cand_begin has n + 1
+ * entries, cand_begin[0] = 0, every operator at least one candidate.  The slices of an operator are priced
+ * like osdp_plan_expand_slices prices them and planned one by one; since they are identical only their
+ * number in DP matters.  Returns, for the batch size of least time per sample, k_out[i] (the granularity
+ * chosen for operator i) and dp_slices[i] (how many of its slices run in DP: the first dp_slices[i], say;
+ * the others run in ZDP).
+ * surge_factor (>= 0): Section 3.3 names the gathered parameters of a ZDP operator as the memory surge
+ * that splitting cuts from size(operator) to size(operator) / granularity.  The sums of Section 3.1 have
+ * no term for it, so it is counted here on top of them: a plan fits if
+ *     sum_i M_i + surge_factor * max over operators with a ZDP slice of (S_i / k_i)  <=  mem_limit,
+ * e.g. 2 for a double-buffered gather, 0 for the paper's memory model as it stands.
+ * Batch loop, *batch, *time_per_sample, max_nodes, nodes_visited and the return value as for
+ * osdp_plan_search; exact unless OSDP_ERR_SEARCH_LIMIT is returned (a multiple-choice knapsack per value
+ * of the largest gathered slice, solved depth first with the memory and best-so-far prunings and a
+ * fractional relaxation as bound). */
+int osdp_plan_search_granularity(const double *ops, int n, const int *cand_begin, const int *cand_k,
+                                 const double *cand_overhead, int world, double alpha, double beta,
+                                 double mem_limit, double surge_factor, int max_batch, int64_t max_nodes,
+                                 int *k_out, int *dp_slices, int *batch, double *time_per_sample,
+                                 int64_t *nodes_visited);
+
 #ifdef __cplusplus
 }
 #endif

@@ -78,12 +78,18 @@ def expand_slices(op, k, overhead=0.0):
     return [(model / k, act / k, extra / k, S / k, gamma * (1.0 + overhead) / k) for _ in range(k)]
 
 
-def search_granularity(ops, candidates, world, alpha, beta, mem_limit, max_batch):
+def search_granularity(ops, candidates, world, alpha, beta, mem_limit, max_batch, surge_factor=0.0):
     """Section 3.3, last paragraph, with the slice granularity of every operator left free as well (the
     paper takes it as given): candidates[i] lists the (k, overhead) pairs allowed for operator i.  For
     each batch size of Algorithm 1 every combination of granularities is tried, each operator replaced by
-    its slices (expand_slices) and the slices planned one by one by the exhaustive inner loop.  Returns
-    (ks, dp_counts, b, time per sample, candidates_per_batch): ks[i] the granularity chosen for operator i,
+    its slices (expand_slices) and every assignment of DP / ZDP to the slices priced.
+
+    surge_factor: Section 3.3 describes the gathered parameters of a ZDP operator as a memory surge that
+    splitting cuts from size(operator) to size(operator) / granularity; the sums of Section 3.1 have no
+    term for it.  Here the largest gathered slice S_i / k_i among the operators with at least one ZDP
+    slice, times surge_factor, is added to the memory a plan needs (0: the paper's model as it stands).
+
+    Returns (ks, dp_counts, b, time per sample, per_batch): ks[i] the granularity chosen for operator i,
     dp_counts[i] how many of its slices run in DP; (None, None, 0, inf, []) if nothing fits at b = 1.
     Tiny instances only: the work is prod_i |candidates[i]| * 2^(sum of k)."""
     per_batch = []
@@ -94,12 +100,18 @@ def search_granularity(ops, candidates, world, alpha, beta, mem_limit, max_batch
             for i, (op, (k, overhead)) in enumerate(zip(ops, choice)):
                 expanded += expand_slices(op, k, overhead)
                 owner += [i] * k
-            t, modes = best_plan_for_batch(expanded, b, world, alpha, beta, mem_limit)
-            if modes is not None and (best is None or t < best[0]):
-                dp = [0] * len(ops)
+            for modes in itertools.product((DP, ZDP), repeat=len(expanded)):
+                surge = 0.0
                 for i, p in zip(owner, modes):
-                    dp[i] += 1 if p == DP else 0
-                best = (t, [k for k, _ in choice], dp)
+                    if p == ZDP:
+                        surge = max(surge, ops[i][3] / choice[i][0])
+                m = memory_cost(expanded, modes, b, world) + surge_factor * surge
+                t = time_cost(expanded, modes, b, world, alpha, beta)
+                if m <= mem_limit and (best is None or t < best[0]):
+                    dp = [0] * len(ops)
+                    for i, p in zip(owner, modes):
+                        dp[i] += 1 if p == DP else 0
+                    best = (t, [k for k, _ in choice], dp)
         if best is None:
             break
         per_batch.append((best[0] / b, best[1], best[2], b))

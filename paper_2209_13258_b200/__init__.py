@@ -12,7 +12,7 @@ from .binding import (  # noqa: F401
     osdp_split_linear_workspace_bytes, osdp_split_mlp_bwd, osdp_split_mlp_fwd, osdp_status_string,
     osdp_version, new_workspace, osdp_bias_grad_noalloc, osdp_debug_wait_probe, osdp_suggest_granularity,
     osdp_zdp_shard_layout, osdp_zdp_linear_fwd_slice, osdp_zdp_linear_bwd_slice,
-    osdp_plan_cost, osdp_plan_search, osdp_plan_expand_slices,
+    osdp_plan_cost, osdp_plan_search, osdp_plan_expand_slices, osdp_plan_search_granularity,
     osdp_split_linear_fwd_f8, osdp_split_linear_bwd_f8, osdp_zdp_linear_bwd_slice_scatter,
     osdp_zdp_mlp_fwd_slice, osdp_zdp_mlp_bwd_slice,
 )

@@ -24,7 +24,7 @@ EXPORTS = [
     "osdp_split_linear_bwd", "osdp_split_linear_bwd_slice", "osdp_split_mlp_fwd", "osdp_split_mlp_bwd",
     "osdp_read_device_status", "osdp_bias_grad_noalloc", "osdp_debug_wait_probe", "osdp_suggest_granularity",
     "osdp_zdp_shard_layout", "osdp_zdp_linear_fwd_slice", "osdp_zdp_linear_bwd_slice",
-    "osdp_plan_cost", "osdp_plan_search", "osdp_plan_expand_slices",
+    "osdp_plan_cost", "osdp_plan_search", "osdp_plan_expand_slices", "osdp_plan_search_granularity",
     "osdp_split_linear_fwd_f8", "osdp_split_linear_bwd_f8", "osdp_zdp_linear_bwd_slice_scatter",
     "osdp_zdp_mlp_fwd_slice", "osdp_zdp_mlp_bwd_slice",
 ]
@@ -83,6 +83,9 @@ def lib():
         L.osdp_plan_cost.argtypes = [pd, ci, ci, dbl, dbl, pu8, ci, pd, pd]
         L.osdp_plan_search.argtypes = [pd, ci, ci, dbl, dbl, dbl, ci, i64, pu8, ctypes.POINTER(ci), pd, p64]
         L.osdp_plan_expand_slices.argtypes = [pd, ci, dbl, pd]
+        pci = ctypes.POINTER(ci)
+        L.osdp_plan_search_granularity.argtypes = [pd, ci, pci, pci, pd, ci, dbl, dbl, dbl, dbl, ci, i64, pci, pci, pci, pd,
+                                                   p64]
         f32 = ctypes.c_float
         pvp = ctypes.POINTER(vp)
         L.osdp_zdp_mlp_fwd_slice.argtypes = [vp, vp, vp, i64, vp, vp, i64, i64, i64, ci, ci, ci, ci, vp, vp, vp, sz, vp]
@@ -314,6 +317,31 @@ def osdp_plan_expand_slices(op, k, overhead=0.0):
     out = (ctypes.c_double * (5 * max(int(k), 1)))()
     rc = lib().osdp_plan_expand_slices((ctypes.c_double * 5)(*[float(v) for v in op]), int(k), float(overhead), out)
     return rc, [tuple(out[5 * s:5 * s + 5]) for s in range(max(int(k), 1))] if rc == 0 else []
+
+
+def osdp_plan_search_granularity(ops, candidates, world, alpha, beta, mem_limit, max_batch, max_nodes=0,
+                                 surge_factor=0.0):
+    """candidates[i] = [(k, overhead), ...] allowed for operator i.  Returns (status, ks, dp_slices, batch,
+    time_per_sample, nodes_visited): ks[i] slices for operator i, the first dp_slices[i] of them in DP.
+    surge_factor * (largest gathered slice among operators with a ZDP slice) counts against mem_limit."""
+    n = len(ops)
+    if len(candidates) != n:
+        raise ValueError("one candidate list per operator")
+    begin, ks, ov = [0], [], []
+    for c in candidates:
+        for k, o in c:
+            ks.append(int(k))
+            ov.append(float(o))
+        begin.append(len(ks))
+    ci = ctypes.c_int
+    k_out, dp = (ci * n)(), (ci * n)()
+    b, t, nodes = ci(), ctypes.c_double(), ctypes.c_int64()
+    rc = lib().osdp_plan_search_granularity(_ops_array(ops), n, (ci * len(begin))(*begin), (ci * max(len(ks), 1))(*ks),
+                                            (ctypes.c_double * max(len(ov), 1))(*ov), int(world), float(alpha),
+                                            float(beta), float(mem_limit), float(surge_factor), int(max_batch),
+                                            int(max_nodes), k_out, dp,
+                                            ctypes.byref(b), ctypes.byref(t), ctypes.byref(nodes))
+    return rc, list(k_out), list(dp), b.value, t.value, nodes.value
 
 
 def osdp_split_linear_fwd_f8(x8, w8_flat, w_offset, scale, bias, M, N, K, k_split, split_dim, act, out, z_save, ws,

@@ -151,6 +151,110 @@ bool solve_batch(const Op *ops, int n, int world, double alpha, double beta, dou
   return true;
 }
 
+
+// ---- granularity left free: every operator picks one of its allowed granularities and how many of its
+// slices run in DP (Section 3.3, last paragraph).  For one batch size this is a multiple-choice knapsack:
+// one option (k, j) per operator, least total time within the memory limit.
+
+struct Option { double mem, time; int k, dp; };
+
+// Memory and time of an operator cut k ways with its first j slices in DP, summed slice by slice.
+void sliced_cost(const Op &o, int k, double overhead, int j, int world, double alpha, double beta, int b, double *mem,
+                 double *time) {
+  const Op s{o.model / (double)k, o.act / (double)k, o.extra / (double)k, o.S / (double)k,
+             o.gamma * (1.0 + overhead) / (double)k};
+  double m = 0.0, t = 0.0;
+  for (int i = 0; i < k; ++i) {
+    const bool zdp = i >= j;
+    m += (zdp ? s.model / (double)world : s.model) + (double)b * s.act + s.extra;
+    t += (zdp ? 3.0 : 2.0) * collective_cost(s, world, alpha, beta) + (double)b * s.gamma;
+  }
+  *mem = m;
+  *time = t;
+}
+
+struct Choice {
+  std::vector<Option> opts;   // undominated, memory ascending, time strictly descending
+  std::vector<int> hull;      // indices into opts: lower convex hull, for the relaxation
+};
+
+struct Segment { double dm, dt; int pos; };   // one hull step of the operator at visiting position pos
+
+struct GranSearch {
+  std::vector<const Choice *> ch;        // per visiting position
+  std::vector<char> same_as_prev;        // identical operator at pos - 1: options in non-decreasing index order
+  std::vector<double> min_mem, min_time; // suffix sums over the least-memory options
+  std::vector<Segment> segs;             // all hull steps, steepest time saving per byte first
+  std::vector<int> pick, best_pick;
+  double best;
+  int64_t nodes, max_nodes;
+  bool cut_short;
+
+  // least time of positions pos.. within cap if options could be mixed fractionally; +inf if nothing fits
+  double bound(int pos, double cap) const {
+    if (min_mem[pos] > cap) return std::numeric_limits<double>::infinity();
+    double room = cap - min_mem[pos], t = min_time[pos];
+    for (const Segment &g : segs) {
+      if (g.pos < pos) continue;
+      if (g.dm <= room) { room -= g.dm; t += g.dt; }
+      else { t += g.dt * (room / g.dm); break; }
+    }
+    return t;
+  }
+
+  void dfs(int pos, double cap, double t) {
+    if (cut_short) return;
+    if (++nodes > max_nodes) { cut_short = true; return; }
+    const int n = (int)ch.size();
+    if (pos == n) {
+      if (t < best) { best = t; best_pick = pick; }
+      return;
+    }
+    const double lb = t + bound(pos, cap);
+    if (!(lb * (1.0 - 1e-12) < best)) return;                      // pruning 2 (time), relaxed
+    const std::vector<Option> &o = ch[pos]->opts;
+    const int lo = same_as_prev[pos] ? pick[pos - 1] : 0;
+    for (int i = (int)o.size() - 1; i >= lo; --i) {                // fastest (largest) option first
+      if (o[i].mem + min_mem[pos + 1] > cap) continue;             // pruning 1 (memory)
+      pick[pos] = i;
+      dfs(pos + 1, cap - o[i].mem, t + o[i].time);
+      if (cut_short) return;
+    }
+  }
+};
+
+// Options of one operator whose gathered slice, if any slice is in ZDP, is at most `tau` bytes.
+void build_choice(const Op &op, const int *ks, const double *ovh, int ncand, int world, double alpha, double beta, int b,
+                  double tau, Choice *c) {
+  std::vector<Option> all;
+  for (int a = 0; a < ncand; ++a)
+    for (int j = 0; j <= ks[a]; ++j) {
+      if (j < ks[a] && op.S / (double)ks[a] > tau) continue;
+      Option o{0.0, 0.0, ks[a], j};
+      sliced_cost(op, ks[a], ovh[a], j, world, alpha, beta, b, &o.mem, &o.time);
+      all.push_back(o);
+    }
+  std::stable_sort(all.begin(), all.end(), [](const Option &x, const Option &y) {
+    return x.mem != y.mem ? x.mem < y.mem : x.time < y.time;
+  });
+  c->opts.clear();
+  for (const Option &o : all)
+    if (c->opts.empty() || o.time < c->opts.back().time) {
+      if (!c->opts.empty() && o.mem == c->opts.back().mem) continue;
+      c->opts.push_back(o);
+    }
+  c->hull.clear();
+  for (int i = 0; i < (int)c->opts.size(); ++i) {
+    while (c->hull.size() >= 2) {
+      const Option &p = c->opts[c->hull[c->hull.size() - 2]], &q = c->opts[c->hull.back()], &r = c->opts[i];
+      // q lies on or above the chord p-r: drop it
+      if ((q.time - p.time) * (r.mem - p.mem) >= (r.time - p.time) * (q.mem - p.mem)) c->hull.pop_back();
+      else break;
+    }
+    c->hull.push_back(i);
+  }
+}
+
 int check_inputs(const double *ops, int n, int world, double alpha, double beta) {
   if (!ops) return OSDP_ERR_NULL_POINTER;
   if (n < 1 || n > 16384 || world < 1) return OSDP_ERR_BAD_SHAPE;
@@ -215,6 +319,141 @@ int osdp_plan_expand_slices(const double *op, int k, double overhead, double *sl
     slices[5 * s + 4] = op[4] * (1.0 + overhead) / (double)k;
   }
   return OSDP_OK;
+}
+
+int osdp_plan_search_granularity(const double *ops, int n, const int *cand_begin, const int *cand_k,
+                                 const double *cand_overhead, int world, double alpha, double beta, double mem_limit,
+                                 double surge_factor, int max_batch, int64_t max_nodes, int *k_out, int *dp_slices,
+                                 int *batch, double *time_per_sample, int64_t *nodes_visited) {
+  int rc = check_inputs(ops, n, world, alpha, beta);
+  if (rc) return rc;
+  if (!cand_begin || !cand_k || !cand_overhead || !k_out || !dp_slices || !batch || !time_per_sample)
+    return OSDP_ERR_NULL_POINTER;
+  if (max_batch < 1 || !(mem_limit >= 0.0) || cand_begin[0] != 0) return OSDP_ERR_BAD_SHAPE;
+  if (!(surge_factor >= 0.0) || !std::isfinite(surge_factor)) return OSDP_ERR_BAD_SHAPE;
+  for (int i = 0; i < n; ++i) {
+    if (cand_begin[i + 1] <= cand_begin[i]) return OSDP_ERR_BAD_SHAPE;     // every operator needs a candidate
+    for (int a = cand_begin[i]; a < cand_begin[i + 1]; ++a) {
+      if (cand_k[a] < 1 || cand_k[a] > OSDP_MAX_SPLIT) return OSDP_ERR_BAD_SPLIT;
+      if (!(cand_overhead[a] > -1.0) || !std::isfinite(cand_overhead[a])) return OSDP_ERR_BAD_SHAPE;
+    }
+  }
+  if (max_nodes <= 0) max_nodes = (int64_t)200 * 1000 * 1000;
+  const Op *o = reinterpret_cast<const Op *>(ops);
+
+  // visiting order: identical operators (same five figures, same candidates) next to each other
+  auto same = [&](int a, int b) {
+    if (std::memcmp(&o[a], &o[b], sizeof(Op)) != 0) return false;
+    const int na = cand_begin[a + 1] - cand_begin[a];
+    if (na != cand_begin[b + 1] - cand_begin[b]) return false;
+    for (int j = 0; j < na; ++j)
+      if (cand_k[cand_begin[a] + j] != cand_k[cand_begin[b] + j] ||
+          cand_overhead[cand_begin[a] + j] != cand_overhead[cand_begin[b] + j]) return false;
+    return true;
+  };
+  std::vector<int> cls((size_t)n), reps;             // class of each operator, representative of each class
+  for (int i = 0; i < n; ++i) {
+    int c = -1;
+    for (size_t r = 0; r < reps.size() && c < 0; ++r)
+      if (same(i, reps[r])) c = (int)r;
+    if (c < 0) { c = (int)reps.size(); reps.push_back(i); }
+    cls[i] = c;
+  }
+  std::vector<int> order((size_t)n);
+  for (int i = 0; i < n; ++i) order[i] = i;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return cls[a] < cls[b]; });
+
+  // The gathered slice of a ZDP operator is transient memory on top of the sums of Section 3.1: the largest
+  // one, times surge_factor, counts against the limit.  A maximum does not fit a knapsack, so the search
+  // runs once per possible value tau of that maximum, with only the options whose gathered slice is at
+  // most tau and with the limit lowered by surge_factor * tau; the best over all tau is the optimum.
+  std::vector<double> taus;
+  if (surge_factor > 0.0) {
+    taus.push_back(0.0);
+    for (int i = 0; i < n; ++i)
+      for (int a = cand_begin[i]; a < cand_begin[i + 1]; ++a) taus.push_back(o[i].S / (double)cand_k[a]);
+    std::sort(taus.begin(), taus.end());
+    taus.erase(std::unique(taus.begin(), taus.end()), taus.end());
+  } else {
+    taus.push_back(std::numeric_limits<double>::infinity());
+  }
+
+  double best = std::numeric_limits<double>::infinity();
+  int best_b = 0;
+  int64_t nodes = 0;
+  bool any_cut = false;
+  std::vector<Choice> choice(reps.size());
+  for (int b = 1; b <= max_batch; ++b) {             // Algorithm 1: grow the batch until nothing fits
+    double best_t = std::numeric_limits<double>::infinity();   // least time at this batch size, over all tau
+    std::vector<int> best_k((size_t)n), best_dp((size_t)n);
+    for (double tau : taus) {
+      const double cap = surge_factor > 0.0 ? mem_limit - surge_factor * tau : mem_limit;
+      if (!(cap >= 0.0)) break;
+      for (size_t r = 0; r < reps.size(); ++r) {
+        const int i = reps[r];
+        build_choice(o[i], cand_k + cand_begin[i], cand_overhead + cand_begin[i], cand_begin[i + 1] - cand_begin[i],
+                     world, alpha, beta, b, tau, &choice[r]);
+      }
+      GranSearch S;
+      S.ch.resize((size_t)n);
+      S.same_as_prev.assign((size_t)n, 0);
+      S.min_mem.assign((size_t)n + 1, 0.0);
+      S.min_time.assign((size_t)n + 1, 0.0);
+      for (int p = 0; p < n; ++p) {
+        S.ch[p] = &choice[cls[order[p]]];
+        S.same_as_prev[p] = p > 0 && cls[order[p]] == cls[order[p - 1]];
+        const Choice &c = *S.ch[p];
+        for (size_t h = 1; h < c.hull.size(); ++h)
+          S.segs.push_back(Segment{c.opts[c.hull[h]].mem - c.opts[c.hull[h - 1]].mem,
+                                   c.opts[c.hull[h]].time - c.opts[c.hull[h - 1]].time, p});
+      }
+      for (int p = n - 1; p >= 0; --p) {
+        S.min_mem[p] = S.min_mem[p + 1] + S.ch[p]->opts.front().mem;
+        S.min_time[p] = S.min_time[p + 1] + S.ch[p]->opts.front().time;
+      }
+      if (S.min_mem[0] > cap) continue;
+      std::stable_sort(S.segs.begin(), S.segs.end(),
+                       [](const Segment &x, const Segment &y) { return x.dt * y.dm < y.dt * x.dm; });
+      S.pick.assign((size_t)n, 0);
+      S.best_pick.assign((size_t)n, 0);
+      S.best = std::numeric_limits<double>::infinity();
+      S.nodes = 0;
+      S.max_nodes = max_nodes;
+      S.cut_short = false;
+      S.dfs(0, cap, 0.0);
+      nodes += S.nodes;
+      any_cut = any_cut || S.cut_short;
+      // (if the budget ran out before the first leaf, best_pick is the least-memory options, which fit)
+      // verdict in the caller's operator order, summed the way a plan is priced; if the last bit of the
+      // memory sum lands above the limit, fall back to least-memory options one operator at a time
+      std::vector<int> pick((size_t)n);
+      for (int p = 0; p < n; ++p) pick[order[p]] = S.best_pick[p];
+      double mem = 0.0, t = 0.0;
+      auto price = [&]() {
+        mem = 0.0; t = 0.0;
+        for (int i = 0; i < n; ++i) { const Option &q = choice[cls[i]].opts[pick[i]]; mem += q.mem; t += q.time; }
+      };
+      price();
+      for (int i = n - 1; i >= 0 && mem > cap; --i)
+        if (pick[i] != 0) { pick[i] = 0; price(); }
+      if (mem > cap) continue;
+      if (t < best_t) {
+        best_t = t;
+        for (int i = 0; i < n; ++i) { const Option &q = choice[cls[i]].opts[pick[i]]; best_k[i] = q.k; best_dp[i] = q.dp; }
+      }
+    }
+    if (!(best_t < std::numeric_limits<double>::infinity())) break;
+    const double per_sample = best_t / (double)b;
+    if (per_sample < best) {
+      best = per_sample;
+      best_b = b;
+      for (int i = 0; i < n; ++i) { k_out[i] = best_k[i]; dp_slices[i] = best_dp[i]; }
+    }
+  }
+  *batch = best_b;
+  *time_per_sample = best;
+  if (nodes_visited) *nodes_visited = nodes;
+  return any_cut ? OSDP_ERR_SEARCH_LIMIT : OSDP_OK;
 }
 
 }  // extern "C"

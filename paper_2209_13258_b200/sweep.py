@@ -440,6 +440,29 @@ def plan_from_measurements(hidden, layers, tokens, world, mem_gb, ks, alpha=10e-
                "gamma_ms": {name: gamma[(name, k)] * 1e3 for name, _, _ in shapes}}
         rows.append(row)
         print(json.dumps(row), flush=True)
+    # every operator free to take any of the measured granularities, its slices planned one by one
+    ops, cands, names = [], [], []
+    for _ in range(layers):
+        for name, N, K in shapes:
+            params = float(N * K)
+            ops.append((16.0 * params, 2.0 * tokens * (N + K), 0.0, 2.0 * params, gamma[(name, 1)]))
+            cands.append([(k, gamma[(name, k)] / gamma[(name, 1)] - 1.0) for k in ks if (name, k) in gamma])
+            names.append(name)
+    # surge 0: the memory model of Section 3.1 as it stands; surge 2: the double-buffered gathered slice of the
+    # sharded slice loop counted as well (what Section 3.3 says splitting divides by the granularity)
+    for surge in ((0.0, 2.0) if all(cands) else ()):
+        rc, kk, dps, b, t, nodes = P.osdp_plan_search_granularity(ops, cands, world, alpha, beta, limit, 4096,
+                                                                  surge_factor=surge)
+        chosen = {}
+        for name, k, d in zip(names, kk, dps):
+            if b:
+                key = "k=%d dp=%d" % (k, d)
+                chosen.setdefault(name, {})[key] = chosen.setdefault(name, {}).get(key, 0) + 1
+        row = {"k": "free", "surge_factor": surge, "status": rc, "operators": len(ops), "batch": b, "chosen": chosen,
+               "time_per_sample_ms": t * 1e3 if b else None, "samples_per_s_per_gpu": 1.0 / t if b else 0.0,
+               "nodes": nodes}
+        rows.append(row)
+        print(json.dumps(row), flush=True)
     return rows
 
 

@@ -136,6 +136,19 @@ def test_hand_worked_granularity_instance():
         assert tt == pytest.approx(t, rel=1e-13)
 
 
+def test_hand_worked_instance_with_the_gathered_slice_counted():
+    op = (8.0, 3.0, 0.0, 4.0, 10.0)
+    rows = []
+    with open(os.path.join(os.path.dirname(__file__), "golden", "plan_granularity_example.txt")) as f:
+        rows = [line.split()[1:] for line in f if line.startswith("surge")]
+    assert len(rows) == 3
+    for factor, limit, alpha, k, dp, b, t in rows:
+        ks, dps, bb, tt, _ = OP.search_granularity([op], [[(1, 0.0), (2, 0.02)]], 2, float(alpha), 1.0, float(limit), 8,
+                                                   surge_factor=float(factor))
+        assert (ks, dps, bb) == ([int(k)], [int(dp)], int(b))
+        assert tt == pytest.approx(float(t), rel=1e-13)
+
+
 def test_one_whole_candidate_reduces_to_the_plain_search():
     rng = random.Random(77)
     for _ in range(20):

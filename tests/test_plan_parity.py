@@ -149,3 +149,109 @@ def test_argument_errors(P):
     assert P.osdp_plan_search([(1.0, 1.0, float("nan"), 1.0, 1.0)], 2, 1.0, 0.5, 100.0, 5)[0] == 2
     assert P.osdp_plan_cost([A], 2, 1.0, 0.5, (0,), 0)[0] == 2
     assert P.lib().osdp_plan_search(None, 1, 2, 1.0, 0.5, 100.0, 5, 0, None, None, None, None) == 1
+
+
+# ---- granularity left free (osdp_plan_search_granularity)
+
+def _priced(ops, ks, dps, ovh_of, b, world, alpha, beta):
+    """Memory and time of a (granularity, DP count) assignment, priced by the oracle on the expanded slices."""
+    expanded, modes = [], []
+    for op, k, dp, i in zip(ops, ks, dps, range(len(ops))):
+        expanded += OP.expand_slices(op, k, ovh_of(i, k))
+        modes += [0] * dp + [1] * (k - dp)
+    return OP.memory_cost(expanded, modes, b, world), OP.time_cost(expanded, modes, b, world, alpha, beta)
+
+
+@pytest.mark.parametrize("seed", range(60))
+def test_granularity_search_matches_exhaustive_enumeration(P, seed):
+    rng = random.Random(5000 + seed)
+    n = rng.randint(1, 3)
+    kinds = [(rng.uniform(5, 200), rng.uniform(0, 20), rng.uniform(0, 5), rng.uniform(1, 100), rng.uniform(0.05, 3))
+             for _ in range(2)]
+    ops = [rng.choice(kinds) for _ in range(n)]
+    pool = [(1, 0.0), (2, rng.uniform(0, 0.1)), (3, rng.uniform(0, 0.2)), (4, rng.uniform(0, 0.3))]
+    shared = sorted(rng.sample(pool, rng.randint(1, 3)))
+    cands = [shared if rng.random() < 0.6 else sorted(rng.sample(pool, rng.randint(1, 3))) for _ in range(n)]
+    world = rng.choice([2, 3, 4, 8])
+    alpha, beta = rng.choice([0.0, rng.uniform(0, 1.5)]), rng.uniform(0, 0.5)
+    lo = OP.memory_cost(ops, [1] * n, 1, world)
+    hi = OP.memory_cost(ops, [0] * n, 3, world)
+    limit = rng.uniform(0.9 * lo, 1.05 * hi)
+    factor = rng.choice([0.0, 0.0, 1.0, 2.0, rng.uniform(0, 3)])
+    ks_o, dps_o, b_o, t_o, _ = OP.search_granularity(ops, cands, world, alpha, beta, limit, 4, surge_factor=factor)
+    rc, ks, dps, b, t, nodes = P.osdp_plan_search_granularity(ops, cands, world, alpha, beta, limit, 4,
+                                                              surge_factor=factor)
+    assert rc == 0 and b == b_o
+    if b_o == 0:
+        assert t == float("inf")
+        return
+    assert t == pytest.approx(t_o, rel=1e-12)
+    ovh = lambda i, k: dict(cands[i])[k]
+    assert all(k in dict(c) for k, c in zip(ks, cands)) and all(0 <= d <= k for d, k in zip(dps, ks))
+    mem, tt = _priced(ops, ks, dps, ovh, b, world, alpha, beta)
+    surge = max([op[3] / k for op, k, d in zip(ops, ks, dps) if d < k] + [0.0])
+    assert mem + factor * surge <= limit * (1 + 1e-12) and tt / b == pytest.approx(t, rel=1e-12)
+
+
+def test_granularity_hand_worked_instance(P):
+    op = (8.0, 3.0, 0.0, 4.0, 10.0)
+    assert P.osdp_plan_search_granularity([op], [[(1, 0.0), (2, 0.02)]], 2, 0.25, 1.0, 9.5, 8)[:5] == \
+        (0, [2], [1], 1, pytest.approx(16.45, rel=1e-13))
+    assert P.osdp_plan_search_granularity([op], [[(1, 0.0), (2, 0.02)]], 2, 1.0, 1.0, 9.5, 8)[:5] == \
+        (0, [1], [0], 1, pytest.approx(19.0, rel=1e-13))
+    for limit, want in ((9.5, ([2], [0], 1, 17.7)), (11.0, ([1], [1], 1, 14.5)), (10.5, ([2], [0], 1, 17.7))):
+        got = P.osdp_plan_search_granularity([op], [[(1, 0.0), (2, 0.02)]], 2, 0.25, 1.0, limit, 8, surge_factor=1.0)
+        assert got[0] == 0 and tuple(got[1:4]) == want[:3] and got[4] == pytest.approx(want[3], rel=1e-13)
+
+
+def test_granularity_with_whole_operators_only_is_the_plain_search(P):
+    rng = random.Random(11)
+    for _ in range(30):
+        ops, world, alpha, beta, limit = random_instance(rng, rng.randint(1, 12))
+        rc, modes, b, t, _ = P.osdp_plan_search(ops, world, alpha, beta, limit, 8)
+        rc2, ks, dps, b2, t2, _ = P.osdp_plan_search_granularity(ops, [[(1, 0.0)]] * len(ops), world, alpha, beta,
+                                                                 limit, 8)
+        assert rc == 0 and rc2 == 0 and b2 == b
+        if b:
+            assert t2 == pytest.approx(t, rel=1e-12) and ks == [1] * len(ops)
+
+
+def test_granularity_on_a_transformer_sized_instance(P):
+    ops = gpt_layers(24, 2048)
+    world, alpha, beta = 8, 10e-6, 1 / 400e9
+    dp = OP.memory_cost(ops, [0] * len(ops), 1, world)
+    zdp = OP.memory_cost(ops, [1] * len(ops), 1, world)
+    limit = zdp + 0.37 * (dp - zdp)
+    cands = [[(1, 0.0), (2, 0.01), (4, 0.03), (8, 0.08)]] * len(ops)
+    t0 = time.time()
+    rc, ks, dps, b, t, nodes = P.osdp_plan_search_granularity(ops, cands, world, alpha, beta, limit, 64)
+    assert rc in (0, 10) and b >= 1 and time.time() - t0 < 60.0
+    mem, tt = _priced(ops, ks, dps, lambda i, k: dict(cands[i])[k], b, world, alpha, beta)
+    assert mem <= limit * (1 + 1e-12) and tt / b == pytest.approx(t, rel=1e-12)
+    # the whole-operator plan is among the candidates: leaving the granularity free cannot cost more
+    rc1, _, b1, t1, _ = P.osdp_plan_search(ops, world, alpha, beta, limit, 64)
+    assert rc1 == 0 and (rc != 0 or t <= t1 * (1 + 1e-12))
+    # without latency and overhead, finer slices only add choices: at least as good as the uniform k = 4 plan
+    free = [[(1, 0.0), (4, 0.0)]] * len(ops)
+    sliced = [s for op in ops for s in OP.expand_slices(op, 4)]
+    rc4, _, _, t4, _ = P.osdp_plan_search(sliced, world, 0.0, beta, limit, 64)
+    rcf, _, _, _, tf, _ = P.osdp_plan_search_granularity(ops, free, world, 0.0, beta, limit, 64)
+    assert rc4 == 0 and (rcf != 0 or tf <= t4 * (1 + 1e-12))
+
+
+def test_granularity_node_budget_and_argument_errors(P):
+    rng = random.Random(4)
+    ops = [(rng.uniform(10, 20), 1.0, 0.0, rng.uniform(10, 20), 1.0) for _ in range(30)]
+    cands = [[(1, 0.0), (2, 0.0), (4, 0.01)]] * 30
+    limit = OP.memory_cost(ops, [1] * 30, 1, 4) + 77.7
+    rc, ks, dps, b, t, nodes = P.osdp_plan_search_granularity(ops, cands, 4, 0.0, 1.0, limit, 1, max_nodes=40)
+    assert rc == 10 and b == 1
+    mem, _ = _priced(ops, ks, dps, lambda i, k: dict(cands[i])[k], 1, 4, 0.0, 1.0)
+    assert mem <= limit * (1 + 1e-12)
+    A = (40.0, 5.0, 2.0, 8.0, 3.0)
+    assert P.osdp_plan_search_granularity([A], [[]], 2, 1.0, 0.5, 100.0, 5)[0] == 2          # no candidate
+    assert P.osdp_plan_search_granularity([A], [[(0, 0.0)]], 2, 1.0, 0.5, 100.0, 5)[0] == 3   # k < 1
+    assert P.osdp_plan_search_granularity([A], [[(2, -1.0)]], 2, 1.0, 0.5, 100.0, 5)[0] == 2  # overhead <= -1
+    assert P.osdp_plan_search_granularity([A], [[(1, 0.0)]], 0, 1.0, 0.5, 100.0, 5)[0] == 2   # world < 1
+    assert P.osdp_plan_search_granularity([A], [[(1, 0.0)]], 2, 1.0, 0.5, 1.0, 5)[3] == 0     # nothing fits
+    assert P.osdp_plan_search_granularity([A], [[(1, 0.0)]], 2, 1.0, 0.5, 100.0, 5, surge_factor=-1.0)[0] == 2
