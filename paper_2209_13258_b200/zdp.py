@@ -120,6 +120,16 @@ class DistComm:
 DP, ZDP = 0, 1
 
 
+def slice_modes_from_plan(k, dp_slices):
+    """Per-slice modes for `ZdpSplitLinear(slice_modes=...)` from the plan search's answer for one operator
+    (`osdp_plan_search_granularity`: k slices, dp_slices of them replicated).  The slices are identical, so
+    which ones stay replicated does not matter to the cost; the first dp_slices do."""
+    k, dp_slices = int(k), int(dp_slices)
+    if k < 1 or not 0 <= dp_slices <= k:
+        raise ValueError("need k >= 1 and 0 <= dp_slices <= k")
+    return [DP] * dp_slices + [ZDP] * (k - dp_slices)
+
+
 class ZdpSplitLinear:
     """Y = act(X W^T + b) with W cut into k slices, each slice either sharded over the ranks (ZDP: gathered
     for use, gradient reduce-scattered) or replicated (DP: resident, gradient all-reduced).  `comm` supplies

@@ -73,6 +73,15 @@ def test_shard_and_unshard_round_trip(P, case, world):
     assert sum(int((sh != 0).sum()) for sh in shards) == N * K - 1      # element 0 is the only zero payload
 
 
+def test_slice_modes_from_plan():
+    from paper_2209_13258_b200.zdp import slice_modes_from_plan, DP, ZDP
+    assert slice_modes_from_plan(4, 3) == [DP, DP, DP, ZDP]
+    assert slice_modes_from_plan(1, 0) == [ZDP] and slice_modes_from_plan(2, 2) == [DP, DP]
+    for bad in ((0, 0), (2, 3), (2, -1)):
+        with pytest.raises(ValueError):
+            slice_modes_from_plan(*bad)
+
+
 def test_runtime_refuses_to_run_without_a_gpu(P):
     if torch.cuda.is_available():
         pytest.skip("CUDA device present")
