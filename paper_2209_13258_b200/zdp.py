@@ -434,17 +434,20 @@ class ZdpSplitLinear:
 
 
 class ZdpSplitMLP:
-    """Linear -> activation -> Linear with both weights sharded over the ranks, split along ffn (first layer OUT,
-    second layer RED) and gathered slice by slice: only W1[F_s,:] and W2[:,F_s] of the slice in use (and of the
-    next one, being gathered) exist in full; the slice's dW1 and dW2 are reduce-scattered as soon as they
-    exist, by a collective from slice-sized staging or, with fused_scatter, by the GEMMs' epilogues.
+    """Linear -> activation -> Linear split along ffn (first layer OUT, second layer RED), slice by slice.  A ZDP
+    slice has both its weights, W1[F_s,:] and W2[:,F_s], sharded over the ranks and gathered for use: only those
+    of the slice in use (and of the next one, being gathered) exist in full; its dW1 and dW2 are reduce-scattered
+    as soon as they exist, by a collective from slice-sized staging or, with fused_scatter, by the GEMMs'
+    epilogues.  A DP slice (`slice_modes`, one mode per slice, default all ZDP) keeps both weights whole on every
+    rank and has its gradients all-reduced.
 
     param_shard[0/1], grad_shard[0/1]: this rank's parts of W1 [ffn, hidden] / W2 [hidden, ffn] and of the summed
-    gradients, slice after slice (ShardLayout of each).
+    gradients, ZDP slice after ZDP slice (ShardLayout of each); dp_weight[0/1][s], dp_grad[0/1][s]: the compact
+    matrices of DP slice s.
     """
 
     def __init__(self, hidden, ffn, k_split, act=B.ACT_GELU_TANH, dw_dtype=B.DTYPE_FP32, comm=None, device="cuda",
-                 flags=0, fused_scatter=False):
+                 flags=0, fused_scatter=False, slice_modes=None):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("ZdpSplitMLP needs a CUDA device: there is no CPU path")
@@ -454,21 +457,36 @@ class ZdpSplitMLP:
         self.layouts = [ShardLayout(ffn, hidden, k_split, B.SPLIT_OUT, world),
                         ShardLayout(hidden, ffn, k_split, B.SPLIT_RED, world)]
         self.k = self.layouts[0].k
+        self.modes = [ZDP] * self.k if slice_modes is None else [int(m) for m in slice_modes]
+        if len(self.modes) != self.k or any(m not in (DP, ZDP) for m in self.modes):
+            raise ValueError("slice_modes needs one mode (0 = DP, 1 = ZDP) per slice")
+        self.zdp_slices = [s for s in range(self.k) if self.modes[s] == ZDP]
+        self._zord = {s: i for i, s in enumerate(self.zdp_slices)}
+        self._zoff, totals = [{}, {}], [0, 0]          # where slice s's part starts in this rank's shard buffers
+        for i, l in enumerate(self.layouts):
+            for s in self.zdp_slices:
+                self._zoff[i][s] = totals[i]
+                totals[i] += l.slices[s][3]
         self.device = torch.device(device)
         gdt = torch.float32 if dw_dtype == B.DTYPE_FP32 else torch.bfloat16
-        self.param_shard = [torch.zeros(l.shard_total, dtype=torch.bfloat16, device=self.device) for l in self.layouts]
+        self.param_shard = [torch.zeros(max(t, 8), dtype=torch.bfloat16, device=self.device) for t in totals]
         self.fused_scatter = bool(fused_scatter)
         if self.fused_scatter:
-            self.peer_grad_shards = [self.comm.peer_buffers(l.shard_total, gdt, self.device) for l in self.layouts]
+            self.peer_grad_shards = [self.comm.peer_buffers(max(t, 8), gdt, self.device) for t in totals]
             self.grad_shard = [p[self.comm.rank] for p in self.peer_grad_shards]
             for t in self.grad_shard:
                 t.zero_()
         else:
-            self.grad_shard = [torch.zeros(l.shard_total, dtype=gdt, device=self.device) for l in self.layouts]
-        nb = min(2, self.k)
+            self.grad_shard = [torch.zeros(max(t, 8), dtype=gdt, device=self.device) for t in totals]
+        dp = [s for s in range(self.k) if self.modes[s] == DP]
+        self.dp_weight = [{s: torch.zeros(l.slices[s][2], dtype=torch.bfloat16, device=self.device) for s in dp}
+                          for l in self.layouts]
+        self.dp_grad = [{s: torch.zeros(l.slices[s][2], dtype=gdt, device=self.device) for s in dp}
+                        for l in self.layouts]
+        nb = min(2, len(self.zdp_slices))
         self.w_stage = [[torch.zeros(l.stage_elems, dtype=torch.bfloat16, device=self.device) for _ in range(nb)]
                         for l in self.layouts]
-        need = any(not self._scatter_ok(s) for s in range(self.k))
+        need = any(self.modes[s] == ZDP and not self._scatter_ok(s) for s in range(self.k))
         self.dw_stage = [[torch.zeros(l.stage_elems, dtype=gdt, device=self.device) for _ in range(nb if need else 0)]
                          for l in self.layouts]
         self.comm_stream = torch.cuda.Stream(device=self.device)
@@ -477,15 +495,41 @@ class ZdpSplitMLP:
     def _scatter_ok(self, s):
         ls = self.layouts[0].slices[s][1] - self.layouts[0].slices[s][0]
         m = 32 * self.comm.world
-        return self.fused_scatter and ls % m == 0 and self.hidden % m == 0
+        return self.fused_scatter and self.modes[s] == ZDP and ls % m == 0 and self.hidden % m == 0
 
     def load_full_weights(self, w1_full, w2_full):
         for i, w in enumerate((w1_full, w2_full)):
-            self.param_shard[i].copy_(self.layouts[i].shard_of(w.to(self.device), self.comm.rank))
+            l = self.layouts[i]
+            w = w.to(self.device)
+            shard = l.shard_of(w, self.comm.rank)
+            for s in self.zdp_slices:
+                n, off = l.slices[s][3], l.slices[s][4]
+                self.param_shard[i][self._zoff[i][s]:self._zoff[i][s] + n].copy_(shard[off:off + n])
+            for s, t in self.dp_weight[i].items():
+                t.copy_(l.slice_matrix(w, s).contiguous().reshape(-1))
+
+    def full_from_parts(self, i, shard_bufs, dp_parts):
+        """The full matrix i (0: [ffn, hidden], 1: [hidden, ffn]) from all ranks' shard buffers (laid out like
+        param_shard[i] / grad_shard[i]) and the DP slices' compact tensors (checkpoint save; copies only)."""
+        import torch
+        l = self.layouts[i]
+        ref = shard_bufs[0] if shard_bufs else next(iter(dp_parts.values()))
+        full = torch.empty(l.N, l.K, dtype=ref.dtype, device=ref.device)
+        for s, (b, e, elems, n, _, ld) in enumerate(l.slices):
+            if self.modes[s] == ZDP:
+                o = self._zoff[i][s]
+                flat = torch.cat([sh[o:o + n] for sh in shard_bufs])[:elems]
+            else:
+                flat = dp_parts[s][:elems]
+            l.slice_matrix(full, s).copy_(flat.reshape(-1, ld))
+        return full
 
     def zero_grad(self):
         for t in self.grad_shard:
             t.zero_()
+        for d in self.dp_grad:
+            for t in d.values():
+                t.zero_()
 
     def staging_bytes(self, M):
         nbytes = lambda ts: sum(t.numel() * t.element_size() for t in ts)
@@ -496,24 +540,41 @@ class ZdpSplitMLP:
         return {"weight_staging": nbytes(self.w_stage[0] + self.w_stage[1]),
                 "grad_staging": nbytes(self.dw_stage[0] + self.dw_stage[1]), "workspace": max(f, b)}
 
+    def state_bytes(self):
+        """Bytes of weights and gradients resident on this rank (shards of ZDP slices, whole DP slices)."""
+        nbytes = lambda ts: sum(t.numel() * t.element_size() for t in ts)
+        return {"weights": nbytes(self.param_shard + [t for d in self.dp_weight for t in d.values()]),
+                "grads": nbytes(self.grad_shard + [t for d in self.dp_grad for t in d.values()])}
+
     def _workspace(self, M):
         n = self.staging_bytes(M)["workspace"]
         if self._ws is None or self._ws.numel() != max(n, 256):
             self._ws = B.new_workspace(n, device=self.device)
         return self._ws
 
-    def _gather(self, s, free_events):
-        """Both weights of slice s into staging buffer s & 1, on the communication stream."""
+    def _gather(self, i, free_events):
+        """Both weights of the i-th ZDP slice into staging buffer i & 1, on the communication stream."""
         import torch
+        s = self.zdp_slices[i]
         with torch.cuda.stream(self.comm_stream):
             for ev in free_events:
                 self.comm_stream.wait_event(ev)
-            for i, l in enumerate(self.layouts):
-                _, _, _, n, off, _ = l.slices[s]
-                self.comm.all_gather_slice(self.w_stage[i][s & 1], self.param_shard[i], off, n)
+            for m, l in enumerate(self.layouts):
+                self.comm.all_gather_slice(self.w_stage[m][i & 1], self.param_shard[m], self._zoff[m][s], l.slices[s][3])
             ev = torch.cuda.Event()
             ev.record(self.comm_stream)
         return ev
+
+    def _weights(self, s, ready, free, cur):
+        """The two compact weight matrices of slice s, valid on `cur`: resident (DP), or gathered one ZDP slice
+        ahead of use.  Returns (w1, w2, staging buffer index or None)."""
+        if self.modes[s] == DP:
+            return self.dp_weight[0][s], self.dp_weight[1][s], None
+        i = self._zord[s]
+        if i + 1 < len(self.zdp_slices):
+            ready[i + 1] = self._gather(i + 1, free[(i + 1) & 1])   # buffer (i + 1) & 1 was last read by ordinal i - 1
+        cur.wait_event(ready[i])
+        return self.w_stage[0][i & 1], self.w_stage[1][i & 1], i & 1
 
     def forward(self, x, b1=None, b2=None, out=None, z1_save=None):
         import torch
@@ -523,24 +584,25 @@ class ZdpSplitMLP:
             out = torch.empty(M, self.hidden, dtype=torch.bfloat16, device=self.device)
         ws = self._workspace(M)
         self.comm_stream.wait_stream(cur)
-        free = [[], []]
-        ready = self._gather(0, [])
+        free, ready = [[], []], {}
+        if self.zdp_slices:
+            ready[0] = self._gather(0, [])
         for s in range(self.k):
-            nxt = self._gather(s + 1, free[(s + 1) & 1]) if s + 1 < self.k else None
-            cur.wait_event(ready)
-            B.osdp_zdp_mlp_fwd_slice(x, self.w_stage[0][s & 1], self.w_stage[1][s & 1], self.layouts[1].slices[s][5], b1,
-                                     b2, M, self.hidden, self.ffn, self.k, self.act, s, out, z1_save, ws, stream=cur,
-                                     check=True, flags=self.flags & B.FLAG_CARRY_BF16)
-            ev = torch.cuda.Event()
-            ev.record(cur)
-            free[s & 1] = [ev]
-            ready = nxt
+            w1, w2, j = self._weights(s, ready, free, cur)
+            B.osdp_zdp_mlp_fwd_slice(x, w1, w2, self.layouts[1].slices[s][5], b1, b2, M, self.hidden, self.ffn, self.k,
+                                     self.act, s, out, z1_save, ws, stream=cur, check=True,
+                                     flags=self.flags & B.FLAG_CARRY_BF16)
+            if j is not None:
+                ev = torch.cuda.Event()
+                ev.record(cur)
+                free[j] = [ev]
         cur.wait_stream(self.comm_stream)                   # join (also what a stream capture needs)
         return out
 
     def backward(self, dy, x, z1_saved=None, b1=None, dx=None, db1=None, db2=None):
         """z1_saved None: the pre-activation is recomputed per slice (needs b1).  Gradients of the weights are
-        summed over ranks into grad_shard (with fused_scatter they add to what is there: zero_grad first)."""
+        summed over ranks into grad_shard (with fused_scatter they add to what is there: zero_grad first) and,
+        for DP slices, into dp_grad."""
         import torch
         M = x.shape[0]
         cur = torch.cuda.current_stream(self.device)
@@ -551,20 +613,27 @@ class ZdpSplitMLP:
             self.flags |= B.FLAG_RECOMPUTE          # the workspace plan has one more slice-sized buffer
         ws = self._workspace(M)
         self.comm_stream.wait_stream(cur)
-        w_free, dw_free = [[], []], [None, None]
-        ready = self._gather(0, [])
+        w_free, dw_free, ready = [[], []], [None, None], {}
+        if self.zdp_slices:
+            ready[0] = self._gather(0, [])
         for s in range(self.k):
-            nxt = self._gather(s + 1, w_free[(s + 1) & 1]) if s + 1 < self.k else None
-            j = s & 1
-            cur.wait_event(ready)
+            w1, w2, j = self._weights(s, ready, w_free, cur)
             ld2 = self.layouts[1].slices[s][5]
-            args = (dy, x, self.w_stage[0][j], self.w_stage[1][j], ld2, b1, z1_saved, M, self.hidden, self.ffn, self.k,
-                    self.act, s, dx)
+            args = (dy, x, w1, w2, ld2, b1, z1_saved, M, self.hidden, self.ffn, self.k, self.act, s, dx)
+            if j is None:
+                # DP slice: the kernels write the slice's gradients where they live, then they are summed over ranks
+                B.osdp_zdp_mlp_bwd_slice(*args, self.dp_grad[0][s], self.dp_grad[1][s], ld2, None, None, self.dw_dtype,
+                                         flags, db1, db2, ws, stream=cur, check=True)
+                done = torch.cuda.Event()
+                done.record(cur)
+                with torch.cuda.stream(self.comm_stream):
+                    self.comm_stream.wait_event(done)
+                    for m in range(2):
+                        self.comm.all_reduce(self.dp_grad[m][s], tag=(m, s))
+                continue
             if self._scatter_ok(s):
-                peers = []
-                for i, l in enumerate(self.layouts):
-                    off = l.slices[s][4]
-                    peers.append([int(t.data_ptr()) + off * t.element_size() for t in self.peer_grad_shards[i]])
+                peers = [[int(t.data_ptr()) + self._zoff[m][s] * t.element_size() for t in self.peer_grad_shards[m]]
+                         for m in range(2)]
                 B.osdp_zdp_mlp_bwd_slice(*args, None, None, 0, peers[0], peers[1], self.dw_dtype, flags, db1, db2, ws,
                                          stream=cur, check=True)
                 done = torch.cuda.Event()
@@ -578,12 +647,11 @@ class ZdpSplitMLP:
                 done.record(cur)
                 with torch.cuda.stream(self.comm_stream):
                     self.comm_stream.wait_event(done)
-                    for i, l in enumerate(self.layouts):
-                        _, _, _, n, off, _ = l.slices[s]
-                        self.comm.reduce_scatter_slice(self.grad_shard[i], off, n, self.dw_stage[i][j])
+                    for m, l in enumerate(self.layouts):
+                        self.comm.reduce_scatter_slice(self.grad_shard[m], self._zoff[m][s], l.slices[s][3],
+                                                       self.dw_stage[m][j])
                     dw_free[j] = torch.cuda.Event()
                     dw_free[j].record(self.comm_stream)
             w_free[j] = [done]
-            ready = nxt
         cur.wait_stream(self.comm_stream)
         return dx

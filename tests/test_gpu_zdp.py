@@ -299,6 +299,24 @@ def test_slices_in_mixed_dp_and_zdp_modes_match_oracle(P, world, split, case, mo
     assert len(layer.w_stage) == min(2, modes.count(1))
 
 
+def test_planned_granularity_and_modes_run_in_the_slice_loop(P):
+    """The plan search's answer for one operator (granularity and how many slices stay replicated) drives the
+    slice loop: states held are what the plan priced, results match the oracle."""
+    from paper_2209_13258_b200.zdp import slice_modes_from_plan
+    M, N, K, world = 256, 2048, 512, 2
+    params = float(N * K)
+    op = (2.0 * params, 2.0 * M * (N + K), 0.0, 2.0 * params, 1e-4)        # states = the bf16 weights alone
+    # room for three quarters of the weights replicated: only a 4-way cut can use it
+    limit = 2.0 * params * (0.75 + 0.25 / world) + op[1] + 1.0
+    rc, ks, dps, b, t, _ = P.osdp_plan_search_granularity([op], [[(1, 0.0), (2, 0.0), (4, 0.0)]], world, 0.0, 1e-9,
+                                                          limit, 1)
+    assert (rc, ks, dps, b) == (0, [4], [3], 1)
+    modes = slice_modes_from_plan(ks[0], dps[0])
+    c, y, dx, dW, db, layer = run_emulated_ranks(P, world, M, N, K, ks[0], 0, 0, modes)
+    check_against_oracle(c, y, dx, dW, db, 0, ks[0], 0)
+    assert layer.state_bytes()["weights"] <= limit - op[1]
+
+
 def test_slice_loop_on_a_one_rank_nccl_group(P):
     """The product's own communicator (torch.distributed, NCCL) with world size 1: every collective
     of the loop runs, on its own stream, and the result matches the oracle."""

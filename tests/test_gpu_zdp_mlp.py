@@ -103,6 +103,10 @@ class EmulatedComm:
         for q in range(self.world):
             self.shared["acc"][i][q][off:off + n] += src[q * n:(q + 1) * n].double()
 
+    def all_reduce(self, t, tag=None):
+        acc = self.shared.setdefault("dp_acc", {})
+        acc[tag] = t.double().clone() if tag not in acc else acc[tag] + t.double()
+
     def barrier(self):
         pass
 
@@ -186,6 +190,86 @@ def test_mlp_slice_loop_over_emulated_ranks_matches_oracle(P, world, fused, shap
     # gathered weights: two slices' worth of each matrix
     per = sum(max(sl[3] for sl in lay.slices) for lay in layers[0].layouts) * world * 2
     assert st["weight_staging"] == (2 if k > 1 else 1) * per
+
+
+MIXED = [((512, 512, 2048), 4, [0, 1, 1, 0]), ((512, 512, 2048), 4, [1, 0, 0, 0]), ((300, 264, 520), 3, [0, 0, 1]),
+         ((384, 1024, 4096), 8, [1, 0, 1, 1, 0, 0, 1, 0]), ((256, 512, 1024), 2, [0, 0])]
+
+
+@pytest.mark.parametrize("world", [2, 3])
+@pytest.mark.parametrize("fused,recompute", [(False, False), (True, True)])
+@pytest.mark.parametrize("shape,k,modes", MIXED)
+def test_mlp_slices_in_mixed_dp_and_zdp_modes_match_oracle(P, world, fused, recompute, shape, k, modes):
+    """Section 3.3, last paragraph, for the block: some slices (both their weights) replicated, the others sharded."""
+    from paper_2209_13258_b200.zdp import ZdpSplitMLP
+    M, H, F = shape
+    c = inputs.mlp_case(M, H, F, w_std=0.05, bias_std=0.1, layer=9)
+    wf = to_dev(c["w_flat"])
+    W1 = wf[c["off_w1"]:c["off_w1"] + F * H].view(F, H)
+    W2 = wf[c["off_w2"]:c["off_w2"] + H * F].view(H, F)
+    b1, b2 = to_dev(c["b1"]), to_dev(c["b2"])
+    shared = {"param": [[None] * world, [None] * world], "grad": [[None] * world, [None] * world],
+              "acc": [[None] * world, [None] * world], "peer_next": [0] * world}
+    layers = []
+    for r in range(world):
+        layer = ZdpSplitMLP(H, F, k, comm=EmulatedComm(r, world, shared), fused_scatter=fused, slice_modes=modes)
+        layer.load_full_weights(W1, W2)
+        for i in range(2):
+            shared["param"][i][r] = layer.param_shard[i]
+            shared["grad"][i][r] = layer.grad_shard[i]
+            shared["acc"][i][r] = torch.zeros(layer.grad_shard[i].numel(), dtype=torch.float64, device="cuda")
+        layers.append(layer)
+    # checkpoint round trip: the full weights come back from the ranks' parts
+    for i, W in enumerate((W1, W2)):
+        assert torch.equal(layers[0].full_from_parts(i, [l.param_shard[i] for l in layers], layers[0].dp_weight[i]), W)
+    y = torch.empty(M, H, dtype=torch.bfloat16, device="cuda")
+    dx = torch.empty(M, H, dtype=torch.bfloat16, device="cuda")
+    db1 = torch.zeros(F, dtype=torch.float64, device="cuda")
+    db2 = torch.zeros(H, dtype=torch.float64, device="cuda")
+    x_all, dy_all = to_dev(c["x"]), to_dev(c["dy"])
+    for r, layer in enumerate(layers):
+        rows = torch.arange(r, M, world, device="cuda")
+        xr, dyr = x_all[rows].contiguous(), dy_all[rows].contiguous()
+        z1 = None if recompute else torch.empty(rows.numel(), F, dtype=torch.bfloat16, device="cuda")
+        yr = layer.forward(xr, b1, b2, z1_save=z1)
+        d1 = torch.empty(F, dtype=torch.float32, device="cuda")
+        d2 = torch.empty(H, dtype=torch.float32, device="cuda")
+        dxr = layer.backward(dyr, xr, z1_saved=z1, b1=b1, db1=d1, db2=d2)
+        torch.cuda.synchronize()
+        rc, st = P.osdp_read_device_status(layer._ws)
+        assert rc == 0 and st == 0
+        y[rows], dx[rows] = yr, dxr
+        db1 += d1.double()
+        db2 += d2.double()
+    full = []
+    for i in range(2):
+        lay = layers[0].layouts[i]
+        shards = []
+        for q, l in enumerate(layers):
+            t = shared["acc"][i][q].clone()
+            for s in l.zdp_slices:
+                if l._scatter_ok(s):      # scattered by the epilogue: complete in the rank's own shard
+                    n, o = lay.slices[s][3], l._zoff[i][s]
+                    t[o:o + n] = l.grad_shard[i][o:o + n].double()
+            shards.append(t)
+        dp_parts = {s: shared["dp_acc"][(i, s)] for s in range(k) if modes[s] == 0}
+        full.append(layers[0].full_from_parts(i, shards, dp_parts))
+    _, yo = oracle.mlp_fwd(c["x"], c["w1"], c["b1"], c["w2"], c["b2"], oracle.ACT_GELU_TANH, k)
+    dXo, dW1o, db1o, dW2o, db2o = oracle.mlp_bwd(c["dy"], c["x"], c["w1"], c["b1"], c["w2"], oracle.ACT_GELU_TANH, k)
+    assert_close(to_f64(y), yo, "Y")
+    assert_close(to_f64(dx), dXo, "dX")
+    assert_close(full[0].cpu().numpy(), dW1o, "dW1 (sum over ranks)")
+    assert_close(full[1].cpu().numpy(), dW2o, "dW2 (sum over ranks)")
+    assert_close(db1.cpu().numpy(), db1o, "db1 (sum over ranks)")
+    assert_close(db2.cpu().numpy(), db2o, "db2 (sum over ranks)")
+    # resident weights: whole DP slices plus 1/world of the ZDP slices (up to the 8-element padding), both matrices
+    want = 0
+    for lay in layers[0].layouts:
+        dp_elems = sum(lay.slices[s][2] for s in range(k) if modes[s] == 0)
+        zdp_shard = sum(lay.slices[s][3] for s in range(k) if modes[s] == 1)
+        want += 2 * (dp_elems + max(zdp_shard, 8))
+    assert layers[0].state_bytes()["weights"] == want
+    assert all(len(st) == min(2, modes.count(1)) for st in layers[0].w_stage)
 
 
 def test_sharded_loop_replays_from_a_cuda_graph(P):
