@@ -113,3 +113,107 @@ class SplitLinear(torch.nn.Module):
         if x.dtype != torch.bfloat16:
             raise TypeError("SplitLinear takes bf16 activations")
         return _SplitLinearFn.apply(x, self.weight, self.bias, self)
+
+
+class _SplitMLPFn(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, x, flat, b1, b2, layer):
+        H, F, k = layer.hidden, layer.ffn, layer.k_split
+        M = x.numel() // H
+        x2 = x.reshape(M, H)
+        if not x2.is_contiguous():
+            x2 = x2.contiguous()
+        out = torch.empty(M, H, dtype=torch.bfloat16, device=x.device)
+        need_grad = x.requires_grad or flat.requires_grad
+        # with recomputation no [M, ffn] activation is kept between forward and backward
+        z1 = torch.empty(M, F, dtype=torch.bfloat16, device=x.device) if need_grad and not layer.recompute else None
+        ws = layer._workspace(M)
+        B.osdp_split_mlp_fwd(x2, layer.flat, layer.off_w1, b1, layer.off_w2, b2, M, H, F, k, layer.act, out, z1, ws,
+                             check=True, flags=layer.flags & B.FLAG_CARRY_BF16)
+        ctx.layer, ctx.M, ctx.x_shape = layer, M, x.shape
+        ctx.has_b = (b1 is not None, b2 is not None)
+        empty = torch.empty(0, device=x.device)
+        ctx.save_for_backward(x2, z1 if z1 is not None else empty, b1 if b1 is not None else empty)
+        return out.reshape(*x.shape[:-1], H)
+
+    @staticmethod
+    def backward(ctx, dy):
+        layer, M = ctx.layer, ctx.M
+        H, F, k = layer.hidden, layer.ffn, layer.k_split
+        x2, z1, b1 = ctx.saved_tensors
+        dy2 = dy.reshape(M, H)
+        if not dy2.is_contiguous():
+            dy2 = dy2.contiguous()
+        need_dx, need_dw = ctx.needs_input_grad[0], ctx.needs_input_grad[1]
+        dx = torch.empty(M, H, dtype=torch.bfloat16, device=dy.device) if need_dx else None
+        # the gradient of the flat parameter buffer, laid out like it: dW1 and dW2 at the offsets of W1 and W2
+        dflat = torch.zeros_like(layer.flat) if need_dw else None
+        db1 = torch.empty(F, dtype=torch.float32, device=dy.device) if ctx.has_b[0] and ctx.needs_input_grad[2] else None
+        db2 = torch.empty(H, dtype=torch.float32, device=dy.device) if ctx.has_b[1] and ctx.needs_input_grad[3] else None
+        flags = (layer.flags & B.FLAG_CARRY_BF16) | (B.FLAG_RECOMPUTE if layer.recompute else 0)
+        ws = layer._workspace(M)
+        B.osdp_split_mlp_bwd(dy2, x2, layer.flat, layer.off_w1, layer.off_w2, z1 if z1.numel() else None, M, H, F, k,
+                             layer.act, dx, dflat, layer.off_w1, layer.off_w2, B.DTYPE_BF16, flags, db1, db2, ws,
+                             check=True, b1=b1 if b1.numel() else None)
+        return (dx.reshape(ctx.x_shape) if need_dx else None), dflat, db1, db2, None
+
+
+class SplitMLP(torch.nn.Module):
+    """y = act(x W1^T + b1) W2^T + b2, the transformer MLP block computed as `k_split` sequential slices of the
+    ffn dimension (Section 3.3 applied to both MatMuls: the first layer's output slice feeds the second layer's
+    reduction slice, so only an [M, ffn / k] intermediate exists at a time).  W1 [ffn, hidden] and W2 [hidden, ffn]
+    live in one flat bf16 parameter buffer (`flat_param`, W1 first), biases are fp32.
+
+    recompute=True is the activation-checkpointing setting of Section 2.3: the forward saves no [M, ffn]
+    pre-activation and the backward recomputes it slice by slice.
+    """
+
+    def __init__(self, hidden, ffn, bias=True, k_split=1, act=B.ACT_GELU_TANH, recompute=False, flags=0, device="cuda"):
+        super().__init__()
+        if hidden % 8 or ffn % 8:
+            raise ValueError("hidden and ffn must be multiples of 8")
+        self.hidden, self.ffn, self.k_split, self.act = int(hidden), int(ffn), int(k_split), int(act)
+        self.recompute, self.flags = bool(recompute), int(flags)
+        self.off_w1, self.off_w2 = 0, self.hidden * self.ffn
+        w = torch.empty(2 * self.hidden * self.ffn, dtype=torch.bfloat16, device=device)
+        torch.nn.init.normal_(w, std=0.02)
+        self.flat_param = torch.nn.Parameter(w)
+        mk = lambda n: torch.nn.Parameter(torch.zeros(n, dtype=torch.float32, device=device)) if bias else None
+        self.b1, self.b2 = mk(self.ffn), mk(self.hidden)
+        self._ws = None
+        rc, _ = B.osdp_split_linear_workspace_bytes(1, self.ffn, self.hidden, self.k_split, B.SPLIT_OUT, self.act,
+                                                    B.OP_MLP_FWD, self.flags)
+        if rc:
+            raise B.OsdpError(rc, "SplitMLP")
+
+    @property
+    def flat(self):
+        return self.flat_param
+
+    @property
+    def w1(self):
+        return self.flat_param[:self.off_w2].view(self.ffn, self.hidden)
+
+    @property
+    def w2(self):
+        return self.flat_param[self.off_w2:].view(self.hidden, self.ffn)
+
+    def _workspace(self, M):
+        need = 0
+        for op, fl in ((B.OP_MLP_FWD, self.flags & B.FLAG_CARRY_BF16),
+                       (B.OP_MLP_BWD, (self.flags & B.FLAG_CARRY_BF16) | (B.FLAG_RECOMPUTE if self.recompute else 0))):
+            rc, n = B.osdp_split_linear_workspace_bytes(M, self.ffn, self.hidden, self.k_split, B.SPLIT_OUT, self.act,
+                                                        op, fl)
+            if rc:
+                raise B.OsdpError(rc, "osdp_split_linear_workspace_bytes")
+            need = max(need, n)
+        if self._ws is None or self._ws.numel() < need or self._ws.device != self.flat.device:
+            self._ws = B.new_workspace(need, device=self.flat.device)
+        return self._ws
+
+    def forward(self, x):
+        if not x.is_cuda:
+            raise RuntimeError("SplitMLP runs on CUDA only: there is no CPU path")
+        if x.dtype != torch.bfloat16:
+            raise TypeError("SplitMLP takes bf16 activations")
+        return _SplitMLPFn.apply(x, self.flat_param, self.b1, self.b2, self)

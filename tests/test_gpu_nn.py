@@ -74,3 +74,48 @@ def test_module_argument_errors(P):
         m(torch.zeros(8, 64, device="cuda"))
     with pytest.raises(RuntimeError):
         m(torch.zeros(8, 64, dtype=torch.bfloat16))
+
+
+@pytest.mark.parametrize("k,recompute", [(1, False), (4, False), (4, True), (3, True)])
+def test_mlp_module(P, k, recompute):
+    """SplitMLP through autograd: forward, dX, the flat parameter's gradient (dW1 then dW2) and both bias
+    gradients against the oracle; with recomputation nothing of size [M, ffn] is saved for the backward."""
+    from paper_2209_13258_b200.nn import SplitMLP
+    B_, S, H, F = 2, 150, 264, 1032
+    if P.osdp_slice_range(F, k, 0)[0] != 0:
+        pytest.skip("invalid split")
+    c = inputs.mlp_case(B_ * S, H, F, w_std=0.05, bias_std=0.1, layer=13)
+    m = SplitMLP(H, F, bias=True, k_split=k, recompute=recompute)
+    with torch.no_grad():
+        m.w1.copy_(to_dev(c["w1"]))
+        m.w2.copy_(to_dev(c["w2"]))
+        m.b1.copy_(to_dev(c["b1"]))
+        m.b2.copy_(to_dev(c["b2"]))
+    x = to_dev(c["x"]).view(B_, S, H).requires_grad_(True)
+    y = m(x)
+    assert y.shape == (B_, S, H) and y.dtype == torch.bfloat16
+    saved = [t for t in y.grad_fn.saved_tensors if t.numel() == B_ * S * F]
+    assert len(saved) == (0 if recompute else 1)
+    y.backward(to_dev(c["dy"]).view(B_, S, H))
+    _, yo = oracle.mlp_fwd(c["x"], c["w1"], c["b1"], c["w2"], c["b2"], oracle.ACT_GELU_TANH, k)
+    dXo, dW1o, db1o, dW2o, db2o = oracle.mlp_bwd(c["dy"], c["x"], c["w1"], c["b1"], c["w2"], oracle.ACT_GELU_TANH, k)
+    assert_close(to_f64(y).reshape(-1, H), yo, "Y")
+    assert_close(to_f64(x.grad).reshape(-1, H), dXo, "dX")
+    g = m.flat_param.grad
+    assert_close(to_f64(g[:H * F]).reshape(F, H), dW1o, "dW1")
+    assert_close(to_f64(g[H * F:]).reshape(H, F), dW2o, "dW2")
+    assert_close(to_f64(m.b1.grad), db1o, "db1")
+    assert_close(to_f64(m.b2.grad), db2o, "db2")
+
+
+def test_mlp_module_argument_errors(P):
+    from paper_2209_13258_b200.nn import SplitMLP
+    with pytest.raises(ValueError):
+        SplitMLP(100, 64)
+    with pytest.raises(P.OsdpError):
+        SplitMLP(64, 256, k_split=100)
+    m = SplitMLP(64, 256)
+    with pytest.raises(TypeError):
+        m(torch.zeros(8, 64, device="cuda"))
+    with pytest.raises(RuntimeError):
+        m(torch.zeros(8, 64, dtype=torch.bfloat16))
