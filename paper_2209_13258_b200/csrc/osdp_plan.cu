@@ -385,6 +385,7 @@ int osdp_plan_search_granularity(const double *ops, int n, const int *cand_begin
   std::vector<Choice> choice(reps.size());
   for (int b = 1; b <= max_batch; ++b) {             // Algorithm 1: grow the batch until nothing fits
     double best_t = std::numeric_limits<double>::infinity();   // least time at this batch size, over all tau
+    int64_t nodes_b = 0;
     std::vector<int> best_k((size_t)n), best_dp((size_t)n);
     for (double tau : taus) {
       const double cap = surge_factor > 0.0 ? mem_limit - surge_factor * tau : mem_limit;
@@ -416,14 +417,35 @@ int osdp_plan_search_granularity(const double *ops, int n, const int *cand_begin
                        [](const Segment &x, const Segment &y) { return x.dt * y.dm < y.dt * x.dm; });
       S.pick.assign((size_t)n, 0);
       S.best_pick.assign((size_t)n, 0);
-      S.best = std::numeric_limits<double>::infinity();
+      S.best = best_t;                               // only plans faster than the best of the earlier tau matter
+      {
+        // first plan: from the least-memory options, hull steps by decreasing time saved per byte while they fit
+        // (the relaxation's solution without its fractional step); it makes the time pruning bite at once
+        std::vector<int> h((size_t)n, 0);
+        std::vector<char> stuck((size_t)n, 0);
+        double room = cap - S.min_mem[0], t = S.min_time[0];
+        for (const Segment &g : S.segs) {
+          if (stuck[g.pos]) continue;
+          if (g.dm <= room) { room -= g.dm; t += g.dt; ++h[g.pos]; }
+          else stuck[g.pos] = 1;                       // an operator's steps come in order: skip its later ones
+        }
+        if (t < S.best) {
+          S.best = t;
+          for (int p = 0; p < n; ++p) S.best_pick[p] = S.ch[p]->hull[h[p]];
+        }
+      }
       S.nodes = 0;
-      S.max_nodes = max_nodes;
+      S.max_nodes = std::max<int64_t>(1, max_nodes - nodes_b);   // one node budget per batch size
       S.cut_short = false;
       S.dfs(0, cap, 0.0);
       nodes += S.nodes;
+      nodes_b += S.nodes;
       any_cut = any_cut || S.cut_short;
-      // (if the budget ran out before the first leaf, best_pick is the least-memory options, which fit)
+      if (!(S.best < best_t)) {
+        // nothing faster under this tau; if no plan is known yet because the budget ran out before the
+        // first leaf, take the least-memory options (best_pick all zero), which fit
+        if (best_t < std::numeric_limits<double>::infinity() || !S.cut_short) continue;
+      }
       // verdict in the caller's operator order, summed the way a plan is priced; if the last bit of the
       // memory sum lands above the limit, fall back to least-memory options one operator at a time
       std::vector<int> pick((size_t)n);
