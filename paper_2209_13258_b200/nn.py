@@ -217,3 +217,77 @@ class SplitMLP(torch.nn.Module):
         if x.dtype != torch.bfloat16:
             raise TypeError("SplitMLP takes bf16 activations")
         return _SplitMLPFn.apply(x, self.flat_param, self.b1, self.b2, self)
+
+
+class _ZdpLinearFn(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, x, shard, bias, layer, *dp_parts):
+        impl = layer.impl
+        M = x.numel() // impl.K
+        x2 = x.reshape(M, impl.K)
+        if not x2.is_contiguous():
+            x2 = x2.contiguous()
+        need_grad = any(ctx.needs_input_grad)
+        z = torch.empty(M, impl.N, dtype=torch.bfloat16, device=x.device) if impl.act != B.ACT_NONE and need_grad else None
+        out = impl.forward(x2, bias=bias, z_save=z)
+        ctx.layer, ctx.M, ctx.x_shape, ctx.has_bias = layer, M, x.shape, bias is not None
+        ctx.save_for_backward(x2, z if z is not None else torch.empty(0, device=x.device))
+        return out.reshape(*x.shape[:-1], impl.N)
+
+    @staticmethod
+    def backward(ctx, dy):
+        layer, M = ctx.layer, ctx.M
+        impl = layer.impl
+        x2, z = ctx.saved_tensors
+        dy2 = dy.reshape(M, impl.N)
+        if not dy2.is_contiguous():
+            dy2 = dy2.contiguous()
+        need_dx = ctx.needs_input_grad[0]
+        need_db = ctx.has_bias and ctx.needs_input_grad[2]
+        db = torch.empty(impl.N, dtype=torch.float32, device=dy.device) if need_db else None
+        dx = impl.backward(dy2, x2, z_saved=z if z.numel() else None, dbias=db, need_dx=need_dx)
+        if need_db:
+            impl.comm.all_reduce(db, tag="bias")       # the bias is replicated: its gradient is summed over ranks
+        # The loop leaves the summed gradients in its own buffers, which the next backward overwrites:
+        # autograd gets copies (shard-sized for the ZDP slices, slice-sized for the DP ones).
+        g_shard = impl.grad_shard.clone() if ctx.needs_input_grad[1] else None
+        g_dp = [impl.dp_grad[s].clone() for s in layer._dp_order]
+        return (dx.reshape(ctx.x_shape) if need_dx else None), g_shard, db, None, *g_dp
+
+
+class ZdpLinear(torch.nn.Module):
+    """The split linear layer with its weight sharded over the ranks of a process group, the counterpart of the
+    paper's wrapper around a sharded module (Section 3.2, implementation; Section 3.3 for the slices): W is cut
+    into `k_split` slices; a ZDP slice is stored as 1 / world of its elements per rank, gathered for use slice by
+    slice in forward and backward, and its gradient reduce-scattered; a DP slice (`slice_modes`, e.g. from
+    `zdp.slice_modes_from_plan`) is whole on every rank and has its gradient all-reduced.
+
+    Parameters: `shard` (bf16, this rank's part of every ZDP slice), `dp_parts` (the DP slices' compact matrices),
+    `bias` (fp32, replicated).  After backward their `.grad` hold this rank's part of the gradient summed over
+    ranks (bf16 for the weights, fp32 for the bias), ready for a sharded optimiser step.  Every rank passes its
+    own tokens.  Collectives run on the layer's communication stream, overlapped with the slice GEMMs.
+    """
+
+    def __init__(self, in_features, out_features, bias=True, k_split=1, split_dim=B.SPLIT_OUT, act=B.ACT_NONE,
+                 slice_modes=None, comm=None, flags=0, device="cuda"):
+        super().__init__()
+        from .zdp import ZdpSplitLinear
+        self.impl = ZdpSplitLinear(out_features, in_features, k_split, split_dim, act=act, dw_dtype=B.DTYPE_BF16, comm=comm,
+                                   device=device, flags=flags, slice_modes=slice_modes)
+        self.in_features, self.out_features = int(in_features), int(out_features)
+        self.shard = torch.nn.Parameter(self.impl.param_shard)            # same storage: an optimiser step updates the loop's shard
+        self._dp_order = sorted(self.impl.dp_weight)
+        self.dp_parts = torch.nn.ParameterList([torch.nn.Parameter(self.impl.dp_weight[s]) for s in self._dp_order])
+        self.bias = torch.nn.Parameter(torch.zeros(self.out_features, dtype=torch.float32, device=device)) if bias else None
+
+    def load_full_weight(self, w_full):
+        """Keeps this rank's part of a full [out_features, in_features] weight."""
+        with torch.no_grad():
+            self.impl.load_full_weight(w_full)
+
+    def forward(self, x):
+        if not x.is_cuda:
+            raise RuntimeError("ZdpLinear runs on CUDA only: there is no CPU path")
+        if x.dtype != torch.bfloat16:
+            raise TypeError("ZdpLinear takes bf16 activations")
+        return _ZdpLinearFn.apply(x, self.shard, self.bias, self, *self.dp_parts)

@@ -353,6 +353,29 @@ def test_slice_loop_on_a_one_rank_nccl_group(P):
             layer.backward(dy, x, z_saved=z, dbias=db, accumulate=True)
             torch.cuda.synchronize()
             assert_close(to_f64(layer.full_from_parts([layer.grad_shard], layer.dp_grad)), 2 * dWo, "dW accumulated")
+        # the autograd wrapper over the same loop: parameters are the shard and the DP slices, their .grad the
+        # summed gradients; a second backward accumulates like any torch parameter
+        from paper_2209_13258_b200.nn import ZdpLinear
+        for split, modes in ((0, None), (1, [1, 0, 0, 1])):
+            c = inputs.linear_case(M, N, K, w_std=0.05, bias_std=0.2, layer=5)
+            W = to_dev(c["w_flat"])[c["w_offset"]:c["w_offset"] + N * K].view(N, K)
+            m = ZdpLinear(K, N, bias=True, k_split=k, split_dim=split, act=1, slice_modes=modes)
+            m.load_full_weight(W)
+            with torch.no_grad():
+                m.bias.copy_(to_dev(c["bias"]))
+            assert m.shard.data_ptr() == m.impl.param_shard.data_ptr()
+            x = to_dev(c["x"]).view(4, M // 4, K).requires_grad_(True)
+            for _ in range(2):
+                y = m(x)
+                y.backward(to_dev(c["dy"]).view(4, M // 4, N))
+            torch.cuda.synchronize()
+            zo, yo = oracle.linear_fwd(c["x"], c["w"], c["bias"], 1, k, split)
+            dXo, dWo, dbo = oracle.linear_bwd(c["dy"], c["x"], c["w"], zo, 1, k, split)
+            assert_close(to_f64(y).reshape(M, N), yo, "Y (module)")
+            assert_close(to_f64(x.grad).reshape(M, K), 2 * dXo, "dX (module, two backward passes)")
+            dp = {s: p.grad for s, p in zip(m._dp_order, m.dp_parts)}
+            assert_close(to_f64(m.impl.full_from_parts([m.shard.grad], dp)), 2 * dWo, "dW (module)")
+            assert_close(to_f64(m.bias.grad), 2 * dbo, "db (module)")
         # the epilogue's scatter into a shard allocated as symmetric memory (one rank: its own buffer)
         try:
             layer = ZdpSplitLinear(N, K, k, 0, act=0, fused_scatter=True)
