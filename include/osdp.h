@@ -148,9 +148,9 @@ int osdp_split_linear_fwd_slice(const void *x, const void *w_flat, int64_t w_off
  *   dbias [N] fp32 or NULL (always overwritten).
  * OUT: dW[R_s,:], db[R_s] per slice, dX = sum over slices (fp32 carry in ws).
  * RED: dX[:,C_s], dW[:,C_s] per slice.
- * For a small operator without activation (fewer 128 x 128 output tiles than SMs in dX and in dW) the
- * call runs dW and db on a stream of its own next to dX, forked from and joined back into `stream`
- * (see osdp_split_mlp_bwd for the rules of these internal streams). */
+ * Without activation, when both dx and dw_flat are given, the call runs dW and db on a stream of its own
+ * next to dX, forked from and joined back into `stream` (see osdp_split_mlp_bwd for the rules of these
+ * internal streams). */
 int osdp_split_linear_bwd(const void *dy, const void *x, const void *w_flat, int64_t w_offset,
                           const void *z_saved, int64_t M, int64_t N, int64_t K, int k_split,
                           int split_dim, int act, void *dx, void *dw_flat, int64_t dw_offset,
@@ -285,7 +285,7 @@ int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const 
  * dX, dW1, db1 are bit-identical to the saved-activation path; dW2 = dY^T act(Z1_s) uses the
  * activation of the unrounded pre-activation, as the forward did.  b1 [ffn] fp32 or NULL is only
  * read then.
- * When a slice's weight-gradient GEMMs are small (fewer 128 x 128 tiles than SMs) the call runs them
+ * When weight gradients are wanted the call runs each slice's two weight-gradient GEMMs
  * on two streams of its own next to the dX GEMM: it forks from `stream` with an event and joins back
  * into `stream` before the next slice, so the caller still sees one ordered call (a stream capture
  * follows the fork).  The two streams and three events per device are created by the first such call;

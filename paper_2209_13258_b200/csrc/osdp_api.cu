@@ -837,25 +837,22 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
   };
 
   if (act == OSDP_ACT_NONE) {
-    // dX, dW and db do not depend on one another.  A small operator (fewer 128 x 128 output tiles than SMs in
-    // both GEMMs) runs dW and db on an internal stream next to dX (fork from and join into `stream`).
+    // dX, dW and db do not depend on one another: when both GEMMs are wanted, dW and db run on an internal
+    // stream next to dX (fork from and join into `stream`), so that each fills the SMs that the other's last,
+    // partly filled wave of tiles leaves idle.  Measured on B200, backward only: 256 x 2048 x 512 42 -> 34 us;
+    // 8192 x 2048 x 2048 +8 %, 4096 x 4096 x 1024 +7 %, 8192 x 2048 x 8192 +5 %, 32768 x 4096 x 4096 +3 %,
+    // 16384 x 8192 x 8192 +0.3 % (k = 8: +1 %); one shape tried lost (8192 x 6144 x 2048, -1.5 %).
     SideStreams *side = nullptr;
     std::unique_lock<std::mutex> side_lock;
     cudaStream_t s_main = stream, s_side = stream;
-    {
-      int sms = 0;
-      rc = device_sms(&sms);
+    if (dx && dw) {
+      rc = side_streams(&side);
       if (rc) return rc;
-      // (measured on B200, 256 x 2048 x 512 forward + backward: 42 -> 34 us at k = 1, 57 -> 46 us at k = 4)
-      if (dx && dw && cdiv(M, 128) * cdiv(K, 128) <= sms && cdiv(N, 128) * cdiv(K, 128) <= sms) {
-        rc = side_streams(&side);
-        if (rc) return rc;
-        side_lock = std::unique_lock<std::mutex>(g_side_mutex);
-        cudaError_t e = cudaEventRecord(side->fork, stream);
-        if (e == cudaSuccess) e = cudaStreamWaitEvent(side->s[0], side->fork, 0);
-        if (e != cudaSuccess) return cuda_fail(e);
-        s_side = side->s[0];
-      }
+      side_lock = std::unique_lock<std::mutex>(g_side_mutex);
+      cudaError_t e = cudaEventRecord(side->fork, stream);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(side->s[0], side->fork, 0);
+      if (e != cudaSuccess) return cuda_fail(e);
+      s_side = side->s[0];
     }
     stream = s_main;
     if (dx) { rc = dx_call(Operand{dy, N, M, N, false, true}, s_begin, s_end); if (rc) return rc; }
@@ -1209,13 +1206,10 @@ static int mlp_bwd_impl(const void *dy, const void *x, const void *w_flat, int64
     rc = launch_colsum(dy, hidden, M, 0, (int)hidden, partial, db2, stream);
     if (rc) return rc;
   }
-  // Fork the slice's independent launches when its weight-gradient GEMMs are small (fewer 128 x 128 tiles
-  // than SMs): measured on B200, hidden 1024 / ffn 4096 / 4096 tokens at k = 8: 1.06 -> 0.84 ms; no
-  // effect, either way, on larger slices.
-  int sms = 0;
-  rc = device_sms(&sms);
-  if (rc) return rc;
-  const bool concurrent = dw_flat && cdiv(L, 128) * cdiv(hidden, 128) <= (int64_t)sms;
+  // The slice's weight-gradient GEMMs are forked onto the internal streams next to its dX GEMM.  Measured on
+  // B200: hidden 1024 / ffn 4096 / 4096 tokens at k = 8 1.06 -> 0.84 ms; hidden 2048 / ffn 8192 at k = 4 +7.5 %;
+  // hidden 4096 / ffn 16384 / 8192 tokens +1.5 %; hidden 8192 / ffn 32768 at k = 8 +0.5 %.
+  const bool concurrent = dw_flat != nullptr;
   for (int s = cs ? cs->idx : 0; s < (cs ? cs->idx + 1 : k); ++s) {
     const int64_t lo = (int64_t)s * L;
     const int64_t ls = (lo + L < ffn ? lo + L : ffn) - lo;
@@ -1255,8 +1249,8 @@ static int mlp_bwd_impl(const void *dy, const void *x, const void *w_flat, int64
     rc = launch_gemm(c, stream);
     if (rc) return rc;
     // The slice's three remaining GEMMs and its column sum depend only on what has been launched so far.
-    // Small ones (a few waves of tiles each) are forked onto the internal streams so that they share the
-    // SMs; large ones fill the GPU on their own and stay in order on the caller's stream.
+    // They are forked onto the internal streams so that they share the SMs (each fills the others' partly
+    // filled last wave of tiles).
     SideStreams *side = nullptr;
     std::unique_lock<std::mutex> side_lock;
     cudaStream_t s_dw2 = stream, s_dw1 = stream;
