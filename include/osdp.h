@@ -148,7 +148,7 @@ int osdp_split_linear_fwd_slice(const void *x, const void *w_flat, int64_t w_off
  *   dbias [N] fp32 or NULL (always overwritten).
  * OUT: dW[R_s,:], db[R_s] per slice, dX = sum over slices (fp32 carry in ws).
  * RED: dX[:,C_s], dW[:,C_s] per slice.
- * Without activation, when both dx and dw_flat are given, the call runs dW and db on a stream of its own
+ * When both dx and dw_flat are given, the call runs dW and db on a stream of its own
  * next to dX, forked from and joined back into `stream` (see osdp_split_mlp_bwd for the rules of these
  * internal streams). */
 int osdp_split_linear_bwd(const void *dy, const void *x, const void *w_flat, int64_t w_offset,

@@ -877,6 +877,32 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
     return OSDP_OK;
   }
 
+  // With an activation the GEMMs read G = dY (.) act'(Z) from staging.  As above, when both are wanted dW (and
+  // db) run on the internal stream next to dX; they join before the staging is written again.
+  SideStreams *side = nullptr;
+  std::unique_lock<std::mutex> side_lock;
+  if (dx && dw) {
+    rc = side_streams(&side);
+    if (rc) return rc;
+    side_lock = std::unique_lock<std::mutex>(g_side_mutex);
+  }
+  cudaStream_t s_main = stream;
+  auto fork = [&]() -> int {
+    if (!side) return OSDP_OK;
+    cudaError_t e = cudaEventRecord(side->fork, s_main);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(side->s[0], side->fork, 0);
+    if (e != cudaSuccess) return cuda_fail(e);
+    stream = side->s[0];
+    return OSDP_OK;
+  };
+  auto join = [&]() -> int {
+    stream = s_main;
+    if (!side) return OSDP_OK;
+    cudaError_t e = cudaEventRecord(side->join[0], side->s[0]);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s_main, side->join[0], 0);
+    return e == cudaSuccess ? OSDP_OK : cuda_fail(e);
+  };
+
   if (out_split) {
     // Slice by slice: G_s = dY[:,R_s] (.) act'(Z[:,R_s]) into slice-sized staging, then the slice's GEMMs.
     for (int s = s_begin; s < s_end; ++s) {
@@ -884,9 +910,14 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
       const int64_t ls = (c0 + L < N ? c0 + L : N) - c0;
       rc = launch_act_backward(dy, N, z_saved, N, stage, L, M, (int)c0, (int)ls, act, stream);
       if (rc) return rc;
-      if (dx) { rc = dx_call(Operand{stage, ls, M, L, false, false}, s, s + 1); if (rc) return rc; }
+      rc = fork();                                     // from here on `stream` is the internal one, if any
+      if (rc) return rc;
       if (dw) { rc = dw_call(Operand{stage, ls, M, L, true, false}, s, s + 1); if (rc) return rc; }
       if (dbias) { rc = launch_colsum(stage, L, M, 0, (int)ls, partial, dbias + c0, stream); if (rc) return rc; }
+      stream = s_main;
+      if (dx) { rc = dx_call(Operand{stage, ls, M, L, false, false}, s, s + 1); if (rc) return rc; }
+      rc = join();
+      if (rc) return rc;
     }
     return OSDP_OK;
   }
@@ -894,11 +925,14 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
   if (s_begin == 0) {
     rc = launch_act_backward(dy, N, z_saved, N, stage, N, M, 0, (int)N, act, stream);
     if (rc) return rc;
-    if (dbias) { rc = launch_colsum(stage, N, M, 0, (int)N, partial, dbias, stream); if (rc) return rc; }
   }
-  if (dx) { rc = dx_call(Operand{stage, N, M, N, false, true}, s_begin, s_end); if (rc) return rc; }
+  rc = fork();
+  if (rc) return rc;
+  if (s_begin == 0 && dbias) { rc = launch_colsum(stage, N, M, 0, (int)N, partial, dbias, stream); if (rc) return rc; }
   if (dw) { rc = dw_call(Operand{stage, N, M, N, true, true}, s_begin, s_end); if (rc) return rc; }
-  return OSDP_OK;
+  stream = s_main;
+  if (dx) { rc = dx_call(Operand{stage, N, M, N, false, true}, s_begin, s_end); if (rc) return rc; }
+  return join();
 }
 
 }  // namespace
