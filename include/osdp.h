@@ -13,8 +13,16 @@
  *      OSDP_SPLIT_RED : the K columns of W and X.  This is the split Section 3.3 describes: the
  *                       input is cut along its last dimension, the operator along the matching
  *                       one, and the slice products are added up.  Y is summed; dX, dW concatenate.
- * Slices are visited in ascending order (slice-major).  A summed output is carried between
- * slices as an fp32 running sum in the caller's workspace.
+ * Slices are visited in ascending order and their products are added in fp32.  Where the sum is kept
+ * between two slices depends on who owns the loop over the slices:
+ *  - one slice per call (the *_slice entry points, the MLP block, OSDP_FLAG_SLICE_MAJOR): the whole
+ *    operator is swept once per slice, and a summed output travels from slice to slice as an fp32
+ *    running sum [rows x cols of that output] in the caller's workspace;
+ *  - all slices in one call (default): the call walks the output in panels of one tile per CTA pair
+ *    (256 x 512 elements each, 148 SMs: about 38 MB of fp32 sums, which is the tensor memory of the
+ *    whole GPU) and visits the slices in order inside a panel, so the running sum of a tile stays in
+ *    tensor memory from its first slice to its last and never goes through global memory.  Same
+ *    products, same ascending order per output element; no carry buffer.
  *
  * Slice rule (the paper gives none for non-divisible extents): slice length
  * L = ceil(D/k) rounded up to a multiple of 8 elements; slice s = [s*L, min(D,(s+1)*L)); a
@@ -90,6 +98,11 @@ extern "C" {
                                      * adjacent slices in one pass, so two slices are read at a time (what a
                                      * double-buffered slice gather holds anyway) and the running sum is carried
                                      * half as often.  Exact fp32, but not bit-identical to the unpaired result. */
+#define OSDP_FLAG_SLICE_MAJOR 16    /* all-slices calls of a summed output: sweep the whole operator once per slice
+                                     * (slice s of every output tile before slice s + 1 of any), the running sum
+                                     * carried in fp32 through the workspace, exactly as a sequence of *_slice
+                                     * calls does.  In a workspace query: include that carry, i.e. size the
+                                     * workspace for the *_slice entry points (which accept and ignore the flag). */
 #define OSDP_FLAG_RECOMPUTE 4       /* osdp_split_mlp_bwd: recompute the first layer's pre-activation slice by
                                      * slice instead of reading z1_saved (activation checkpointing). */
 

@@ -5,7 +5,7 @@ marshals arguments.  There is no CPU fallback: if the library is missing, loadin
 ``paper_2209_13258_b200.inputs`` (seeded synthetic inputs) does not need the library.
 """
 from .binding import (  # noqa: F401
-    ACT_GELU_ERF, ACT_GELU_TANH, ACT_NONE, DTYPE_BF16, DTYPE_FP32, FLAG_ACCUMULATE_DW, FLAG_CARRY_BF16, FLAG_RECOMPUTE, FLAG_PAIR_SLICES, OP_LINEAR_BWD, OP_LINEAR_FWD,
+    ACT_GELU_ERF, ACT_GELU_TANH, ACT_NONE, DTYPE_BF16, DTYPE_FP32, FLAG_ACCUMULATE_DW, FLAG_CARRY_BF16, FLAG_RECOMPUTE, FLAG_PAIR_SLICES, FLAG_SLICE_MAJOR, OP_LINEAR_BWD, OP_LINEAR_FWD,
     OP_MLP_BWD, OP_MLP_FWD, SPLIT_OUT, SPLIT_RED, OsdpError, lib, lib_path,
     osdp_last_cuda_error, osdp_read_device_status, osdp_slice_range, osdp_split_linear_bwd,
     osdp_split_linear_bwd_slice, osdp_split_linear_fwd, osdp_split_linear_fwd_slice,

@@ -16,7 +16,7 @@ SPLIT_OUT, SPLIT_RED = 0, 1
 ACT_NONE, ACT_GELU_TANH, ACT_GELU_ERF = 0, 1, 2
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 OP_LINEAR_FWD, OP_LINEAR_BWD, OP_MLP_FWD, OP_MLP_BWD = 0, 1, 2, 3
-FLAG_ACCUMULATE_DW, FLAG_CARRY_BF16, FLAG_RECOMPUTE, FLAG_PAIR_SLICES = 1, 2, 4, 8
+FLAG_ACCUMULATE_DW, FLAG_CARRY_BF16, FLAG_RECOMPUTE, FLAG_PAIR_SLICES, FLAG_SLICE_MAJOR = 1, 2, 4, 8, 16
 
 EXPORTS = [
     "osdp_version", "osdp_status_string", "osdp_last_cuda_error", "osdp_slice_range",

@@ -140,6 +140,11 @@ struct WsPlan {
 
 int plan_workspace(int64_t M, int64_t N, int64_t K, int k, int split_dim, int act, int op, int flags, WsPlan *w) {
   const bool fp32_carry = !(flags & OSDP_FLAG_CARRY_BF16);
+  // The linear ops carry a running sum through memory only when the operator is swept once per slice: the
+  // *_slice entry points and all-slices calls in slice-major order (both ask with OSDP_FLAG_SLICE_MAJOR), paired
+  // slices, and the backward with an activation (its G_s is staged slice by slice).  Otherwise an all-slices
+  // call keeps every tile's sum in tensor memory across the slices.
+  const bool swept = (flags & (OSDP_FLAG_SLICE_MAJOR | OSDP_FLAG_PAIR_SLICES)) != 0;
   memset(w, 0, sizeof(*w));
   if (M <= 0 || N <= 0 || K <= 0) return OSDP_ERR_BAD_SHAPE;
   if (k == 0) k = 1;
@@ -157,13 +162,15 @@ int plan_workspace(int64_t M, int64_t N, int64_t K, int k, int split_dim, int ac
       if (split_dim != OSDP_SPLIT_OUT && split_dim != OSDP_SPLIT_RED) return OSDP_ERR_BAD_SPLIT;
       rc = slice_len(split_dim == OSDP_SPLIT_OUT ? N : K, k, &L);
       if (rc) return rc;
-      if (split_dim == OSDP_SPLIT_RED && k > 1 && fp32_carry) take((size_t)M * N * 4, &w->carry_off, &w->carry_bytes);
+      if (split_dim == OSDP_SPLIT_RED && k > 1 && fp32_carry && swept)
+        take((size_t)M * N * 4, &w->carry_off, &w->carry_bytes);
       break;
     case OSDP_OP_LINEAR_BWD:
       if (split_dim != OSDP_SPLIT_OUT && split_dim != OSDP_SPLIT_RED) return OSDP_ERR_BAD_SPLIT;
       rc = slice_len(split_dim == OSDP_SPLIT_OUT ? N : K, k, &L);
       if (rc) return rc;
-      if (split_dim == OSDP_SPLIT_OUT && k > 1 && fp32_carry) take((size_t)M * K * 4, &w->carry_off, &w->carry_bytes);
+      if (split_dim == OSDP_SPLIT_OUT && k > 1 && fp32_carry && (swept || act != OSDP_ACT_NONE))
+        take((size_t)M * K * 4, &w->carry_off, &w->carry_bytes);
       if (act != OSDP_ACT_NONE)
         take((size_t)M * (split_dim == OSDP_SPLIT_OUT ? L : N) * 2, &w->stage0_off, &w->stage0_bytes);
       take(chunks * (size_t)N * 4, &w->part_off, &w->part_bytes);
@@ -213,6 +220,7 @@ struct GemmCall {
   Epilogue epi;
   int carry_bf16;   // MODE_RED: running sum in `out` (bf16) instead of the fp32 carry buffer
   int pair_slices;  // MODE_RED: accumulate two adjacent slices per pass
+  int slice_major;  // MODE_RED, all slices in the launch: sweep slice by slice with the carry (else: slices inside a tile)
   int out_is_slice; // MODE_ROWS / MODE_COLS: `epi.out` is the slice's own compact matrix, not the whole output
   int fp8;          // operands are fp8 e4m3 (1 byte per element) instead of bf16
   int n_peers;      // > 0: the output slice is reduce-added row block by row block into peer_out[0..n_peers)
@@ -425,7 +433,11 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   // letting the CTAs drift across slices inside one launch (16384 x 8192 x 8192: k = 16 4.5 -> 3.9 ms,
   // k = 32 7.8 -> 7.1 ms; no gain at k <= 8, a loss with the bf16 running sum, and a loss of 20 % on
   // operators with only a few tiles per pair such as 8192 x 2048 x 2048).  Same arithmetic, same bits.
-  if (c.mode == MODE_RED && c.s_end - c.s_begin > 1 && !c.pair_slices && !c.carry_bf16 && c.L <= 512 &&
+  // Summed output, every slice in this launch, no option that concerns the carry: a tile walks the slices'
+  // k-blocks in order with its accumulator kept in tensor memory; nothing is carried through memory.
+  const bool in_tmem = c.mode == MODE_RED && c.k_total > 1 && c.s_begin == 0 && c.s_end == c.k_total &&
+                       !c.slice_major && !c.pair_slices && !c.carry_bf16;
+  if (c.mode == MODE_RED && !in_tmem && c.s_end - c.s_begin > 1 && !c.pair_slices && !c.carry_bf16 && c.L <= 512 &&
       cdiv(c.P, 2 * BM) * cdiv(c.Q, 256) >= (int64_t)16 * (sms / 2)) {
     for (int s = c.s_begin; s < c.s_end; ++s) {
       GemmCall one = c;
@@ -454,9 +466,10 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   // a ragged last wave.  Measured model, per tile and CTA pair: 256-wide 6.5 ns per reduction
   // element (epilogue hidden), 512-wide 11.5 ns per element plus 5 us of exposed epilogue; time =
   // rounds of the persistent schedule x tile time.  Both tiles produce the same bits per element
-  // (same k-block order), so the choice may differ between launches.  Summed outputs keep 256.
+  // (same k-block order), so the choice may differ between launches.  Summed outputs that carry their
+  // running sum through memory keep 256 (the carry traffic needs the overlapped epilogue).
   // So does the GEMM whose epilogue reads a second tensor element-wise (direct stores, slower: better hidden).
-  if (pair && c.mode != MODE_RED && c.epi.gz == nullptr) {
+  if (pair && (c.mode != MODE_RED || in_tmem) && c.epi.gz == nullptr) {
     const int64_t units = sms / 2;
     const double red_len = (double)c.R * (c.fp8 ? 0.5 : 1.0);   // an fp8 k-step covers twice the elements
     const double t_n = (double)cdiv(count_items(c, 2 * BM, 256), units) * (6.5e-3 * red_len) + 5.0;
@@ -477,7 +490,7 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   if (p.epi.scale == 0.0f) p.epi.scale = 1.0f;   // callers that zero-fill the call leave it unset
   p.status = c.status;
   p.carry_bf16 = (c.mode == MODE_RED && c.k_total > 1) ? c.carry_bf16 : 0;
-  p.red_group = (c.mode == MODE_RED && c.pair_slices && c.s_end - c.s_begin > 1) ? 2 : 1;
+  p.red_group = in_tmem ? c.k_total : ((c.mode == MODE_RED && c.pair_slices && c.s_end - c.s_begin > 1) ? 2 : 1);
   // Outputs leave through TMA.  The epilogue that reads a second tensor element-wise (gz) does too
   // (its input arrives by TMA as well) when the launch is unsliced and writes bf16, which is how the MLP
   // backward uses it; otherwise that epilogue falls back to direct stores from registers.
@@ -521,7 +534,7 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
                             nullptr);
       if (rc) return rc;
     }
-    if (c.mode == MODE_RED && c.k_total > 1 && !p.carry_bf16) {
+    if (c.mode == MODE_RED && c.k_total > 1 && !p.carry_bf16 && !in_tmem) {
       CUtensorMap unused;
       rc = make_output_maps(c.epi.carry, true, c.P, c.Q, c.epi.ld_carry, MODE_NONE, c.L, 1, &unused, &p.carry_map,
                             nullptr);
@@ -670,9 +683,11 @@ int fwd_impl(const void *x, const void *w_flat, int64_t w_offset, const float *b
   // fp8: x and W are e4m3 bytes (16 elements per 16 bytes: extents, offset and slice length multiples of 16)
   if (!x || !w_flat || !out) return OSDP_ERR_NULL_POINTER;
   {
-    const int frc = check_flags(flags, OSDP_FLAG_CARRY_BF16 | (single ? 0 : OSDP_FLAG_PAIR_SLICES), act, z_save);
+    const int frc = check_flags(flags, OSDP_FLAG_CARRY_BF16 | OSDP_FLAG_SLICE_MAJOR | (single ? 0 : OSDP_FLAG_PAIR_SLICES),
+                                act, z_save);
     if (frc) return frc;
   }
+  if (single) flags |= OSDP_FLAG_SLICE_MAJOR;   // one slice per call is slice-major by construction
   int64_t L = 0;
   int rc = check_common(M, N, K, k, split_dim, act, &L);
   if (rc) return rc;
@@ -724,6 +739,7 @@ int fwd_impl(const void *x, const void *w_flat, int64_t w_offset, const float *b
   c.epi.ld_carry = N;
   c.carry_bf16 = (flags & OSDP_FLAG_CARRY_BF16) ? 1 : 0;
   c.pair_slices = (flags & OSDP_FLAG_PAIR_SLICES) ? 1 : 0;
+  c.slice_major = (flags & OSDP_FLAG_SLICE_MAJOR) ? 1 : 0;
   c.status = static_cast<int *>(ws);
   return launch_gemm(c, static_cast<cudaStream_t>(stream));
 }
@@ -740,8 +756,10 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
   // ld_dw_slice > 0: dW of the slice is written as a compact matrix of the same shape.
   if (!dy || !x || !w_flat) return OSDP_ERR_NULL_POINTER;
   // the bf16 running sum concerns dX only, which has neither bias nor activation of its own
-  if (flags & ~(OSDP_FLAG_ACCUMULATE_DW | OSDP_FLAG_CARRY_BF16 | (single ? 0 : OSDP_FLAG_PAIR_SLICES)))
+  if (flags & ~(OSDP_FLAG_ACCUMULATE_DW | OSDP_FLAG_CARRY_BF16 | OSDP_FLAG_SLICE_MAJOR |
+                (single ? 0 : OSDP_FLAG_PAIR_SLICES)))
     return OSDP_ERR_UNSUPPORTED;
+  if (single) flags |= OSDP_FLAG_SLICE_MAJOR;   // one slice per call is slice-major by construction
   if ((flags & OSDP_FLAG_PAIR_SLICES) && ((flags & OSDP_FLAG_CARRY_BF16) || act != OSDP_ACT_NONE))
     return OSDP_ERR_UNSUPPORTED;   // with an activation the backward runs slice by slice (staged G_s)
   const int accumulate = (flags & OSDP_FLAG_ACCUMULATE_DW) ? 1 : 0;
@@ -812,6 +830,7 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
     c.epi.ld_carry = K;
     c.carry_bf16 = (flags & OSDP_FLAG_CARRY_BF16) ? 1 : 0;
     c.pair_slices = (flags & OSDP_FLAG_PAIR_SLICES) ? 1 : 0;
+    c.slice_major = (flags & OSDP_FLAG_SLICE_MAJOR) ? 1 : 0;
     c.status = status;
     return launch_gemm(c, stream);
   };
@@ -979,10 +998,12 @@ int osdp_split_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int k_spl
                                       int flags, size_t *bytes) {
   if (!bytes) return OSDP_ERR_NULL_POINTER;
   if (act != OSDP_ACT_NONE && act != OSDP_ACT_GELU_TANH && act != OSDP_ACT_GELU_ERF) return OSDP_ERR_UNSUPPORTED;
-  if (flags & ~(OSDP_FLAG_ACCUMULATE_DW | OSDP_FLAG_CARRY_BF16 | OSDP_FLAG_RECOMPUTE | OSDP_FLAG_PAIR_SLICES))
+  if (flags & ~(OSDP_FLAG_ACCUMULATE_DW | OSDP_FLAG_CARRY_BF16 | OSDP_FLAG_RECOMPUTE | OSDP_FLAG_PAIR_SLICES |
+                OSDP_FLAG_SLICE_MAJOR))
     return OSDP_ERR_UNSUPPORTED;
   if ((flags & OSDP_FLAG_RECOMPUTE) && op != OSDP_OP_MLP_BWD) return OSDP_ERR_UNSUPPORTED;
-  if ((flags & OSDP_FLAG_PAIR_SLICES) && op != OSDP_OP_LINEAR_FWD && op != OSDP_OP_LINEAR_BWD) return OSDP_ERR_UNSUPPORTED;
+  if ((flags & (OSDP_FLAG_PAIR_SLICES | OSDP_FLAG_SLICE_MAJOR)) && op != OSDP_OP_LINEAR_FWD && op != OSDP_OP_LINEAR_BWD)
+    return OSDP_ERR_UNSUPPORTED;
   WsPlan plan;
   int rc = plan_workspace(M, N, K, k_split, split_dim, act, op, flags, &plan);
   if (rc) return rc;

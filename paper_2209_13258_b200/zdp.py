@@ -233,9 +233,9 @@ class ZdpSplitLinear:
     def staging_bytes(self, M):
         """Bytes this layer holds besides its weights and gradients: staging plus the kernels' workspace."""
         _, f = B.osdp_split_linear_workspace_bytes(M, self.N, self.K, self.k, self.split_dim, self.act,
-                                                   B.OP_LINEAR_FWD, self.flags & B.FLAG_CARRY_BF16)
+                                                   B.OP_LINEAR_FWD, (self.flags & B.FLAG_CARRY_BF16) | B.FLAG_SLICE_MAJOR)
         _, b = B.osdp_split_linear_workspace_bytes(M, self.N, self.K, self.k, self.split_dim, self.act,
-                                                   B.OP_LINEAR_BWD, self.flags & B.FLAG_CARRY_BF16)
+                                                   B.OP_LINEAR_BWD, (self.flags & B.FLAG_CARRY_BF16) | B.FLAG_SLICE_MAJOR)
         nbytes = lambda ts: sum(t.numel() * t.element_size() for t in ts)
         return {"weight_staging": nbytes(self.w_stage), "grad_staging": nbytes(self.dw_stage), "workspace": max(f, b)}
 

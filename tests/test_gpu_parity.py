@@ -33,8 +33,9 @@ def run_linear(P, c, k, split, act=0, dw_fp32=True, use_bias=True, accumulate=0,
     if dw_init is not None:
         dwf.t.copy_(dw_init)
     db = Guarded((N,), torch.float32)
-    rc, n1 = P.osdp_split_linear_workspace_bytes(M, N, K, k, split, act, P.OP_LINEAR_FWD, flags)
-    rc2, n2 = P.osdp_split_linear_workspace_bytes(M, N, K, k, split, act, P.OP_LINEAR_BWD, flags)
+    qflags = flags | (P.FLAG_SLICE_MAJOR if per_slice else 0)     # one slice per call carries the sum in ws
+    rc, n1 = P.osdp_split_linear_workspace_bytes(M, N, K, k, split, act, P.OP_LINEAR_FWD, qflags)
+    rc2, n2 = P.osdp_split_linear_workspace_bytes(M, N, K, k, split, act, P.OP_LINEAR_BWD, qflags)
     assert rc == 0 and rc2 == 0
     ws = P.new_workspace(max(n1, n2))
     accumulate = accumulate | flags
@@ -111,14 +112,17 @@ RAGGED = [(200, 264, 136), (300, 520, 328), (77, 1032, 72), (513, 8, 520), (130,
 
 @pytest.mark.parametrize("shape", RAGGED)
 @pytest.mark.parametrize("split", [0, 1])
-def test_ragged_shapes_all_k(P, shape, split):
+@pytest.mark.parametrize("order", ["tile", "slice_major"])
+def test_ragged_shapes_all_k(P, shape, split, order):
+    # both orders of an all-slices call: slices inside a tile (sum kept in tensor memory) and
+    # slice-major (sum carried through the workspace)
     M, N, K = shape
     c = inputs.linear_case(M, N, K, w_std=0.1, bias_std=0.3, w_offset=72, flat_pad=8, layer=2)
     D = N if split == 0 else K
     for k in (1, 2, 3, 5, 8, D // 8):
         if k < 1 or P.osdp_slice_range(D, k, 0)[0] != 0:
             continue
-        g = run_linear(P, c, k, split)
+        g = run_linear(P, c, k, split, flags=P.FLAG_SLICE_MAJOR if order == "slice_major" else 0)
         compare(g, oracle_linear(c, 0, k, split), 0)
 
 
@@ -228,11 +232,35 @@ def test_bit_identity_of_concatenated_outputs(P, shape):
 @pytest.mark.parametrize("split", [0, 1])
 @pytest.mark.parametrize("act", [0, 1])
 def test_per_slice_calls_equal_whole_call(P, split, act):
+    # one call per slice == one slice-major call over all slices, bit for bit; the default order of an
+    # all-slices call gives the same concatenated outputs and a summed output equal up to fp32 rounding order
     c = inputs.linear_case(300, 520, 328, w_std=0.1, bias_std=0.2, layer=7)
-    a = run_linear(P, c, 3, split, act=act)
+    a = run_linear(P, c, 3, split, act=act, flags=P.FLAG_SLICE_MAJOR)
     b = run_linear(P, c, 3, split, act=act, per_slice=True)
     for name in ("y", "dx", "dw", "db"):
         assert torch.equal(_bits(a[name]), _bits(b[name])), name
+    d = run_linear(P, c, 3, split, act=act)
+    for name in (("y", "dw", "db") if split == 0 else ("dx", "dw", "db")):
+        assert torch.equal(_bits(a[name]), _bits(d[name])), name
+    summed = "dx" if split == 0 else "y"
+    assert_close(to_f64(d[summed]), to_f64(a[summed]), summed + " tile order vs slice-major", relf_tol=3e-3)
+
+
+@pytest.mark.parametrize("shape", [(512, 2048, 1024), (2048, 4096, 4096)])
+def test_summed_output_in_tensor_memory_is_bit_identical_to_unsplit(P, shape):
+    # default order, slice length a multiple of the 64-element k-block: a tile meets exactly the k-blocks
+    # of the unsplit GEMM in the same order, so even the summed output has the unsplit result's bits
+    M, N, K = shape
+    c = inputs.linear_case(M, N, K, bias_std=0.1, layer=19)
+    g1 = run_linear(P, c, 1, 0)
+    for k in (2, 4, 8, 16):
+        for split in (0, 1):
+            g = run_linear(P, c, k, split)
+            for name in ("y", "dx", "dw", "db"):
+                assert torch.equal(_bits(g[name]), _bits(g1[name])), (name, k, split)
+    # and the workspace of such a call holds no carry
+    _, n = P.osdp_split_linear_workspace_bytes(M, N, K, 8, 1, 0, P.OP_LINEAR_FWD)
+    assert n == 256
 
 
 def test_repeated_runs_are_bitwise_equal(P):
@@ -515,6 +543,8 @@ def _random_cases(n, seed):
         k = int(rng.choice([1, 2, 3, 4, 5, 7, 8, 12, 16, max(1, D // 8)]))
         act = int(rng.choice([0, 0, 1, 2]))
         flags = 2 if (act == 0 and 1 < k <= 8 and rng.random() < 0.3) else 0   # bf16 running sum: k <= 8 only
+        if flags == 0 and rng.random() < 0.4:
+            flags = 16                                                          # slice-major order, fp32 carry
         cases.append((M, N, K, k, split, act, flags))
     return cases
 
@@ -528,7 +558,7 @@ def test_random_shapes_against_oracle(P, chunk):
                                layer=100 + chunk * 10 + idx)
         g = run_linear(P, c, k, split, act=act, flags=flags, dw_fp32=bool(idx % 2))
         o = oracle_linear(c, act, k, split)
-        loose = 3e-2 * (2 * k) ** 0.5 if flags else 3e-2
+        loose = 3e-2 * (2 * k) ** 0.5 if flags == 2 else 3e-2
         try:
             compare(g, o, act, y_abs_tol=loose if split == 1 else 3e-2, dx_abs_tol=loose if split == 0 else 3e-2)
         except AssertionError as e:

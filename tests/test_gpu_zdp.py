@@ -44,8 +44,8 @@ def test_gathered_slice_entry_points_match_flat_buffer_ones_bit_for_bit(P, shape
     off = c["w_offset"]
     W = wf[off:off + N * K].view(N, K)
     lay = ShardLayout(N, K, k, split, 1)
-    _, n1 = P.osdp_split_linear_workspace_bytes(M, N, K, k, split, act, P.OP_LINEAR_FWD)
-    _, n2 = P.osdp_split_linear_workspace_bytes(M, N, K, k, split, act, P.OP_LINEAR_BWD)
+    _, n1 = P.osdp_split_linear_workspace_bytes(M, N, K, k, split, act, P.OP_LINEAR_FWD, P.FLAG_SLICE_MAJOR)
+    _, n2 = P.osdp_split_linear_workspace_bytes(M, N, K, k, split, act, P.OP_LINEAR_BWD, P.FLAG_SLICE_MAJOR)
     res = {}
     for staged in (False, True):
         ws = P.new_workspace(max(n1, n2))
@@ -92,7 +92,7 @@ def test_gathered_slice_argument_errors(P):
     x = torch.zeros(M, K, dtype=torch.bfloat16, device="cuda")
     w = torch.zeros(N // k, K, dtype=torch.bfloat16, device="cuda")
     out = torch.zeros(M, N, dtype=torch.bfloat16, device="cuda")
-    _, n = P.osdp_split_linear_workspace_bytes(M, N, K, k, 0, 0, P.OP_LINEAR_BWD)
+    _, n = P.osdp_split_linear_workspace_bytes(M, N, K, k, 0, 0, P.OP_LINEAR_BWD, P.FLAG_SLICE_MAJOR)
     ws = P.new_workspace(n)
     f = P.osdp_zdp_linear_fwd_slice
     assert f(x, w, 0, None, M, N, K, k, 0, 0, 0, out, None, ws) == 2        # ld_w <= 0
@@ -262,7 +262,7 @@ def test_scatter_argument_errors(P):
     x = torch.zeros(M, K, dtype=torch.bfloat16, device="cuda")
     w = torch.zeros(N // k, K, dtype=torch.bfloat16, device="cuda")
     dy = torch.zeros(M, N, dtype=torch.bfloat16, device="cuda")
-    _, n = P.osdp_split_linear_workspace_bytes(M, N, K, k, 0, 0, P.OP_LINEAR_BWD)
+    _, n = P.osdp_split_linear_workspace_bytes(M, N, K, k, 0, 0, P.OP_LINEAR_BWD, P.FLAG_SLICE_MAJOR)
     ws = P.new_workspace(n)
     g = P.osdp_zdp_linear_bwd_slice_scatter
     sh = [torch.zeros(N // k * K // 2, dtype=torch.float32, device="cuda") for _ in range(2)]

@@ -41,18 +41,28 @@ def test_slice_range_matches_golden_table():
 
 def test_workspace_plan():
     M, N, K = 16384, 8192, 8192
-    q = lambda k, split, act, op: P.osdp_split_linear_workspace_bytes(M, N, K, k, split, act, op)
-    # forward: nothing but the status block unless the reduction dim is split (fp32 carry of Y)
+    q = lambda k, split, act, op, fl=0: P.osdp_split_linear_workspace_bytes(M, N, K, k, split, act, op, fl)
+    SM = P.FLAG_SLICE_MAJOR
+    # forward, all slices in one call: nothing but the status block (a summed output stays in tensor memory)
     assert q(1, 0, 0, P.OP_LINEAR_FWD) == (0, 256)
     assert q(8, 0, 0, P.OP_LINEAR_FWD) == (0, 256)
-    assert q(8, 1, 0, P.OP_LINEAR_FWD) == (0, 256 + M * N * 4)
-    # backward: column-sum partials always; fp32 carry of dX when the output dim is split
+    assert q(8, 1, 0, P.OP_LINEAR_FWD) == (0, 256)
+    # slice-major order / one slice per call: fp32 carry of Y when the reduction dim is split
+    assert q(8, 0, 0, P.OP_LINEAR_FWD, SM) == (0, 256)
+    assert q(8, 1, 0, P.OP_LINEAR_FWD, SM) == (0, 256 + M * N * 4)
+    assert q(8, 1, 0, P.OP_LINEAR_FWD, P.FLAG_PAIR_SLICES) == (0, 256 + M * N * 4)
+    assert q(1, 1, 0, P.OP_LINEAR_FWD, SM) == (0, 256)
+    # backward: column-sum partials always; fp32 carry of dX when the output dim is split slice-major
     part = 16 * N * 4
     assert q(1, 0, 0, P.OP_LINEAR_BWD) == (0, 256 + part)
-    assert q(8, 0, 0, P.OP_LINEAR_BWD) == (0, 256 + M * K * 4 + part)
+    assert q(8, 0, 0, P.OP_LINEAR_BWD) == (0, 256 + part)
+    assert q(8, 0, 0, P.OP_LINEAR_BWD, SM) == (0, 256 + M * K * 4 + part)
     assert q(8, 1, 0, P.OP_LINEAR_BWD) == (0, 256 + part)
-    # activation backward stages G for one slice (output split) or whole (reduction split)
-    assert q(8, 0, 1, P.OP_LINEAR_BWD)[1] - q(8, 0, 0, P.OP_LINEAR_BWD)[1] == M * (N // 8) * 2
+    assert q(8, 1, 0, P.OP_LINEAR_BWD, SM) == (0, 256 + part)
+    # activation backward stages G for one slice (output split; the call then goes slice by slice and
+    # carries dX whatever the flags) or whole (reduction split)
+    assert q(8, 0, 1, P.OP_LINEAR_BWD)[1] == 256 + M * K * 4 + M * (N // 8) * 2 + part
+    assert q(8, 0, 1, P.OP_LINEAR_BWD, SM) == q(8, 0, 1, P.OP_LINEAR_BWD)
     assert q(8, 1, 1, P.OP_LINEAR_BWD)[1] - q(8, 1, 0, P.OP_LINEAR_BWD)[1] == M * N * 2
     # MLP chain: slice-sized intermediates shrink as 1/k
     f = lambda k: P.osdp_split_linear_workspace_bytes(8192, 32768, 8192, k, 0, 1, P.OP_MLP_FWD)[1]
@@ -60,12 +70,12 @@ def test_workspace_plan():
     assert f(1) == 256 + 8192 * 32768 * 2
     for k in (2, 4, 8, 16):
         assert f(k) == 256 + carry + 8192 * (32768 // k) * 2
-    assert q(8, 1, 0, P.OP_LINEAR_FWD) != (0, 256)
-    assert P.osdp_split_linear_workspace_bytes(M, N, K, 8, 1, 0, P.OP_LINEAR_FWD, P.FLAG_CARRY_BF16) == (0, 256)
-    assert P.osdp_split_linear_workspace_bytes(M, N, K, 8, 0, 0, P.OP_LINEAR_BWD, P.FLAG_CARRY_BF16) == (0, 256 + part)
+    assert q(8, 1, 0, P.OP_LINEAR_FWD, SM | P.FLAG_CARRY_BF16) == (0, 256)
+    assert q(8, 0, 0, P.OP_LINEAR_BWD, SM | P.FLAG_CARRY_BF16) == (0, 256 + part)
     assert P.osdp_split_linear_workspace_bytes(8192, 32768, 8192, 8, 0, 1, P.OP_MLP_FWD, P.FLAG_CARRY_BF16) == (
         0, 256 + 8192 * 4096 * 2)
-    assert P.osdp_split_linear_workspace_bytes(8, 8, 8, 1, 0, 0, 0, 16)[0] == 6
+    assert P.osdp_split_linear_workspace_bytes(8, 8, 8, 1, 0, 0, 0, 32)[0] == 6
+    assert P.osdp_split_linear_workspace_bytes(8, 8, 8, 1, 0, 0, P.OP_MLP_FWD, SM)[0] == 6
     assert P.osdp_split_linear_workspace_bytes(8, 8, 8, 1, 0, 0, 9)[0] == 6
     assert P.osdp_split_linear_workspace_bytes(8, 8, 8, 1, 0, 7, 0)[0] == 6
     assert P.osdp_split_linear_workspace_bytes(8, 16, 8, 3, 0, 0, 0)[0] == 3
@@ -96,7 +106,9 @@ def test_forward_argument_checks():
     assert _fwd(x=A + 2) == 4 and _fwd(out=A + 8) == 4 and _fwd(ws=(A + 16, 1 << 30)) == 4
     assert _fwd(k_split=-1) == 3 and _fwd(k_split=9) == 3 and _fwd(split_dim=2) == 3
     assert _fwd(act=3) == 6
-    assert _fwd(split_dim=1, ws=(A, 256)) == 5          # the carry does not fit
+    assert _fwd(split_dim=1, ws=(A, 256)) in (0, 7)     # all slices in one call: the sum stays in tensor memory
+    assert _fwd(split_dim=1, ws=(A, 256), flags=P.FLAG_SLICE_MAJOR) == 5   # slice-major: the carry does not fit
+    assert P.osdp_split_linear_fwd_slice(A, A, 0, None, 64, 64, 64, 2, 1, 0, 0, A, None, (A, 256), stream=0) == 5
     assert _fwd(split_dim=1, ws=(A, 256), flags=P.FLAG_CARRY_BF16) in (0, 7)   # bf16 running sum: no carry needed
     assert _fwd(flags=P.FLAG_CARRY_BF16, act=1) == 6    # the bf16 running sum excludes an activation ...
     assert _fwd(flags=P.FLAG_CARRY_BF16, z_save=A) == 6  # ... and a saved pre-activation
@@ -117,7 +129,8 @@ def test_backward_argument_checks():
     assert _bwd(dw_dtype=2) == 6
     assert _bwd(dw_offset=12) == 4 and _bwd(dx=A + 4) == 4 and _bwd(dbias=A + 4) == 4
     assert _bwd(k_split=9) == 3
-    assert _bwd(ws=(A, 1024)) == 5
+    assert _bwd(ws=(A, 64)) == 5
+    assert _bwd(ws=(A, 1024)) in (0, 7) and _bwd(ws=(A, 1024), flags=P.FLAG_SLICE_MAJOR) == 5
     assert _bwd(flags=32) == 6
     # pairing of adjacent slices: all-slices calls only, not together with the bf16 running sum or an activation
     assert _bwd(flags=P.FLAG_PAIR_SLICES) in (0, 7)
@@ -143,7 +156,7 @@ def test_mlp_argument_checks():
     assert b(z1_saved=None) == 1 and b(dw_dtype=5) == 6 and b(dw_off_w1=4) == 4 and b(ws=(A, 4096)) == 5
     # with recomputation no saved activation is needed, but one more slice-sized buffer is
     assert b(z1_saved=None, flags=P.FLAG_RECOMPUTE) in (0, 7)
-    assert b(flags=16) == 6 and b(flags=P.FLAG_RECOMPUTE, b1=A + 4) == 4
+    assert b(flags=32) == 6 and b(flags=P.FLAG_SLICE_MAJOR) == 6 and b(flags=P.FLAG_RECOMPUTE, b1=A + 4) == 4
     plain = P.osdp_split_linear_workspace_bytes(32, 256, 64, 4, 0, 1, P.OP_MLP_BWD)[1]
     assert P.osdp_split_linear_workspace_bytes(32, 256, 64, 4, 0, 1, P.OP_MLP_BWD, P.FLAG_RECOMPUTE)[1] == plain + 32 * 64 * 2
     assert P.osdp_split_linear_workspace_bytes(32, 256, 64, 4, 0, 1, P.OP_MLP_FWD, P.FLAG_RECOMPUTE)[0] == 6
