@@ -240,9 +240,14 @@ def test_per_slice_calls_equal_whole_call(P, split, act):
     for name in ("y", "dx", "dw", "db"):
         assert torch.equal(_bits(a[name]), _bits(b[name])), name
     d = run_linear(P, c, 3, split, act=act)
+    summed = "dx" if split == 0 else "y"
+    if split == 1 and act:
+        # the saved pre-activation is itself the summed output here, so the whole backward sees other bits
+        for name in ("y", "dx", "dw", "db"):
+            assert_close(to_f64(d[name]), to_f64(a[name]), name + " tile order vs slice-major", relf_tol=3e-3)
+        return
     for name in (("y", "dw", "db") if split == 0 else ("dx", "dw", "db")):
         assert torch.equal(_bits(a[name]), _bits(d[name])), name
-    summed = "dx" if split == 0 else "y"
     assert_close(to_f64(d[summed]), to_f64(a[summed]), summed + " tile order vs slice-major", relf_tol=3e-3)
 
 
