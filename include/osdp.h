@@ -31,7 +31,16 @@
  *
  * Conventions for every call
  *  - All tensor pointers are DEVICE pointers unless stated; they stay owned by the caller and
- *    must stay valid until the stream has passed the call.  Nothing is allocated or freed.
+ *    must stay valid until the stream has passed the call.  No device memory is allocated or
+ *    freed by any call.  Two things are created once per device at first use and kept until the
+ *    process ends: each kernel variant's attributes (shared-memory size), and, by the first
+ *    backward call that asks for dX and dW together (or the first osdp_split_mlp_bwd with weight
+ *    gradients), two internal non-blocking streams and three events.  Such a call forks its
+ *    weight-gradient launches onto those streams and joins them back into `stream` before it
+ *    returns to the caller's ordering; while it enqueues that fork / join section it holds a
+ *    host-side lock, so concurrent callers on one device are serialised on the host for the
+ *    few microseconds of enqueueing (the GPU work is not serialised).  Make the first call on a
+ *    device outside any stream capture.
  *  - bf16 tensors are row-major, 16-byte aligned; N and K must be multiples of 8.
  *  - W lives inside a flat bf16 parameter buffer `w_flat` at ELEMENT offset `w_offset`
  *    (multiple of 8); it is read in place through TMA descriptors, never copied or unflattened.
@@ -117,10 +126,14 @@ int osdp_last_cuda_error(void);
  * or s is out of range. */
 int osdp_slice_range(int64_t D, int k_split, int slice_idx, int64_t *begin, int64_t *end);
 
-/* Exact scratch bytes a call with these arguments uses (the "staging" figure).  For the linear
+/* Section 3.3 states the memory effect of splitting as size(MatMul) / slice granularity: only one slice of
+ * the operator and of its intermediates is live at a time.  This query makes that figure concrete.
+ * Exact scratch bytes a call with these arguments uses (the "staging" figure).  For the linear
  * ops (M,N,K) are the layer's; for the MLP ops pass M = tokens, N = ffn, K = hidden.
  * The query assumes every optional output (dx, dbias, ...) is requested.  `flags` as for the call
- * (OSDP_FLAG_CARRY_BF16 removes the fp32 carry). */
+ * (OSDP_FLAG_SLICE_MAJOR: sized for the *_slice entry points, i.e. with the fp32 carry of a summed
+ * output; OSDP_FLAG_CARRY_BF16 removes that carry).  Host-only arithmetic.
+ * Errors: NULL bytes, bad shape / split / activation / op / flags as for the call itself. */
 int osdp_split_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int k_split, int split_dim,
                                       int act, int op, int flags, size_t *bytes);
 
@@ -134,12 +147,15 @@ int osdp_split_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int k_spl
 int osdp_suggest_granularity(int64_t M, int64_t N, int64_t K, int split_dim, int act, int op, int flags,
                              size_t budget_bytes, int max_k, int *k_split);
 
-/* Forward of all k slices in slice-major order (Section 3.3 steps 1-3).
+/* Forward of all k slices (Section 3.3 steps 1-3: partition, process the slices one after another, add
+ * the results).
  *   x [M,K] bf16; bias [N] fp32 or NULL; out [M,N] bf16 = act(X W^T + bias);
  *   z_save [M,N] bf16 or NULL: receives the pre-activation (what the backward needs when act != NONE).
- * OUT: slice s writes columns R_s of out.  RED: partial products are summed (fp32 carry in ws, or
- * in `out` itself with OSDP_FLAG_CARRY_BF16); bias and activation are applied once.
- * flags: 0, OSDP_FLAG_CARRY_BF16, OSDP_FLAG_PAIR_SLICES. */
+ * OUT: slice s writes columns R_s of out.  RED: the slices' products are added in ascending order in fp32
+ * (in tensor memory, tile by tile; with OSDP_FLAG_SLICE_MAJOR slice by slice over the whole operator with
+ * the running sum in ws, or in `out` itself with OSDP_FLAG_CARRY_BF16); bias and activation are applied once.
+ * flags: 0, OSDP_FLAG_SLICE_MAJOR, OSDP_FLAG_CARRY_BF16, OSDP_FLAG_PAIR_SLICES (the last two imply the
+ * slice-major order: they are options of its carry). */
 int osdp_split_linear_fwd(const void *x, const void *w_flat, int64_t w_offset, const float *bias,
                           int64_t M, int64_t N, int64_t K, int k_split, int split_dim, int act,
                           int flags, void *out, void *z_save, void *ws, size_t ws_bytes, void *stream);
@@ -147,20 +163,27 @@ int osdp_split_linear_fwd(const void *x, const void *w_flat, int64_t w_offset, c
 /* One slice of the forward (Section 3.3 step 2: the slices are computed one after another):
  * lets a caller put other work between slices.  Slices must be issued in
  * ascending order on one stream with the same arguments and workspace: under RED slice 0
- * starts the carry and slice k-1 writes `out`. */
+ * starts the carry and slice k-1 writes `out`.  The workspace must be sized with
+ * OSDP_FLAG_SLICE_MAJOR in the query's flags (OSDP_ERR_WORKSPACE_TOO_SMALL otherwise). */
 int osdp_split_linear_fwd_slice(const void *x, const void *w_flat, int64_t w_offset, const float *bias,
                                 int64_t M, int64_t N, int64_t K, int k_split, int split_dim, int act,
                                 int flags, int slice_idx, void *out, void *z_save, void *ws,
                                 size_t ws_bytes, void *stream);
 
-/* Backward of all k slices in slice-major order.
+/* Backward of all k slices.  The paper states the forward only (Section 3.3) and leaves the backward to
+ * automatic differentiation; differentiating  Y = act(sum_s X[:,C_s] W[:,C_s]^T + b)  (RED)  or
+ * Y[:,R_s] = act(X W[R_s,:]^T + b[R_s])  (OUT)  slice by slice gives, with G = dY (.) act'(Z):
+ *   OUT: dW[R_s,:] = G[:,R_s]^T X, db[R_s] = colsum G[:,R_s], dX = sum_s G[:,R_s] W[R_s,:]
+ *   RED: dX[:,C_s] = G W[:,C_s], dW[:,C_s] = G^T X[:,C_s], db = colsum G
+ * i.e. the split that concatenates in the forward sums in the backward and vice versa.
  *   dy [M,N] bf16; x [M,K] bf16; z_saved [M,N] bf16 (pre-activation; required iff act != NONE);
  *   dx [M,K] bf16 or NULL; dw_flat + dw_offset: dW [N,K] in dw_dtype (bf16 or fp32), NULL to skip;
  *   flags: OSDP_FLAG_ACCUMULATE_DW (dW += ... instead of dW = ...), OSDP_FLAG_CARRY_BF16 (dX's running
  *   sum in dx itself under OUT split), OSDP_FLAG_PAIR_SLICES (dX under OUT split);
  *   dbias [N] fp32 or NULL (always overwritten).
- * OUT: dW[R_s,:], db[R_s] per slice, dX = sum over slices (fp32 carry in ws).
- * RED: dX[:,C_s], dW[:,C_s] per slice.
+ *   flags also: OSDP_FLAG_SLICE_MAJOR (dX under OUT split swept slice by slice, fp32 carry in ws).
+ * With an activation under OUT split the call stages G_s = dY[:,R_s] (.) act'(Z[:,R_s]) one slice at a
+ * time (slice-sized staging) and therefore always runs slice-major with the fp32 carry of dX.
  * When both dx and dw_flat are given, the call runs dW and db on a stream of its own
  * next to dX, forked from and joined back into `stream` (see osdp_split_mlp_bwd for the rules of these
  * internal streams). */
@@ -170,8 +193,10 @@ int osdp_split_linear_bwd(const void *dy, const void *x, const void *w_flat, int
                           int dw_dtype, int flags, float *dbias, void *ws, size_t ws_bytes,
                           void *stream);
 
-/* One slice of the backward; same ordering rule as osdp_split_linear_fwd_slice.  Under RED
- * dbias is produced by slice 0. */
+/* One slice of the backward (the per-slice terms of the derivation above; Section 3.3 step 2 applied to
+ * the backward); same ordering rule as osdp_split_linear_fwd_slice: under OUT slice 0 starts the carry
+ * of dX and slice k-1 writes dx.  Under RED dbias is produced by slice 0.  The workspace must be sized
+ * with OSDP_FLAG_SLICE_MAJOR in the query's flags. */
 int osdp_split_linear_bwd_slice(const void *dy, const void *x, const void *w_flat, int64_t w_offset,
                                 const void *z_saved, int64_t M, int64_t N, int64_t K, int k_split,
                                 int split_dim, int act, int slice_idx, void *dx, void *dw_flat,
@@ -309,9 +334,12 @@ int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_
                        int64_t dw_off_w2, int dw_dtype, int flags, float *db1, float *db2,
                        void *ws, size_t ws_bytes, void *stream);
 
-/* Synchronises `stream`, copies the device status word at the start of `ws` to *status
- * (OSDP_OK, or OSDP_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel ran out) and
- * clears it.  Every device-side wait in this library is bounded; none can hang the GPU. */
+/* Failure detection (no counterpart in the paper, which does not discuss faults: the slices of Section
+ * 3.3 "executed sequentially" are pipelines of asynchronous copies and tensor-core work whose stages
+ * wait on one another, and every such wait here is bounded).  Synchronises `stream`, copies the device
+ * status word at the start of `ws` to *status (OSDP_OK, or OSDP_ERR_DEVICE_TIMEOUT if a bounded wait
+ * inside a kernel ran out) and clears it.  Every device-side wait in this library is bounded; none can
+ * hang the GPU.  This is the one call that synchronises. */
 int osdp_read_device_status(void *ws, int *status, void *stream);
 
 /* Diagnostic for the failure-detection path (no counterpart in the paper): launches one warp that
@@ -333,14 +361,17 @@ int osdp_debug_wait_probe(void *ws, int64_t limit_us, void *stream);
  *
  * The partial sums live in a 4 MiB array built into the library image
  * (OSDP_NOALLOC_MAX_PARTIALS floats); every GPU on which the library is loaded holds it until
- * the process exits.  Limit: ceil(M/1024) * N <= OSDP_NOALLOC_MAX_PARTIALS, else
- * OSDP_ERR_EXCEEDS_STATIC_SCRATCH and nothing is launched.
+ * the process exits.  Limit: ceil(M/1024) * N <= OSDP_NOALLOC_MAX_PARTIALS and ceil(M/1024) <= 65535,
+ * else OSDP_ERR_EXCEEDS_STATIC_SCRATCH and nothing is launched.
  *
  *   dy [M,N] bf16 device, row-major, 16-byte aligned, N a multiple of 8; dbias [N] fp32 device.
  *   Asynchronous on `stream`; caller keeps the buffers alive until the stream has passed it.
  *
  * The first call on each device looks up the array's device address (with that device
- * current); make that first call before starting any stream capture.  All calls on a device
+ * current).  With CUDA's lazy module loading that look-up is also what loads the library's device
+ * code and reserves the array on that GPU, so the first call is not itself allocation-free: make it
+ * once per device at start-up, before the region where allocation is forbidden and before starting
+ * any stream capture.  All calls on a device
  * share the one array, which keeps whatever the last call left in it; each call overwrites the
  * part it reads, so no clearing is needed, but two calls that may run at the same time on one
  * GPU (different streams, different threads) race on it: serialise them. */

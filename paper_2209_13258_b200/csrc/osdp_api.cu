@@ -109,6 +109,60 @@ int side_streams(SideStreams **out) {
   return OSDP_OK;
 }
 
+// One fork / join section: launches that may run next to the caller's stream go to the internal streams
+// between begin() and end().  end() always runs (the destructor calls it on an early return), so the caller's
+// stream is joined with whatever was queued on the internal streams even when a launch in between failed.
+// If the internal streams are in use by a stream capture other than the caller's own (a capture that pulled
+// them in and has not ended yet), the section does not fork: everything goes to the caller's stream.
+struct ForkJoin {
+  SideStreams *side = nullptr;
+  std::unique_lock<std::mutex> lock;
+  cudaStream_t main = nullptr;
+  int n = 0;
+  bool open = false;
+
+  static bool foreign_capture(cudaStream_t caller, cudaStream_t internal) {
+    cudaStreamCaptureStatus si = cudaStreamCaptureStatusNone, sc = cudaStreamCaptureStatusNone;
+    unsigned long long idi = 0, idc = 0;
+    if (cudaStreamGetCaptureInfo(internal, &si, &idi) != cudaSuccess) { cudaGetLastError(); return true; }
+    if (si == cudaStreamCaptureStatusNone) return false;
+    if (cudaStreamGetCaptureInfo(caller, &sc, &idc) != cudaSuccess) { cudaGetLastError(); return true; }
+    return !(sc == cudaStreamCaptureStatusActive && si == cudaStreamCaptureStatusActive && idc == idi);
+  }
+  // acquire the internal streams (first use creates them); no GPU work is queued yet
+  int acquire(cudaStream_t caller, int n_streams) {
+    int rc = side_streams(&side);
+    if (rc) return rc;
+    lock = std::unique_lock<std::mutex>(g_side_mutex);
+    main = caller;
+    n = n_streams;
+    for (int i = 0; i < n; ++i)
+      if (foreign_capture(caller, side->s[i])) { n = 0; break; }
+    return OSDP_OK;
+  }
+  int begin() {
+    if (!side || n == 0) return OSDP_OK;
+    cudaError_t e = cudaEventRecord(side->fork, main);
+    for (int i = 0; i < n && e == cudaSuccess; ++i) e = cudaStreamWaitEvent(side->s[i], side->fork, 0);
+    if (e != cudaSuccess) return cuda_fail(e);
+    open = true;
+    return OSDP_OK;
+  }
+  cudaStream_t stream(int i) const { return (open && i < n) ? side->s[i] : main; }
+  int end() {
+    if (!open) return OSDP_OK;
+    open = false;
+    cudaError_t first = cudaSuccess;
+    for (int i = 0; i < n; ++i) {
+      cudaError_t e = cudaEventRecord(side->join[i], side->s[i]);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(main, side->join[i], 0);
+      if (e != cudaSuccess && first == cudaSuccess) first = e;
+    }
+    return first == cudaSuccess ? OSDP_OK : cuda_fail(first);
+  }
+  ~ForkJoin() { end(); }
+};
+
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -775,6 +829,7 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
     s_end = k;
   }
   if (act != OSDP_ACT_NONE && !z_saved) return OSDP_ERR_NULL_POINTER;
+  if (dbias && cdiv(M, COLSUM_ROWS_PER_CHUNK) > 65535) return OSDP_ERR_BAD_SHAPE;   // the column sum's grid limit
   if (fp8) {
     if (act != OSDP_ACT_NONE || dbias || ld_w_slice > 0 || ld_dw_slice > 0 || !std::isfinite(scale_dx) ||
         !std::isfinite(scale_dw))
@@ -861,18 +916,15 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
     // partly filled wave of tiles leaves idle.  Measured on B200, backward only: 256 x 2048 x 512 42 -> 34 us;
     // 8192 x 2048 x 2048 +8 %, 4096 x 4096 x 1024 +7 %, 8192 x 2048 x 8192 +5 %, 32768 x 4096 x 4096 +3 %,
     // 16384 x 8192 x 8192 +0.3 % (k = 8: +1 %); one shape tried lost (8192 x 6144 x 2048, -1.5 %).
-    SideStreams *side = nullptr;
-    std::unique_lock<std::mutex> side_lock;
-    cudaStream_t s_main = stream, s_side = stream;
+    ForkJoin fj;
+    cudaStream_t s_main = stream;
     if (dx && dw) {
-      rc = side_streams(&side);
+      rc = fj.acquire(stream, 1);
       if (rc) return rc;
-      side_lock = std::unique_lock<std::mutex>(g_side_mutex);
-      cudaError_t e = cudaEventRecord(side->fork, stream);
-      if (e == cudaSuccess) e = cudaStreamWaitEvent(side->s[0], side->fork, 0);
-      if (e != cudaSuccess) return cuda_fail(e);
-      s_side = side->s[0];
+      rc = fj.begin();
+      if (rc) return rc;
     }
+    cudaStream_t s_side = fj.stream(0);
     stream = s_main;
     if (dx) { rc = dx_call(Operand{dy, N, M, N, false, true}, s_begin, s_end); if (rc) return rc; }
     stream = s_side;
@@ -888,38 +940,26 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
       if (rc) return rc;
     }
     stream = s_main;
-    if (side) {
-      cudaError_t e = cudaEventRecord(side->join[0], side->s[0]);
-      if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, side->join[0], 0);
-      if (e != cudaSuccess) return cuda_fail(e);
-    }
-    return OSDP_OK;
+    return fj.end();
   }
 
   // With an activation the GEMMs read G = dY (.) act'(Z) from staging.  As above, when both are wanted dW (and
   // db) run on the internal stream next to dX; they join before the staging is written again.
-  SideStreams *side = nullptr;
-  std::unique_lock<std::mutex> side_lock;
+  ForkJoin fj;
   if (dx && dw) {
-    rc = side_streams(&side);
+    rc = fj.acquire(stream, 1);
     if (rc) return rc;
-    side_lock = std::unique_lock<std::mutex>(g_side_mutex);
   }
   cudaStream_t s_main = stream;
   auto fork = [&]() -> int {
-    if (!side) return OSDP_OK;
-    cudaError_t e = cudaEventRecord(side->fork, s_main);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(side->s[0], side->fork, 0);
-    if (e != cudaSuccess) return cuda_fail(e);
-    stream = side->s[0];
+    int r = fj.begin();
+    if (r) return r;
+    stream = fj.stream(0);
     return OSDP_OK;
   };
   auto join = [&]() -> int {
     stream = s_main;
-    if (!side) return OSDP_OK;
-    cudaError_t e = cudaEventRecord(side->join[0], side->s[0]);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(s_main, side->join[0], 0);
-    return e == cudaSuccess ? OSDP_OK : cuda_fail(e);
+    return fj.end();
   };
 
   if (out_split) {
@@ -1306,20 +1346,14 @@ static int mlp_bwd_impl(const void *dy, const void *x, const void *w_flat, int64
     // The slice's three remaining GEMMs and its column sum depend only on what has been launched so far.
     // They are forked onto the internal streams so that they share the SMs (each fills the others' partly
     // filled last wave of tiles).
-    SideStreams *side = nullptr;
-    std::unique_lock<std::mutex> side_lock;
-    cudaStream_t s_dw2 = stream, s_dw1 = stream;
+    ForkJoin fj;
     if (concurrent) {
-      rc = side_streams(&side);
+      rc = fj.acquire(stream, 2);
       if (rc) return rc;
-      side_lock = std::unique_lock<std::mutex>(g_side_mutex);
-      cudaError_t e = cudaEventRecord(side->fork, stream);
-      if (e == cudaSuccess) e = cudaStreamWaitEvent(side->s[0], side->fork, 0);
-      if (e == cudaSuccess) e = cudaStreamWaitEvent(side->s[1], side->fork, 0);
-      if (e != cudaSuccess) return cuda_fail(e);
-      s_dw2 = side->s[0];
-      s_dw1 = side->s[1];
+      rc = fj.begin();
+      if (rc) return rc;
     }
+    cudaStream_t s_dw2 = fj.stream(0), s_dw1 = fj.stream(1);
     if (dw_flat) {
       // dW2[:,F_s] = dY^T A_s
       memset(&c, 0, sizeof(c));
@@ -1371,15 +1405,9 @@ static int mlp_bwd_impl(const void *dy, const void *x, const void *w_flat, int64
       rc = launch_gemm(c, stream);
       if (rc) return rc;
     }
-    if (concurrent) {
-      // join: the next slice reuses the staging buffers these launches read
-      cudaError_t e = cudaSuccess;
-      for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
-        e = cudaEventRecord(side->join[i], side->s[i]);
-        if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, side->join[i], 0);
-      }
-      if (e != cudaSuccess) return cuda_fail(e);
-    }
+    // join: the next slice reuses the staging buffers these launches read
+    rc = fj.end();
+    if (rc) return rc;
   }
   return OSDP_OK;
 }
@@ -1521,7 +1549,8 @@ extern "C" int osdp_bias_grad_noalloc(const void *dy, int64_t M, int64_t N, floa
   if (N & 7) return OSDP_ERR_ALIGNMENT;
   if (!aligned16(dy) || !aligned16(dbias)) return OSDP_ERR_ALIGNMENT;
   const int64_t chunks = cdiv(M, COLSUM_ROWS_PER_CHUNK);
-  if (chunks * N > (int64_t)OSDP_NOALLOC_MAX_PARTIALS) return OSDP_ERR_EXCEEDS_STATIC_SCRATCH;
+  // the chunk count is also a grid dimension of the first pass (at most 65535)
+  if (chunks > 65535 || chunks * N > (int64_t)OSDP_NOALLOC_MAX_PARTIALS) return OSDP_ERR_EXCEEDS_STATIC_SCRATCH;
   float *partials = nullptr;
   int rc = noalloc_scratch(&partials);   // first call on a device: looks the address up
   if (rc) return rc;

@@ -432,6 +432,25 @@ class ZdpSplitLinear:
         cur.wait_stream(self.comm_stream)                   # gradients are complete for whoever runs next on `cur`
         return dx
 
+    def backward_step(self, *args, **kwargs):
+        """One gradient step with the ordering the epilogue-fused scatter needs.  Every rank zeroes its gradient
+        shards; the ranks meet at a barrier (no rank may add into a shard that its owner has not zeroed yet);
+        `backward(*args, **kwargs)` runs; the ranks meet again (every rank's terms have arrived) and only then
+        are the shards valid to read.  The host waits for the device before each barrier, so the barrier orders
+        the ranks' device work, not just their hosts.  Without fused_scatter the collectives order everything
+        themselves and this is `backward` (gradients overwritten, or added with accumulate=True)."""
+        import torch
+        if not self.fused_scatter:
+            return self.backward(*args, **kwargs)
+        cur = torch.cuda.current_stream(self.device)
+        self.zero_grad()
+        cur.synchronize()
+        self.comm.barrier()
+        out = self.backward(*args, **kwargs)
+        cur.synchronize()
+        self.comm.barrier()
+        return out
+
 
 class ZdpSplitMLP:
     """Linear -> activation -> Linear split along ffn (first layer OUT, second layer RED), slice by slice.  A ZDP
@@ -655,3 +674,22 @@ class ZdpSplitMLP:
             w_free[j] = [done]
         cur.wait_stream(self.comm_stream)
         return dx
+
+    def backward_step(self, *args, **kwargs):
+        """One gradient step with the ordering the epilogue-fused scatter needs.  Every rank zeroes its gradient
+        shards; the ranks meet at a barrier (no rank may add into a shard that its owner has not zeroed yet);
+        `backward(*args, **kwargs)` runs; the ranks meet again (every rank's terms have arrived) and only then
+        are the shards valid to read.  The host waits for the device before each barrier, so the barrier orders
+        the ranks' device work, not just their hosts.  Without fused_scatter the collectives order everything
+        themselves and this is `backward` (gradients overwritten, or added with accumulate=True)."""
+        import torch
+        if not self.fused_scatter:
+            return self.backward(*args, **kwargs)
+        cur = torch.cuda.current_stream(self.device)
+        self.zero_grad()
+        cur.synchronize()
+        self.comm.barrier()
+        out = self.backward(*args, **kwargs)
+        cur.synchronize()
+        self.comm.barrier()
+        return out

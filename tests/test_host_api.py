@@ -196,3 +196,14 @@ def test_suggest_granularity():
     assert P.osdp_suggest_granularity(64, 40, 64, 0, 0, P.OP_LINEAR_BWD, 0, 1 << 30, 64) == (0, 1)
     assert P.osdp_suggest_granularity(64, 40, 64, 0, 0, P.OP_LINEAR_BWD, 0, 1 << 30, 0)[0] == 3
     assert P.osdp_suggest_granularity(0, 40, 64, 0, 0, P.OP_LINEAR_BWD, 0, 1 << 30, 8)[0] == 2
+
+
+def test_noalloc_bias_grad_argument_checks():
+    # refusals come before anything touches a device
+    assert P.osdp_bias_grad_noalloc(A, 65536, 32768, A, stream=0) == 9            # 2^21 partials > 2^20
+    assert P.osdp_bias_grad_noalloc(A, 65536 * 1024 + 1, 8, A, stream=0) == 9     # 65537 row chunks: grid limit
+    assert P.osdp_bias_grad_noalloc(None, 8, 8, A, stream=0) == 1
+    assert P.osdp_bias_grad_noalloc(A, 8, 12, A, stream=0) == 4
+    assert P.osdp_bias_grad_noalloc(A, 0, 8, A, stream=0) == 2
+    # the regular backward refuses the same row count when a bias gradient is asked for
+    assert _bwd(M=65536 * 1024 + 8, dx=None, dw_flat=None) == 2

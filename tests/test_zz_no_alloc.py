@@ -48,6 +48,8 @@ def test_noalloc_rejects_sizes_beyond_the_built_in_scratch():
     # ceil(M/1024) * N = 64 * 32768 = 2^21 > 2^20 partials
     assert P.osdp_bias_grad_noalloc(A, 65536, 32768, A, stream=0) == 9
     assert "scratch" in P.osdp_status_string(9)
+    # few columns, very many rows: the partials would fit, but the first pass's grid would not
+    assert P.osdp_bias_grad_noalloc(A, 65536 * 1024 + 1, 8, A, stream=0) == 9
     assert P.osdp_bias_grad_noalloc(None, 8, 8, A, stream=0) == 1
     assert P.osdp_bias_grad_noalloc(A, 8, 12, A, stream=0) == 4
     assert P.osdp_bias_grad_noalloc(A, 0, 8, A, stream=0) == 2
