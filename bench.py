@@ -40,9 +40,12 @@ UNIT = "TFLOP/s"
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the three GEMM launches of a
 # step at this workload's full size, k = 8, output split, from one ncu capture of
-# `bench.py --case linear:16384:8192:8192:8:out` (metrics named above only: one pass).  Refreshed
-# whenever the kernel or its tile choice changes.
-NCU_TRAFFIC_BYTES = {}
+# `bench.py --case linear:16384:8192:8192:8:out`.  Refreshed whenever the kernel or its tile choice changes.
+NCU_TRAFFIC_BYTES = {
+    ("fwd", 8, "out"): 2793704000 + 259512320,
+    ("dx", 8, "out"): 2375177000 + 257772288,
+    ("dw", 8, "out"): 3149494000 + 124363008,
+}
 
 
 def peaks():
@@ -536,15 +539,27 @@ def run_ours(args):
     # ---- MLP blocks split along ffn (Linear -> GeLU -> Linear, fc1 output-split + fc2 reduction-split):
     # the wide-layer stress (hidden 8192, ffn 32768, 4 x 2048 tokens; k = 1, 8) and the small block
     # (hidden 1024, ffn 4096, 8 x 512 tokens; k = 1, 2, 4, 8)
-    def mlp_block(Mm, Hh, Ff, ks, reps, rounds):
+    def mlp_block(Mm, Hh, Ff, ks, reps, rounds, graphs=False):
         t = _mlp_tensors(torch, dev, Mm, Hh, Ff)
         wsm = {}
         for kk in ks:
             n1 = P.osdp_split_linear_workspace_bytes(Mm, Ff, Hh, kk, P.SPLIT_OUT, P.ACT_GELU_TANH, P.OP_MLP_FWD)[1]
             n2 = P.osdp_split_linear_workspace_bytes(Mm, Ff, Hh, kk, P.SPLIT_OUT, P.ACT_GELU_TANH, P.OP_MLP_BWD)[1]
             wsm[kk] = (P.new_workspace(max(n1, n2), dev), n1, n2)
-        med = interleaved({kk: (lambda kk=kk: _mlp_step(P, t, Mm, Hh, Ff, kk, wsm[kk][0], stream)) for kk in ks},
-                          rounds=rounds, warm=2, reps=reps)
+        fns = {kk: (lambda kk=kk: _mlp_step(P, t, Mm, Hh, Ff, kk, wsm[kk][0], stream)) for kk in ks}
+        if graphs:
+            # the same calls captured once into a CUDA graph and replayed: what a launch-bound loop of small
+            # operators does in production (the calls are plain stream work, internal fork / join included)
+            side = torch.cuda.Stream(dev)
+            for kk in ks:
+                fns[kk]()                                   # first use outside the capture
+                torch.cuda.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.stream(side):
+                    with torch.cuda.graph(g, stream=side):
+                        _mlp_step(P, t, Mm, Hh, Ff, kk, wsm[kk][0], torch.cuda.current_stream())
+                fns["graph_k%d" % kk] = g.replay
+        med = interleaved(fns, rounds=rounds, warm=2, reps=reps)
         flm = 6 * 2.0 * Mm * Hh * Ff
         res = {}
         for kk in ks:
@@ -552,12 +567,16 @@ def run_ours(args):
                                "frac_of_measured_sustained_peak": flm / med[kk] / 1e9 / pk["bf16_tflops_sustained"],
                                "staging_fwd_bytes": wsm[kk][1], "staging_bwd_bytes": wsm[kk][2],
                                "overhead_vs_k1": med[kk] / med[ks[0]] - 1.0}
+            if graphs:
+                g = med["graph_k%d" % kk]
+                res["k%d" % kk].update({"graph_replay_ms_per_step": g, "graph_replay_tflops": flm / g / 1e9,
+                                        "graph_replay_overhead_vs_k1": g / med["graph_k%d" % ks[0]] - 1.0})
         return res
 
     mlp_wide, mlp_small = {}, {}
     if rank == 0 and not args.no_sweep:
         mlp_wide = mlp_block(8192, 8192, 32768, (1, 8), 1, 7)
-        mlp_small = mlp_block(4096, 1024, 4096, (1, 2, 4, 8), 6, 10)
+        mlp_small = mlp_block(4096, 1024, 4096, (1, 2, 4, 8), 6, 10, graphs=True)
 
     # ---- the skinny single layer (X [256,512], W [2048,512], k = 4 along the output dimension): latency of one
     # forward + backward issued to an idle GPU, with the operands left in L2 by the previous step and after a flush
