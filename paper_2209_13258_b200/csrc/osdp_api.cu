@@ -663,7 +663,7 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
       if (rc) return rc;
       const cuuint64_t dims[3] = {(cuuint64_t)c.Q, (cuuint64_t)c.P, 1};
       const cuuint64_t str[2] = {(cuuint64_t)c.epi.ld_carry * 4, (cuuint64_t)c.epi.ld_carry * 4 * (cuuint64_t)c.P};
-      const cuuint32_t box[3] = {(cuuint32_t)bn, 32, 1};
+      const cuuint32_t box[3] = {(cuuint32_t)(bn > 256 ? 256 : bn), 32, 1};   // a box dimension is at most 256
       rc = encode3d(&p.carry_pf_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, c.epi.carry, dims, str, box, false);
       if (rc) return rc;
       if (!c.epi.out_fp32) {

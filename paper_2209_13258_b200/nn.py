@@ -21,7 +21,9 @@ class _SplitLinearFn(torch.autograd.Function):
             x2 = x2.contiguous()
         N, K, k = layer.out_features, layer.in_features, layer.k_split
         out = torch.empty(M, N, dtype=torch.bfloat16, device=x.device)
-        need_z = layer.act != B.ACT_NONE and (x.requires_grad or weight.requires_grad)
+        # any gradient of an activated layer, the bias gradient included, is taken through act'(Z)
+        need_z = layer.act != B.ACT_NONE and (x.requires_grad or weight.requires_grad or
+                                              (bias is not None and bias.requires_grad))
         z = torch.empty(M, N, dtype=torch.bfloat16, device=x.device) if need_z else None
         ws = layer._workspace(M)
         # the parameter is read in place from the flat buffer it lives in (element offset of the view)
