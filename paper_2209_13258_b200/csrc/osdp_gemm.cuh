@@ -1224,8 +1224,10 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
         else mbar_arrive(tempty_bar(buf));
       }
     }
-    // Nothing this warp handed to TMA may still be reading shared memory (or be in flight) at exit.
-    if (lane == 0) bulk_wait_all();
+    // Nothing this warp handed to TMA may still be reading shared memory at exit.  (The writes themselves are
+    // complete and visible when the grid is: waiting for them here would only put their latency in front of
+    // the next kernel on the stream.)
+    if (lane == 0) bulk_wait_read<0>();
     __syncwarp();
   }
 
