@@ -1002,7 +1002,9 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
     if (dx) { rc = dx_call(Operand{dy, N, M, N, false, true}, s_begin, s_end); if (rc) return rc; }
     stream = s_side;
     if (dw) { rc = dw_call(Operand{dy, N, M, N, true, true}, s_begin, s_end); if (rc) return rc; }
-    if (dx) stream = s_main;   // the short column sum follows dX rather than lengthening the dW chain
+    // The short column sum goes behind the shorter of the two GEMM chains: dX reduces over N, dW over the M
+    // tokens, and with equal flops the longer reduction has the fewer tiles and takes longer.
+    if (dx && M >= N) stream = s_main;
     if (dbias) {
       if (out_split) {
         const int64_t c0 = (int64_t)s_begin * L;
