@@ -63,7 +63,7 @@
 extern "C" {
 #endif
 
-#define OSDP_VERSION 100
+#define OSDP_VERSION 110
 
 /* status codes */
 #define OSDP_OK 0

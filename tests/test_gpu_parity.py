@@ -658,3 +658,54 @@ def test_calls_allocate_no_device_memory(P):
     # the reported staging is what the call needs: one byte less is refused, nothing is launched
     assert P.osdp_split_linear_bwd(dy, x, wf, 0, None, M, N, K, k, 0, 0, dx, dw, 0, P.DTYPE_FP32, 0, db,
                                    (ws.data_ptr(), n2 - 1)) == 5
+
+
+# ---------------------------------------------------------------------------------------------
+# two host threads, two streams, backward calls that fork onto the library's internal streams: the calls are
+# serialised on the host while they enqueue, each is joined back into its own stream, results as when run alone
+
+def test_two_threads_calling_backward_on_their_own_streams(P):
+    import threading
+    M, N, K, k = 1024, 1024, 512, 4
+    jobs = []
+    for t in range(2):
+        c = inputs.linear_case(M, N, K, w_std=0.05, layer=22 + t)
+        x, dy, wf = to_dev(c["x"]), to_dev(c["dy"]), to_dev(c["w_flat"])
+        _, n = P.osdp_split_linear_workspace_bytes(M, N, K, k, 0, 0, P.OP_LINEAR_BWD)
+        jobs.append({"x": x, "dy": dy, "wf": wf, "ws": P.new_workspace(n), "stream": torch.cuda.Stream(),
+                     "dx": torch.empty(M, K, dtype=torch.bfloat16, device="cuda"),
+                     "dw": torch.empty(N * K, dtype=torch.float32, device="cuda"),
+                     "db": torch.empty(N, dtype=torch.float32, device="cuda")})
+
+    def call(j, stream):
+        P.osdp_split_linear_bwd(j["dy"], j["x"], j["wf"], 0, None, M, N, K, k, P.SPLIT_OUT, 0, j["dx"], j["dw"], 0,
+                                P.DTYPE_FP32, 0, j["db"], j["ws"], stream=stream, check=True)
+
+    want = []
+    for j in jobs:                                   # alone, one after the other
+        call(j, torch.cuda.current_stream())
+        torch.cuda.synchronize()
+        want.append([j[n].clone() for n in ("dx", "dw", "db")])
+        for n in ("dx", "dw", "db"):
+            j[n].fill_(float("nan"))
+    errors = []
+
+    def worker(j):
+        try:
+            torch.cuda.set_device(0)
+            for _ in range(20):
+                call(j, j["stream"])
+            j["stream"].synchronize()
+        except Exception as e:      # pragma: no cover
+            errors.append(e)
+    threads = [threading.Thread(target=worker, args=(j,)) for j in jobs]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    torch.cuda.synchronize()
+    for j, w in zip(jobs, want):
+        for n, ref in zip(("dx", "dw", "db"), w):
+            assert torch.equal(_bits(j[n]), _bits(ref)), n
+        assert P.osdp_read_device_status(j["ws"]) == (0, 0)
