@@ -749,6 +749,7 @@ def run_ours(args):
                "sample": "%d of %d token rows, full N and K, k=%d %s, one fwd+bwd" % (args.ref_rows, M, k, args.split)}
 
     burst_value = aggregate_value(fl, args.steps, 1, burst_ms)
+    clocks = sampler.summary() if sampler else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -774,7 +775,11 @@ def run_ours(args):
                        "pinned host; copy-in / compute / copy-out on three streams over two buffer sets; the flat "
                        "weight buffer stays resident on the device (parameters are not an input of a step)"},
         "gpu_launches": launches_per_step * args.steps,
-        "clocks": sampler.summary() if sampler else None,
+        "clocks": clocks,
+        # time x clock: what is left of a comparison between runs once the power cap's clock is divided out
+        "clock_normalised": ({"ms_per_step_x_sm_ghz": ms_total / args.steps * clocks["sm_mhz"] / 1e3,
+                              "tflops_per_sm_ghz": value / world / (clocks["sm_mhz"] / 1e3)}
+                             if clocks and clocks.get("sm_mhz") else None),
     }
     print(json.dumps(line), flush=True)
     if world > 1:
