@@ -279,6 +279,7 @@ struct GemmCall {
   int slice_major;  // MODE_RED, all slices in the launch: sweep slice by slice with the carry (else: slices inside a tile)
   int out_is_slice; // MODE_ROWS / MODE_COLS: `epi.out` is the slice's own compact matrix, not the whole output
   int fp8;          // operands are fp8 e4m3 (1 byte per element) instead of bf16
+  int compact;      // the launch runs next to another GEMM of the call: CTA pairs on 256-wide tiles even when few
   int n_peers;      // > 0: the output slice is reduce-added row block by row block into peer_out[0..n_peers)
   void *peer_out[8];
   int *status;
@@ -518,7 +519,8 @@ void make_key(const GemmCall &c, PreparedKey *k) {
       ((uint64_t)(uint32_t)e.gz_act << 24));
   putf(e.scale);
   put(((uint64_t)(uint32_t)c.carry_bf16) | ((uint64_t)(uint32_t)c.pair_slices << 8) | ((uint64_t)(uint32_t)c.slice_major << 16) |
-      ((uint64_t)(uint32_t)c.out_is_slice << 24) | ((uint64_t)(uint32_t)c.fp8 << 32) | ((uint64_t)(uint32_t)c.n_peers << 40));
+      ((uint64_t)(uint32_t)c.out_is_slice << 24) | ((uint64_t)(uint32_t)c.fp8 << 32) | ((uint64_t)(uint32_t)c.n_peers << 40) |
+      ((uint64_t)(uint32_t)c.compact << 48));
   for (int q = 0; q < 8; ++q) putp(q < c.n_peers ? c.peer_out[q] : nullptr);
   putp(c.status);
   uint64_t h = 1469598103934665603ull;
@@ -577,7 +579,13 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   // tiles on (49 pairs of 74): measured on B200, operators with 64 pair tiles (4096 x 1024 and 2048 x 2048
   // outputs) run 8-11 % faster on 64 CTA pairs than on 128 single CTAs, with 32 pair tiles there is no
   // difference, with 16 the narrower single-CTA tiles win.
-  const bool pair = cdiv(c.bn_P, 2 * BM) * cdiv(c.bn_Q, 256) >= (int64_t)sms / 3;
+  // A GEMM that the call runs next to another one (a weight-gradient GEMM forked beside dX) takes pair tiles from 8
+  // tiles on: the same latency on a quarter of the SMs (a 1024 x 512 slice gradient over 4096 tokens: 28 us on 16
+  // SMs instead of 26 us on 64), which leaves the SMs to its neighbour.  Measured on B200, backward of the MLP
+  // block: 4096 tokens, hidden 1024, ffn 4096 k = 2 0.26 -> 0.21 ms, k = 4 0.41 -> 0.32 ms (k = 8 unchanged);
+  // 8192 tokens, hidden 2048, ffn 8192 k = 8 1.60 -> 1.28 ms; linear layers of 1024 to 2048 outputs -1 to -7 %.
+  const int64_t pair_tiles = cdiv(c.bn_P, 2 * BM) * cdiv(c.bn_Q, 256);
+  const bool pair = pair_tiles >= (int64_t)sms / 3 || (c.compact && pair_tiles >= 8 && !c.fp8);
   int bn = 64;
   const int64_t want = (int64_t)sms * 4 / 5;
   if (pair || cdiv(c.bn_P, BM) * cdiv(c.bn_Q, 256) >= want) bn = 256;
@@ -975,6 +983,7 @@ int bwd_impl(const void *dy, const void *x, const void *w_flat, int64_t w_offset
     c.epi.scale = scale_dw;
     c.epi.accumulate = accumulate;
     c.out_is_slice = (ld_dw_slice > 0 && k > 1) ? 1 : 0;
+    c.compact = (dx && dw) ? 1 : 0;   // runs next to the dX GEMM
     if (n_peers > 0) {
       c.n_peers = n_peers;
       for (int q = 0; q < n_peers && q < 8; ++q) c.peer_out[q] = dw_peers[q];
@@ -1445,6 +1454,7 @@ static int mlp_bwd_impl(const void *dy, const void *x, const void *w_flat, int64
       c.epi = cs ? plain_epilogue(cs->dw2_peers ? cs->dw2_peers[0] : cs->dw2, cs->ld_dw2, fp32)
                  : plain_epilogue(dw_ptr(dw_off_w2 + lo), ffn, fp32);
       c.epi.accumulate = accumulate;
+      c.compact = concurrent ? 1 : 0;
       if (cs && cs->dw2_peers) {
         c.n_peers = cs->world;
         for (int q = 0; q < cs->world && q < 8; ++q) c.peer_out[q] = cs->dw2_peers[q];
@@ -1461,6 +1471,7 @@ static int mlp_bwd_impl(const void *dy, const void *x, const void *w_flat, int64
       c.epi = cs ? plain_epilogue(cs->dw1_peers ? cs->dw1_peers[0] : cs->dw1, hidden, fp32)
                  : plain_epilogue(dw_ptr(dw_off_w1 + lo * hidden), hidden, fp32);
       c.epi.accumulate = accumulate;
+      c.compact = concurrent ? 1 : 0;
       if (cs && cs->dw1_peers) {
         c.n_peers = cs->world;
         for (int q = 0; q < cs->world && q < 8; ++q) c.peer_out[q] = cs->dw1_peers[q];
