@@ -35,7 +35,7 @@
  *    freed by any call.  Two things are created once per device at first use and kept until the
  *    process ends: each kernel variant's attributes (shared-memory size), and, by the first
  *    backward call that asks for dX and dW together (or the first osdp_split_mlp_bwd with weight
- *    gradients), two internal non-blocking streams and three events.  Such a call forks its
+ *    gradients), two internal non-blocking streams and nine events.  Such a call forks its
  *    weight-gradient launches onto those streams and joins them back into `stream` before it
  *    returns to the caller's ordering; while it enqueues that fork / join section it holds a
  *    host-side lock, so concurrent callers on one device are serialised on the host for the
@@ -319,7 +319,12 @@ int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const 
 /* Backward of the split MLP block, slice by slice, from the saved pre-activation z1_saved
  * [M,ffn] bf16:  dA_s = dY W2[:,F_s]; dZ_s = dA_s (.) act'(Z1_s); dW2[:,F_s] = dY^T act(Z1_s);
  * dW1[F_s,:] = dZ_s^T X; db1[F_s] = colsum dZ_s; dX = sum_s dZ_s W1[F_s,:]; db2 = colsum dY.
- * dW1/dW2 land at dw_off_w1/dw_off_w2 of dw_flat (dw_dtype).  Slice-sized dZ_s and A_s live in ws.
+ * dW1/dW2 land at dw_off_w1/dw_off_w2 of dw_flat (dw_dtype).  Slice-sized dZ_s and A_s live in ws: one set
+ * of them, or two sets used in turn when k > 2 and a slice is small (ceil(M/256) * ceil(L/256) <= 74, L the
+ * slice length: each GEMM of a slice is then at most one wave of tiles and the call is bound by the latency of
+ * its kernel chain).  With two sets a slice's weight-gradient GEMMs need not finish before the next slice
+ * starts, only before the slice after that; the staging is still ~ 1/k, and
+ * osdp_split_linear_workspace_bytes reports it.
  * With OSDP_FLAG_RECOMPUTE (the paper's Section 2.3 setting, activation checkpointing) z1_saved is
  * not read (may be NULL): Z1_s = X W1[F_s,:]^T + b1[F_s] is recomputed per slice (one more GEMM,
  * one more slice-sized buffer), so that no [M,ffn] activation exists between forward and backward.
@@ -328,8 +333,9 @@ int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const 
  * read then.
  * When weight gradients are wanted the call runs each slice's two weight-gradient GEMMs
  * on two streams of its own next to the dX GEMM: it forks from `stream` with an event and joins back
- * into `stream` before the next slice, so the caller still sees one ordered call (a stream capture
- * follows the fork).  The two streams and three events per device are created by the first such call;
+ * into `stream` before the next slice (with two sets of slice buffers: before the slice after the next, and
+ * at the end of the call), so the caller still sees one ordered call (a stream capture
+ * follows the fork).  The two streams and nine events per device are created by the first such call;
  * such calls on one device are serialised on the host while they enqueue. */
 int osdp_split_mlp_bwd(const void *dy, const void *x, const void *w_flat, int64_t off_w1, const float *b1,
                        int64_t off_w2, const void *z1_saved, int64_t M, int64_t hidden, int64_t ffn,

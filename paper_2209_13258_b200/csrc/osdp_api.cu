@@ -80,6 +80,7 @@ int device_sms(int *sms) {
 struct SideStreams {
   cudaStream_t s[2];
   cudaEvent_t fork, join[2];
+  cudaEvent_t ring[3][2];   // "this stream (0: the caller's, 1, 2: internal) is done with slice s", by the parity of s
 };
 SideStreams g_side[64];
 std::atomic<bool> g_side_ready[64];
@@ -98,6 +99,10 @@ int side_streams(SideStreams **out) {
         e = cudaStreamCreateWithFlags(&S.s[i], cudaStreamNonBlocking);
         if (e != cudaSuccess) return cuda_fail(e);
         e = cudaEventCreateWithFlags(&S.join[i], cudaEventDisableTiming);
+        if (e != cudaSuccess) return cuda_fail(e);
+      }
+      for (int i = 0; i < 6; ++i) {
+        e = cudaEventCreateWithFlags(&S.ring[i / 2][i % 2], cudaEventDisableTiming);
         if (e != cudaSuccess) return cuda_fail(e);
       }
       e = cudaEventCreateWithFlags(&S.fork, cudaEventDisableTiming);
@@ -149,6 +154,20 @@ struct ForkJoin {
     return OSDP_OK;
   }
   cudaStream_t stream(int i) const { return (open && i < n) ? side->s[i] : main; }
+  // Edges inside a section whose work is pipelined over slices: mark(q, b) records "stream q (0: the caller's,
+  // 1, 2: internal) has got this far" under parity b; after(q, b, t) makes stream t wait for the latest such mark.
+  // Without a fork everything is on the caller's stream and both do nothing: program order holds.
+  cudaStream_t lane(int q) const { return q == 0 ? main : stream(q - 1); }
+  int mark(int q, int b) {
+    if (!open) return OSDP_OK;
+    cudaError_t e = cudaEventRecord(side->ring[q][b], lane(q));
+    return e == cudaSuccess ? OSDP_OK : cuda_fail(e);
+  }
+  int after(int q, int b, int t) {
+    if (!open || lane(q) == lane(t)) return OSDP_OK;
+    cudaError_t e = cudaStreamWaitEvent(lane(t), side->ring[q][b], 0);
+    return e == cudaSuccess ? OSDP_OK : cuda_fail(e);
+  }
   int end() {
     if (!open) return OSDP_OK;
     open = false;
@@ -191,8 +210,14 @@ struct WsPlan {
   size_t stage1_off, stage1_bytes;    // second bf16 slice staging (dZ_s)
   size_t stage2_off, stage2_bytes;    // third bf16 slice staging (recomputed Z1_s)
   size_t part_off, part_bytes;        // column-sum partials
+  size_t stage_stride;                // distance between the two sets of slice staging buffers (0: one set)
   size_t total;
 };
+
+// The backward of an MLP block whose slices are small (each GEMM of a slice at most one wave of 256 x 256 tiles on
+// 74 CTA pairs) is bound by the latency of its chain of small kernels.  An all-slices call then keeps two sets of
+// slice staging buffers, so that a slice's weight-gradient GEMMs run beside the next slice's first GEMM.
+inline bool mlp_bwd_pipelined(int64_t M, int64_t L, int k) { return k > 2 && cdiv(M, 256) * cdiv(L, 256) <= 74; }
 
 int plan_workspace(int64_t M, int64_t N, int64_t K, int k, int split_dim, int act, int op, int flags, WsPlan *w) {
   const bool fp32_carry = !(flags & OSDP_FLAG_CARRY_BF16);
@@ -241,10 +266,12 @@ int plan_workspace(int64_t M, int64_t N, int64_t K, int k, int split_dim, int ac
       rc = slice_len(N, k, &L);
       if (rc) return rc;
       if (k > 1 && fp32_carry) take((size_t)M * K * 4, &w->carry_off, &w->carry_bytes);
-      take((size_t)M * L * 2, &w->stage0_off, &w->stage0_bytes);
-      take((size_t)M * L * 2, &w->stage1_off, &w->stage1_bytes);
-      if (flags & OSDP_FLAG_RECOMPUTE) take((size_t)M * L * 2, &w->stage2_off, &w->stage2_bytes);
-      take(chunks * (size_t)(L + K) * 4, &w->part_off, &w->part_bytes);   // db1's slice and db2 side by side
+      w->stage_stride = mlp_bwd_pipelined(M, L, k) ? align_up((size_t)M * L * 2, 256) : 0;
+      take(w->stage_stride + (size_t)M * L * 2, &w->stage0_off, &w->stage0_bytes);
+      take(w->stage_stride + (size_t)M * L * 2, &w->stage1_off, &w->stage1_bytes);
+      if (flags & OSDP_FLAG_RECOMPUTE) take(w->stage_stride + (size_t)M * L * 2, &w->stage2_off, &w->stage2_bytes);
+      // db1's slice (one set of partial sums per set of staging buffers) and db2 side by side
+      take(chunks * (size_t)((w->stage_stride ? 2 : 1) * L + K) * 4, &w->part_off, &w->part_bytes);
       break;
     default:
       return OSDP_ERR_UNSUPPORTED;
@@ -1374,7 +1401,8 @@ static int mlp_bwd_impl(const void *dy, const void *x, const void *w_flat, int64
   __nv_bfloat16 *z1_s = reinterpret_cast<__nv_bfloat16 *>(wsb + plan.stage2_off);
   float *carry = reinterpret_cast<float *>(wsb + plan.carry_off);
   float *partial = reinterpret_cast<float *>(wsb + plan.part_off);
-  float *partial2 = partial + ((size_t)((M + COLSUM_ROWS_PER_CHUNK - 1) / COLSUM_ROWS_PER_CHUNK)) * (size_t)L;   // db2's
+  const size_t part_set = ((size_t)((M + COLSUM_ROWS_PER_CHUNK - 1) / COLSUM_ROWS_PER_CHUNK)) * (size_t)L;
+  float *partial2 = partial + (plan.stage_stride ? 2 : 1) * part_set;   // db2's
   int *status = static_cast<int *>(ws);
   const int fp32 = dw_dtype == OSDP_DTYPE_FP32;
   auto dw_ptr = [&](int64_t off) -> void * {
@@ -1389,9 +1417,38 @@ static int mlp_bwd_impl(const void *dy, const void *x, const void *w_flat, int64
   // B200: hidden 1024 / ffn 4096 / 4096 tokens at k = 8 1.06 -> 0.84 ms; hidden 2048 / ffn 8192 at k = 4 +7.5 %;
   // hidden 4096 / ffn 16384 / 8192 tokens +1.5 %; hidden 8192 / ffn 32768 at k = 8 +0.5 %.
   const bool concurrent = dw_flat != nullptr;
+  // Small slices, all of them in this call: two sets of staging buffers, used in turn.  The slice's weight-gradient
+  // GEMMs then need not finish before the next slice's first GEMM writes its buffers, only before the slice after
+  // that does; the caller's stream carries dZ_s -> dX -> db1 slice after slice without waiting for them.
+  // Measured on B200 (backward, 4096 tokens, hidden 1024, ffn 4096): k = 4 0.32 -> 0.29 ms, k = 8 0.52 -> 0.40 ms;
+  // 8192 tokens: k = 8 0.83 -> 0.64 ms.
+  const bool piped = !cs && concurrent && plan.stage_stride != 0;
+  ForkJoin pipe;
+  if (piped) {
+    rc = pipe.acquire(stream, 2);
+    if (rc) return rc;
+    rc = pipe.begin();
+    if (rc) return rc;
+  }
+  __nv_bfloat16 *const a_s0 = a_s, *const dz_s0 = dz_s, *const z1_s0 = z1_s;
+  float *const partial0 = partial;
   for (int s = cs ? cs->idx : 0; s < (cs ? cs->idx + 1 : k); ++s) {
     const int64_t lo = (int64_t)s * L;
     const int64_t ls = (lo + L < ffn ? lo + L : ffn) - lo;
+    const int par = s & 1;
+    if (piped) {
+      const size_t shift = (size_t)par * plan.stage_stride;
+      a_s = reinterpret_cast<__nv_bfloat16 *>(reinterpret_cast<char *>(a_s0) + shift);
+      dz_s = reinterpret_cast<__nv_bfloat16 *>(reinterpret_cast<char *>(dz_s0) + shift);
+      z1_s = reinterpret_cast<__nv_bfloat16 *>(reinterpret_cast<char *>(z1_s0) + shift);
+      partial = partial0 + (size_t)par * part_set;
+      if (s >= 2) {   // slice s - 2's weight-gradient GEMMs have read this set of buffers
+        rc = pipe.after(1, par, 0);
+        if (rc) return rc;
+        rc = pipe.after(2, par, 0);
+        if (rc) return rc;
+      }
+    }
     const __nv_bfloat16 *w1s = cs ? static_cast<const __nv_bfloat16 *>(cs->w1) : w1 + lo * hidden;   // [ls, hidden]
     const __nv_bfloat16 *w2s = cs ? static_cast<const __nv_bfloat16 *>(cs->w2) : w2 + lo;            // [hidden, ls]
     const int64_t ld_w2s = cs ? cs->ld_w2 : ffn;
@@ -1425,19 +1482,27 @@ static int mlp_bwd_impl(const void *dy, const void *x, const void *w_flat, int64
     c.epi.act_out = recompute ? nullptr : a_s;
     c.epi.ld_act_out = L;
     c.status = status;
+    c.compact = piped ? 1 : 0;   // the previous slice's weight-gradient GEMMs are still running beside it
     rc = launch_gemm(c, stream);
     if (rc) return rc;
     // The slice's three remaining GEMMs and its column sum depend only on what has been launched so far.
     // They are forked onto the internal streams so that they share the SMs (each fills the others' partly
     // filled last wave of tiles).
     ForkJoin fj;
-    if (concurrent) {
+    if (piped) {
+      rc = pipe.mark(0, par);
+      if (rc) return rc;
+      rc = pipe.after(0, par, 1);
+      if (rc) return rc;
+      rc = pipe.after(0, par, 2);
+      if (rc) return rc;
+    } else if (concurrent) {
       rc = fj.acquire(stream, 2);
       if (rc) return rc;
       rc = fj.begin();
       if (rc) return rc;
     }
-    cudaStream_t s_dw2 = fj.stream(0), s_dw1 = fj.stream(1);
+    cudaStream_t s_dw2 = piped ? pipe.stream(0) : fj.stream(0), s_dw1 = piped ? pipe.stream(1) : fj.stream(1);
     if (db2_pending) {
       // its partial sums use the part of the scratch past the slice's own (db1's) columns
       rc = launch_colsum(dy, hidden, M, 0, (int)hidden, partial2, db2, s_dw2);
@@ -1500,11 +1565,17 @@ static int mlp_bwd_impl(const void *dy, const void *x, const void *w_flat, int64
       if (rc) return rc;
       if (db1) { rc = launch_colsum(dz_s, L, M, 0, (int)ls, partial, db1 + lo, stream); if (rc) return rc; }
     }
+    if (piped) {
+      rc = pipe.mark(1, par);
+      if (rc) return rc;
+      rc = pipe.mark(2, par);
+      if (rc) return rc;
+    }
     // join: the next slice reuses the staging buffers these launches read
     rc = fj.end();
     if (rc) return rc;
   }
-  return OSDP_OK;
+  return pipe.end();
 }
 
 int osdp_split_mlp_fwd(const void *x, const void *w_flat, int64_t off_w1, const float *b1, int64_t off_w2,

@@ -530,6 +530,56 @@ def test_cuda_graph_replay_matches_eager(P):
     assert P.osdp_read_device_status(ws) == (0, 0)
 
 
+@pytest.mark.parametrize("k", [2, 5])
+def test_mlp_cuda_graph_replay_matches_eager(P, k):
+    """The MLP block's backward forks onto the library's internal streams (k = 5, small slices: pipelined over
+    two sets of slice buffers; k = 2: one fork / join per slice); a capture follows them and replays the same bits."""
+    M, H, F = 300, 264, 520
+    c = inputs.mlp_case(M, H, F, w_std=0.08, layer=23)
+    x, dy, wf = to_dev(c["x"]), to_dev(c["dy"]), to_dev(c["w_flat"])
+    b1, b2 = to_dev(c["b1"]), to_dev(c["b2"])
+    _, n1 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, 1, P.OP_MLP_FWD)
+    _, n2 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, 1, P.OP_MLP_BWD)
+    ws = P.new_workspace(max(n1, n2))
+    y = torch.empty(M, H, dtype=torch.bfloat16, device="cuda")
+    z1 = torch.empty(M, F, dtype=torch.bfloat16, device="cuda")
+    dx = torch.empty(M, H, dtype=torch.bfloat16, device="cuda")
+    dwf = torch.empty(2 * F * H, dtype=torch.float32, device="cuda")
+    db1 = torch.empty(F, dtype=torch.float32, device="cuda")
+    db2 = torch.empty(H, dtype=torch.float32, device="cuda")
+    outs = [y, z1, dx, dwf, db1, db2]
+
+    def step():
+        P.osdp_split_mlp_fwd(x, wf, c["off_w1"], b1, c["off_w2"], b2, M, H, F, k, 1, y, z1, ws, check=True)
+        P.osdp_split_mlp_bwd(dy, x, wf, c["off_w1"], c["off_w2"], z1, M, H, F, k, 1, dx, dwf, c["off_w1"], c["off_w2"],
+                             P.DTYPE_FP32, 0, db1, db2, ws, check=True)
+
+    step()
+    step()   # the second call reuses the events of the first
+    torch.cuda.synchronize()
+    eager = [o.clone() for o in outs]
+    grads = oracle.mlp_bwd(c["dy"], c["x"], c["w1"], c["b1"], c["w2"], oracle.ACT_GELU_TANH, k)
+    assert_close(to_f64(dx), grads[0], "dx")
+    assert_close(to_f64(dwf[c["off_w1"]:c["off_w1"] + F * H].view(F, H)), grads[1], "dw1")
+    s = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(graph, stream=s):
+            step()
+    for rep in range(2):
+        for o in outs:
+            o.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        for e, o in zip(eager, outs):
+            assert torch.equal(_bits(e), _bits(o)), rep
+    step()   # eager again after the capture ended: the internal streams are free again
+    torch.cuda.synchronize()
+    for e, o in zip(eager, outs):
+        assert torch.equal(_bits(e), _bits(o))
+    assert P.osdp_read_device_status(ws) == (0, 0)
+
+
 # ---------------------------------------------------------------------------------------------
 # seeded random shapes / splits / activations / flags: every tile-shape variant of the kernel
 # (CTA pairs, single CTAs with 256-, 128- and 64-wide tiles), slices narrower than a tile, one-row

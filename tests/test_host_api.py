@@ -157,8 +157,11 @@ def test_mlp_argument_checks():
     # with recomputation no saved activation is needed, but one more slice-sized buffer is
     assert b(z1_saved=None, flags=P.FLAG_RECOMPUTE) in (0, 7)
     assert b(flags=32) == 6 and b(flags=P.FLAG_SLICE_MAJOR) == 6 and b(flags=P.FLAG_RECOMPUTE, b1=A + 4) == 4
+    # small slices with k > 2: two sets of the slice-sized buffers (consecutive slices overlap), so two more here
     plain = P.osdp_split_linear_workspace_bytes(32, 256, 64, 4, 0, 1, P.OP_MLP_BWD)[1]
-    assert P.osdp_split_linear_workspace_bytes(32, 256, 64, 4, 0, 1, P.OP_MLP_BWD, P.FLAG_RECOMPUTE)[1] == plain + 32 * 64 * 2
+    assert P.osdp_split_linear_workspace_bytes(32, 256, 64, 4, 0, 1, P.OP_MLP_BWD, P.FLAG_RECOMPUTE)[1] == plain + 2 * 32 * 64 * 2
+    plain = P.osdp_split_linear_workspace_bytes(32, 256, 64, 2, 0, 1, P.OP_MLP_BWD)[1]
+    assert P.osdp_split_linear_workspace_bytes(32, 256, 64, 2, 0, 1, P.OP_MLP_BWD, P.FLAG_RECOMPUTE)[1] == plain + 32 * 128 * 2
     assert P.osdp_split_linear_workspace_bytes(32, 256, 64, 4, 0, 1, P.OP_MLP_FWD, P.FLAG_RECOMPUTE)[0] == 6
 
 
@@ -207,3 +210,28 @@ def test_noalloc_bias_grad_argument_checks():
     assert P.osdp_bias_grad_noalloc(A, 0, 8, A, stream=0) == 2
     # the regular backward refuses the same row count when a bias gradient is asked for
     assert _bwd(M=65536 * 1024 + 8, dx=None, dw_flat=None) == 2
+
+
+def test_mlp_backward_staging_sets():
+    """Slice-sized buffers of the MLP backward: one set, except two sets for k > 2 when a slice's GEMMs are at
+    most one wave of 256 x 256 tiles on 74 CTA pairs (the slices are then pipelined); always ~ 1/k."""
+    def parts(M, H, F, k):
+        L = -(-(-(-F // k)) // 8) * 8
+        chunks = -(-M // 1024)
+        carry = M * H * 4 if k > 1 else 0
+        sets = 2 if (k > 2 and -(-M // 256) * -(-L // 256) <= 74) else 1
+        up = lambda v: -(-v // 256) * 256
+        stage = up(M * L * 2) + M * L * 2 if sets == 2 else M * L * 2
+        total = 256 + (up(carry) if carry else 0) + 2 * up(stage) + up(chunks * (sets * L + H) * 4)
+        return total, sets
+    for (M, H, F) in ((4096, 1024, 4096), (8192, 8192, 32768), (8192, 2048, 8192)):
+        for k in (1, 2, 4, 8, 16):
+            want, sets = parts(M, H, F, k)
+            rc, got = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, 1, P.OP_MLP_BWD)
+            assert rc == 0 and got == want, (M, H, F, k, got, want, sets)
+    assert parts(4096, 1024, 4096, 8)[1] == 2 and parts(4096, 1024, 4096, 2)[1] == 1
+    assert parts(8192, 8192, 32768, 8)[1] == 1 and parts(8192, 8192, 32768, 16)[1] == 1
+    assert parts(8192, 2048, 8192, 8)[1] == 1 and parts(8192, 2048, 8192, 16)[1] == 2
+    # the forward keeps one set whatever the size
+    assert P.osdp_split_linear_workspace_bytes(4096, 4096, 1024, 8, 0, 1, P.OP_MLP_FWD)[1] == \
+        256 + 4096 * 1024 * 4 + 4096 * 512 * 2
