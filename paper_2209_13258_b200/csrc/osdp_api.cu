@@ -651,6 +651,8 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   p.status = c.status;
   p.carry_bf16 = (c.mode == MODE_RED && c.k_total > 1) ? c.carry_bf16 : 0;
   p.red_group = in_tmem ? c.k_total : ((c.mode == MODE_RED && c.pair_slices && c.s_end - c.s_begin > 1) ? 2 : 1);
+  // Two k-blocks per barrier round of the operand ring, except where the epilogue carries a running sum through memory.
+  p.round_kblocks = (c.mode == MODE_RED && c.k_total > 1 && !in_tmem) ? 1 : 2;
   // Outputs leave through TMA.  The epilogue that reads a second tensor element-wise (gz) does too
   // (its input arrives by TMA as well) when the launch is unsliced and writes bf16, which is how the MLP
   // backward uses it; otherwise that epilogue falls back to direct stores from registers.

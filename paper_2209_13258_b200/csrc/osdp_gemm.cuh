@@ -80,6 +80,7 @@ struct GemmParams {
   int n_peers, rows_per_peer;
   int out_sc_mul;
   int red_group;             // MODE_RED: slices whose products a tile accumulates in one pass (1, or 2 = adjacent pairs)
+  int round_kblocks;         // k-blocks per barrier round of the operand ring that the launch asks for (1 or 2)
   int carry_bf16;            // MODE_RED: the running sum is kept in `out` itself, in bf16 (no fp32 carry buffer)
   int tma_epilogue;          // 1: outputs leave through shared-memory staging + TMA; 0: direct stores
   int bk;                    // reduction elements per k-block: 128 / (bytes per operand element)
@@ -372,6 +373,18 @@ struct SmemLayout {
   static constexpr int STG_BYTES = EPI_WARPS * STG_BUFS * 4096;
   static constexpr int RING_BYTES = 229376 - STG_BYTES;
   static constexpr int STAGES = (RING_BYTES / STAGE_BYTES) > 8 ? 8 : (RING_BYTES / STAGE_BYTES);
+  // Stages are handed from the producer to the MMA thread, and back, UNIT at a time (one barrier round per UNIT
+  // k-blocks).  The thread that issues the tcgen05.mma instructions is the pace-setter of the main loop: an
+  // instruction occupies it for about as long as the tensor pipe works on it, so every other instruction it
+  // executes per round (barrier poll, fence, commit: about 100 cycles that cannot be hidden behind the last MMA)
+  // is time the pipe idles.  Measured on B200 with time stamps in the MMA thread: a k-block of the 256 x 256 pair
+  // tile takes 512 cycles of tensor work; 546-566 with no barrier traffic at all, 630-675 with one round per
+  // k-block, 570-610 with one round per two k-blocks.  With six or more stages two k-blocks share a round (the ring still has three or four rounds in
+  // flight); the rings with four stages keep one k-block per round (two rounds in flight would not cover the
+  // latency of the copies).
+  // Launches whose epilogue moves a running sum through the same path to the L2 keep one k-block per round
+  // (finer refill of the ring: measured +5 % with two), so the launch chooses; UNIT is the most a variant allows.
+  static constexpr int UNIT = (STAGES >= 6) ? 2 : 1;
   static constexpr int STG_OFFSET = STAGES * STAGE_BYTES;
   static constexpr int BAR_OFFSET = STG_OFFSET + STG_BYTES;
   static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;   // barriers + alignment slack
@@ -651,6 +664,8 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const int unit = (SL::UNIT > 1 && p.round_kblocks > 1) ? SL::UNIT : 1;   // k-blocks per barrier round
+  const int groups = SL::STAGES / unit;                                     // rounds in the ring
 
   // Programmatic dependent launch: the next kernel on the stream may be scheduled as soon as this
   // grid's CTAs retire and may run its own prologue; it touches global memory only after its
@@ -658,9 +673,9 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (threadIdx.x == 0) {
-    for (int st = 0; st < SL::STAGES; ++st) {
-      mbar_init(full_bar(st), 1);
-      mbar_init(empty_bar(st), 1);
+    for (int g = 0; g < SL::STAGES; ++g) {   // a launch uses the first STAGES / unit of them
+      mbar_init(full_bar(g), 1);
+      mbar_init(empty_bar(g), 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull_bar(b), 1);
@@ -706,14 +721,15 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
     // ------------------------------------------------------------------ TMA producer(s)
     const bool load_a = (warp == 0);
     const bool load_b = SPLIT_PRODUCER ? (warp == 3) : true;
-    int stage = 0;
+    int grp = 0, sub = 0, n_sub = 0;       // round of the ring being filled, k-block inside it, k-blocks it will hold
     uint32_t phase = 0;
-    uint32_t armed = 0, armed_phase = 0;   // per-stage bookkeeping for the unwind path
+    uint32_t armed = 0, armed_phase = 0;   // per-round bookkeeping for the unwind path
     bool ok = true;
     Work w;
     for (int i = 0; ok && get_work<TM, BN>(p, i, bid, G, w); ++i) {
       w.a_row += (int)rank * BM;            // this CTA's rows of the pair's tile
       w.b_col += (int)rank * SL::GB_ROWS * (CTA2 ? 1 : 0);   // ... and its half of each 256-column group of B
+      int tile_left = w.kblocks;            // k-blocks of this tile still to load (a round never spans two tiles)
       for (int sl = 0; sl < w.s_count && ok; ++sl) {
       const int ss = w.s + sl;               // the slice whose operand boxes are loaded now
       const bool tail = (ss == p.k_total - 1);
@@ -723,13 +739,19 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
       const int b_sc = (b_sliced && !tail) ? ss * p.b_sc_mul : 0;
       const int nkb = (p.mode == MODE_RED) ? ceil_div(min(p.L, p.R - ss * p.L), BKE) : w.kblocks;
       for (int kb = 0; kb < nkb; ++kb) {
-        ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER);
-        if (!ok) break;
+        if (sub == 0) {
+          ok = mbar_wait(empty_bar(grp), phase ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER);
+          if (!ok) break;
+          n_sub = min(unit, tile_left);
+          if (lane == 0 && load_a && (!CTA2 || rank == 0))
+            mbar_expect_tx(full_bar(grp), (uint32_t)n_sub * SL::STAGE_BYTES * (CTA2 ? 2 : 1));
+          armed |= 1u << grp;
+          armed_phase = (armed_phase & ~(1u << grp)) | (phase << grp);
+        }
         if (lane == 0) {
-          const uint32_t sa = smem_base + stage * SL::STAGE_BYTES;
+          const uint32_t sa = smem_base + (uint32_t)(grp * unit + sub) * SL::STAGE_BYTES;
           const uint32_t sb = sa + SL::A_BYTES;
-          const uint32_t fb = full_bar(stage);
-          if (load_a && (!CTA2 || rank == 0)) mbar_expect_tx(fb, SL::STAGE_BYTES * (CTA2 ? 2 : 1));
+          const uint32_t fb = full_bar(grp);
           const int kc = kb * BKE;
           auto tma_load = [&](uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2) {
             if (CTA2) tma_load_3d_pair(dst, map, fb, c0, c1, c2);
@@ -765,16 +787,18 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
             }
           }
         }
-        armed |= 1u << stage;
-        armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
         __syncwarp();
-        if (++stage == SL::STAGES) { stage = 0; phase ^= 1u; }
+        --tile_left;
+        if (++sub == n_sub) {
+          sub = 0;
+          if (++grp == groups) { grp = 0; phase ^= 1u; }
+        }
       }
       }
     }
     if (!ok && rank == 0 && load_a) {
       // Unwinding: let the copies already issued land before the CTA's shared memory goes away.
-      for (int st = 0; st < SL::STAGES; ++st) {
+      for (int st = 0; st < groups; ++st) {
         if (!((armed >> st) & 1u)) continue;
         const unsigned long long t0 = globaltimer_ns();
         while (!mbar_try_wait(full_bar(st), (armed_phase >> st) & 1u)) {
@@ -784,45 +808,54 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
     }
   } else if (warp == 1 && rank == 0) {
     // ------------------------------------------------------------------ MMA issuer (even CTA of a pair)
+    // One thread runs the whole role: it waits for a round of the ring (UNIT k-blocks), issues their MMAs and
+    // hands the round back with one commit.
     constexpr uint32_t idesc = make_idesc<TM, SL::UMMA_N, A_MN, B_MN, EB>();
-    int stage = 0;
-    uint32_t phase = 0;
-    bool ok = true;
-    Work w;
-    for (int i = 0; ok && get_work<TM, BN>(p, i, bid, G, w); ++i) {
-      const int buf = i % SL::NBUF;
-      const uint32_t bphase = (uint32_t)(i / SL::NBUF) & 1u;
-      ok = mbar_wait(tempty_bar(buf), bphase ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA);
-      if (!ok) break;
-      tc_fence_after();
-      const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-      for (int kb = 0; kb < w.kblocks; ++kb) {
-        ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status, STATUS_TIMEOUT_MMA);
+    if (lane == 0) {
+      int grp = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      Work w;
+      for (int i = 0; ok && get_work<TM, BN>(p, i, bid, G, w); ++i) {
+        const int buf = i % SL::NBUF;
+        const uint32_t bphase = (uint32_t)(i / SL::NBUF) & 1u;
+        ok = mbar_wait(tempty_bar(buf), bphase ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA);
         if (!ok) break;
-        tc_fence_after();
-        if (lane == 0) {
-          const uint32_t sa = smem_base + stage * SL::STAGE_BYTES;
-          const uint32_t sb = sa + SL::A_BYTES;
-          const uint64_t adesc = make_smem_desc<A_MN, EB>(sa);
-          const uint64_t bdesc = make_smem_desc<B_MN, EB>(sb);
+        tc_fence_after();   // the epilogue's tensor-memory loads of this accumulator set are complete
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+        for (int kb = 0; kb < w.kblocks; kb += unit) {
+          const int n_sub = min(unit, w.kblocks - kb);
+          ok = mbar_wait(full_bar(grp), phase, abort_flag, p.status, STATUS_TIMEOUT_MMA);
+          if (!ok) break;
+          tc_fence_after();
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {   // four tcgen05.mma of 32 bytes of reduction each per k-block
+          for (int sub = 0; sub < SL::UNIT; ++sub) {
+            if (sub < n_sub) {
+              const uint32_t sa = smem_base + (uint32_t)(grp * unit + sub) * SL::STAGE_BYTES;
+              const uint32_t sb = sa + SL::A_BYTES;
+              const uint64_t adesc = make_smem_desc<A_MN, EB>(sa);
+              const uint64_t bdesc = make_smem_desc<B_MN, EB>(sb);
 #pragma unroll
-            for (int g = 0; g < SL::NG; ++g) {
-              const uint32_t d = d_tmem + (uint32_t)(g * SL::UMMA_N);
-              const uint64_t ad = adesc + (uint64_t)((kk * desc_k_advance<A_MN, EB>()) >> 4);
-              const uint64_t bd = bdesc + (uint64_t)((g * SL::GB_ROWS * 128 + kk * desc_k_advance<B_MN, EB>()) >> 4);
-              if (EB == 2) umma_bf16<CTA2>(d, ad, bd, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
-              else umma_f8<CTA2>(d, ad, bd, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+              for (int kk = 0; kk < 4; ++kk) {   // four tcgen05.mma of 32 bytes of reduction each per k-block
+#pragma unroll
+                for (int g = 0; g < SL::NG; ++g) {
+                  const uint32_t d = d_tmem + (uint32_t)(g * SL::UMMA_N);
+                  const uint64_t ad = adesc + (uint64_t)((kk * desc_k_advance<A_MN, EB>()) >> 4);
+                  const uint64_t bd = bdesc + (uint64_t)((g * SL::GB_ROWS * 128 + kk * desc_k_advance<B_MN, EB>()) >> 4);
+                  const uint32_t acc = (kb + sub > 0 || kk > 0) ? 1u : 0u;
+                  if (EB == 2) umma_bf16<CTA2>(d, ad, bd, idesc, acc);
+                  else umma_f8<CTA2>(d, ad, bd, idesc, acc);
+                }
+              }
             }
           }
-          umma_commit<CTA2>(empty_bar(stage));                      // frees the stage when the MMAs retire
-          if (kb == w.kblocks - 1) umma_commit<CTA2>(tfull_bar(buf));   // accumulator complete
+          umma_commit<CTA2>(empty_bar(grp));                               // frees the round when its MMAs retire
+          if (kb + unit >= w.kblocks) umma_commit<CTA2>(tfull_bar(buf));   // accumulator complete
+          if (++grp == groups) { grp = 0; phase ^= 1u; }
         }
-        __syncwarp();
-        if (++stage == SL::STAGES) { stage = 0; phase ^= 1u; }
       }
     }
+    __syncwarp();
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ epilogue
     // Each warp owns 32 rows of the tile and two 4 KB staging buffers (32 rows x 128 bytes, 128-byte
