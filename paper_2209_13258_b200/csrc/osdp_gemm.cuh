@@ -890,6 +890,20 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
       const int wrow0 = w.row0 + quarter * 32;
       const long long row = (long long)wrow0 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
+      // Hands the accumulator set back to the MMA thread: at the end of the tile's epilogue, or, where one tile
+      // fills the tensor memory (nothing else for the tensor pipe to do meanwhile), as soon as this warp's last
+      // columns are in registers, so that converting and storing them overlaps the next tile's first k-blocks.
+      bool released = false;
+      auto release_accumulator = [&]() {
+        if (released) return;
+        released = true;
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          if (CTA2 && rank != 0) mbar_arrive_remote(tempty_bar(buf), 0);   // the even CTA's MMA thread waits on it
+          else mbar_arrive(tempty_bar(buf));
+        }
+      };
       if (p.tma_epilogue && p.mode == MODE_RED && lane == 0) {
         // The carry of this CTA's next tile is touched one main loop from now: have it in L2 by then.
         Work nx;
@@ -1153,6 +1167,7 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
             uint32_t v[32];
             tmem_ld_x32(taddr + (uint32_t)(c * 32), v);
             tmem_ld_wait();
+            if (SL::NBUF == 1 && (c + 1 == (wg + 1) * (BN / 32 / EG) || cbase + 32 >= w.col_end)) release_accumulator();
             scale_acc(v, p.epi.scale);
             if (p.epi.bias) {
 #pragma unroll
@@ -1197,6 +1212,7 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
               tmem_ld_x32(taddr + (uint32_t)(c * 64), lo);
               if (BN >= 64) tmem_ld_x32(taddr + (uint32_t)(c * 64 + 32), hi);
               tmem_ld_wait();
+              if (SL::NBUF == 1 && (c + 1 == (wg + 1) * ((BN + 63) / 64 / EG) || cbase + 64 >= w.col_end)) release_accumulator();
               scale_acc(lo, p.epi.scale);
               if (BN >= 64) scale_acc(hi, p.epi.scale);
 #pragma unroll
@@ -1250,12 +1266,7 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
           }
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) {
-        if (CTA2 && rank != 0) mbar_arrive_remote(tempty_bar(buf), 0);   // the even CTA's MMA thread waits on it
-        else mbar_arrive(tempty_bar(buf));
-      }
+      release_accumulator();
     }
     // Nothing this warp handed to TMA may still be reading shared memory at exit.  (The writes themselves are
     // complete and visible when the grid is: waiting for them here would only put their latency in front of
