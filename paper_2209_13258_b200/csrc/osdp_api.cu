@@ -219,6 +219,9 @@ struct WsPlan {
 // slice staging buffers, so that a slice's weight-gradient GEMMs run beside the next slice's first GEMM.
 inline bool mlp_bwd_pipelined(int64_t M, int64_t L, int k) { return k > 2 && cdiv(M, 256) * cdiv(L, 256) <= 74; }
 
+// fp32 running sum of a P x Q output, kept as boxes of 32 x 32 (both extents padded to whole boxes)
+inline size_t carry_bytes(int64_t P, int64_t Q) { return (size_t)(cdiv(P, 32) * 32) * (size_t)(cdiv(Q, 32) * 32) * 4; }
+
 int plan_workspace(int64_t M, int64_t N, int64_t K, int k, int split_dim, int act, int op, int flags, WsPlan *w) {
   const bool fp32_carry = !(flags & OSDP_FLAG_CARRY_BF16);
   // The linear ops carry a running sum through memory only when the operator is swept once per slice: the
@@ -244,14 +247,14 @@ int plan_workspace(int64_t M, int64_t N, int64_t K, int k, int split_dim, int ac
       rc = slice_len(split_dim == OSDP_SPLIT_OUT ? N : K, k, &L);
       if (rc) return rc;
       if (split_dim == OSDP_SPLIT_RED && k > 1 && fp32_carry && swept)
-        take((size_t)M * N * 4, &w->carry_off, &w->carry_bytes);
+        take(carry_bytes(M, N), &w->carry_off, &w->carry_bytes);
       break;
     case OSDP_OP_LINEAR_BWD:
       if (split_dim != OSDP_SPLIT_OUT && split_dim != OSDP_SPLIT_RED) return OSDP_ERR_BAD_SPLIT;
       rc = slice_len(split_dim == OSDP_SPLIT_OUT ? N : K, k, &L);
       if (rc) return rc;
       if (split_dim == OSDP_SPLIT_OUT && k > 1 && fp32_carry && (swept || act != OSDP_ACT_NONE))
-        take((size_t)M * K * 4, &w->carry_off, &w->carry_bytes);
+        take(carry_bytes(M, K), &w->carry_off, &w->carry_bytes);
       if (act != OSDP_ACT_NONE)
         take((size_t)M * (split_dim == OSDP_SPLIT_OUT ? L : N) * 2, &w->stage0_off, &w->stage0_bytes);
       take(chunks * (size_t)N * 4, &w->part_off, &w->part_bytes);
@@ -259,13 +262,13 @@ int plan_workspace(int64_t M, int64_t N, int64_t K, int k, int split_dim, int ac
     case OSDP_OP_MLP_FWD:   // N = ffn, K = hidden
       rc = slice_len(N, k, &L);
       if (rc) return rc;
-      if (k > 1 && fp32_carry) take((size_t)M * K * 4, &w->carry_off, &w->carry_bytes);
+      if (k > 1 && fp32_carry) take(carry_bytes(M, K), &w->carry_off, &w->carry_bytes);
       take((size_t)M * L * 2, &w->stage0_off, &w->stage0_bytes);
       break;
     case OSDP_OP_MLP_BWD:
       rc = slice_len(N, k, &L);
       if (rc) return rc;
-      if (k > 1 && fp32_carry) take((size_t)M * K * 4, &w->carry_off, &w->carry_bytes);
+      if (k > 1 && fp32_carry) take(carry_bytes(M, K), &w->carry_off, &w->carry_bytes);
       w->stage_stride = mlp_bwd_pipelined(M, L, k) ? align_up((size_t)M * L * 2, 256) : 0;
       take(w->stage_stride + (size_t)M * L * 2, &w->stage0_off, &w->stage0_bytes);
       take(w->stage_stride + (size_t)M * L * 2, &w->stage1_off, &w->stage1_bytes);
@@ -700,15 +703,18 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
       if (rc) return rc;
     }
     if (c.mode == MODE_RED && c.k_total > 1 && !p.carry_bf16 && !in_tmem) {
-      CUtensorMap unused;
-      rc = make_output_maps(c.epi.carry, true, c.P, c.Q, c.epi.ld_carry, MODE_NONE, c.L, 1, &unused, &p.carry_map,
-                            nullptr);
+      // the carry, box by box (see GemmParams): [boxes * 32 rows, 32 columns], 128 bytes per row
+      const int64_t cb = cdiv(c.Q, 32), boxes = cdiv(c.P, 32) * cb;
+      p.carry_cb = (int)cb;
+      const cuuint64_t cdims[3] = {32, (cuuint64_t)boxes * 32, 1};
+      const cuuint64_t cstr[2] = {128, (cuuint64_t)boxes * 32 * 128};
+      const cuuint32_t cbox[3] = {32, 32, 1};
+      rc = encode3d(&p.carry_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, c.epi.carry, cdims, cstr, cbox, true);
+      if (rc) return rc;
+      const cuuint32_t pbox[3] = {32, (cuuint32_t)(bn > 256 ? 256 : bn), 1};   // the bn / 32 boxes of a warp's tile rows
+      rc = encode3d(&p.carry_pf_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, c.epi.carry, cdims, cstr, pbox, false);
       if (rc) return rc;
       const cuuint64_t dims[3] = {(cuuint64_t)c.Q, (cuuint64_t)c.P, 1};
-      const cuuint64_t str[2] = {(cuuint64_t)c.epi.ld_carry * 4, (cuuint64_t)c.epi.ld_carry * 4 * (cuuint64_t)c.P};
-      const cuuint32_t box[3] = {(cuuint32_t)(bn > 256 ? 256 : bn), 32, 1};   // a box dimension is at most 256
-      rc = encode3d(&p.carry_pf_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, c.epi.carry, dims, str, box, false);
-      if (rc) return rc;
       if (!c.epi.out_fp32) {
         // the last slice's bf16 results leave as unswizzled boxes of 32 rows x 32 columns
         const cuuint32_t box32[3] = {32, 32, 1};

@@ -67,7 +67,11 @@ struct GemmParams {
   int a_sc_mul, b_sc_mul;    // 1: the operand map has a slice coordinate; 0: the operand is one slice already
   // Output-side maps (3-D, same slice-coordinate scheme): final output, saved pre-activation, fp32 carry.
   CUtensorMap out_main, out_tail, z_main, z_tail, carry_map;
-  CUtensorMap carry_pf_map;  // same tensor as carry_map, unswizzled box of 32 rows x BN columns, for L2 prefetch
+  // The fp32 carry of a summed output belongs to this kernel alone (written by slice s, read by slice s + 1 of the
+  // same tile), so it is not kept as an [P, Q] matrix but box by box: box (rb, cb) = rows 32 rb .., columns 32 cb ..
+  // is one contiguous 4 KB block at index rb * carry_cb + cb, and a warp's boxes of a tile are adjacent (whole
+  // DRAM pages instead of 128-byte row segments 4 Q bytes apart).  carry_map: a [boxes * 32, 32] matrix, box 32 x 32.
+  CUtensorMap carry_pf_map;  // the same memory, box of (tile width / 32) * 32 rows: a warp's boxes of a tile, for L2 prefetch
   CUtensorMap out32_map, z32_map;   // bf16 out / second bf16 output (z_save, act_out) as unswizzled boxes of 32 x 32:
                                     // the last slice of a summed output and the epilogue that reads gz
   CUtensorMap gz32_map;             // the element-wise second input gz, same boxes
@@ -81,6 +85,7 @@ struct GemmParams {
   int out_sc_mul;
   int red_group;             // MODE_RED: slices whose products a tile accumulates in one pass (1, or 2 = adjacent pairs)
   int round_kblocks;         // k-blocks per barrier round of the operand ring that the launch asks for (1 or 2)
+  int carry_cb;              // fp32 carry: boxes of 32 columns per row block (the carry is stored box by box, see carry_map)
   int carry_bf16;            // MODE_RED: the running sum is kept in `out` itself, in bf16 (no fp32 carry buffer)
   int tma_epilogue;          // 1: outputs leave through shared-memory staging + TMA; 0: direct stores
   int bk;                    // reduction elements per k-block: 128 / (bytes per operand element)
@@ -873,6 +878,8 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
     const uint32_t swz = (uint32_t)(lane & 7);
     const bool out_sliced = (p.mode == MODE_COLS) || (p.mode == MODE_ROWS);
     const bool out_mid = (p.mode == MODE_COLS);
+    // first row, in the carry's box-by-box layout, of the box that holds rows row .. row + 31, columns col .. col + 31
+    auto carry_box = [&](int row, int col) { return ((row >> 5) * p.carry_cb + (col >> 5)) << 5; };
     uint32_t n_store = 0;   // staged boxes issued by this warp (selects the staging buffer)
     uint32_t n_cload = 0;   // carry boxes loaded by this warp
     bool ok = true;
@@ -908,7 +915,7 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
         // The carry of this CTA's next tile is touched one main loop from now: have it in L2 by then.
         Work nx;
         if (get_work<TM, BN>(p, i + 1, bid, G, nx) && nx.carry_in)
-          tma_prefetch_l2_3d(&p.carry_pf_map, nx.col0, nx.row0 + (int)rank * BM + quarter * 32, 0);
+          tma_prefetch_l2_3d(&p.carry_pf_map, 0, carry_box(nx.row0 + (int)rank * BM + quarter * 32, nx.col0), 0);
       }
       if (p.tma_epilogue && p.epi.gz && lane == 0) {
         // likewise the next tile's rows of gz
@@ -964,10 +971,12 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
             } else if (out_mid && map != &p.carry_map) {
               if (reduce) tma_reduce_add_3d(map, src, col_in, sc, r_in);
               else tma_store_3d(map, src, col_in, sc, r_in);
+            } else if (map == &p.carry_map) {
+              if (reduce) tma_reduce_add_3d(map, src, 0, carry_box(r_in, col_in), 0);
+              else tma_store_3d(map, src, 0, carry_box(r_in, col_in), 0);
             } else {
-              const int c2 = (map == &p.carry_map) ? 0 : sc;
-              if (reduce) tma_reduce_add_3d(map, src, col_in, r_in, c2);
-              else tma_store_3d(map, src, col_in, r_in, c2);
+              if (reduce) tma_reduce_add_3d(map, src, col_in, r_in, sc);
+              else tma_store_3d(map, src, col_in, r_in, sc);
             }
             bulk_commit();
           }
@@ -1014,7 +1023,7 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
               if (staged_out) bulk_wait_read<0>();   // the store that last left from this buffer
               const uint32_t b = n_cload % NB;
               mbar_expect_tx(cbar + 8u * b, 4096u);
-              tma_load_3d(stg + b * 4096u, &p.carry_map, cbar + 8u * b, w.col0 + c * 32, wrow0, 0);
+              tma_load_3d(stg + b * 4096u, &p.carry_map, cbar + 8u * b, 0, carry_box(wrow0, w.col0 + c * 32), 0);
             }
             ++n_cload;
           };
