@@ -66,7 +66,7 @@
 extern "C" {
 #endif
 
-#define OSDP_VERSION 110
+#define OSDP_VERSION 111
 
 /* status codes */
 #define OSDP_OK 0

@@ -18,7 +18,7 @@ def test_library_exports_every_declared_symbol():
     L = P.lib()
     for name in declared:
         assert hasattr(L, name), name
-    assert P.osdp_version() == 110
+    assert P.osdp_version() == 111
     assert P.osdp_status_string(0) == "ok" and "split" in P.osdp_status_string(3)
 
 
