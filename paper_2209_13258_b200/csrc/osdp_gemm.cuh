@@ -86,7 +86,6 @@ struct GemmParams {
   int red_group;             // MODE_RED: slices whose products a tile accumulates in one pass (1, or 2 = adjacent pairs)
   int round_kblocks;         // k-blocks per barrier round of the operand ring that the launch asks for (1 or 2)
   int carry_cb;              // fp32 carry: boxes of 32 columns per row block (the carry is stored box by box, see carry_map)
-  int unit_shift;            // second problem of a two-problem launch: tiles of the first problem (see gemm_body)
   int carry_bf16;            // MODE_RED: the running sum is kept in `out` itself, in bf16 (no fp32 carry buffer)
   int tma_epilogue;          // 1: outputs leave through shared-memory staging + TMA; 0: direct stores
   int bk;                    // reduction elements per k-block: 128 / (bytes per operand element)
@@ -646,25 +645,16 @@ __device__ __forceinline__ void epilogue8(const Epilogue &e, long long row, int 
 // of the B tile (BN/2 rows), holds the accumulator of its 128 rows in its own tensor memory and
 // runs its own epilogue.  Per CTA a stage is 32 KB instead of 48 KB (6 stages instead of 4) and
 // half as many B bytes cross from L2 to shared memory per flop.
-// The kernel body works through one or two GEMM problems (pa, then pb) in one launch: the ring, the tensor-memory
-// accumulator sets and the staging buffers simply carry on from the first problem's last tile to the second
-// problem's first.  Two problems are launched together when they are independent and small (a slice's second GEMM
-// and the next slice's first GEMM of the MLP block): one launch instead of two in a chain of dependent launches,
-// and the persistent CTAs fill up with the second problem's tiles where the first leaves them idle.
-template <int BN, bool A_MN, bool B_MN, bool CTA2, bool HEAVY, int EB>
-__device__ __forceinline__ void gemm_body(const GemmParams &pa, const GemmParams &pb, const int nprob) {
-  const GemmParams &p = pa;   // what is not per problem: status word, ring granularity
+template <int BN, bool A_MN, bool B_MN, bool CTA2, bool HEAVY = false, int EB = 2>
+__global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
   using SL = SmemLayout<BN, CTA2, HEAVY>;
   constexpr int BKE = 128 / EB;   // reduction elements per k-block
   constexpr int CW = 128 / EB;    // output rows / columns per 128-byte chunk of an MN-major operand
   constexpr int TM = CTA2 ? 2 * BM : BM;
   constexpr int BNL = SL::BNL;
   const uint32_t rank = CTA2 ? cluster_ctarank() : 0u;
-  const int bid0 = CTA2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int bid = CTA2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
   const int G = CTA2 ? (int)(gridDim.x >> 1) : (int)gridDim.x;
-  // The second problem's tiles are dealt starting with the unit after the one that got the first problem's last
-  // tile, so that the units with one tile less take the first ones.
-  const int bid1 = (nprob > 1) ? (bid0 + G - pb.unit_shift % G) % G : bid0;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -708,11 +698,6 @@ __device__ __forceinline__ void gemm_body(const GemmParams &pa, const GemmParams
       prefetch_tmap(&p.out_tail);
       prefetch_tmap(&p.carry_map);
     }
-    if (nprob > 1) {
-      prefetch_tmap(&pb.a_main);
-      prefetch_tmap(&pb.b_main);
-      prefetch_tmap(&pb.out_main);
-    }
   }
   if (warp == 2) {
     tmem_alloc<CTA2>(smem_u32(tmem_holder), SL::TMEM_COLS);
@@ -727,6 +712,12 @@ __device__ __forceinline__ void gemm_body(const GemmParams &pa, const GemmParams
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const uint32_t tmem_base = *tmem_holder;
 
+  // Which operand dimension the slice coordinate belongs to (fixed by mode and operand major).
+  const bool a_sliced = (p.mode == MODE_ROWS) || (p.mode == MODE_RED);
+  const bool b_sliced = (p.mode == MODE_COLS) || (p.mode == MODE_RED);
+  const bool a_mid = A_MN ? (p.mode == MODE_ROWS) : (p.mode == MODE_RED);   // slice cuts A's contiguous dim
+  const bool b_mid = B_MN ? (p.mode == MODE_COLS) : (p.mode == MODE_RED);
+
   // With both operands MN-major a stage takes four to six copies; two warps then walk the ring in
   // lock step (warp 0 arms the stage's barrier and loads A, warp 3 loads B) so that two threads issue
   // them in parallel.  Otherwise warp 0 does it all (measured: the split costs 1-2 % there).
@@ -740,14 +731,6 @@ __device__ __forceinline__ void gemm_body(const GemmParams &pa, const GemmParams
     uint32_t armed = 0, armed_phase = 0;   // per-round bookkeeping for the unwind path
     bool ok = true;
     Work w;
-    for (int pr = 0; pr < nprob && ok; ++pr) {
-    const GemmParams &p = pr ? pb : pa;
-    const int bid = pr ? bid1 : bid0;
-    // Which operand dimension the slice coordinate belongs to (fixed by mode and operand major).
-    const bool a_sliced = (p.mode == MODE_ROWS) || (p.mode == MODE_RED);
-    const bool b_sliced = (p.mode == MODE_COLS) || (p.mode == MODE_RED);
-    const bool a_mid = A_MN ? (p.mode == MODE_ROWS) : (p.mode == MODE_RED);   // slice cuts A's contiguous dim
-    const bool b_mid = B_MN ? (p.mode == MODE_COLS) : (p.mode == MODE_RED);
     for (int i = 0; ok && get_work<TM, BN>(p, i, bid, G, w); ++i) {
       w.a_row += (int)rank * BM;            // this CTA's rows of the pair's tile
       w.b_col += (int)rank * SL::GB_ROWS * (CTA2 ? 1 : 0);   // ... and its half of each 256-column group of B
@@ -818,7 +801,6 @@ __device__ __forceinline__ void gemm_body(const GemmParams &pa, const GemmParams
       }
       }
     }
-    }
     if (!ok && rank == 0 && load_a) {
       // Unwinding: let the copies already issued land before the CTA's shared memory goes away.
       for (int st = 0; st < groups; ++st) {
@@ -839,13 +821,9 @@ __device__ __forceinline__ void gemm_body(const GemmParams &pa, const GemmParams
       uint32_t phase = 0;
       bool ok = true;
       Work w;
-      int it = 0;   // tiles of this unit so far, over both problems
-      for (int pr = 0; pr < nprob && ok; ++pr) {
-      const GemmParams &p = pr ? pb : pa;
-      const int bid = pr ? bid1 : bid0;
-      for (int i = 0; ok && get_work<TM, BN>(p, i, bid, G, w); ++i, ++it) {
-        const int buf = it % SL::NBUF;
-        const uint32_t bphase = (uint32_t)(it / SL::NBUF) & 1u;
+      for (int i = 0; ok && get_work<TM, BN>(p, i, bid, G, w); ++i) {
+        const int buf = i % SL::NBUF;
+        const uint32_t bphase = (uint32_t)(i / SL::NBUF) & 1u;
         ok = mbar_wait(tempty_bar(buf), bphase ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA);
         if (!ok) break;
         tc_fence_after();   // the epilogue's tensor-memory loads of this accumulator set are complete
@@ -881,7 +859,6 @@ __device__ __forceinline__ void gemm_body(const GemmParams &pa, const GemmParams
           if (++grp == groups) { grp = 0; phase ^= 1u; }
         }
       }
-      }
     }
     __syncwarp();
   } else if (warp >= 4) {
@@ -899,25 +876,21 @@ __device__ __forceinline__ void gemm_body(const GemmParams &pa, const GemmParams
     const uint32_t stg = smem_base + SL::STG_OFFSET + (uint32_t)(warp - 4) * (NB * 4096u);
     const uint32_t row_off = (uint32_t)lane * 128u;
     const uint32_t swz = (uint32_t)(lane & 7);
-    uint32_t n_store = 0;   // staged boxes issued by this warp (selects the staging buffer)
-    uint32_t n_cload = 0;   // carry boxes loaded by this warp
-    bool ok = true;
-    Work w;
-    int it = 0;             // tiles of this unit so far, over both problems
-    for (int pr = 0; pr < nprob && ok; ++pr) {
-    const GemmParams &p = pr ? pb : pa;
-    const int bid = pr ? bid1 : bid0;
     const bool out_sliced = (p.mode == MODE_COLS) || (p.mode == MODE_ROWS);
     const bool out_mid = (p.mode == MODE_COLS);
     // first row, in the carry's box-by-box layout, of the box that holds rows row .. row + 31, columns col .. col + 31
     auto carry_box = [&](int row, int col) { return ((row >> 5) * p.carry_cb + (col >> 5)) << 5; };
-    for (int i = 0; ok && get_work<TM, BN>(p, i, bid, G, w); ++i, ++it) {
+    uint32_t n_store = 0;   // staged boxes issued by this warp (selects the staging buffer)
+    uint32_t n_cload = 0;   // carry boxes loaded by this warp
+    bool ok = true;
+    Work w;
+    for (int i = 0; ok && get_work<TM, BN>(p, i, bid, G, w); ++i) {
       w.a_row += (int)rank * BM;
       w.row0 += (int)rank * BM;
       if (i == 0 && p.tma_epilogue && p.epi.gz && lane == 0)   // this CTA's first tile: while its main loop runs
         tma_prefetch_l2_3d(&p.gz_pf_map, w.b_col, w.a_row + quarter * 32, 0);
-      const int buf = it % SL::NBUF;
-      const uint32_t bphase = (uint32_t)(it / SL::NBUF) & 1u;
+      const int buf = i % SL::NBUF;
+      const uint32_t bphase = (uint32_t)(i / SL::NBUF) & 1u;
       ok = mbar_wait(tfull_bar(buf), bphase, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE);
       if (!ok) break;
       tc_fence_after();
@@ -1304,7 +1277,6 @@ __device__ __forceinline__ void gemm_body(const GemmParams &pa, const GemmParams
       }
       release_accumulator();
     }
-    }   // (nothing to wait for between the problems: they are independent, so they touch different memory)
     // Nothing this warp handed to TMA may still be reading shared memory at exit.  (The writes themselves are
     // complete and visible when the grid is: waiting for them here would only put their latency in front of
     // the next kernel on the stream.)
@@ -1319,17 +1291,6 @@ __device__ __forceinline__ void gemm_body(const GemmParams &pa, const GemmParams
     tc_fence_after();
     tmem_dealloc<CTA2>(tmem_base, SL::TMEM_COLS);
   }
-}
-
-template <int BN, bool A_MN, bool B_MN, bool CTA2, bool HEAVY = false, int EB = 2>
-__global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
-  gemm_body<BN, A_MN, B_MN, CTA2, HEAVY, EB>(p, p, 1);
-}
-// Two independent problems of the same variant in one launch (see gemm_body).
-template <int BN, bool A_MN, bool B_MN, bool CTA2, bool HEAVY = false, int EB = 2>
-__global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1)
-gemm_kernel_dual(const __grid_constant__ GemmParams pa, const __grid_constant__ GemmParams pb) {
-  gemm_body<BN, A_MN, B_MN, CTA2, HEAVY, EB>(pa, pb, 2);
 }
 
 // Diagnostic: one warp waits, with the same bounded wait the GEMM uses, on a barrier that nothing
