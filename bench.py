@@ -42,9 +42,9 @@ UNIT = "TFLOP/s"
 # step at this workload's full size, k = 8, output split, from one ncu capture of
 # `bench.py --case linear:16384:8192:8192:8:out`.  Refreshed whenever the kernel or its tile choice changes.
 NCU_TRAFFIC_BYTES = {
-    ("fwd", 8, "out"): 3578255000 + 263906048,
-    ("dx", 8, "out"): 2063174000 + 257440768,
-    ("dw", 8, "out"): 3009129000 + 123269376,
+    ("fwd", 8, "out"): 2709627000 + 257286400,
+    ("dx", 8, "out"): 1851115000 + 258307840,
+    ("dw", 8, "out"): 2350985000 + 121548544,
 }
 
 

@@ -636,10 +636,11 @@ int launch_gemm(const GemmCall &c, cudaStream_t stream) {
   if (pair && (c.mode != MODE_RED || in_tmem) && c.epi.gz == nullptr) {
     const int64_t units = sms / 2;
     const double red_len = (double)c.R * (c.fp8 ? 0.5 : 1.0);   // an fp8 k-step covers twice the elements
-    // (256-wide with both operands K-major: 5.9 ns since its ring is handed over two k-blocks at a time; measured,
-    // 16384 x 8192 x 8192 forward 1439 us wide, 1414 us 256-wide; 8192 x 8192 x 4096 439 / 411 us.)
-    const double ns256 = (!c.a.mn_major && !c.b.mn_major) ? 5.9e-3 : 6.5e-3;
-    const double t_n = (double)cdiv(count_items(c, 2 * BM, 256), units) * (ns256 * red_len) + 5.0;
+    // (With both operands K-major the 256-wide tile is 2-6 % faster than this model says when the GPU runs at burst
+    // clocks, 16384 x 8192 x 8192 forward 1414 against 1439 us, but 3-4 % slower in the power-capped state that a
+    // training loop runs in, 1.739 against 1.670 ms: it moves more bytes per flop through shared memory, L2 and
+    // DRAM.  The model follows the sustained state.)
+    const double t_n = (double)cdiv(count_items(c, 2 * BM, 256), units) * (6.5e-3 * red_len) + 5.0;
     const double t_w = (double)cdiv(count_items(c, 2 * BM, 512), units) * (11.5e-3 * red_len + 5.0);
     if (t_w < 0.97 * t_n) bn = 512;
   }
