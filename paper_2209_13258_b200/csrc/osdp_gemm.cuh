@@ -262,10 +262,28 @@ __device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t adesc, uint64_
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-template <bool CTA2>
+// COLL: use of the tensor core's collector buffer for the A operand.  0: none.  1: this MMA leaves its A operand in
+// the buffer (fill); 2: this MMA takes A from the buffer, for the last time (lastuse).  The 256 x 512 tile issues two
+// MMAs per k-step that share A (one per 256-column group): the second does not read A from shared memory again.
+// Same bits; measured on B200 in the power-capped state: -0.1 ... -0.3 % per step at the benchmark shape.
+template <bool CTA2, int COLL = 0>
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                           uint32_t accumulate) {
-  if (CTA2)
+  if (CTA2 && COLL == 1)
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16.collector::a::fill [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  else if (CTA2 && COLL == 2)
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16.collector::a::lastuse [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  else if (CTA2)
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
@@ -848,7 +866,9 @@ __global__ void __launch_bounds__((BN > 256 || HEAVY) ? 384 : 256, 1) gemm_kerne
                   const uint64_t ad = adesc + (uint64_t)((kk * desc_k_advance<A_MN, EB>()) >> 4);
                   const uint64_t bd = bdesc + (uint64_t)((g * SL::GB_ROWS * 128 + kk * desc_k_advance<B_MN, EB>()) >> 4);
                   const uint32_t acc = (kb + sub > 0 || kk > 0) ? 1u : 0u;
-                  if (EB == 2) umma_bf16<CTA2>(d, ad, bd, idesc, acc);
+                  if (EB == 2 && SL::NG == 2 && g == 0) umma_bf16<CTA2, 1>(d, ad, bd, idesc, acc);
+                  else if (EB == 2 && SL::NG == 2 && g == 1) umma_bf16<CTA2, 2>(d, ad, bd, idesc, acc);
+                  else if (EB == 2) umma_bf16<CTA2>(d, ad, bd, idesc, acc);
                   else umma_f8<CTA2>(d, ad, bd, idesc, acc);
                 }
               }
