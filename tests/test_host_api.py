@@ -235,3 +235,17 @@ def test_mlp_backward_staging_sets():
     # the forward keeps one set whatever the size
     assert P.osdp_split_linear_workspace_bytes(4096, 4096, 1024, 8, 0, 1, P.OP_MLP_FWD)[1] == \
         256 + 4096 * 1024 * 4 + 4096 * 512 * 2
+
+
+def test_carry_is_sized_in_boxes_of_32_by_32():
+    """The fp32 running sum of a slice-major summed output is stored as 32 x 32 boxes: both extents are padded."""
+    up = lambda v, a: -(-v // a) * a
+    for (M, N, K) in ((200, 264, 520), (4096, 1024, 4096), (33, 40, 72)):
+        # forward under RED, slice-major: status block + carry [M, N] + nothing else
+        rc, got = P.osdp_split_linear_workspace_bytes(M, N, K, 3, P.SPLIT_RED, 0, P.OP_LINEAR_FWD, P.FLAG_SLICE_MAJOR)
+        assert rc == 0 and got == 256 + up(up(M, 32) * up(N, 32) * 4, 256), (M, N, K, got)
+        # default order: the sum stays in tensor memory, no carry
+        assert P.osdp_split_linear_workspace_bytes(M, N, K, 3, P.SPLIT_RED, 0, P.OP_LINEAR_FWD, 0) == (0, 256)
+        # backward under OUT, slice-major: carry [M, K] + column-sum partials
+        rc, got = P.osdp_split_linear_workspace_bytes(M, N, K, 3, P.SPLIT_OUT, 0, P.OP_LINEAR_BWD, P.FLAG_SLICE_MAJOR)
+        assert rc == 0 and got == 256 + up(up(M, 32) * up(K, 32) * 4, 256) + up(-(-M // 1024) * N * 4, 256), (M, N, K, got)
