@@ -531,6 +531,45 @@ def test_cuda_graph_replay_matches_eager(P):
 
 
 @pytest.mark.parametrize("k", [2, 5])
+def test_mlp_backward_with_subsets_of_outputs(P, k):
+    """Every output of the MLP block's backward is optional; whatever is asked for has the same bits as in the call
+    that asks for everything (k = 5: the slices are pipelined over two sets of slice buffers, with the weight
+    gradients on the internal streams; without weight gradients nothing is forked)."""
+    M, H, F = 300, 264, 520
+    c = inputs.mlp_case(M, H, F, w_std=0.08, layer=29)
+    x, dy, wf = to_dev(c["x"]), to_dev(c["dy"]), to_dev(c["w_flat"])
+    b1, b2 = to_dev(c["b1"]), to_dev(c["b2"])
+    _, n1 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, 1, P.OP_MLP_FWD)
+    _, n2 = P.osdp_split_linear_workspace_bytes(M, F, H, k, 0, 1, P.OP_MLP_BWD)
+    ws = P.new_workspace(max(n1, n2))
+    y = torch.empty(M, H, dtype=torch.bfloat16, device="cuda")
+    z1 = torch.empty(M, F, dtype=torch.bfloat16, device="cuda")
+    P.osdp_split_mlp_fwd(x, wf, c["off_w1"], b1, c["off_w2"], b2, M, H, F, k, 1, y, z1, ws, check=True)
+
+    def bwd(want_dx, want_dw, want_db):
+        dx = torch.full((M, H), 7.0, dtype=torch.bfloat16, device="cuda") if want_dx else None
+        dwf = torch.full((2 * F * H,), 7.0, dtype=torch.float32, device="cuda") if want_dw else None
+        db1 = torch.full((F,), 7.0, dtype=torch.float32, device="cuda") if want_db else None
+        db2 = torch.full((H,), 7.0, dtype=torch.float32, device="cuda") if want_db else None
+        P.osdp_split_mlp_bwd(dy, x, wf, c["off_w1"], c["off_w2"], z1, M, H, F, k, 1, dx, dwf, c["off_w1"], c["off_w2"],
+                             P.DTYPE_FP32, 0, db1, db2, ws, check=True)
+        torch.cuda.synchronize()
+        return {"dx": dx, "dw": dwf, "db1": db1, "db2": db2}
+
+    full = bwd(True, True, True)
+    grads = oracle.mlp_bwd(c["dy"], c["x"], c["w1"], c["b1"], c["w2"], oracle.ACT_GELU_TANH, k)
+    assert_close(to_f64(full["dx"]), grads[0], "dx")
+    assert_close(to_f64(full["db1"]), grads[2], "db1")
+    for want in ((True, False, False), (False, True, False), (False, False, True), (True, False, True),
+                 (False, True, True), (True, True, False)):
+        part = bwd(*want)
+        for name, t in part.items():
+            if t is not None:
+                assert torch.equal(_bits(t), _bits(full[name])), (want, name)
+    assert P.osdp_read_device_status(ws) == (0, 0)
+
+
+@pytest.mark.parametrize("k", [2, 5])
 def test_mlp_cuda_graph_replay_matches_eager(P, k):
     """The MLP block's backward forks onto the library's internal streams (k = 5, small slices: pipelined over
     two sets of slice buffers; k = 2: one fork / join per slice); a capture follows them and replays the same bits."""
